@@ -1,0 +1,188 @@
+/*
+ * pipesd.h -- C ABI of the cloud-side non-autoregressive verification (NAV) pass of speculative
+ * decoding, implemented as hand-written CUDA kernels for sm_100a.
+ *
+ * The operation (paper Sec. 2.2 and Sec. 3.1 step 4): the edge sends k draft tokens; the cloud
+ * validates them with ONE forward pass of the target model against the already accepted prefix,
+ * accepts drafts up to the first failure, lets the target model correct that token, and -- when
+ * every draft passes -- contributes one extra token (App. B).  The accepted and corrected tokens
+ * become the prefix of the next round, the rejected tail is discarded (App. B).  The acceptance
+ * test is the speculative-sampling rule of the works the paper builds on, which is what keeps
+ * the target model's output distribution unchanged (Sec. 1): accept draft x_i while
+ * u_i < min(1, p(x_i)/q(x_i)), otherwise draw from norm(max(0, p - q)).
+ *
+ * Conventions
+ *   - Every function returns PIPESD_OK (0) or a negative pipesd_status.  Nothing throws, aborts or
+ *     traps; after an error the context stays usable unless the error is PIPESD_E_CUDA.
+ *   - "host" / "device" in a comment says where a pointer must live.  The library allocates no
+ *     device memory: the caller provides the three device buffers sized by pipesd_query_sizes and
+ *     owns them until pipesd_ctx_destroy.  The library owns small pinned host staging buffers.
+ *   - All device work is enqueued on the stream given to pipesd_ctx_create (a cudaStream_t passed
+ *     as void*).  A context is not thread-safe.
+ *   - Model: Llama-style decoder (RMSNorm, rotary embedding with "rotate-half" pairing, grouped
+ *     query attention, SwiGLU FFN, untied LM head), bf16 weights, fp32 activations, bf16 KV cache.
+ *     d_model, d_ffn, vocab and the head widths must be multiples of 16; head_dim is 64 or 128.
+ */
+#ifndef PIPESD_H
+#define PIPESD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum pipesd_status {
+    PIPESD_OK = 0,
+    PIPESD_E_INVALID = -1,     /* null pointer, out-of-range argument, unsupported shape      */
+    PIPESD_E_FULL = -2,        /* no free request slot                                        */
+    PIPESD_E_OOM_PAGES = -3,   /* KV page pool exhausted; the call changed nothing            */
+    PIPESD_E_STATE = -4,       /* call order violated (e.g. verify with an uncommitted tail)  */
+    PIPESD_E_RANGE = -5,       /* length / count outside what the request state allows        */
+    PIPESD_E_CUDA = -6,        /* a CUDA runtime call failed; see pipesd_last_error           */
+    PIPESD_E_NOMEM = -7        /* a caller-provided buffer is smaller than pipesd_query_sizes */
+} pipesd_status;
+
+#define PIPESD_MODE_STOCHASTIC 0 /* u_i < min(1, p/q), residual resample, extra token ~ p */
+#define PIPESD_MODE_GREEDY 1     /* accept while draft == argmax (Sec. 2.2 prose); emit the argmax */
+
+#define PIPESD_Q_HOST 1u /* verify flag: item.q pointers are host memory; the library copies them */
+
+typedef struct pipesd_model_cfg {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    float rms_eps;
+    float rope_base;
+    int32_t page_size;    /* tokens per KV page (16)                                           */
+    int32_t n_pages;      /* pages in the pool; one page holds page_size positions of ALL layers */
+    int32_t max_requests; /* request slots                                                     */
+    int32_t max_draft;    /* largest k accepted by pipesd_verify (<= 31)                       */
+    int32_t max_rows;     /* largest sum of (k+1) over the items of one verify call            */
+    int32_t max_seq;      /* largest number of cached positions per request                    */
+    int32_t device;       /* CUDA device ordinal                                               */
+} pipesd_model_cfg;
+
+/* Device pointers to row-major [out, in] bf16 matrices; norm gains are fp32 [d_model]. */
+typedef struct pipesd_layer_weights {
+    const void *wq, *wk, *wv; /* [n_q_heads*head_dim, d_model], [n_kv_heads*head_dim, d_model] x2 */
+    const void *wo;           /* [d_model, n_q_heads*head_dim]                                    */
+    const void *wg, *wu;      /* [d_ffn, d_model]                                                 */
+    const void *wd;           /* [d_model, d_ffn]                                                 */
+    const float *attn_norm, *ffn_norm;
+} pipesd_layer_weights;
+
+typedef struct pipesd_weights {
+    const void *tok_emb;                /* device, bf16 [vocab, d_model]         */
+    const void *lm_head;                /* device, bf16 [vocab, d_model]         */
+    const float *final_norm;            /* device, fp32 [d_model]                */
+    const pipesd_layer_weights *layers; /* HOST array of n_layers entries        */
+} pipesd_weights;
+
+typedef struct pipesd_sizes {
+    uint64_t weights_bytes;   /* repacked weights                    */
+    uint64_t kv_bytes;        /* paged bf16 KV pool                  */
+    uint64_t workspace_bytes; /* activations, partial sums, metadata */
+} pipesd_sizes;
+
+/* Caller-allocated device buffers (256-byte aligned), at least as large as pipesd_query_sizes says. */
+typedef struct pipesd_mem {
+    void *weights; uint64_t weights_bytes;
+    void *kv; uint64_t kv_bytes;
+    void *workspace; uint64_t workspace_bytes;
+} pipesd_mem;
+
+/* One request of a verify call.  tokens[0] is the pending token (the previous round's correction
+ * or extra token, whose KV is not cached yet), tokens[1..k] the drafts.  Row i of the forward
+ * scores draft i+1; row k gives the extra-token distribution. */
+typedef struct pipesd_verify_item {
+    int32_t req;           /* request slot from pipesd_req_open                                  */
+    int32_t k;             /* number of drafts, 1..max_draft                                     */
+    int32_t mode;          /* PIPESD_MODE_*                                                      */
+    int32_t reserved;
+    const int32_t *tokens; /* host, k+1 ids                                                      */
+    const float *q;        /* device (host with PIPESD_Q_HOST), fp32 [k, vocab] row-major draft  */
+                           /* probabilities; ignored (may be null) in greedy mode                */
+    const float *u;        /* host, k+1 uniforms in [0,1): u[0..k-1] acceptance tests, u[k] the  */
+                           /* single final draw (correction or extra token)                      */
+} pipesd_verify_item;
+
+typedef struct pipesd_verify_result {
+    int32_t n_accepted; /* 0..k                                                            */
+    int32_t next_token; /* correction token if n_accepted < k, else the extra token        */
+    int32_t status;     /* PIPESD_OK, or the device-side error of this request             */
+    int32_t reserved;
+} pipesd_verify_result;
+
+typedef struct pipesd_ctx pipesd_ctx;
+
+const char *pipesd_strerror(int32_t status);
+/* Text of the most recent error on this context (host string owned by the context). */
+const char *pipesd_last_error(const pipesd_ctx *ctx);
+
+/* Bytes the caller must provide for a configuration.  Pure function of cfg. */
+int32_t pipesd_query_sizes(const pipesd_model_cfg *cfg, pipesd_sizes *out);
+
+/* Create a context: validates cfg, repacks the caller's weights into mem->weights (the caller may
+ * free its own weight tensors once pipesd_ctx_sync has returned), zero-initialises metadata.
+ * `cuda_stream` is a cudaStream_t (null = the legacy default stream). */
+int32_t pipesd_ctx_create(const pipesd_model_cfg *cfg, const pipesd_weights *w, const pipesd_mem *mem,
+                          void *cuda_stream, pipesd_ctx **out);
+/* Releases host state and pinned staging; the caller's device buffers are untouched. */
+int32_t pipesd_ctx_destroy(pipesd_ctx *ctx);
+/* Waits for the stream; delivers pending verify results to the caller's array. */
+int32_t pipesd_ctx_sync(pipesd_ctx *ctx);
+
+/* Request slots: an empty block table / return of all its pages to the pool. */
+int32_t pipesd_req_open(pipesd_ctx *ctx, int32_t *req);
+int32_t pipesd_req_close(pipesd_ctx *ctx, int32_t req);
+/* Committed length (cached positions) of a request. */
+int32_t pipesd_req_len(pipesd_ctx *ctx, int32_t req, int32_t *len);
+
+/* Append n prompt tokens (host ids) to the request's cache: the same layer stack as verify run in
+ * chunks of max_rows rows, no acceptance step.  If last_logits (host, vocab floats) is non-null it
+ * receives the logits of the final position; the call then synchronises. */
+int32_t pipesd_prefill(pipesd_ctx *ctx, int32_t req, const int32_t *tokens, int32_t n, float *last_logits);
+
+/* The NAV pass over n_req requests in one batch (Sec. 2.2; multi-edge serving, App. I): forward of
+ * each item's k+1 tokens against its cached prefix, the accept/correct rule, K/V of all k+1
+ * positions written speculatively.  results (host, n_req entries) is filled when the next
+ * pipesd_ctx_sync returns.  Each request must then be committed with pipesd_kv_rollback before it
+ * can be verified again (PIPESD_E_STATE otherwise). */
+int32_t pipesd_verify(pipesd_ctx *ctx, int32_t n_req, const pipesd_verify_item *items,
+                      pipesd_verify_result *results, uint32_t flags);
+
+/* Commit / rollback (App. B: rejected drafts are discarded, generation restarts after the last
+ * accepted token): length <- base + 1 + n_accepted[i] with 0 <= n_accepted[i] <= k of the
+ * request's last verify; pages wholly beyond the new length return to the pool.  No KV bytes move;
+ * rows of the rejected tail are never read again. */
+int32_t pipesd_kv_rollback(pipesd_ctx *ctx, int32_t n_req, const int32_t *reqs, const int32_t *n_accepted);
+
+/* ---- component entry points (used for per-kernel parity and bandwidth measurements) ---- */
+
+/* fp32 logits [rows, vocab] of the most recent verify / prefill chunk -> host buffer. Synchronises. */
+int32_t pipesd_debug_get_logits(pipesd_ctx *ctx, float *dst, int32_t rows);
+/* Read / write cached K and V rows of one layer as bf16 bit patterns, host [n_pos, n_kv_heads*head_dim].
+ * Writing beyond the committed length extends it (pages are allocated).  Synchronises. */
+int32_t pipesd_debug_read_kv(pipesd_ctx *ctx, int32_t req, int32_t layer, int32_t pos0, int32_t n_pos,
+                             uint16_t *k, uint16_t *v);
+int32_t pipesd_debug_write_kv(pipesd_ctx *ctx, int32_t req, int32_t layer, int32_t pos0, int32_t n_pos,
+                              const uint16_t *k, const uint16_t *v);
+/* The accept/correct rule alone on caller-supplied logits (host fp32 [k+1, vocab]), q (host fp32
+ * [k, vocab]), drafts (host, k ids), u (host, k+1).  Synchronises. */
+int32_t pipesd_reject_from_logits(pipesd_ctx *ctx, int32_t k, int32_t mode, const float *logits,
+                                  const float *q, const int32_t *drafts, const float *u,
+                                  pipesd_verify_result *result);
+
+/* Small-M weight-streaming GEMM on its own: y[M,N] = x[M,K] . W[N,K]^T with bf16 W, fp32 x and y.
+ * pipesd_gemm_packed_bytes: size of the repacked copy of W.  pipesd_gemm_pack: W (device, row-major
+ * bf16 [N,K]) -> packed (device).  pipesd_gemm_run: x, y device; scratch device of
+ * pipesd_gemm_scratch_bytes(M,N,K) bytes (split-K partial sums).  N, K multiples of 16. */
+uint64_t pipesd_gemm_packed_bytes(int32_t N, int32_t K);
+uint64_t pipesd_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
+int32_t pipesd_gemm_pack(const void *W, void *packed, int32_t N, int32_t K, void *cuda_stream);
+int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scratch, int32_t M, int32_t N,
+                        int32_t K, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PIPESD_H */

@@ -1,0 +1,835 @@
+// Host engine and C ABI of the NAV verify library: context, paged-KV bookkeeping, launch plan.
+// Every step of the pass runs in the kernels of this directory; the host only validates, keeps the
+// page tables and request lengths, uploads the per-call metadata and launches.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/pipesd.h"
+#include "attention.cuh"
+#include "common.cuh"
+#include "gemm.cuh"
+#include "layers.cuh"
+#include "reject.cuh"
+
+using namespace pipesd;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+struct Request {
+    bool open = false;
+    int len = 0;        // committed positions
+    int tentative = 0;  // rows written by a verify that has not been committed yet (k+1), else 0
+    std::vector<int> pages;
+};
+
+struct GemmW {
+    uint4* packed = nullptr;
+    int N = 0, K = 0;
+};
+
+struct LayerW {
+    GemmW qkv, o, gu, dn;
+    float *n1 = nullptr, *n2 = nullptr;
+};
+
+// Fixed offsets of the per-call metadata block (same layout in pinned host staging and on device).
+struct MetaLayout {
+    size_t row_item, row_pos, row_tok, it_slot, it_row0, it_rows, it_base, it_nsplit, it_chunk, it_part0, u, rej, total;
+};
+
+MetaLayout meta_layout(int max_rows, int max_items) {
+    MetaLayout m;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 16); return r; };
+    m.row_item = take(4 * (size_t)max_rows);
+    m.row_pos = take(4 * (size_t)max_rows);
+    m.row_tok = take(4 * (size_t)max_rows);
+    m.it_slot = take(4 * (size_t)max_items);
+    m.it_row0 = take(4 * (size_t)max_items);
+    m.it_rows = take(4 * (size_t)max_items);
+    m.it_base = take(4 * (size_t)max_items);
+    m.it_nsplit = take(4 * (size_t)max_items);
+    m.it_chunk = take(4 * (size_t)max_items);
+    m.it_part0 = take(4 * (size_t)max_items);
+    m.u = take(4 * (size_t)max_rows);
+    m.rej = take(sizeof(RejectItem) * (size_t)max_items);
+    m.total = align_up(o);
+    return m;
+}
+
+struct Derived {
+    int Nqkv, qd, kvd, max_pages, max_items;
+    size_t part_floats;  // largest split-K partial array over all GEMMs and row counts
+};
+
+Derived derive(const pipesd_model_cfg& c) {
+    Derived d;
+    d.qd = c.n_q_heads * c.head_dim;
+    d.kvd = c.n_kv_heads * c.head_dim;
+    d.Nqkv = d.qd + 2 * d.kvd;
+    d.max_pages = (c.max_seq + c.page_size - 1) / c.page_size;
+    d.max_items = std::min(c.max_requests, c.max_rows);
+    size_t best = 0;
+    const int shapes[5][2] = {{d.Nqkv, c.d_model}, {c.d_model, d.qd}, {2 * c.d_ffn, c.d_model},
+                              {c.d_model, c.d_ffn}, {c.vocab, c.d_model}};
+    for (int m = 1; m <= c.max_rows; ++m)
+        for (auto& s : shapes) {
+            GemmPlan p = gemm_plan(m, s[0], s[1]);
+            best = std::max(best, (size_t)p.S * m * s[0]);
+        }
+    d.part_floats = best;
+    return d;
+}
+
+struct WsLayout {
+    size_t x, h, qbuf, attn, act, logits, partA, partB, o_part, m_part, l_part, cs, sn, stats, results, meta,
+        block_tab, qstage, total;
+};
+
+WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
+    WsLayout w;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
+    const size_t M = c.max_rows;
+    w.x = take(4 * M * c.d_model);
+    w.h = take(4 * M * c.d_model);
+    w.qbuf = take(4 * M * d.qd);
+    w.attn = take(4 * M * d.qd);
+    w.act = take(4 * M * c.d_ffn);
+    w.logits = take(4 * M * c.vocab);
+    w.partA = take(4 * d.part_floats);
+    w.partB = take(4 * d.part_floats);
+    const size_t slots = M * c.n_q_heads * kMaxSplits;
+    w.o_part = take(4 * slots * c.head_dim);
+    w.m_part = take(4 * slots);
+    w.l_part = take(4 * slots);
+    w.cs = take(4 * M * (c.head_dim / 2));
+    w.sn = take(4 * M * (c.head_dim / 2));
+    w.stats = take(sizeof(RowStat) * M * kStatSplits);
+    w.results = take(sizeof(RejectOut) * d.max_items);
+    w.meta = take(meta_layout(c.max_rows, d.max_items).total);
+    w.block_tab = take(4 * (size_t)c.max_requests * d.max_pages);
+    w.qstage = take(4 * M * c.vocab);
+    w.total = o;
+    return w;
+}
+
+size_t packed_bytes(int N, int K) { return align_up((size_t)N * K * 2); }
+
+size_t weights_bytes(const pipesd_model_cfg& c, const Derived& d) {
+    size_t per_layer = packed_bytes(d.Nqkv, c.d_model) + packed_bytes(c.d_model, d.qd) +
+                       packed_bytes(2 * c.d_ffn, c.d_model) + packed_bytes(c.d_model, c.d_ffn) +
+                       2 * align_up(4 * (size_t)c.d_model);
+    return (size_t)c.n_layers * per_layer + align_up((size_t)c.vocab * c.d_model * 2) +
+           packed_bytes(c.vocab, c.d_model) + align_up(4 * (size_t)c.d_model);
+}
+
+size_t kv_bytes(const pipesd_model_cfg& c) {
+    return (size_t)c.n_layers * c.n_pages * 2 * c.n_kv_heads * c.page_size * c.head_dim * 2;
+}
+
+int check_cfg(const pipesd_model_cfg* c) {
+    if (!c) return PIPESD_E_INVALID;
+    if (c->n_layers < 1 || c->d_model < 16 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->d_ffn < 16 ||
+        c->vocab < 16)
+        return PIPESD_E_INVALID;
+    if (c->head_dim != 64 && c->head_dim != 128) return PIPESD_E_INVALID;
+    if (c->d_model % 16 || c->d_ffn % 16 || c->vocab % 16) return PIPESD_E_INVALID;
+    if (c->n_q_heads % c->n_kv_heads) return PIPESD_E_INVALID;
+    if (c->page_size < 1 || c->page_size > 256 || c->n_pages < 1 || c->max_requests < 1) return PIPESD_E_INVALID;
+    if (c->max_draft < 1 || c->max_draft > kMaxItemRows - 1) return PIPESD_E_INVALID;
+    if (c->max_rows < c->max_draft + 1 || c->max_rows > 4096 || c->max_seq < 1) return PIPESD_E_INVALID;
+    if (!(c->rms_eps >= 0.f) || !(c->rope_base > 1.f)) return PIPESD_E_INVALID;
+    return PIPESD_OK;
+}
+
+// Copy rows of one layer between a contiguous [n_pos][Hkv*hd] bf16 staging array and the pages.
+__global__ void kv_copy_kernel(uint16_t* __restrict__ kv_pool, uint16_t* __restrict__ stage_k,
+                               uint16_t* __restrict__ stage_v, const int32_t* __restrict__ bt, int pos0, int n_pos,
+                               int layer, int n_pages, int page_size, int Hkv, int hd, int to_pool) {
+    const int w = Hkv * hd;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)n_pos * w;
+         i += (size_t)gridDim.x * blockDim.x) {
+        int p = (int)(i / w), c = (int)(i % w), head = c / hd, e = c % hd;
+        int pos = pos0 + p, page = bt[pos / page_size], slot = pos % page_size;
+        size_t ko = kv_index(layer, n_pages, page, 0, Hkv, head, page_size, slot, hd, e);
+        size_t vo = kv_index(layer, n_pages, page, 1, Hkv, head, page_size, slot, hd, e);
+        if (to_pool) { kv_pool[ko] = stage_k[i]; kv_pool[vo] = stage_v[i]; }
+        else { stage_k[i] = kv_pool[ko]; stage_v[i] = kv_pool[vo]; }
+    }
+}
+
+}  // namespace
+
+struct pipesd_ctx {
+    pipesd_model_cfg cfg;
+    Derived dv;
+    WsLayout ws;
+    MetaLayout ml;
+    cudaStream_t st = nullptr;
+    // device
+    uint16_t* emb = nullptr;
+    GemmW lm;
+    float* final_norm = nullptr;
+    std::vector<LayerW> layers;
+    uint16_t* kv_pool = nullptr;
+    char* wsp = nullptr;
+    // host
+    std::vector<Request> reqs;
+    std::vector<int> free_pages;
+    static constexpr int kStages = 4;
+    char* h_meta[kStages] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ev_meta[kStages] = {nullptr, nullptr, nullptr, nullptr};
+    int stage = 0;
+    RejectOut* h_results = nullptr;
+    pipesd_verify_result* pend_dst = nullptr;
+    int pend_n = 0;
+    int last_rows = 0;
+    std::string err;
+
+    template <typename T>
+    T* W(size_t off) const { return reinterpret_cast<T*>(wsp + off); }
+    PassMeta pass_meta() const {
+        PassMeta m;
+        const char* b = wsp + ws.meta;
+        m.row_item = (const int32_t*)(b + ml.row_item);
+        m.row_pos = (const int32_t*)(b + ml.row_pos);
+        m.row_tok = (const int32_t*)(b + ml.row_tok);
+        m.it_slot = (const int32_t*)(b + ml.it_slot);
+        m.it_row0 = (const int32_t*)(b + ml.it_row0);
+        m.it_rows = (const int32_t*)(b + ml.it_rows);
+        m.it_base = (const int32_t*)(b + ml.it_base);
+        m.it_nsplit = (const int32_t*)(b + ml.it_nsplit);
+        m.it_chunk = (const int32_t*)(b + ml.it_chunk);
+        m.it_part0 = (const int32_t*)(b + ml.it_part0);
+        m.block_tab = W<int32_t>(ws.block_tab);
+        m.max_pages = dv.max_pages;
+        return m;
+    }
+};
+
+namespace {
+
+int fail(pipesd_ctx* c, int code, const char* what) {
+    if (c) c->err = std::string(pipesd_strerror(code)) + ": " + what;
+    return code;
+}
+
+int cuda_fail(pipesd_ctx* c, cudaError_t e, const char* where) {
+    if (c) c->err = std::string("CUDA error at ") + where + ": " + cudaGetErrorString(e);
+    return PIPESD_E_CUDA;
+}
+
+#define CU(call)                                                    \
+    do {                                                            \
+        cudaError_t e_ = (call);                                    \
+        if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);    \
+    } while (0)
+
+struct ItemDesc {
+    int slot, rows, mode, k;
+    const int32_t* tokens;  // host, rows ids
+    const float* q;         // device
+    const float* u;         // host, k+1 (null when mode == 2)
+};
+
+// Make sure the request owns pages for `need_len` positions. All-or-nothing is checked by the caller.
+int pages_needed(const pipesd_ctx* c, const Request& r, int need_len) {
+    int need = (need_len + c->cfg.page_size - 1) / c->cfg.page_size;
+    return std::max(0, need - (int)r.pages.size());
+}
+
+int grow_pages(pipesd_ctx* ctx, int slot, int need_len) {
+    Request& r = ctx->reqs[slot];
+    int add = pages_needed(ctx, r, need_len);
+    if (add == 0) return PIPESD_OK;
+    int first = (int)r.pages.size();
+    for (int i = 0; i < add; ++i) {
+        r.pages.push_back(ctx->free_pages.back());
+        ctx->free_pages.pop_back();
+    }
+    int32_t* dst = ctx->W<int32_t>(ctx->ws.block_tab) + (size_t)slot * ctx->dv.max_pages + first;
+    CU(cudaMemcpyAsync(dst, r.pages.data() + first, 4 * (size_t)add, cudaMemcpyHostToDevice, ctx->st));
+    return PIPESD_OK;
+}
+
+void shrink_pages(pipesd_ctx* c, Request& r, int keep_len) {
+    int keep = (keep_len + c->cfg.page_size - 1) / c->cfg.page_size;
+    while ((int)r.pages.size() > keep) {
+        c->free_pages.push_back(r.pages.back());
+        r.pages.pop_back();
+    }
+}
+
+// Upload the metadata of one pass and run the layer stack over M rows.
+int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logits, bool want_reject) {
+    const pipesd_model_cfg& c = ctx->cfg;
+    const Derived& dv = ctx->dv;
+    const int n_items = (int)items.size();
+    int M = 0;
+    for (auto& it : items) M += it.rows;
+
+    // ---- metadata
+    const int sidx = ctx->stage;
+    ctx->stage = (ctx->stage + 1) % pipesd_ctx::kStages;
+    CU(cudaEventSynchronize(ctx->ev_meta[sidx]));
+    char* hm = ctx->h_meta[sidx];
+    const MetaLayout& ml = ctx->ml;
+    auto I = [&](size_t off) { return reinterpret_cast<int32_t*>(hm + off); };
+    float* hu = reinterpret_cast<float*>(hm + ml.u);
+    RejectItem* hr = reinterpret_cast<RejectItem*>(hm + ml.rej);
+    // split policy: aim at two waves of CTAs over all (item, head, split) triples
+    int target = std::max(1, (2 * kWaveCtas + n_items * c.n_q_heads - 1) / (n_items * c.n_q_heads));
+    int row = 0, part0 = 0, max_nsplit = 1, u0 = 0;
+    for (int i = 0; i < n_items; ++i) {
+        const ItemDesc& it = items[i];
+        const Request& r = ctx->reqs[it.slot];
+        const int total = r.len + it.rows;
+        int chunk = (total + target - 1) / target;
+        chunk = std::max(chunk, 64);
+        chunk = std::max(chunk, (total + kMaxSplits - 1) / kMaxSplits);
+        chunk = (chunk + c.page_size - 1) / c.page_size * c.page_size;
+        int nsplit = (total + chunk - 1) / chunk;
+        I(ml.it_slot)[i] = it.slot;
+        I(ml.it_row0)[i] = row;
+        I(ml.it_rows)[i] = it.rows;
+        I(ml.it_base)[i] = r.len;
+        I(ml.it_nsplit)[i] = nsplit;
+        I(ml.it_chunk)[i] = chunk;
+        I(ml.it_part0)[i] = part0;
+        max_nsplit = std::max(max_nsplit, nsplit);
+        part0 += it.rows * c.n_q_heads * nsplit;
+        hr[i].row0 = row;
+        hr[i].k = it.k;
+        hr[i].mode = it.mode;
+        hr[i].u0 = u0;
+        hr[i].q = it.q;
+        for (int j = 0; j < it.rows; ++j) {
+            I(ml.row_item)[row + j] = i;
+            I(ml.row_pos)[row + j] = r.len + j;
+            I(ml.row_tok)[row + j] = it.tokens[j];
+        }
+        for (int j = 0; j <= it.k; ++j) hu[u0 + j] = it.u ? it.u[j] : 0.f;
+        u0 += it.k + 1;
+        row += it.rows;
+    }
+    CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.meta, hm, ml.total, cudaMemcpyHostToDevice, ctx->st));
+    CU(cudaEventRecord(ctx->ev_meta[sidx], ctx->st));
+
+    // ---- layer stack
+    const PassMeta meta = ctx->pass_meta();
+    cudaStream_t st = ctx->st;
+    float* x = ctx->W<float>(ctx->ws.x);
+    float* h = ctx->W<float>(ctx->ws.h);
+    float* qbuf = ctx->W<float>(ctx->ws.qbuf);
+    float* attn = ctx->W<float>(ctx->ws.attn);
+    float* act = ctx->W<float>(ctx->ws.act);
+    float* partA = ctx->W<float>(ctx->ws.partA);
+    float* partB = ctx->W<float>(ctx->ws.partB);
+    float* o_part = ctx->W<float>(ctx->ws.o_part);
+    float* m_part = ctx->W<float>(ctx->ws.m_part);
+    float* l_part = ctx->W<float>(ctx->ws.l_part);
+    float* cs = ctx->W<float>(ctx->ws.cs);
+    float* sn = ctx->W<float>(ctx->ws.sn);
+    const int hd = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads, d = c.d_model, F = c.d_ffn;
+
+    {
+        int n = M * hd / 2;
+        rope_table_kernel<<<(n + 127) / 128, 128, 0, st>>>(meta.row_pos, M, hd, log((double)c.rope_base), cs, sn);
+    }
+    const float* part = nullptr;
+    int S = 0;
+    const size_t asmem = attn_smem_bytes(hd);
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerW& lw = ctx->layers[l];
+        add_norm_kernel<<<M, 256, 0, st>>>(x, l == 0 ? ctx->emb : nullptr, meta.row_tok, part, S, M, lw.n1,
+                                           c.rms_eps, d, h);
+        GemmPlan p = gemm_plan(M, dv.Nqkv, d);
+        CU(gemm_launch(p, lw.qkv.packed, h, d, partA, M, dv.Nqkv, d, st));
+        rope_kv_kernel<<<dim3(M, Hq + 2 * Hkv), hd / 2, 0, st>>>(partA, p.S, M, Hq, Hkv, hd, cs, sn, meta, qbuf,
+                                                                 ctx->kv_pool, l, c.n_pages, c.page_size);
+        dim3 ag(max_nsplit, Hq, n_items);
+        if (hd == 128)
+            attn_split_kernel<128><<<ag, kAttnThreads, asmem, st>>>(qbuf, meta, ctx->kv_pool, l, c.n_pages,
+                                                                    c.page_size, Hq, Hkv, o_part, m_part, l_part);
+        else
+            attn_split_kernel<64><<<ag, kAttnThreads, asmem, st>>>(qbuf, meta, ctx->kv_pool, l, c.n_pages,
+                                                                   c.page_size, Hq, Hkv, o_part, m_part, l_part);
+        attn_combine_kernel<<<dim3(M, Hq), hd, 0, st>>>(o_part, m_part, l_part, meta, Hq, hd, attn);
+        p = gemm_plan(M, d, dv.qd);
+        CU(gemm_launch(p, lw.o.packed, attn, dv.qd, partB, M, d, dv.qd, st));
+        add_norm_kernel<<<M, 256, 0, st>>>(x, nullptr, nullptr, partB, p.S, M, lw.n2, c.rms_eps, d, h);
+        p = gemm_plan(M, 2 * F, d);
+        CU(gemm_launch(p, lw.gu.packed, h, d, partA, M, 2 * F, d, st));
+        {
+            size_t n = (size_t)M * F;
+            int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
+            silu_mul_kernel<<<blocks, 256, 0, st>>>(partA, p.S, M, F, act);
+        }
+        p = gemm_plan(M, d, F);
+        CU(gemm_launch(p, lw.dn.packed, act, F, partB, M, d, F, st));
+        part = partB;
+        S = p.S;
+    }
+    if (want_logits) {
+        float* logits = ctx->W<float>(ctx->ws.logits);
+        RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
+        add_norm_kernel<<<M, 256, 0, st>>>(x, nullptr, nullptr, part, S, M, ctx->final_norm, c.rms_eps, d, h);
+        GemmPlan p = gemm_plan(M, c.vocab, d);
+        float* dst = p.S == 1 ? logits : partA;
+        CU(gemm_launch(p, ctx->lm.packed, h, d, dst, M, c.vocab, d, st));
+        row_stats_kernel<<<dim3(M, kStatSplits), 256, 0, st>>>(p.S == 1 ? nullptr : partA, p.S, M, c.vocab, logits,
+                                                               stats);
+        ctx->last_rows = M;
+        if (want_reject) {
+            accept_sample_kernel<<<n_items, kSampleThreads, 0, st>>>(
+                logits, c.vocab, stats, reinterpret_cast<const RejectItem*>(ctx->wsp + ctx->ws.meta + ml.rej),
+                meta.row_tok, reinterpret_cast<const float*>(ctx->wsp + ctx->ws.meta + ml.u),
+                ctx->W<RejectOut>(ctx->ws.results));
+        }
+    }
+    CU(cudaGetLastError());
+    return PIPESD_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------- C ABI
+extern "C" {
+
+const char* pipesd_strerror(int32_t s) {
+    switch (s) {
+        case PIPESD_OK: return "ok";
+        case PIPESD_E_INVALID: return "invalid argument";
+        case PIPESD_E_FULL: return "no free request slot";
+        case PIPESD_E_OOM_PAGES: return "KV page pool exhausted";
+        case PIPESD_E_STATE: return "call order violated";
+        case PIPESD_E_RANGE: return "length out of range";
+        case PIPESD_E_CUDA: return "CUDA failure";
+        case PIPESD_E_NOMEM: return "caller buffer too small";
+        default: return "unknown status";
+    }
+}
+
+const char* pipesd_last_error(const pipesd_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int32_t pipesd_query_sizes(const pipesd_model_cfg* cfg, pipesd_sizes* out) {
+    int rc = check_cfg(cfg);
+    if (rc != PIPESD_OK || !out) return PIPESD_E_INVALID;
+    Derived d = derive(*cfg);
+    out->weights_bytes = weights_bytes(*cfg, d);
+    out->kv_bytes = kv_bytes(*cfg);
+    out->workspace_bytes = ws_layout(*cfg, d).total;
+    return PIPESD_OK;
+}
+
+int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, const pipesd_mem* mem,
+                          void* cuda_stream, pipesd_ctx** out) {
+    int rc = check_cfg(cfg);
+    if (rc != PIPESD_OK) return rc;
+    if (!w || !mem || !out || !w->tok_emb || !w->lm_head || !w->final_norm || !w->layers) return PIPESD_E_INVALID;
+    if (!mem->weights || !mem->kv || !mem->workspace) return PIPESD_E_INVALID;
+    pipesd_ctx* ctx = new (std::nothrow) pipesd_ctx();
+    if (!ctx) return PIPESD_E_INVALID;
+    ctx->cfg = *cfg;
+    ctx->dv = derive(*cfg);
+    ctx->ws = ws_layout(*cfg, ctx->dv);
+    ctx->ml = meta_layout(cfg->max_rows, ctx->dv.max_items);
+    ctx->st = (cudaStream_t)cuda_stream;
+    const pipesd_model_cfg& c = ctx->cfg;
+    const Derived& dv = ctx->dv;
+    auto bail = [&](int code) { pipesd_ctx_destroy(ctx); return code; };
+    if (mem->weights_bytes < weights_bytes(c, dv) || mem->kv_bytes < kv_bytes(c) ||
+        mem->workspace_bytes < ctx->ws.total)
+        return bail(PIPESD_E_NOMEM);
+    if (((uintptr_t)mem->weights | (uintptr_t)mem->kv | (uintptr_t)mem->workspace) & 255) return bail(PIPESD_E_INVALID);
+    cudaError_t e = cudaSetDevice(c.device);
+    if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
+    if ((e = gemm_init_attrs()) != cudaSuccess) return bail(PIPESD_E_CUDA);
+    e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes(128));
+    if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
+    e = cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes(64));
+    if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
+
+    ctx->kv_pool = (uint16_t*)mem->kv;
+    ctx->wsp = (char*)mem->workspace;
+    for (int i = 0; i < pipesd_ctx::kStages; ++i) {
+        if (cudaHostAlloc((void**)&ctx->h_meta[i], ctx->ml.total, cudaHostAllocDefault) != cudaSuccess)
+            return bail(PIPESD_E_CUDA);
+        if (cudaEventCreateWithFlags(&ctx->ev_meta[i], cudaEventDisableTiming) != cudaSuccess)
+            return bail(PIPESD_E_CUDA);
+    }
+    if (cudaHostAlloc((void**)&ctx->h_results, sizeof(RejectOut) * dv.max_items, cudaHostAllocDefault) != cudaSuccess)
+        return bail(PIPESD_E_CUDA);
+
+    // ---- repack the weights into the library's own layout
+    cudaStream_t st = ctx->st;
+    char* wp = (char*)mem->weights;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* p = wp + off; off += align_up(bytes); return p; };
+    auto pack = [&](GemmW& g, int N, int K, std::initializer_list<std::pair<const void*, int>> srcs) {
+        g.packed = (uint4*)take((size_t)N * K * 2);
+        g.N = N;
+        g.K = K;
+        int r0 = 0;
+        for (auto& s : srcs) {
+            size_t total = (size_t)(s.second / 16) * (K / 16) * 32;
+            int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
+            gemm_pack_kernel<<<blocks, 256, 0, st>>>((const uint16_t*)s.first,
+                                                     g.packed + (size_t)(r0 / 16) * (K / 16) * 32, s.second, K);
+            r0 += s.second;
+        }
+    };
+    ctx->emb = (uint16_t*)take((size_t)c.vocab * c.d_model * 2);
+    if (cudaMemcpyAsync(ctx->emb, w->tok_emb, (size_t)c.vocab * c.d_model * 2, cudaMemcpyDeviceToDevice, st) !=
+        cudaSuccess)
+        return bail(PIPESD_E_CUDA);
+    ctx->layers.resize(c.n_layers);
+    for (int l = 0; l < c.n_layers; ++l) {
+        const pipesd_layer_weights& s = w->layers[l];
+        if (!s.wq || !s.wk || !s.wv || !s.wo || !s.wg || !s.wu || !s.wd || !s.attn_norm || !s.ffn_norm)
+            return bail(PIPESD_E_INVALID);
+        LayerW& lw = ctx->layers[l];
+        pack(lw.qkv, dv.Nqkv, c.d_model, {{s.wq, dv.qd}, {s.wk, dv.kvd}, {s.wv, dv.kvd}});
+        pack(lw.o, c.d_model, dv.qd, {{s.wo, c.d_model}});
+        pack(lw.gu, 2 * c.d_ffn, c.d_model, {{s.wg, c.d_ffn}, {s.wu, c.d_ffn}});
+        pack(lw.dn, c.d_model, c.d_ffn, {{s.wd, c.d_model}});
+        lw.n1 = (float*)take(4 * (size_t)c.d_model);
+        lw.n2 = (float*)take(4 * (size_t)c.d_model);
+        cudaMemcpyAsync(lw.n1, s.attn_norm, 4 * (size_t)c.d_model, cudaMemcpyDeviceToDevice, st);
+        cudaMemcpyAsync(lw.n2, s.ffn_norm, 4 * (size_t)c.d_model, cudaMemcpyDeviceToDevice, st);
+    }
+    pack(ctx->lm, c.vocab, c.d_model, {{w->lm_head, c.vocab}});
+    ctx->final_norm = (float*)take(4 * (size_t)c.d_model);
+    cudaMemcpyAsync(ctx->final_norm, w->final_norm, 4 * (size_t)c.d_model, cudaMemcpyDeviceToDevice, st);
+    if (cudaGetLastError() != cudaSuccess) return bail(PIPESD_E_CUDA);
+
+    ctx->reqs.resize(c.max_requests);
+    ctx->free_pages.resize(c.n_pages);
+    for (int i = 0; i < c.n_pages; ++i) ctx->free_pages[i] = c.n_pages - 1 - i;
+    *out = ctx;
+    return PIPESD_OK;
+}
+
+int32_t pipesd_ctx_destroy(pipesd_ctx* ctx) {
+    if (!ctx) return PIPESD_E_INVALID;
+    if (ctx->wsp) cudaStreamSynchronize(ctx->st);
+    for (int i = 0; i < pipesd_ctx::kStages; ++i) {
+        if (ctx->h_meta[i]) cudaFreeHost(ctx->h_meta[i]);
+        if (ctx->ev_meta[i]) cudaEventDestroy(ctx->ev_meta[i]);
+    }
+    if (ctx->h_results) cudaFreeHost(ctx->h_results);
+    delete ctx;
+    return PIPESD_OK;
+}
+
+int32_t pipesd_ctx_sync(pipesd_ctx* ctx) {
+    if (!ctx) return PIPESD_E_INVALID;
+    CU(cudaStreamSynchronize(ctx->st));
+    if (ctx->pend_dst) {
+        for (int i = 0; i < ctx->pend_n; ++i) {
+            ctx->pend_dst[i].n_accepted = ctx->h_results[i].n_accepted;
+            ctx->pend_dst[i].next_token = ctx->h_results[i].next_token;
+            ctx->pend_dst[i].status = ctx->h_results[i].status;
+            ctx->pend_dst[i].reserved = 0;
+        }
+        ctx->pend_dst = nullptr;
+        ctx->pend_n = 0;
+    }
+    return PIPESD_OK;
+}
+
+int32_t pipesd_req_open(pipesd_ctx* ctx, int32_t* req) {
+    if (!ctx || !req) return PIPESD_E_INVALID;
+    for (int i = 0; i < (int)ctx->reqs.size(); ++i)
+        if (!ctx->reqs[i].open) {
+            ctx->reqs[i] = Request();
+            ctx->reqs[i].open = true;
+            *req = i;
+            return PIPESD_OK;
+        }
+    return fail(ctx, PIPESD_E_FULL, "pipesd_req_open");
+}
+
+static inline bool bad_req(const pipesd_ctx* ctx, int32_t req) {
+    return req < 0 || req >= (int)ctx->reqs.size() || !ctx->reqs[req].open;
+}
+
+int32_t pipesd_req_close(pipesd_ctx* ctx, int32_t req) {
+    if (!ctx || bad_req(ctx, req)) return fail(ctx, PIPESD_E_INVALID, "pipesd_req_close: bad request");
+    Request& r = ctx->reqs[req];
+    shrink_pages(ctx, r, 0);
+    r = Request();
+    return PIPESD_OK;
+}
+
+int32_t pipesd_req_len(pipesd_ctx* ctx, int32_t req, int32_t* len) {
+    if (!ctx || !len || bad_req(ctx, req)) return fail(ctx, PIPESD_E_INVALID, "pipesd_req_len: bad request");
+    *len = ctx->reqs[req].len;
+    return PIPESD_OK;
+}
+
+int32_t pipesd_prefill(pipesd_ctx* ctx, int32_t req, const int32_t* tokens, int32_t n, float* last_logits) {
+    if (!ctx || !tokens || n < 1 || bad_req(ctx, req)) return fail(ctx, PIPESD_E_INVALID, "pipesd_prefill");
+    Request& r = ctx->reqs[req];
+    if (r.tentative) return fail(ctx, PIPESD_E_STATE, "prefill on a request with an uncommitted verify");
+    if (r.len + n > ctx->cfg.max_seq) return fail(ctx, PIPESD_E_RANGE, "prefill beyond max_seq");
+    for (int i = 0; i < n; ++i)
+        if (tokens[i] < 0 || tokens[i] >= ctx->cfg.vocab) return fail(ctx, PIPESD_E_INVALID, "token id out of range");
+    if (pages_needed(ctx, r, r.len + n) > (int)ctx->free_pages.size())
+        return fail(ctx, PIPESD_E_OOM_PAGES, "pipesd_prefill");
+    int rc = grow_pages(ctx, req, r.len + n);
+    if (rc != PIPESD_OK) return rc;
+    const int chunk = std::min(ctx->cfg.max_rows, kMaxItemRows);
+    for (int done = 0; done < n; done += chunk) {
+        int rows = std::min(chunk, n - done);
+        bool last = done + rows == n;
+        std::vector<ItemDesc> items(1);
+        items[0] = ItemDesc{req, rows, 2, 0, tokens + done, nullptr, nullptr};
+        rc = run_pass(ctx, items, last && last_logits, false);
+        if (rc != PIPESD_OK) return rc;
+        r.len += rows;
+        if (last && last_logits) {
+            CU(cudaMemcpyAsync(last_logits, ctx->W<float>(ctx->ws.logits) + (size_t)(rows - 1) * ctx->cfg.vocab,
+                               4 * (size_t)ctx->cfg.vocab, cudaMemcpyDeviceToHost, ctx->st));
+            CU(cudaStreamSynchronize(ctx->st));
+        }
+    }
+    return PIPESD_OK;
+}
+
+int32_t pipesd_verify(pipesd_ctx* ctx, int32_t n_req, const pipesd_verify_item* items_in,
+                      pipesd_verify_result* results, uint32_t flags) {
+    if (!ctx || !items_in || !results || n_req < 1 || n_req > ctx->dv.max_items)
+        return fail(ctx, PIPESD_E_INVALID, "pipesd_verify: arguments");
+    const pipesd_model_cfg& c = ctx->cfg;
+    if (ctx->pend_dst) {  // deliver the previous call's results before their staging is reused
+        int rc = pipesd_ctx_sync(ctx);
+        if (rc != PIPESD_OK) return rc;
+    }
+    int M = 0, pages = 0;
+    std::vector<char> seen(c.max_requests, 0);
+    for (int i = 0; i < n_req; ++i) {
+        const pipesd_verify_item& it = items_in[i];
+        if (bad_req(ctx, it.req) || seen[it.req]) return fail(ctx, PIPESD_E_INVALID, "verify: bad or repeated request");
+        seen[it.req] = 1;
+        if (it.k < 1 || it.k > c.max_draft || !it.tokens) return fail(ctx, PIPESD_E_INVALID, "verify: item");
+        if (it.mode == PIPESD_MODE_STOCHASTIC && !it.u) return fail(ctx, PIPESD_E_INVALID, "verify: uniforms missing");
+        if (it.mode != PIPESD_MODE_STOCHASTIC && it.mode != PIPESD_MODE_GREEDY)
+            return fail(ctx, PIPESD_E_INVALID, "verify: mode");
+        if (it.mode == PIPESD_MODE_STOCHASTIC && !it.q) return fail(ctx, PIPESD_E_INVALID, "verify: q missing");
+        for (int j = 0; j <= it.k; ++j) {
+            if (it.tokens[j] < 0 || it.tokens[j] >= c.vocab) return fail(ctx, PIPESD_E_INVALID, "verify: token id");
+            if (it.u && !(it.u[j] >= 0.f && it.u[j] < 1.f)) return fail(ctx, PIPESD_E_INVALID, "verify: uniform outside [0,1)");
+        }
+        const Request& r = ctx->reqs[it.req];
+        if (r.tentative) return fail(ctx, PIPESD_E_STATE, "verify on a request with an uncommitted tail");
+        if (r.len + it.k + 1 > c.max_seq) return fail(ctx, PIPESD_E_RANGE, "verify beyond max_seq");
+        M += it.k + 1;
+        pages += pages_needed(ctx, r, r.len + it.k + 1);
+    }
+    if (M > c.max_rows) return fail(ctx, PIPESD_E_RANGE, "verify: more rows than max_rows");
+    if (pages > (int)ctx->free_pages.size()) return fail(ctx, PIPESD_E_OOM_PAGES, "pipesd_verify");
+
+    std::vector<ItemDesc> items(n_req);
+    float* qstage = ctx->W<float>(ctx->ws.qstage);
+    size_t qrow = 0;
+    for (int i = 0; i < n_req; ++i) {
+        const pipesd_verify_item& it = items_in[i];
+        int rc = grow_pages(ctx, it.req, ctx->reqs[it.req].len + it.k + 1);
+        if (rc != PIPESD_OK) return rc;
+        const float* q = it.q;
+        if (it.mode == PIPESD_MODE_STOCHASTIC && (flags & PIPESD_Q_HOST)) {
+            float* dst = qstage + qrow * c.vocab;
+            CU(cudaMemcpyAsync(dst, it.q, 4 * (size_t)it.k * c.vocab, cudaMemcpyHostToDevice, ctx->st));
+            q = dst;
+            qrow += it.k;
+        }
+        items[i] = ItemDesc{it.req, it.k + 1, it.mode, it.k, it.tokens, q, it.u};
+    }
+    int rc = run_pass(ctx, items, true, true);
+    if (rc != PIPESD_OK) return rc;
+    CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut) * n_req,
+                       cudaMemcpyDeviceToHost, ctx->st));
+    ctx->pend_dst = results;
+    ctx->pend_n = n_req;
+    for (int i = 0; i < n_req; ++i) ctx->reqs[items_in[i].req].tentative = items_in[i].k + 1;
+    return PIPESD_OK;
+}
+
+int32_t pipesd_kv_rollback(pipesd_ctx* ctx, int32_t n_req, const int32_t* reqs, const int32_t* n_accepted) {
+    if (!ctx || !reqs || !n_accepted || n_req < 1) return fail(ctx, PIPESD_E_INVALID, "pipesd_kv_rollback");
+    for (int i = 0; i < n_req; ++i) {
+        if (bad_req(ctx, reqs[i])) return fail(ctx, PIPESD_E_INVALID, "rollback: bad request");
+        const Request& r = ctx->reqs[reqs[i]];
+        if (!r.tentative) return fail(ctx, PIPESD_E_STATE, "rollback without a preceding verify");
+        if (n_accepted[i] < 0 || n_accepted[i] > r.tentative - 1)
+            return fail(ctx, PIPESD_E_RANGE, "rollback: n_accepted outside 0..k");
+    }
+    for (int i = 0; i < n_req; ++i) {
+        Request& r = ctx->reqs[reqs[i]];
+        r.len += 1 + n_accepted[i];
+        r.tentative = 0;
+        shrink_pages(ctx, r, r.len);
+    }
+    return PIPESD_OK;
+}
+
+int32_t pipesd_debug_get_logits(pipesd_ctx* ctx, float* dst, int32_t rows) {
+    if (!ctx || !dst || rows < 1 || rows > ctx->last_rows) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_get_logits");
+    CU(cudaMemcpyAsync(dst, ctx->W<float>(ctx->ws.logits), 4 * (size_t)rows * ctx->cfg.vocab, cudaMemcpyDeviceToHost,
+                       ctx->st));
+    CU(cudaStreamSynchronize(ctx->st));
+    return PIPESD_OK;
+}
+
+static int32_t kv_rw(pipesd_ctx* ctx, int32_t req, int32_t layer, int32_t pos0, int32_t n_pos, uint16_t* k,
+                     uint16_t* v, bool write) {
+    if (!ctx || !k || !v || bad_req(ctx, req) || layer < 0 || layer >= ctx->cfg.n_layers || pos0 < 0 || n_pos < 1)
+        return fail(ctx, PIPESD_E_INVALID, "kv read/write");
+    const pipesd_model_cfg& c = ctx->cfg;
+    Request& r = ctx->reqs[req];
+    if (r.tentative) return fail(ctx, PIPESD_E_STATE, "kv read/write with an uncommitted verify");
+    const int end = pos0 + n_pos;
+    if (write) {
+        if (end > c.max_seq) return fail(ctx, PIPESD_E_RANGE, "kv write beyond max_seq");
+        if (pages_needed(ctx, r, end) > (int)ctx->free_pages.size()) return fail(ctx, PIPESD_E_OOM_PAGES, "kv write");
+        int rc = grow_pages(ctx, req, end);
+        if (rc != PIPESD_OK) return rc;
+        r.len = std::max(r.len, end);
+    } else if (end > r.len) {
+        return fail(ctx, PIPESD_E_RANGE, "kv read beyond the committed length");
+    }
+    const int w = ctx->dv.kvd;
+    // staging: the two split-K partial arrays (idle between passes)
+    uint16_t* sk = ctx->W<uint16_t>(ctx->ws.partA);
+    uint16_t* sv = ctx->W<uint16_t>(ctx->ws.partB);
+    const size_t cap = ctx->dv.part_floats * 2 / w;  // positions per round
+    if (cap < 1) return fail(ctx, PIPESD_E_NOMEM, "kv staging");
+    const int32_t* bt = ctx->W<int32_t>(ctx->ws.block_tab) + (size_t)req * ctx->dv.max_pages;
+    const int step = (int)std::min<size_t>(cap, (size_t)1 << 20);
+    for (int done = 0; done < n_pos; done += step) {
+        int n = std::min(step, n_pos - done);
+        size_t bytes = (size_t)n * w * 2;
+        if (write) {
+            CU(cudaMemcpyAsync(sk, k + (size_t)done * w, bytes, cudaMemcpyHostToDevice, ctx->st));
+            CU(cudaMemcpyAsync(sv, v + (size_t)done * w, bytes, cudaMemcpyHostToDevice, ctx->st));
+        }
+        int blocks = (int)std::min<size_t>(((size_t)n * w + 255) / 256, 148 * 8);
+        kv_copy_kernel<<<blocks, 256, 0, ctx->st>>>(ctx->kv_pool, sk, sv, bt, pos0 + done, n, layer, c.n_pages,
+                                                    c.page_size, c.n_kv_heads, c.head_dim, write ? 1 : 0);
+        if (!write) {
+            CU(cudaMemcpyAsync(k + (size_t)done * w, sk, bytes, cudaMemcpyDeviceToHost, ctx->st));
+            CU(cudaMemcpyAsync(v + (size_t)done * w, sv, bytes, cudaMemcpyDeviceToHost, ctx->st));
+        }
+        CU(cudaStreamSynchronize(ctx->st));
+    }
+    return PIPESD_OK;
+}
+
+int32_t pipesd_debug_read_kv(pipesd_ctx* ctx, int32_t req, int32_t layer, int32_t pos0, int32_t n_pos, uint16_t* k,
+                             uint16_t* v) {
+    return kv_rw(ctx, req, layer, pos0, n_pos, k, v, false);
+}
+
+int32_t pipesd_debug_write_kv(pipesd_ctx* ctx, int32_t req, int32_t layer, int32_t pos0, int32_t n_pos,
+                              const uint16_t* k, const uint16_t* v) {
+    return kv_rw(ctx, req, layer, pos0, n_pos, const_cast<uint16_t*>(k), const_cast<uint16_t*>(v), true);
+}
+
+int32_t pipesd_reject_from_logits(pipesd_ctx* ctx, int32_t k, int32_t mode, const float* logits, const float* q,
+                                  const int32_t* drafts, const float* u, pipesd_verify_result* result) {
+    if (!ctx || !logits || !drafts || !u || !result || k < 1 || k > ctx->cfg.max_draft)
+        return fail(ctx, PIPESD_E_INVALID, "pipesd_reject_from_logits");
+    if (mode != PIPESD_MODE_GREEDY && (mode != PIPESD_MODE_STOCHASTIC || !q))
+        return fail(ctx, PIPESD_E_INVALID, "pipesd_reject_from_logits: mode / q");
+    if (ctx->pend_dst) {
+        int rc = pipesd_ctx_sync(ctx);
+        if (rc != PIPESD_OK) return rc;
+    }
+    const int V = ctx->cfg.vocab;
+    for (int i = 0; i < k; ++i)
+        if (drafts[i] < 0 || drafts[i] >= V) return fail(ctx, PIPESD_E_INVALID, "draft id out of range");
+    const int sidx = ctx->stage;
+    ctx->stage = (ctx->stage + 1) % pipesd_ctx::kStages;
+    CU(cudaEventSynchronize(ctx->ev_meta[sidx]));
+    char* hm = ctx->h_meta[sidx];
+    const MetaLayout& ml = ctx->ml;
+    int32_t* tok = reinterpret_cast<int32_t*>(hm + ml.row_tok);
+    tok[0] = 0;
+    for (int i = 0; i < k; ++i) tok[i + 1] = drafts[i];
+    float* hu = reinterpret_cast<float*>(hm + ml.u);
+    for (int i = 0; i <= k; ++i) hu[i] = u[i];
+    float* dl = ctx->W<float>(ctx->ws.logits);
+    float* dq = ctx->W<float>(ctx->ws.qstage);
+    RejectItem* hr = reinterpret_cast<RejectItem*>(hm + ml.rej);
+    hr[0] = RejectItem{0, k, mode, 0, dq};
+    cudaStream_t st = ctx->st;
+    CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.meta, hm, ml.total, cudaMemcpyHostToDevice, st));
+    CU(cudaEventRecord(ctx->ev_meta[sidx], st));
+    CU(cudaMemcpyAsync(dl, logits, 4 * (size_t)(k + 1) * V, cudaMemcpyHostToDevice, st));
+    if (mode == PIPESD_MODE_STOCHASTIC) CU(cudaMemcpyAsync(dq, q, 4 * (size_t)k * V, cudaMemcpyHostToDevice, st));
+    RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
+    row_stats_kernel<<<dim3(k + 1, kStatSplits), 256, 0, st>>>(nullptr, 1, k + 1, V, dl, stats);
+    accept_sample_kernel<<<1, kSampleThreads, 0, st>>>(
+        dl, V, stats, reinterpret_cast<const RejectItem*>(ctx->wsp + ctx->ws.meta + ml.rej),
+        reinterpret_cast<const int32_t*>(ctx->wsp + ctx->ws.meta + ml.row_tok),
+        reinterpret_cast<const float*>(ctx->wsp + ctx->ws.meta + ml.u), ctx->W<RejectOut>(ctx->ws.results));
+    CU(cudaGetLastError());
+    CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut), cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    result->n_accepted = ctx->h_results[0].n_accepted;
+    result->next_token = ctx->h_results[0].next_token;
+    result->status = ctx->h_results[0].status;
+    result->reserved = 0;
+    ctx->last_rows = k + 1;
+    return PIPESD_OK;
+}
+
+uint64_t pipesd_gemm_packed_bytes(int32_t N, int32_t K) { return (uint64_t)N * K * 2; }
+
+uint64_t pipesd_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K) {
+    if (M < 1 || N < 16 || K < 16) return 0;
+    GemmPlan p = gemm_plan(M, N, K);
+    return (uint64_t)p.S * M * N * 4;
+}
+
+int32_t pipesd_gemm_pack(const void* W, void* packed, int32_t N, int32_t K, void* cuda_stream) {
+    if (!W || !packed || N < 16 || K < 16 || N % 16 || K % 16) return PIPESD_E_INVALID;
+    size_t total = (size_t)(N / 16) * (K / 16) * 32;
+    int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
+    gemm_pack_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)W, (uint4*)packed, N, K);
+    return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
+}
+
+int32_t pipesd_gemm_run(const void* packed, const float* x, float* y, void* scratch, int32_t M, int32_t N,
+                        int32_t K, void* cuda_stream) {
+    if (!packed || !x || !y || !scratch || M < 1 || N < 16 || K < 16 || N % 16 || K % 16) return PIPESD_E_INVALID;
+    static bool attrs = false;
+    if (!attrs) {
+        if (gemm_init_attrs() != cudaSuccess) return PIPESD_E_CUDA;
+        attrs = true;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    GemmPlan p = gemm_plan(M, N, K);
+    float* dst = p.S == 1 ? y : (float*)scratch;
+    if (gemm_launch(p, (const uint4*)packed, x, K, dst, M, N, K, st) != cudaSuccess) return PIPESD_E_CUDA;
+    if (p.S > 1) {
+        size_t n = (size_t)M * N;
+        int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
+        reduce_partials_kernel<<<blocks, 256, 0, st>>>((const float*)scratch, y, n, p.S);
+    }
+    return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,216 @@
+// Vocabulary-wide part of the verify pass: row softmax statistics, the sequential accept chain, and
+// the single final draw (residual resample on a rejection, extra token when all drafts pass).
+//
+// Rule: accept draft x_i while u_i < min(1, p_i(x_i) / q_i(x_i)); on the first failure at row r draw
+// the correction from norm(max(0, p_r - q_r)); when all k pass draw the extra token from p_k.
+// Greedy mode: accept while the draft is the row's argmax (lowest index on ties), emit the argmax.
+// Decisions are taken in fp64 on fp32 logits; sums run in a fixed order, so a result is reproducible.
+#pragma once
+#include "common.cuh"
+
+namespace pipesd {
+
+constexpr int kStatSplits = 16;     // column splits per row in the statistics kernel
+constexpr int kSampleThreads = 1024;
+
+struct RowStat {
+    float m;       // max logit in the split
+    int arg;       // its lowest index
+    double z;      // sum exp(l - m) over the split
+};
+
+// logits[row][j] = sum_s part[s][row][j] (written out), and per (row, split): max, argmax, sum-exp.
+// grid (M, kStatSplits), block 256.
+__global__ void __launch_bounds__(256) row_stats_kernel(const float* __restrict__ part, int S, int M, int V,
+                                                        float* __restrict__ logits, RowStat* __restrict__ stats) {
+    const int row = blockIdx.x, sp = blockIdx.y;
+    const int per = (V + kStatSplits - 1) / kStatSplits;
+    const int j0 = sp * per, j1 = min(V, j0 + per);
+    float* lr = logits + (size_t)row * V;
+    float m = -INFINITY;
+    int arg = 0x7fffffff;
+    for (int j = j0 + threadIdx.x; j < j1; j += 256) {
+        float v;
+        if (part) {
+            v = 0.f;
+            for (int s = 0; s < S; ++s) v += part[((size_t)s * M + row) * V + j];
+            lr[j] = v;
+        } else {
+            v = lr[j];
+        }
+        if (v > m) { m = v; arg = j; }
+    }
+    __shared__ float sm_m[8];
+    __shared__ int sm_a[8];
+    __shared__ double sm_z[8];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float om = __shfl_xor_sync(0xffffffffu, m, o);
+        int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+        if (om > m || (om == m && oa < arg)) { m = om; arg = oa; }
+    }
+    if ((threadIdx.x & 31) == 0) { sm_m[threadIdx.x >> 5] = m; sm_a[threadIdx.x >> 5] = arg; }
+    __syncthreads();
+    m = sm_m[0]; arg = sm_a[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w)
+        if (sm_m[w] > m || (sm_m[w] == m && sm_a[w] < arg)) { m = sm_m[w]; arg = sm_a[w]; }
+    double z = 0.0;
+    for (int j = j0 + threadIdx.x; j < j1; j += 256) z += (double)expf(lr[j] - m);
+    z = warp_sum_d(z);
+    if ((threadIdx.x & 31) == 0) sm_z[threadIdx.x >> 5] = z;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double zt = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) zt += sm_z[w];
+        RowStat st;
+        st.m = m; st.arg = arg; st.z = zt;
+        stats[(size_t)row * kStatSplits + sp] = st;
+    }
+}
+
+struct RejectItem {
+    int row0;          // first logits row of the request
+    int k;             // drafts
+    int mode;          // 0 stochastic, 1 greedy, 2 none (prefill)
+    int u0;            // offset of the request's k+1 uniforms
+    const float* q;    // device [k][V]
+};
+
+struct RejectOut { int n_accepted, next_token, status, reserved; };
+
+// One CTA per request: combine the row statistics, run the accept chain, make the final draw.
+__global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const float* __restrict__ logits, int V,
+                                                                       const RowStat* __restrict__ stats,
+                                                                       const RejectItem* __restrict__ items,
+                                                                       const int32_t* __restrict__ row_tok,
+                                                                       const float* __restrict__ u_all,
+                                                                       RejectOut* __restrict__ out) {
+    const RejectItem it = items[blockIdx.x];
+    if (it.mode == 2) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ double s_m[kMaxItemRows], s_z[kMaxItemRows];
+    __shared__ int s_arg[kMaxItemRows];
+    __shared__ int s_nacc, s_tok, s_owner;
+    __shared__ double s_warp[32];
+    __shared__ double s_total;
+    __shared__ double s_incl[kSampleThreads];
+
+    if (tid <= it.k) {   // rows 0..k: merge the column splits
+        const RowStat* st = stats + (size_t)(it.row0 + tid) * kStatSplits;
+        float m = st[0].m;
+        int arg = st[0].arg;
+        for (int s = 1; s < kStatSplits; ++s)
+            if (st[s].m > m || (st[s].m == m && st[s].arg < arg)) { m = st[s].m; arg = st[s].arg; }
+        double z = 0.0;
+        for (int s = 0; s < kStatSplits; ++s)
+            if (st[s].m > -INFINITY) z += st[s].z * exp((double)st[s].m - (double)m);
+        s_m[tid] = (double)m; s_z[tid] = z; s_arg[tid] = arg;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int n = 0;
+        for (int i = 0; i < it.k; ++i) {
+            const int x = row_tok[it.row0 + i + 1];
+            bool ok;
+            if (it.mode == 1) {
+                ok = (x == s_arg[i]);
+            } else {
+                const double p = exp((double)logits[(size_t)(it.row0 + i) * V + x] - s_m[i]) / s_z[i];
+                const double qx = (double)it.q[(size_t)i * V + x];
+                double ratio = qx > 0.0 ? p / qx : (p > 0.0 ? INFINITY : 0.0);
+                ok = (double)u_all[it.u0 + i] < fmin(ratio, 1.0);
+            }
+            if (!ok) break;
+            ++n;
+        }
+        s_nacc = n;
+        s_tok = -1;
+        s_owner = 0x7fffffff;
+    }
+    __syncthreads();
+    const int n_acc = s_nacc;
+    if (it.mode == 1) {
+        if (tid == 0) { RejectOut r{n_acc, s_arg[n_acc], 0, 0}; out[blockIdx.x] = r; }
+        return;
+    }
+    // Final draw from row n_acc: residual max(0, p - q) if a draft was rejected there, else p.
+    const float* lr = logits + (size_t)(it.row0 + n_acc) * V;
+    const double m = s_m[n_acc], inv_z = 1.0 / s_z[n_acc];
+    const double uk = (double)u_all[it.u0 + it.k];
+    const int per = (V + kSampleThreads - 1) / kSampleThreads;
+    const int j0 = min(V, tid * per), j1 = min(V, j0 + per);
+    bool use_q = n_acc < it.k;
+    const float* qr = use_q ? it.q + (size_t)n_acc * V : nullptr;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        double loc = 0.0;
+        for (int j = j0; j < j1; ++j) {
+            double r = exp((double)lr[j] - m) * inv_z;
+            if (use_q) r = fmax(0.0, r - (double)qr[j]);
+            loc += r;
+        }
+        // inclusive scan over threads in index order: warp scan, then scan of warp totals
+        double inc = loc;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            double t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        if (lane == 31) s_warp[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            double w = s_warp[lane], winc = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                double t = __shfl_up_sync(0xffffffffu, winc, o);
+                if (lane >= o) winc += t;
+            }
+            s_warp[lane] = winc - w;     // exclusive prefix of the warp totals
+            if (lane == 31) s_total = winc;
+        }
+        __syncthreads();
+        const double total = s_total;
+        if (use_q && !(total > 0.0)) {   // p <= q everywhere (e.g. p == q): fall back to p
+            use_q = false;
+            __syncthreads();
+            continue;
+        }
+        const double incl = inc + s_warp[warp];
+        s_incl[tid] = incl;
+        const double target = uk * total;
+        // the owner is the first thread whose inclusive prefix exceeds the target
+        if (incl > target) atomicMin(&s_owner, tid);
+        __syncthreads();
+        const int owner = s_owner;
+        const double excl = tid ? s_incl[tid - 1] : 0.0;
+        if (owner == tid) {
+            double run = excl;
+            int tok = -1;
+            for (int j = j0; j < j1; ++j) {
+                double r = exp((double)lr[j] - m) * inv_z;
+                if (use_q) r = fmax(0.0, r - (double)qr[j]);
+                run += r;
+                if (run > target) { tok = j; break; }
+            }
+            if (tok < 0) tok = j1 - 1;   // rounding at the range's upper edge
+            s_tok = tok;
+        }
+        __syncthreads();
+        if (owner == 0x7fffffff && tid == 0) {
+            // target >= every prefix (rounding at the top of the CDF): last token with mass
+            int tok = V - 1;
+            for (int j = V - 1; j >= 0; --j) {
+                double r = exp((double)lr[j] - m) * inv_z;
+                if (use_q) r = fmax(0.0, r - (double)qr[j]);
+                if (r > 0.0) { tok = j; break; }
+            }
+            s_tok = tok;
+        }
+        __syncthreads();
+        break;
+    }
+    if (tid == 0) { RejectOut r{n_acc, s_tok, 0, 0}; out[blockIdx.x] = r; }
+}
+
+}  // namespace pipesd
