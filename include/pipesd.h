@@ -172,6 +172,22 @@ int32_t pipesd_reject_from_logits(pipesd_ctx *ctx, int32_t k, int32_t mode, cons
                                   const float *q, const int32_t *drafts, const float *u,
                                   pipesd_verify_result *result);
 
+/* Truncate a request's committed length to new_len <= its current length (pages beyond return to the
+ * pool).  Lets a harness replay rounds from a recorded point; the serving path uses pipesd_kv_rollback. */
+int32_t pipesd_debug_set_len(pipesd_ctx *ctx, int32_t req, int32_t new_len);
+
+/* Launch accounting.  While enabled, every kernel launch of the context is counted and every
+ * weight-streaming GEMM launch is bracketed by CUDA events on the context's stream.
+ * pipesd_profile_read synchronises, reports the totals since the last read and resets them. */
+typedef struct pipesd_profile_info {
+    int64_t kernel_launches; /* all kernels launched by the context                         */
+    int64_t gemm_launches;   /* weight-streaming GEMM launches among them                    */
+    double gemm_ms;          /* summed device time of those GEMM launches (CUDA events)      */
+    double gemm_bytes;       /* their algorithmic bytes: bf16 W once + fp32 x in + fp32 y out */
+} pipesd_profile_info;
+int32_t pipesd_profile_enable(pipesd_ctx *ctx, int32_t time_gemms);
+int32_t pipesd_profile_read(pipesd_ctx *ctx, pipesd_profile_info *out);
+
 /* Small-M weight-streaming GEMM on its own: y[M,N] = x[M,K] . W[N,K]^T with bf16 W, fp32 x and y.
  * pipesd_gemm_packed_bytes: size of the repacked copy of W.  pipesd_gemm_pack: W (device, row-major
  * bf16 [N,K]) -> packed (device).  pipesd_gemm_run: x, y device; scratch device of

@@ -54,6 +54,11 @@ class VerifyResult(ctypes.Structure):
     _fields_ = [("n_accepted", i32), ("next_token", i32), ("status", i32), ("reserved", i32)]
 
 
+class ProfileInfo(ctypes.Structure):
+    _fields_ = [("kernel_launches", ctypes.c_int64), ("gemm_launches", ctypes.c_int64),
+                ("gemm_ms", ctypes.c_double), ("gemm_bytes", ctypes.c_double)]
+
+
 # name -> (restype, argtypes); mirrors include/pipesd.h one to one
 _SIGNATURES = {
     "pipesd_strerror": (ctypes.c_char_p, [i32]),
@@ -73,6 +78,9 @@ _SIGNATURES = {
     "pipesd_debug_read_kv": (i32, [vp, i32, i32, i32, i32, vp, vp]),
     "pipesd_debug_write_kv": (i32, [vp, i32, i32, i32, i32, vp, vp]),
     "pipesd_reject_from_logits": (i32, [vp, i32, i32, vp, vp, vp, vp, ctypes.POINTER(VerifyResult)]),
+    "pipesd_debug_set_len": (i32, [vp, i32, i32]),
+    "pipesd_profile_enable": (i32, [vp, i32]),
+    "pipesd_profile_read": (i32, [vp, ctypes.POINTER(ProfileInfo)]),
     "pipesd_gemm_packed_bytes": (u64, [i32, i32]),
     "pipesd_gemm_scratch_bytes": (u64, [i32, i32, i32]),
     "pipesd_gemm_pack": (i32, [vp, vp, i32, i32, vp]),
@@ -262,6 +270,18 @@ class Context:
         v = np.ascontiguousarray(v_bf16, np.uint16)
         self._check(lib().pipesd_debug_write_kv(self._h, req, layer, pos0, k.shape[0], _np_ptr(k), _np_ptr(v)),
                     "pipesd_debug_write_kv")
+
+    def debug_set_len(self, req: int, new_len: int):
+        self._check(lib().pipesd_debug_set_len(self._h, req, new_len), "pipesd_debug_set_len")
+
+    def profile_enable(self, time_gemms: bool = False):
+        self._check(lib().pipesd_profile_enable(self._h, int(time_gemms)), "pipesd_profile_enable")
+
+    def profile_read(self) -> dict:
+        info = ProfileInfo()
+        self._check(lib().pipesd_profile_read(self._h, ctypes.byref(info)), "pipesd_profile_read")
+        return dict(kernel_launches=info.kernel_launches, gemm_launches=info.gemm_launches,
+                    gemm_ms=info.gemm_ms, gemm_bytes=info.gemm_bytes)
 
     def reject_from_logits(self, logits, q, drafts, u, mode: int = MODE_STOCHASTIC):
         logits = np.ascontiguousarray(logits, np.float32)

@@ -194,6 +194,12 @@ struct pipesd_ctx {
     int pend_n = 0;
     int last_rows = 0;
     std::string err;
+    // launch accounting
+    int64_t n_launch = 0, n_gemm = 0;
+    double gemm_bytes = 0.0;
+    bool time_gemms = false;
+    std::vector<cudaEvent_t> prof_ev;   // start/stop pairs
+    size_t prof_used = 0;
 
     template <typename T>
     T* W(size_t off) const { return reinterpret_cast<T*>(wsp + off); }
@@ -233,6 +239,31 @@ int cuda_fail(pipesd_ctx* c, cudaError_t e, const char* where) {
         cudaError_t e_ = (call);                                    \
         if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);    \
     } while (0)
+
+// Launch one weight-streaming GEMM with accounting (and event timing when profiling is on).
+int launch_gemm(pipesd_ctx* ctx, const GemmPlan& p, const uint4* W, const float* x, int ldx, float* out, int M,
+                int N, int K) {
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (ctx->time_gemms) {
+        if (ctx->prof_used + 2 > ctx->prof_ev.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                CU(cudaEventCreate(&e));
+                ctx->prof_ev.push_back(e);
+            }
+        }
+        e0 = ctx->prof_ev[ctx->prof_used];
+        e1 = ctx->prof_ev[ctx->prof_used + 1];
+        ctx->prof_used += 2;
+        CU(cudaEventRecord(e0, ctx->st));
+    }
+    CU(gemm_launch(p, W, x, ldx, out, M, N, K, ctx->st));
+    if (e1) CU(cudaEventRecord(e1, ctx->st));
+    ctx->n_launch += 1;
+    ctx->n_gemm += 1;
+    ctx->gemm_bytes += 2.0 * N * K + 4.0 * M * K + 4.0 * M * N;
+    return PIPESD_OK;
+}
 
 struct ItemDesc {
     int slot, rows, mode, k;
@@ -353,7 +384,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         add_norm_kernel<<<M, 256, 0, st>>>(x, l == 0 ? ctx->emb : nullptr, meta.row_tok, part, S, M, lw.n1,
                                            c.rms_eps, d, h);
         GemmPlan p = gemm_plan(M, dv.Nqkv, d);
-        CU(gemm_launch(p, lw.qkv.packed, h, d, partA, M, dv.Nqkv, d, st));
+        { int rc_ = launch_gemm(ctx, p, lw.qkv.packed, h, d, partA, M, dv.Nqkv, d); if (rc_) return rc_; }
         rope_kv_kernel<<<dim3(M, Hq + 2 * Hkv), hd / 2, 0, st>>>(partA, p.S, M, Hq, Hkv, hd, cs, sn, meta, qbuf,
                                                                  ctx->kv_pool, l, c.n_pages, c.page_size);
         dim3 ag(max_nsplit, Hq, n_items);
@@ -365,27 +396,30 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
                                                                    c.page_size, Hq, Hkv, o_part, m_part, l_part);
         attn_combine_kernel<<<dim3(M, Hq), hd, 0, st>>>(o_part, m_part, l_part, meta, Hq, hd, attn);
         p = gemm_plan(M, d, dv.qd);
-        CU(gemm_launch(p, lw.o.packed, attn, dv.qd, partB, M, d, dv.qd, st));
+        { int rc_ = launch_gemm(ctx, p, lw.o.packed, attn, dv.qd, partB, M, d, dv.qd); if (rc_) return rc_; }
         add_norm_kernel<<<M, 256, 0, st>>>(x, nullptr, nullptr, partB, p.S, M, lw.n2, c.rms_eps, d, h);
         p = gemm_plan(M, 2 * F, d);
-        CU(gemm_launch(p, lw.gu.packed, h, d, partA, M, 2 * F, d, st));
+        { int rc_ = launch_gemm(ctx, p, lw.gu.packed, h, d, partA, M, 2 * F, d); if (rc_) return rc_; }
         {
             size_t n = (size_t)M * F;
             int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
             silu_mul_kernel<<<blocks, 256, 0, st>>>(partA, p.S, M, F, act);
         }
         p = gemm_plan(M, d, F);
-        CU(gemm_launch(p, lw.dn.packed, act, F, partB, M, d, F, st));
+        { int rc_ = launch_gemm(ctx, p, lw.dn.packed, act, F, partB, M, d, F); if (rc_) return rc_; }
         part = partB;
         S = p.S;
+        ctx->n_launch += 6;   // add_norm x2, rope_kv, attn_split, attn_combine, silu_mul
     }
+    ctx->n_launch += 1;       // rope_table
     if (want_logits) {
+        ctx->n_launch += 2 + (want_reject ? 1 : 0);   // add_norm, row_stats, accept_sample
         float* logits = ctx->W<float>(ctx->ws.logits);
         RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
         add_norm_kernel<<<M, 256, 0, st>>>(x, nullptr, nullptr, part, S, M, ctx->final_norm, c.rms_eps, d, h);
         GemmPlan p = gemm_plan(M, c.vocab, d);
         float* dst = p.S == 1 ? logits : partA;
-        CU(gemm_launch(p, ctx->lm.packed, h, d, dst, M, c.vocab, d, st));
+        { int rc_ = launch_gemm(ctx, p, ctx->lm.packed, h, d, dst, M, c.vocab, d); if (rc_) return rc_; }
         row_stats_kernel<<<dim3(M, kStatSplits), 256, 0, st>>>(p.S == 1 ? nullptr : partA, p.S, M, c.vocab, logits,
                                                                stats);
         ctx->last_rows = M;
@@ -529,6 +563,7 @@ int32_t pipesd_ctx_destroy(pipesd_ctx* ctx) {
         if (ctx->ev_meta[i]) cudaEventDestroy(ctx->ev_meta[i]);
     }
     if (ctx->h_results) cudaFreeHost(ctx->h_results);
+    for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
     delete ctx;
     return PIPESD_OK;
 }
@@ -793,6 +828,45 @@ int32_t pipesd_reject_from_logits(pipesd_ctx* ctx, int32_t k, int32_t mode, cons
     result->status = ctx->h_results[0].status;
     result->reserved = 0;
     ctx->last_rows = k + 1;
+    return PIPESD_OK;
+}
+
+int32_t pipesd_debug_set_len(pipesd_ctx* ctx, int32_t req, int32_t new_len) {
+    if (!ctx || bad_req(ctx, req)) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_len");
+    Request& r = ctx->reqs[req];
+    if (r.tentative) return fail(ctx, PIPESD_E_STATE, "set_len with an uncommitted verify");
+    if (new_len < 0 || new_len > r.len) return fail(ctx, PIPESD_E_RANGE, "set_len can only truncate");
+    r.len = new_len;
+    shrink_pages(ctx, r, r.len);
+    return PIPESD_OK;
+}
+
+int32_t pipesd_profile_enable(pipesd_ctx* ctx, int32_t time_gemms) {
+    if (!ctx) return PIPESD_E_INVALID;
+    CU(cudaStreamSynchronize(ctx->st));
+    ctx->time_gemms = time_gemms != 0;
+    ctx->n_launch = ctx->n_gemm = 0;
+    ctx->gemm_bytes = 0.0;
+    ctx->prof_used = 0;
+    return PIPESD_OK;
+}
+
+int32_t pipesd_profile_read(pipesd_ctx* ctx, pipesd_profile_info* out) {
+    if (!ctx || !out) return PIPESD_E_INVALID;
+    CU(cudaStreamSynchronize(ctx->st));
+    double ms = 0.0;
+    for (size_t i = 0; i + 1 < ctx->prof_used; i += 2) {
+        float t = 0.f;
+        CU(cudaEventElapsedTime(&t, ctx->prof_ev[i], ctx->prof_ev[i + 1]));
+        ms += t;
+    }
+    out->kernel_launches = ctx->n_launch;
+    out->gemm_launches = ctx->n_gemm;
+    out->gemm_ms = ms;
+    out->gemm_bytes = ctx->gemm_bytes;
+    ctx->n_launch = ctx->n_gemm = 0;
+    ctx->gemm_bytes = 0.0;
+    ctx->prof_used = 0;
     return PIPESD_OK;
 }
 

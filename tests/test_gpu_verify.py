@@ -30,14 +30,19 @@ def test_tiny_config_many_seeds():
     req = ctx.req_open()
     last = ctx.prefill(req, prefix, want_last_logits=True)
     assert ctx.req_len(req) == P
-    # KV written by the GPU prefill equals the oracle's bf16-rounded rows up to one bf16 ulp on rare elements
+    # KV written by the GPU prefill equals the oracle's bf16-rounded rows up to a crossed rounding boundary
     for layer in (0, 1):
         kg, vg = ctx.debug_read_kv(req, layer, 0, P)
         ko = np.stack([orc.get_kv(layer, p)[0] for p in range(P)])
         vo = np.stack([orc.get_kv(layer, p)[1] for p in range(P)])
-        dk = np.abs(synth.bf16_to_f32(kg) - ko); dv = np.abs(synth.bf16_to_f32(vg) - vo)
-        assert dk.max() <= 2.0 ** -7 * max(1.0, np.abs(ko).max()) and (dk > 0).mean() < 0.02
-        assert dv.max() <= 2.0 ** -7 * max(1.0, np.abs(vo).max()) and (dv > 0).mean() < 0.02
+        for got_bits, want in ((kg, ko), (vg, vo)):
+            diff = np.abs(synth.bf16_to_f32(got_bits) - want)
+            # Layer 0 sees identical inputs: a value differs only where the fp32-vs-fp64 difference crosses a
+            # bf16 rounding boundary (one ulp).  Those crossings are the noise later layers start from:
+            # rms sqrt(2 * eps * ulp) ~ 1e-4 of the value scale for eps ~ 3e-6, whatever the kernels do.
+            slack, l1 = (2e-5, 1e-4) if layer == 0 else (5e-4, 5e-4)
+            assert np.all(diff <= 2.0 ** -7 * np.abs(want) + slack)
+            assert diff.sum() / np.abs(want).sum() < l1
     ref_last = oracle.Oracle(shape, w, P + 8)
     ref_last_logits = ref_last.prefill(prefix, want_last_logits=True)
     assert logit_rel_err(last[None], ref_last_logits).max() < LOGIT_TOL
