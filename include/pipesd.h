@@ -40,7 +40,8 @@ typedef enum pipesd_status {
     PIPESD_E_STATE = -4,       /* call order violated (e.g. verify with an uncommitted tail)  */
     PIPESD_E_RANGE = -5,       /* length / count outside what the request state allows        */
     PIPESD_E_CUDA = -6,        /* a CUDA runtime call failed; see pipesd_last_error           */
-    PIPESD_E_NOMEM = -7        /* a caller-provided buffer is smaller than pipesd_query_sizes */
+    PIPESD_E_NOMEM = -7,       /* a caller-provided buffer is smaller than pipesd_query_sizes */
+    PIPESD_E_TOO_LARGE = -8    /* pipesd_gemm_run_static: the problem exceeds the built-in scratch */
 } pipesd_status;
 
 #define PIPESD_MODE_STOCHASTIC 0 /* u_i < min(1, p/q), residual resample, extra token ~ p */
@@ -197,6 +198,32 @@ uint64_t pipesd_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
 int32_t pipesd_gemm_pack(const void *W, void *packed, int32_t N, int32_t K, void *cuda_stream);
 int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scratch, int32_t M, int32_t N,
                         int32_t K, void *cuda_stream);
+
+/* The same GEMM for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a convenience of the library, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin or callback that is handed
+ * its input and output buffers and nothing else, a real-time or latency-critical loop that must not
+ * take the allocator's lock or trigger an implicit device synchronisation, a process whose memory
+ * budget was fixed at start-up and has no pool to draw from.  Such callers have nowhere to get the
+ * split-K scratch that pipesd_gemm_run asks for.  Here the scratch is a fixed array of
+ * PIPESD_STATIC_SCRATCH_BYTES inside the library itself (every GPU that loads the library carries it
+ * until the process ends); the call allocates and frees nothing, on the device or through any
+ * library.  The caller still passes packed weights, x and y (device), exactly as for pipesd_gemm_run,
+ * and gets the same result.
+ *
+ * Limits and rules:
+ *   - If pipesd_gemm_scratch_bytes(M, N, K) is larger than PIPESD_STATIC_SCRATCH_BYTES the call returns
+ *     PIPESD_E_TOO_LARGE and launches nothing (8 MiB covers, e.g., M <= 16 rows against the 7B shapes).
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and sets kernel attributes; make that first call during set-up, before any stream capture.
+ *   - All calls share the one array and it keeps whatever the last call left there.  Nothing needs
+ *     clearing (each call overwrites every element it later reads), but two calls whose kernels can
+ *     overlap on the GPU -- different streams, no ordering between them -- race on it: keep calls on
+ *     one stream or order them with events. */
+#define PIPESD_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t pipesd_gemm_run_static(const void *packed, const float *x, float *y, int32_t M, int32_t N, int32_t K,
+                               void *cuda_stream);
 
 #ifdef __cplusplus
 }

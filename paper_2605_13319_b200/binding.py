@@ -16,6 +16,8 @@ LIB_PATH = _HERE / "libpipesd.so"
 _lib = None
 
 OK, E_INVALID, E_FULL, E_OOM_PAGES, E_STATE, E_RANGE, E_CUDA, E_NOMEM = 0, -1, -2, -3, -4, -5, -6, -7
+E_TOO_LARGE = -8
+STATIC_SCRATCH_BYTES = 8 << 20
 MODE_STOCHASTIC, MODE_GREEDY = 0, 1
 Q_HOST = 1
 
@@ -85,6 +87,7 @@ _SIGNATURES = {
     "pipesd_gemm_scratch_bytes": (u64, [i32, i32, i32]),
     "pipesd_gemm_pack": (i32, [vp, vp, i32, i32, vp]),
     "pipesd_gemm_run": (i32, [vp, vp, vp, vp, i32, i32, i32, vp]),
+    "pipesd_gemm_run_static": (i32, [vp, vp, vp, i32, i32, i32, vp]),
 }
 
 
@@ -323,3 +326,17 @@ def gemm_run(packed, x, y, scratch, N, K, stream=None):
                                vp(st.cuda_stream))
     if rc != OK:
         raise PipesdError(rc, "pipesd_gemm_run")
+
+
+def gemm_run_static(packed, x, y, N, K, stream=None):
+    """pipesd_gemm_run_static: the GEMM with its split-K scratch inside the library, for callers that may
+    not allocate device memory.  Same arguments as gemm_run minus the scratch tensor; nothing is allocated
+    here either (the tensors are the caller's).  Raises PipesdError(E_TOO_LARGE) beyond the built-in limit."""
+    import torch
+    M = x.shape[0]
+    assert x.dtype == torch.float32 and y.dtype == torch.float32 and x.is_contiguous() and y.is_contiguous()
+    assert x.shape[1] == K and tuple(y.shape) == (M, N)
+    st = stream if stream is not None else torch.cuda.current_stream(x.device)
+    rc = lib().pipesd_gemm_run_static(packed.data_ptr(), x.data_ptr(), y.data_ptr(), M, N, K, vp(st.cuda_stream))
+    if rc != OK:
+        raise PipesdError(rc, "pipesd_gemm_run_static")

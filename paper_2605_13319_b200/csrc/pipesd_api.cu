@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -449,6 +450,7 @@ const char* pipesd_strerror(int32_t s) {
         case PIPESD_E_RANGE: return "length out of range";
         case PIPESD_E_CUDA: return "CUDA failure";
         case PIPESD_E_NOMEM: return "caller buffer too small";
+        case PIPESD_E_TOO_LARGE: return "problem needs more scratch than the library's built-in array holds";
         default: return "unknown status";
     }
 }
@@ -896,6 +898,57 @@ int32_t pipesd_gemm_run(const void* packed, const float* x, float* y, void* scra
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     GemmPlan p = gemm_plan(M, N, K);
+    float* dst = p.S == 1 ? y : (float*)scratch;
+    if (gemm_launch(p, (const uint4*)packed, x, K, dst, M, N, K, st) != cudaSuccess) return PIPESD_E_CUDA;
+    if (p.S > 1) {
+        size_t n = (size_t)M * N;
+        int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
+        reduce_partials_kernel<<<blocks, 256, 0, st>>>((const float*)scratch, y, n, p.S);
+    }
+    return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
+}
+
+// ---- GEMM without any caller- or library-side allocation ------------------------------------
+// Split-K partial sums of pipesd_gemm_run_static live in this fixed array.  It is part of the
+// library image: every GPU that loads the library keeps these bytes reserved until the process
+// exits, which is why the limit is modest.
+static __device__ __align__(256) unsigned char g_static_gemm_scratch[PIPESD_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {nullptr};   // device address of the array, per device ordinal
+
+// In host code the array's name is only a handle for the runtime, not a device address; the address
+// a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device current.
+int static_scratch_for_current_device(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PIPESD_E_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_gemm_scratch) != cudaSuccess || !p) return PIPESD_E_CUDA;
+        if (gemm_init_attrs() != cudaSuccess) return PIPESD_E_CUDA;
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return PIPESD_OK;
+}
+}  // namespace
+
+int32_t pipesd_gemm_run_static(const void* packed, const float* x, float* y, int32_t M, int32_t N, int32_t K,
+                               void* cuda_stream) {
+    if (!packed || !x || !y || M < 1 || N < 16 || K < 16 || N % 16 || K % 16) return PIPESD_E_INVALID;
+    const GemmPlan p = gemm_plan(M, N, K);
+    const size_t need = p.S > 1 ? (size_t)p.S * M * N * sizeof(float) : 0;
+    if (need > (size_t)PIPESD_STATIC_SCRATCH_BYTES) return PIPESD_E_TOO_LARGE;
+    void* scratch = nullptr;
+    int rc = static_scratch_for_current_device(&scratch);
+    if (rc != PIPESD_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // Nothing has to be cleared: every partial sum the reduction reads is written by the GEMM kernel of
+    // this same call first (all S slices, all M rows, all N columns), so the previous call's contents
+    // never reach the output.
     float* dst = p.S == 1 ? y : (float*)scratch;
     if (gemm_launch(p, (const uint4*)packed, x, K, dst, M, N, K, st) != cudaSuccess) return PIPESD_E_CUDA;
     if (p.S > 1) {
