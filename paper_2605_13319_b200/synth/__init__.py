@@ -197,14 +197,26 @@ def make_accept_uniforms(k: int, seed: int, request: int = 0, round_: int = 0) -
     return np.ascontiguousarray(u[round_ * 64: round_ * 64 + k + 1])
 
 
+_KV_BASE = {}
+
+
 def make_synthetic_kv(shape: ModelShape, n_pos: int, seed: int, layer: int, request: int = 0,
                       std_k: float = 1.0, std_v: float = 0.1):
-    """Seeded stand-in K and V rows (bf16 bit patterns, [n_pos, n_kv_heads*head_dim] each) for
-    full-size cases where a CPU prefill is out of reach."""
-    base = STREAM_KV + 100 * request + 100000 * (layer + 1)
-    k = normal_bf16((n_pos, shape.kv_dim), seed, base, std_k)
-    v = normal_bf16((n_pos, shape.kv_dim), seed, base + 1, std_v)
-    return k, v
+    """Seeded stand-in K and V rows (bf16 bit patterns, [n_pos, n_kv_heads*head_dim] each) for full-size
+    cases where a CPU prefill is out of reach.  One block of normals is drawn per (seed, request); layer l
+    uses it rotated by 16*l columns and l rows (pure data movement), so that layers differ without
+    drawing 2*n_layers*n_pos*width normals."""
+    key = (shape.kv_dim, n_pos, seed, request, std_k, std_v)
+    if key not in _KV_BASE:
+        if len(_KV_BASE) > 2:
+            _KV_BASE.clear()
+        base = STREAM_KV + 100 * request
+        _KV_BASE[key] = (normal_bf16((n_pos, shape.kv_dim), seed, base, std_k),
+                         normal_bf16((n_pos, shape.kv_dim), seed, base + 1, std_v))
+    k, v = _KV_BASE[key]
+    sh = (16 * layer) % shape.kv_dim
+    return (np.ascontiguousarray(np.roll(np.roll(k, sh, axis=1), layer, axis=0)),
+            np.ascontiguousarray(np.roll(np.roll(v, sh, axis=1), layer, axis=0)))
 
 
 def ragged_requests(seed: int, n_req: int = 32, len_lo: int = 256, len_hi: int = 4096,
