@@ -190,7 +190,7 @@ int32_t pipesd_profile_enable(pipesd_ctx *ctx, int32_t time_gemms);
 int32_t pipesd_profile_read(pipesd_ctx *ctx, pipesd_profile_info *out);
 
 /* Small-M weight-streaming GEMM on its own: y[M,N] = x[M,K] . W[N,K]^T with bf16 W, fp32 x and y.
- * pipesd_gemm_packed_bytes: size of the repacked copy of W.  pipesd_gemm_pack: W (device, row-major
+ * pipesd_gemm_packed_bytes: size of the repacked copy of W (rows padded to a multiple of 128).  pipesd_gemm_pack: W (device, row-major
  * bf16 [N,K]) -> packed (device).  pipesd_gemm_run: x, y device; scratch device of
  * pipesd_gemm_scratch_bytes(M,N,K) bytes (split-K partial sums).  N, K multiples of 16. */
 uint64_t pipesd_gemm_packed_bytes(int32_t N, int32_t K);
@@ -198,6 +198,9 @@ uint64_t pipesd_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
 int32_t pipesd_gemm_pack(const void *W, void *packed, int32_t N, int32_t K, void *cuda_stream);
 int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scratch, int32_t M, int32_t N,
                         int32_t K, void *cuda_stream);
+
+/* Tuning hook: force the number of K slices of every subsequent GEMM plan (0 = choose automatically). */
+int32_t pipesd_debug_gemm_force_split(int32_t S);
 
 /* The same GEMM for callers that cannot allocate device memory.  (The paper has no counterpart: this
  * is a convenience of the library, not a step of the method.)

@@ -88,6 +88,7 @@ _SIGNATURES = {
     "pipesd_gemm_pack": (i32, [vp, vp, i32, i32, vp]),
     "pipesd_gemm_run": (i32, [vp, vp, vp, vp, i32, i32, i32, vp]),
     "pipesd_gemm_run_static": (i32, [vp, vp, vp, i32, i32, i32, vp]),
+    "pipesd_debug_gemm_force_split": (i32, [i32]),
 }
 
 

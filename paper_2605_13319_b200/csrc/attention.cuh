@@ -21,6 +21,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const float* _
                                                                   int Hkv, float* __restrict__ o_part,
                                                                   float* __restrict__ m_part,
                                                                   float* __restrict__ l_part) {
+    pdl_wait();
+    pdl_launch_dependents();
     constexpr int RG = kAttnThreads / HD;          // row groups in the P.V phase
     constexpr int RPT = kMaxItemRows / RG;         // rows per thread in the P.V phase
     const int item = blockIdx.z, h = blockIdx.y, sp = blockIdx.x;
@@ -140,10 +142,13 @@ static inline size_t attn_smem_bytes(int hd) {
            sizeof(size_t) * kAttnTile;
 }
 
-// Merge the splits: out = sum_s e^{m_s - m} o_s / sum_s e^{m_s - m} l_s.  grid (M, n_q_heads), block HD.
+// Merge the splits: out = sum_s e^{m_s - m} o_s / sum_s e^{m_s - m} l_s, stored as split-bf16 B fragments
+// for the output projection (column index = head * hd + e).  grid (M, n_q_heads), block hd.
 __global__ void attn_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ m_part,
-                                    const float* __restrict__ l_part, PassMeta meta, int Hq, int hd,
-                                    float* __restrict__ out) {
+                                    const float* __restrict__ l_part, PassMeta meta, int M, int Hq, int hd,
+                                    uint32_t* __restrict__ xf_out) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int row = blockIdx.x, h = blockIdx.y, e = threadIdx.x;
     const int item = meta.row_item[row];
     const int r = row - meta.it_row0[item], nsplit = meta.it_nsplit[item];
@@ -151,14 +156,16 @@ __global__ void attn_combine_kernel(const float* __restrict__ o_part, const floa
     float m = -INFINITY;
     for (int s = 0; s < nsplit; ++s) m = fmaxf(m, m_part[slot0 + s]);
     float num = 0.f, den = 0.f;
+#pragma unroll 4
     for (int s = 0; s < nsplit; ++s) {
-        float ms = m_part[slot0 + s];
-        if (ms == -INFINITY) continue;       // split lies wholly beyond this row's causal horizon
-        float w = expf(ms - m);
+        const float ms = m_part[slot0 + s];
+        const float w = (ms == -INFINITY) ? 0.f : expf(ms - m);   // a split wholly beyond the causal horizon
         num += w * o_part[(slot0 + s) * hd + e];
         den += w * l_part[slot0 + s];
     }
-    out[((size_t)row * Hq + h) * hd + e] = num / den;
+    const float v = num / den;
+    const float v1 = __shfl_down_sync(0xffffffffu, v, 1);
+    if ((e & 1) == 0) xf_store_pair(xf_out, row, h * hd + e, v, v1, (Hq * hd) / 16, xf_nt(M));
 }
 
 }  // namespace pipesd

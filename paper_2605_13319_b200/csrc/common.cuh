@@ -59,6 +59,90 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     return v;
 }
 
+// ---- shared-memory barriers, bulk asynchronous copies, programmatic dependent launch ----------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for the barrier phase with the given parity.  Bounded: gives up (returns false) after about two
+// seconds so that a protocol error can never hang the GPU; callers then raise the kernel's error word.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if ((it & 1023u) == 1023u) {
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 2000000000ull) return false;
+        }
+    }
+}
+// Contiguous global -> shared copy by the copy engine; completion is counted in bytes on `bar`.
+// Both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
+// while its predecessor drains; pdl_wait() blocks until the predecessor has completed and its writes
+// are visible, pdl_launch_dependents() lets the successor start early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                     Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// ---- split-bf16 activation arrays ("xf"): B fragments of mma.m16n8k16 in global memory ----------
+// Layout [token block][k16 step][n8 tile][lane] of uint4 = {hi.b0, hi.b1, lo.b0, lo.b1} where, for lane
+// = 4*g + t, b0 holds k = 2t, 2t+1 and b1 holds k = 2t+8, 2t+9 of token 8*tile + g.
+// Stores the pair (k, k+1), k even, of one token.  KS = K/16, NT = tiles per token block.
+__device__ __forceinline__ void xf_store_pair(uint32_t* xf, int tok, int k, float v0, float v1, int KS, int NT) {
+    const int tb = tok / (8 * NT), nt = (tok >> 3) % NT, g = tok & 7;
+    const int ks = k >> 4, kk = k & 15, t = (kk & 7) >> 1, half = kk >> 3;
+    const size_t slot = ((size_t)(tb * KS + ks) * NT + nt) * 32 + g * 4 + t;
+    uint16_t h0, l0, h1, l1;
+    split_bf16(v0, h0, l0);
+    split_bf16(v1, h1, l1);
+    xf[slot * 4 + half] = pack2(h0, h1);
+    xf[slot * 4 + 2 + half] = pack2(l0, l1);
+}
+
 // Offset (in elements) of K (kv=0) or V (kv=1) element (slot, e) of a head inside the paged pool:
 // layout [layer][page][kv][head][slot][e].
 __device__ __host__ __forceinline__ size_t kv_index(int layer, int n_pages, int page, int kv, int n_kv_heads,

@@ -2,6 +2,7 @@
 // the residual add and RMSNorm, rotary embedding fused with the KV-page append, SwiGLU gate.
 #pragma once
 #include "common.cuh"
+#include "gemm.cuh"
 
 namespace pipesd {
 
@@ -21,38 +22,71 @@ struct PassMeta {
     int max_pages;
 };
 
-// x_new = (first layer ? bf16 embedding row : x) + sum_s part[s]   (residual stream, fp32)
-// h     = x_new * rsqrt(mean(x_new^2) + eps) * gain
-// One CTA per row.  The sum over split-K partials is taken in slice order (deterministic).
-__global__ void __launch_bounds__(256) add_norm_kernel(float* __restrict__ x, const uint16_t* __restrict__ emb,
-                                                       const int32_t* __restrict__ row_tok,
-                                                       const float* __restrict__ part, int S, int M,
-                                                       const float* __restrict__ gain, float eps, int d,
-                                                       float* __restrict__ h) {
+// x_new = (first layer ? bf16 embedding row : x) + sum_s part[s]   (residual stream, fp32, written back)
+// h     = x_new * rsqrt(mean(x_new^2) + eps) * gain                 (written as split-bf16 B fragments)
+// One CTA of 1024 threads per row, four columns per thread.  The sum over split-K partials is taken in
+// slice order (deterministic); the loads of all slices are independent, so they overlap.
+constexpr int kNormThreads = 1024;
+constexpr int kNormMaxVec = 2;   // float4 per thread: d <= 8192
+__global__ void __launch_bounds__(kNormThreads) add_norm_kernel(float* __restrict__ x, const uint16_t* __restrict__ emb,
+                                                                const int32_t* __restrict__ row_tok,
+                                                                const float* __restrict__ part, int S, int M,
+                                                                const float* __restrict__ gain, float eps, int d,
+                                                                uint32_t* __restrict__ xf_out) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int row = blockIdx.x;
-    __shared__ float red[8];
+    __shared__ float red[kNormThreads / 32];
+    float4 v[kNormMaxVec];
     float ss = 0.f;
     float* xr = x + (size_t)row * d;
-    for (int e = threadIdx.x; e < d; e += 256) {
-        float v = emb ? bf16_bits_to_f32(emb[(size_t)row_tok[row] * d + e]) : xr[e];
-        for (int s = 0; s < S; ++s) v += part[((size_t)s * M + row) * d + e];
-        xr[e] = v;
-        ss += v * v;
+#pragma unroll
+    for (int i = 0; i < kNormMaxVec; ++i) {
+        const int e = (threadIdx.x + i * kNormThreads) * 4;
+        if (e < d) {
+            float4 a;
+            if (emb) {
+                const uint2 b = *reinterpret_cast<const uint2*>(emb + (size_t)row_tok[row] * d + e);
+                a = make_float4(__uint_as_float(b.x << 16), __uint_as_float(b.x & 0xffff0000u),
+                                __uint_as_float(b.y << 16), __uint_as_float(b.y & 0xffff0000u));
+            } else {
+                a = *reinterpret_cast<const float4*>(xr + e);
+            }
+#pragma unroll 4
+            for (int s = 0; s < S; ++s) {
+                const float4 p = *reinterpret_cast<const float4*>(part + ((size_t)s * M + row) * d + e);
+                a.x += p.x; a.y += p.y; a.z += p.z; a.w += p.w;
+            }
+            *reinterpret_cast<float4*>(xr + e) = a;
+            ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+            v[i] = a;
+        }
     }
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
     float tot = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) tot += red[w];
+    for (int w = 0; w < kNormThreads / 32; ++w) tot += red[w];
     const float r = rsqrtf(tot / (float)d + eps);
-    for (int e = threadIdx.x; e < d; e += 256) h[(size_t)row * d + e] = xr[e] * r * gain[e];
+    const int KS = d / 16, NT = xf_nt(M);
+#pragma unroll
+    for (int i = 0; i < kNormMaxVec; ++i) {
+        const int e = (threadIdx.x + i * kNormThreads) * 4;
+        if (e < d) {
+            const float4 g = *reinterpret_cast<const float4*>(gain + e);
+            xf_store_pair(xf_out, row, e, v[i].x * r * g.x, v[i].y * r * g.y, KS, NT);
+            xf_store_pair(xf_out, row, e + 2, v[i].z * r * g.z, v[i].w * r * g.w, KS, NT);
+        }
+    }
 }
 
 // cos/sin of pos * base^(-2j/hd), evaluated in fp64 (positions reach 10^4, fp32 angles would lose
 // three digits), stored fp32 [M][hd/2].
 __global__ void rope_table_kernel(const int32_t* __restrict__ row_pos, int M, int hd, double log_base,
                                   float* __restrict__ cs, float* __restrict__ sn) {
+    pdl_wait();
+    pdl_launch_dependents();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     int half = hd / 2;
     if (i >= M * half) return;
@@ -72,6 +106,8 @@ __global__ void rope_kv_kernel(const float* __restrict__ part, int S, int M, int
                                const float* __restrict__ cs, const float* __restrict__ sn, PassMeta meta,
                                float* __restrict__ qout, uint16_t* __restrict__ kv_pool, int layer,
                                int n_pages, int page_size) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int row = blockIdx.x, head = blockIdx.y, j = threadIdx.x, half = hd / 2;
     const int Nqkv = (Hq + 2 * Hkv) * hd;
     const int col = head * hd + j;
@@ -102,18 +138,23 @@ __global__ void rope_kv_kernel(const float* __restrict__ part, int S, int M, int
     dst[j + half] = f32_to_bf16_bits(b);
 }
 
-// act = silu(sum_s gate_s) * sum_s up_s ; partials are [S][M][2F] with gate in [0,F), up in [F,2F).
-__global__ void silu_mul_kernel(const float* __restrict__ part, int S, int M, int F, float* __restrict__ act) {
-    size_t n = (size_t)M * F;
+// act = silu(sum_s gate_s) * sum_s up_s, stored as split-bf16 B fragments for the down projection.
+// Partials are [S][M][2F] with gate in [0,F), up in [F,2F).  One thread per (row, even column).
+__global__ void silu_mul_kernel(const float* __restrict__ part, int S, int M, int F, uint32_t* __restrict__ xf_out) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const size_t n = (size_t)M * (F / 2);
+    const int KS = F / 16, NT = xf_nt(M);
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        size_t row = i / F, f = i % F;
-        float g = 0.f, u = 0.f;
+        const int row = (int)(i / (F / 2)), f = 2 * (int)(i % (F / 2));
+        float2 g = make_float2(0.f, 0.f), u = make_float2(0.f, 0.f);
+#pragma unroll 4
         for (int s = 0; s < S; ++s) {
-            const float* p = part + ((size_t)s * M + row) * 2 * F;
-            g += p[f];
-            u += p[F + f];
+            const float* p = part + ((size_t)s * M + row) * 2 * F + f;
+            const float2 a = *reinterpret_cast<const float2*>(p), b = *reinterpret_cast<const float2*>(p + F);
+            g.x += a.x; g.y += a.y; u.x += b.x; u.y += b.y;
         }
-        act[i] = g / (1.f + expf(-g)) * u;
+        xf_store_pair(xf_out, row, f, g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y, KS, NT);
     }
 }
 

@@ -91,7 +91,7 @@ Derived derive(const pipesd_model_cfg& c) {
 }
 
 struct WsLayout {
-    size_t x, h, qbuf, attn, act, logits, partA, partB, o_part, m_part, l_part, cs, sn, stats, results, meta,
+    size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, o_part, m_part, l_part, cs, sn, stats, results, meta,
         block_tab, qstage, total;
 };
 
@@ -101,10 +101,11 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
     const size_t M = c.max_rows;
     w.x = take(4 * M * c.d_model);
-    w.h = take(4 * M * c.d_model);
+    // split-bf16 activation arrays: 4 bytes per element, token count padded to whole token blocks
+    w.xf_h = take(4 * (M + 32) * c.d_model);
     w.qbuf = take(4 * M * d.qd);
-    w.attn = take(4 * M * d.qd);
-    w.act = take(4 * M * c.d_ffn);
+    w.xf_attn = take(4 * (M + 32) * d.qd);
+    w.xf_act = take(4 * (M + 32) * c.d_ffn);
     w.logits = take(4 * M * c.vocab);
     w.partA = take(4 * d.part_floats);
     w.partB = take(4 * d.part_floats);
@@ -115,7 +116,7 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     w.cs = take(4 * M * (c.head_dim / 2));
     w.sn = take(4 * M * (c.head_dim / 2));
     w.stats = take(sizeof(RowStat) * M * kStatSplits);
-    w.results = take(sizeof(RejectOut) * d.max_items);
+    w.results = take(sizeof(RejectOut) * d.max_items + 16);   // + the device error word, read back with the results
     w.meta = take(meta_layout(c.max_rows, d.max_items).total);
     w.block_tab = take(4 * (size_t)c.max_requests * d.max_pages);
     w.qstage = take(4 * M * c.vocab);
@@ -123,7 +124,7 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     return w;
 }
 
-size_t packed_bytes(int N, int K) { return align_up((size_t)N * K * 2); }
+size_t packed_bytes(int N, int K) { return align_up(gemm_packed_bytes(N, K)); }
 
 size_t weights_bytes(const pipesd_model_cfg& c, const Derived& d) {
     size_t per_layer = packed_bytes(d.Nqkv, c.d_model) + packed_bytes(c.d_model, d.qd) +
@@ -143,7 +144,7 @@ int check_cfg(const pipesd_model_cfg* c) {
         c->vocab < 16)
         return PIPESD_E_INVALID;
     if (c->head_dim != 64 && c->head_dim != 128) return PIPESD_E_INVALID;
-    if (c->d_model % 16 || c->d_ffn % 16 || c->vocab % 16) return PIPESD_E_INVALID;
+    if (c->d_model % 16 || c->d_ffn % 16 || c->vocab % 16 || c->d_model > 8192) return PIPESD_E_INVALID;
     if (c->n_q_heads % c->n_kv_heads) return PIPESD_E_INVALID;
     if (c->page_size < 1 || c->page_size > 256 || c->n_pages < 1 || c->max_requests < 1) return PIPESD_E_INVALID;
     if (c->max_draft < 1 || c->max_draft > kMaxItemRows - 1) return PIPESD_E_INVALID;
@@ -204,6 +205,7 @@ struct pipesd_ctx {
 
     template <typename T>
     T* W(size_t off) const { return reinterpret_cast<T*>(wsp + off); }
+    int* err_word() const { return reinterpret_cast<int*>(wsp + ws.results + sizeof(RejectOut) * dv.max_items); }
     PassMeta pass_meta() const {
         PassMeta m;
         const char* b = wsp + ws.meta;
@@ -242,8 +244,8 @@ int cuda_fail(pipesd_ctx* c, cudaError_t e, const char* where) {
     } while (0)
 
 // Launch one weight-streaming GEMM with accounting (and event timing when profiling is on).
-int launch_gemm(pipesd_ctx* ctx, const GemmPlan& p, const uint4* W, const float* x, int ldx, float* out, int M,
-                int N, int K) {
+int launch_gemm(pipesd_ctx* ctx, const GemmPlan& p, const uint4* W, const void* xf, float* out, int M, int N,
+                int K) {
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (ctx->time_gemms) {
         if (ctx->prof_used + 2 > ctx->prof_ev.size()) {
@@ -258,7 +260,7 @@ int launch_gemm(pipesd_ctx* ctx, const GemmPlan& p, const uint4* W, const float*
         ctx->prof_used += 2;
         CU(cudaEventRecord(e0, ctx->st));
     }
-    CU(gemm_launch(p, W, x, ldx, out, M, N, K, ctx->st));
+    CU(gemm_launch(p, W, (const uint4*)xf, out, ctx->err_word(), M, N, ctx->st));
     if (e1) CU(cudaEventRecord(e1, ctx->st));
     ctx->n_launch += 1;
     ctx->n_gemm += 1;
@@ -360,10 +362,10 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     const PassMeta meta = ctx->pass_meta();
     cudaStream_t st = ctx->st;
     float* x = ctx->W<float>(ctx->ws.x);
-    float* h = ctx->W<float>(ctx->ws.h);
+    uint32_t* xf_h = ctx->W<uint32_t>(ctx->ws.xf_h);
     float* qbuf = ctx->W<float>(ctx->ws.qbuf);
-    float* attn = ctx->W<float>(ctx->ws.attn);
-    float* act = ctx->W<float>(ctx->ws.act);
+    uint32_t* xf_attn = ctx->W<uint32_t>(ctx->ws.xf_attn);
+    uint32_t* xf_act = ctx->W<uint32_t>(ctx->ws.xf_act);
     float* partA = ctx->W<float>(ctx->ws.partA);
     float* partB = ctx->W<float>(ctx->ws.partB);
     float* o_part = ctx->W<float>(ctx->ws.o_part);
@@ -372,42 +374,49 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     float* cs = ctx->W<float>(ctx->ws.cs);
     float* sn = ctx->W<float>(ctx->ws.sn);
     const int hd = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads, d = c.d_model, F = c.d_ffn;
+    const uint16_t* no_emb = nullptr;
+    const int32_t* no_tok = nullptr;
 
+    // Every kernel of the chain is launched with programmatic stream serialisation: it may start while its
+    // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
     {
         int n = M * hd / 2;
-        rope_table_kernel<<<(n + 127) / 128, 128, 0, st>>>(meta.row_pos, M, hd, log((double)c.rope_base), cs, sn);
+        CU(launch_pdl(rope_table_kernel, dim3((n + 127) / 128), dim3(128), 0, st, meta.row_pos, M, hd,
+                      log((double)c.rope_base), cs, sn));
     }
     const float* part = nullptr;
     int S = 0;
     const size_t asmem = attn_smem_bytes(hd);
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& lw = ctx->layers[l];
-        add_norm_kernel<<<M, 256, 0, st>>>(x, l == 0 ? ctx->emb : nullptr, meta.row_tok, part, S, M, lw.n1,
-                                           c.rms_eps, d, h);
+        CU(launch_pdl(add_norm_kernel, dim3(M), dim3(kNormThreads), 0, st, x, l == 0 ? (const uint16_t*)ctx->emb : no_emb,
+                      meta.row_tok, part, S, M, (const float*)lw.n1, c.rms_eps, d, xf_h));
         GemmPlan p = gemm_plan(M, dv.Nqkv, d);
-        { int rc_ = launch_gemm(ctx, p, lw.qkv.packed, h, d, partA, M, dv.Nqkv, d); if (rc_) return rc_; }
-        rope_kv_kernel<<<dim3(M, Hq + 2 * Hkv), hd / 2, 0, st>>>(partA, p.S, M, Hq, Hkv, hd, cs, sn, meta, qbuf,
-                                                                 ctx->kv_pool, l, c.n_pages, c.page_size);
+        { int rc_ = launch_gemm(ctx, p, lw.qkv.packed, xf_h, partA, M, dv.Nqkv, d); if (rc_) return rc_; }
+        CU(launch_pdl(rope_kv_kernel, dim3(M, Hq + 2 * Hkv), dim3(hd / 2), 0, st, (const float*)partA, p.S, M, Hq, Hkv, hd,
+                      (const float*)cs, (const float*)sn, meta, qbuf, ctx->kv_pool, l, c.n_pages, c.page_size));
         dim3 ag(max_nsplit, Hq, n_items);
         if (hd == 128)
-            attn_split_kernel<128><<<ag, kAttnThreads, asmem, st>>>(qbuf, meta, ctx->kv_pool, l, c.n_pages,
-                                                                    c.page_size, Hq, Hkv, o_part, m_part, l_part);
+            CU(launch_pdl(attn_split_kernel<128>, ag, dim3(kAttnThreads), asmem, st, (const float*)qbuf, meta,
+                          (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, Hq, Hkv, o_part, m_part, l_part));
         else
-            attn_split_kernel<64><<<ag, kAttnThreads, asmem, st>>>(qbuf, meta, ctx->kv_pool, l, c.n_pages,
-                                                                   c.page_size, Hq, Hkv, o_part, m_part, l_part);
-        attn_combine_kernel<<<dim3(M, Hq), hd, 0, st>>>(o_part, m_part, l_part, meta, Hq, hd, attn);
+            CU(launch_pdl(attn_split_kernel<64>, ag, dim3(kAttnThreads), asmem, st, (const float*)qbuf, meta,
+                          (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, Hq, Hkv, o_part, m_part, l_part));
+        CU(launch_pdl(attn_combine_kernel, dim3(M, Hq), dim3(hd), 0, st, (const float*)o_part, (const float*)m_part,
+                      (const float*)l_part, meta, M, Hq, hd, xf_attn));
         p = gemm_plan(M, d, dv.qd);
-        { int rc_ = launch_gemm(ctx, p, lw.o.packed, attn, dv.qd, partB, M, d, dv.qd); if (rc_) return rc_; }
-        add_norm_kernel<<<M, 256, 0, st>>>(x, nullptr, nullptr, partB, p.S, M, lw.n2, c.rms_eps, d, h);
+        { int rc_ = launch_gemm(ctx, p, lw.o.packed, xf_attn, partB, M, d, dv.qd); if (rc_) return rc_; }
+        CU(launch_pdl(add_norm_kernel, dim3(M), dim3(kNormThreads), 0, st, x, no_emb, no_tok, (const float*)partB, p.S, M,
+                      (const float*)lw.n2, c.rms_eps, d, xf_h));
         p = gemm_plan(M, 2 * F, d);
-        { int rc_ = launch_gemm(ctx, p, lw.gu.packed, h, d, partA, M, 2 * F, d); if (rc_) return rc_; }
+        { int rc_ = launch_gemm(ctx, p, lw.gu.packed, xf_h, partA, M, 2 * F, d); if (rc_) return rc_; }
         {
-            size_t n = (size_t)M * F;
+            size_t n = (size_t)M * (F / 2);
             int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
-            silu_mul_kernel<<<blocks, 256, 0, st>>>(partA, p.S, M, F, act);
+            CU(launch_pdl(silu_mul_kernel, dim3(blocks), dim3(256), 0, st, (const float*)partA, p.S, M, F, xf_act));
         }
         p = gemm_plan(M, d, F);
-        { int rc_ = launch_gemm(ctx, p, lw.dn.packed, act, F, partB, M, d, F); if (rc_) return rc_; }
+        { int rc_ = launch_gemm(ctx, p, lw.dn.packed, xf_act, partB, M, d, F); if (rc_) return rc_; }
         part = partB;
         S = p.S;
         ctx->n_launch += 6;   // add_norm x2, rope_kv, attn_split, attn_combine, silu_mul
@@ -417,10 +426,12 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         ctx->n_launch += 2 + (want_reject ? 1 : 0);   // add_norm, row_stats, accept_sample
         float* logits = ctx->W<float>(ctx->ws.logits);
         RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
-        add_norm_kernel<<<M, 256, 0, st>>>(x, nullptr, nullptr, part, S, M, ctx->final_norm, c.rms_eps, d, h);
+        CU(launch_pdl(add_norm_kernel, dim3(M), dim3(kNormThreads), 0, st, x, no_emb, no_tok, part, S, M,
+                      (const float*)ctx->final_norm, c.rms_eps, d, xf_h));
         GemmPlan p = gemm_plan(M, c.vocab, d);
         float* dst = p.S == 1 ? logits : partA;
-        { int rc_ = launch_gemm(ctx, p, ctx->lm.packed, h, d, dst, M, c.vocab, d); if (rc_) return rc_; }
+        { int rc_ = launch_gemm(ctx, p, ctx->lm.packed, xf_h, dst, M, c.vocab, d); if (rc_) return rc_; }
+        // plain launches from here on: they start after the GEMM has fully completed
         row_stats_kernel<<<dim3(M, kStatSplits), 256, 0, st>>>(p.S == 1 ? nullptr : partA, p.S, M, c.vocab, logits,
                                                                stats);
         ctx->last_rows = M;
@@ -505,7 +516,7 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         if (cudaEventCreateWithFlags(&ctx->ev_meta[i], cudaEventDisableTiming) != cudaSuccess)
             return bail(PIPESD_E_CUDA);
     }
-    if (cudaHostAlloc((void**)&ctx->h_results, sizeof(RejectOut) * dv.max_items, cudaHostAllocDefault) != cudaSuccess)
+    if (cudaHostAlloc((void**)&ctx->h_results, sizeof(RejectOut) * dv.max_items + 16, cudaHostAllocDefault) != cudaSuccess)
         return bail(PIPESD_E_CUDA);
 
     // ---- repack the weights into the library's own layout
@@ -514,15 +525,17 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     size_t off = 0;
     auto take = [&](size_t bytes) { char* p = wp + off; off += align_up(bytes); return p; };
     auto pack = [&](GemmW& g, int N, int K, std::initializer_list<std::pair<const void*, int>> srcs) {
-        g.packed = (uint4*)take((size_t)N * K * 2);
+        g.packed = (uint4*)take(gemm_packed_bytes(N, K));
         g.N = N;
         g.K = K;
+        const int padded = (N + 127) / 128 * 128;
         int r0 = 0;
+        size_t left = srcs.size();
         for (auto& s : srcs) {
-            size_t total = (size_t)(s.second / 16) * (K / 16) * 32;
+            const int pad_to = --left == 0 ? padded : r0 + s.second;   // the last source also zero-fills the padding
+            size_t total = (size_t)((pad_to - r0) / 16) * (K / 16) * 32;
             int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
-            gemm_pack_kernel<<<blocks, 256, 0, st>>>((const uint16_t*)s.first,
-                                                     g.packed + (size_t)(r0 / 16) * (K / 16) * 32, s.second, K);
+            gemm_pack_kernel<<<blocks, 256, 0, st>>>((const uint16_t*)s.first, g.packed, r0, s.second, K, pad_to);
             r0 += s.second;
         }
     };
@@ -574,6 +587,14 @@ int32_t pipesd_ctx_sync(pipesd_ctx* ctx) {
     if (!ctx) return PIPESD_E_INVALID;
     CU(cudaStreamSynchronize(ctx->st));
     if (ctx->pend_dst) {
+        const int dev_err = *reinterpret_cast<const int*>(ctx->h_results + ctx->dv.max_items);
+        if (dev_err) {   // a bounded device-side wait gave up: the results of this call are void
+            for (int i = 0; i < ctx->pend_n; ++i) ctx->pend_dst[i].status = PIPESD_E_CUDA;
+            ctx->pend_dst = nullptr;
+            ctx->pend_n = 0;
+            cudaMemsetAsync(ctx->err_word(), 0, 4, ctx->st);
+            return fail(ctx, PIPESD_E_CUDA, "a device-side wait timed out (kernel error word set)");
+        }
         for (int i = 0; i < ctx->pend_n; ++i) {
             ctx->pend_dst[i].n_accepted = ctx->h_results[i].n_accepted;
             ctx->pend_dst[i].next_token = ctx->h_results[i].next_token;
@@ -696,7 +717,7 @@ int32_t pipesd_verify(pipesd_ctx* ctx, int32_t n_req, const pipesd_verify_item* 
     }
     int rc = run_pass(ctx, items, true, true);
     if (rc != PIPESD_OK) return rc;
-    CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut) * n_req,
+    CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut) * ctx->dv.max_items + 4,
                        cudaMemcpyDeviceToHost, ctx->st));
     ctx->pend_dst = results;
     ctx->pend_n = n_req;
@@ -872,19 +893,46 @@ int32_t pipesd_profile_read(pipesd_ctx* ctx, pipesd_profile_info* out) {
     return PIPESD_OK;
 }
 
-uint64_t pipesd_gemm_packed_bytes(int32_t N, int32_t K) { return (uint64_t)N * K * 2; }
+uint64_t pipesd_gemm_packed_bytes(int32_t N, int32_t K) {
+    if (N < 16 || K < 16) return 0;
+    return gemm_packed_bytes(N, K);
+}
+
+static size_t gemm_xf_bytes(int M, int K) { return align_up(xf_elems(M, K) * 16); }
 
 uint64_t pipesd_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K) {
     if (M < 1 || N < 16 || K < 16) return 0;
     GemmPlan p = gemm_plan(M, N, K);
-    return (uint64_t)p.S * M * N * 4;
+    return gemm_xf_bytes(M, K) + (p.S > 1 ? (uint64_t)p.S * M * N * 4 : 0);
 }
 
 int32_t pipesd_gemm_pack(const void* W, void* packed, int32_t N, int32_t K, void* cuda_stream) {
     if (!W || !packed || N < 16 || K < 16 || N % 16 || K % 16) return PIPESD_E_INVALID;
-    size_t total = (size_t)(N / 16) * (K / 16) * 32;
+    const int padded = (N + 127) / 128 * 128;
+    size_t total = (size_t)(padded / 16) * (K / 16) * 32;
     int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
-    gemm_pack_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)W, (uint4*)packed, N, K);
+    gemm_pack_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)W, (uint4*)packed, 0, N, K, padded);
+    return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
+}
+
+// x -> split-bf16 fragments, GEMM, fixed-order sum of the K slices.  scratch = [xf | partial sums].
+static int32_t gemm_run_with_scratch(const void* packed, const float* x, float* y, void* scratch, int M, int N, int K,
+                                     cudaStream_t st) {
+    const GemmPlan p = gemm_plan(M, N, K);
+    uint32_t* xf = (uint32_t*)scratch;
+    float* part = (float*)((char*)scratch + gemm_xf_bytes(M, K));
+    {
+        size_t n = (size_t)M * (K / 2);
+        int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
+        xf_format_kernel<<<blocks, 256, 0, st>>>(x, xf, M, K);
+    }
+    float* dst = p.S == 1 ? y : part;
+    if (gemm_launch(p, (const uint4*)packed, (const uint4*)xf, dst, nullptr, M, N, st) != cudaSuccess) return PIPESD_E_CUDA;
+    if (p.S > 1) {
+        size_t n = (size_t)M * N;
+        int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
+        reduce_partials_kernel<<<blocks, 256, 0, st>>>((const float*)part, y, n, p.S);
+    }
     return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
 }
 
@@ -896,17 +944,17 @@ int32_t pipesd_gemm_run(const void* packed, const float* x, float* y, void* scra
         if (gemm_init_attrs() != cudaSuccess) return PIPESD_E_CUDA;
         attrs = true;
     }
-    cudaStream_t st = (cudaStream_t)cuda_stream;
-    GemmPlan p = gemm_plan(M, N, K);
-    float* dst = p.S == 1 ? y : (float*)scratch;
-    if (gemm_launch(p, (const uint4*)packed, x, K, dst, M, N, K, st) != cudaSuccess) return PIPESD_E_CUDA;
-    if (p.S > 1) {
-        size_t n = (size_t)M * N;
-        int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
-        reduce_partials_kernel<<<blocks, 256, 0, st>>>((const float*)scratch, y, n, p.S);
-    }
-    return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
+    return gemm_run_with_scratch(packed, x, y, scratch, M, N, K, (cudaStream_t)cuda_stream);
 }
+
+int32_t pipesd_debug_gemm_force_split(int32_t S) {
+    g_gemm_force_split = S > 0 ? S : 0;
+    return PIPESD_OK;
+}
+
+}  // extern "C"
+
+extern "C" {
 
 // ---- GEMM without any caller- or library-side allocation ------------------------------------
 // Split-K partial sums of pipesd_gemm_run_static live in this fixed array.  It is part of the
@@ -939,24 +987,13 @@ int static_scratch_for_current_device(void** out) {
 int32_t pipesd_gemm_run_static(const void* packed, const float* x, float* y, int32_t M, int32_t N, int32_t K,
                                void* cuda_stream) {
     if (!packed || !x || !y || M < 1 || N < 16 || K < 16 || N % 16 || K % 16) return PIPESD_E_INVALID;
-    const GemmPlan p = gemm_plan(M, N, K);
-    const size_t need = p.S > 1 ? (size_t)p.S * M * N * sizeof(float) : 0;
-    if (need > (size_t)PIPESD_STATIC_SCRATCH_BYTES) return PIPESD_E_TOO_LARGE;
+    if (pipesd_gemm_scratch_bytes(M, N, K) > (uint64_t)PIPESD_STATIC_SCRATCH_BYTES) return PIPESD_E_TOO_LARGE;
     void* scratch = nullptr;
     int rc = static_scratch_for_current_device(&scratch);
     if (rc != PIPESD_OK) return rc;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
-    // Nothing has to be cleared: every partial sum the reduction reads is written by the GEMM kernel of
-    // this same call first (all S slices, all M rows, all N columns), so the previous call's contents
-    // never reach the output.
-    float* dst = p.S == 1 ? y : (float*)scratch;
-    if (gemm_launch(p, (const uint4*)packed, x, K, dst, M, N, K, st) != cudaSuccess) return PIPESD_E_CUDA;
-    if (p.S > 1) {
-        size_t n = (size_t)M * N;
-        int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
-        reduce_partials_kernel<<<blocks, 256, 0, st>>>((const float*)scratch, y, n, p.S);
-    }
-    return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
+    // Nothing has to be cleared: the activation fragments and every partial sum the reduction reads are
+    // written by this same call first, so the previous call's contents never reach the output.
+    return gemm_run_with_scratch(packed, x, y, scratch, M, N, K, (cudaStream_t)cuda_stream);
 }
 
 }  // extern "C"
