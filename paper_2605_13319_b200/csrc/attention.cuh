@@ -1,7 +1,16 @@
 // Multi-query decode attention over a paged bf16 KV cache: each request contributes a short chunk
 // of query rows (the pending token plus its k drafts) that attend to the cached prefix and, causally,
-// to each other.  The prefix is cut into splits ("split-K"); every split produces an un-normalised
+// to each other.  The keys are cut into splits ("split-K"); every split produces an un-normalised
 // partial output with its running max and sum, and a second kernel merges the splits.
+//
+// One CTA (4 warps) = one KV head of one request x one split x up to 64 query rows, where the rows are
+// all (query head of the group, chunk row) pairs that share the KV head (GQA).  K and V tiles of 64 keys
+// travel global -> shared with 16-byte cp.async in a three-stage ring (page table resolved per key row,
+// rows XOR-swizzled so that ldmatrix is conflict-free).  QK^T and PV run on mma.sync m16n8k16 with fp32
+// accumulation; Q and the softmax probabilities are fp32 values split into bf16 hi + lo terms (two MMAs),
+// K and V are the cache's bf16.  How the 4 warps share a tile depends on the number of 16-row tiles:
+// 1 tile -> 4 key strips of 16, 2 tiles -> 2 x 2 strips of 32, 3-4 tiles -> one tile each over all 64 keys;
+// warps that split the keys keep independent online-softmax states that are merged in shared memory.
 #pragma once
 #include "common.cuh"
 #include "layers.cuh"
@@ -9,137 +18,338 @@
 namespace pipesd {
 
 constexpr int kAttnThreads = 128;
-constexpr int kAttnTile = 128;  // keys per inner tile
+constexpr int kAttnTile = 64;       // keys per tile
+constexpr int kAttnStages = 3;
+constexpr int kAttnMaxRowTiles = 4; // 64 query rows per CTA
 
-// grid (max_nsplit, n_q_heads, n_items), block 128.  One CTA: one query head of one request against
-// one split of its keys.  Thread t scores key t of the tile against all rows, a warp per row does the
-// online-softmax update, then thread (e, row group) accumulates P.V for output dimension e.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+    const int sz = valid ? 16 : 0;   // size 0: the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+template <int HD>
+struct AttnSmem {
+    static constexpr int kRowBytes = HD * 2;
+    static constexpr int kTileBytes = kAttnTile * kRowBytes;            // one K or V tile
+    static constexpr int kStageBytes = 2 * kTileBytes;                  // K then V
+    static constexpr int kQTileBytes = (HD / 16) * 2 * 512;             // A fragments hi+lo of one 16-row tile
+    static constexpr int kRing = kAttnStages * kStageBytes;
+    static size_t bytes(int row_tiles) { return (size_t)kRing + (size_t)row_tiles * kQTileBytes; }
+};
+
+// Per-CTA constants shared by the mode-specialised bodies.
+struct AttnCtx {
+    const uint16_t* kv_pool;
+    const int32_t* bt;
+    int layer, n_pages, page_size, Hkv, kvh;
+    int k0, k1, base, rows, R, rho0;
+};
+
+// Issue the cp.async copies of one 64-key tile (K and V) into a ring stage.
+template <int HD>
+__device__ __forceinline__ void attn_load_tile(const AttnCtx& c, uint32_t stage_addr, int j0) {
+    constexpr int kChunks = HD / 8;                       // 16-byte chunks per row
+    constexpr int kPerThread = kAttnTile * kChunks / kAttnThreads;
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+        const int idx = threadIdx.x + i * kAttnThreads;
+        const int row = idx / kChunks, ch = idx % kChunks;
+        const int j = j0 + row;
+        const bool valid = j < c.k1;
+        size_t ko = 0, vo = 0;
+        if (valid) {
+            const int page = c.bt[j / c.page_size], slot = j % c.page_size;
+            ko = kv_index(c.layer, c.n_pages, page, 0, c.Hkv, c.kvh, c.page_size, slot, HD, ch * 8);
+            vo = kv_index(c.layer, c.n_pages, page, 1, c.Hkv, c.kvh, c.page_size, slot, HD, ch * 8);
+        }
+        const uint32_t off = row * (HD * 2) + ((ch ^ (row & 7)) << 4);
+        cp_async16(stage_addr + off, c.kv_pool + ko, valid);
+        cp_async16(stage_addr + AttnSmem<HD>::kTileBytes + off, c.kv_pool + vo, valid);
+    }
+}
+
+// Main loop for one CTA.  RTW = row-tile groups among the 4 warps (1, 2 or 4); 4/RTW = key strips.
+template <int HD, int RTW>
+__device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem, float* __restrict__ o_part,
+                                          float* __restrict__ m_part, float* __restrict__ l_part, int Hq, int G,
+                                          int nsplit, int sp, int part0) {
+    constexpr int KSW = 4 / RTW;               // key strips per tile
+    constexpr int STRIP = kAttnTile / KSW;     // keys per warp per tile
+    constexpr int NTS = STRIP / 8;             // score n-tiles per warp
+    constexpr int KSTEPS = HD / 16;
+    constexpr int NTO = HD / 8;                // output n-tiles
+    using SM = AttnSmem<HD>;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int rtw = warp % RTW, strip = warp / RTW;
+    const uint32_t ring = smem_u32(smem);
+    const unsigned char* qs = smem + SM::kRing + rtw * SM::kQTileBytes;
+    const int sk0 = strip * STRIP;
+    const bool warp_active = c.rho0 + rtw * 16 < c.R;
+
+    float o[NTO][4];
+#pragma unroll
+    for (int i = 0; i < NTO; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[i][e] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    // rows of this lane: rho = rho0 + rtw*16 + g (+8); r = rho % rows gives the causal horizon base + r
+    int horizon[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const int rho = c.rho0 + rtw * 16 + g + 8 * hh;
+        horizon[hh] = rho < c.R ? c.base + rho % c.rows : -1;   // keys j <= horizon are visible; -1: padding row
+    }
+
+    const int ntiles = (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile;
+    attn_load_tile<HD>(c, ring, c.k0);
+    cp_async_commit();
+    if (ntiles > 1) attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile);
+    cp_async_commit();
+
+    for (int it = 0; it < ntiles; ++it) {
+        cp_async_wait<1>();
+        __syncthreads();          // tile `it` has landed for everyone; everyone is done with tile it-1
+        if (it + 2 < ntiles)
+            attn_load_tile<HD>(c, ring + ((it + 2) % kAttnStages) * SM::kStageBytes, c.k0 + (it + 2) * kAttnTile);
+        cp_async_commit();
+        if (!warp_active) continue;
+        const uint32_t kst = ring + (it % kAttnStages) * SM::kStageBytes;
+        const uint32_t vst = kst + SM::kTileBytes;
+        const int j0 = c.k0 + it * kAttnTile + sk0;    // first key of this warp's strip
+
+        // ---- S = Q K^T over the strip
+        float s[NTS][4];
+#pragma unroll
+        for (int i = 0; i < NTS; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[i][e] = 0.f;
+#pragma unroll
+        for (int kp = 0; kp < KSTEPS / 2; ++kp) {
+            const uint4 qh0 = *reinterpret_cast<const uint4*>(qs + (((2 * kp) * 2 + 0) * 32 + lane) * 16);
+            const uint4 ql0 = *reinterpret_cast<const uint4*>(qs + (((2 * kp) * 2 + 1) * 32 + lane) * 16);
+            const uint4 qh1 = *reinterpret_cast<const uint4*>(qs + (((2 * kp + 1) * 2 + 0) * 32 + lane) * 16);
+            const uint4 ql1 = *reinterpret_cast<const uint4*>(qs + (((2 * kp + 1) * 2 + 1) * 32 + lane) * 16);
+#pragma unroll
+            for (int nt = 0; nt < NTS; ++nt) {
+                const int row = sk0 + nt * 8 + (lane & 7);
+                const int ch = kp * 4 + (lane >> 3);
+                uint32_t b[4];
+                ldmatrix_x4(b, kst + row * (HD * 2) + ((ch ^ (row & 7)) << 4));
+                mma_bf16_16816(s[nt], qh0, b[0], b[1]);
+                mma_bf16_16816(s[nt], ql0, b[0], b[1]);
+                mma_bf16_16816(s[nt], qh1, b[2], b[3]);
+                mma_bf16_16816(s[nt], ql1, b[2], b[3]);
+            }
+        }
+        // ---- mask, online softmax (rows g and g+8 of the tile)
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nt = 0; nt < NTS; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int j = j0 + nt * 8 + 2 * t + (e & 1);
+                const int hh = e >> 1;
+                const float v = (j < c.k1 && j <= horizon[hh]) ? s[nt][e] : -INFINITY;
+                s[nt][e] = v;
+                mx[hh] = fmaxf(mx[hh], v);
+            }
+        float alpha[2];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
+            mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
+            const float m_new = fmaxf(m_run[hh], mx[hh]);
+            alpha[hh] = (m_run[hh] == -INFINITY) ? 0.f : expf(m_run[hh] - m_new);
+            m_run[hh] = m_new;
+            l_run[hh] *= alpha[hh];
+        }
+#pragma unroll
+        for (int nt = 0; nt < NTS; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int hh = e >> 1;
+                const float p = (s[nt][e] == -INFINITY) ? 0.f : expf(s[nt][e] - m_run[hh]);
+                s[nt][e] = p;
+                l_run[hh] += p;      // per-lane partial; the quad is summed once at the end
+            }
+#pragma unroll
+        for (int i = 0; i < NTO; ++i) {
+            o[i][0] *= alpha[0]; o[i][1] *= alpha[0];
+            o[i][2] *= alpha[1]; o[i][3] *= alpha[1];
+        }
+        // ---- O += P V over the strip's keys, P split into bf16 hi + lo
+#pragma unroll
+        for (int kk = 0; kk < STRIP / 16; ++kk) {
+            uint4 ph, pl;
+            {
+                uint16_t h0, l0, h1, l1;
+                split_bf16(s[2 * kk][0], h0, l0); split_bf16(s[2 * kk][1], h1, l1);
+                ph.x = pack2(h0, h1); pl.x = pack2(l0, l1);
+                split_bf16(s[2 * kk][2], h0, l0); split_bf16(s[2 * kk][3], h1, l1);
+                ph.y = pack2(h0, h1); pl.y = pack2(l0, l1);
+                split_bf16(s[2 * kk + 1][0], h0, l0); split_bf16(s[2 * kk + 1][1], h1, l1);
+                ph.z = pack2(h0, h1); pl.z = pack2(l0, l1);
+                split_bf16(s[2 * kk + 1][2], h0, l0); split_bf16(s[2 * kk + 1][3], h1, l1);
+                ph.w = pack2(h0, h1); pl.w = pack2(l0, l1);
+            }
+#pragma unroll
+            for (int np = 0; np < NTO / 2; ++np) {
+                const int row = sk0 + kk * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
+                const int ch = np * 2 + (lane >> 4);
+                uint32_t b[4];
+                ldmatrix_x4_trans(b, vst + row * (HD * 2) + ((ch ^ (row & 7)) << 4));
+                mma_bf16_16816(o[2 * np], ph, b[0], b[1]);
+                mma_bf16_16816(o[2 * np], pl, b[0], b[1]);
+                mma_bf16_16816(o[2 * np + 1], ph, b[2], b[3]);
+                mma_bf16_16816(o[2 * np + 1], pl, b[2], b[3]);
+            }
+        }
+    }
+    cp_async_wait<0>();
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        l_run[hh] += __shfl_xor_sync(0xffffffffu, l_run[hh], 1);
+        l_run[hh] += __shfl_xor_sync(0xffffffffu, l_run[hh], 2);
+    }
+
+    // ---- write the split's partial result: merge the key strips first when the warps split the keys
+    auto emit = [&](int rho, int e, float v0, float v1, float m, float l, bool write_ml) {
+        if (rho >= c.R) return;
+        const int gq = rho / c.rows, r = rho % c.rows;
+        const size_t slot = (size_t)part0 + ((size_t)r * Hq + c.kvh * G + gq) * nsplit + sp;
+        *reinterpret_cast<float2*>(o_part + slot * HD + e) = make_float2(v0, v1);
+        if (write_ml) { m_part[slot] = m; l_part[slot] = l; }
+    };
+    if (KSW == 1) {
+        if (!warp_active) return;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int rho = c.rho0 + rtw * 16 + g + 8 * hh;
+#pragma unroll
+            for (int i = 0; i < NTO; ++i)
+                emit(rho, i * 8 + 2 * t, o[i][2 * hh], o[i][2 * hh + 1], m_run[hh], l_run[hh], i == 0 && t == 0);
+        }
+        return;
+    }
+    __syncthreads();                               // the ring is free: reuse it as the merge buffer
+    float* mo = reinterpret_cast<float*>(smem);    // [warp][16 rows][HD] then [warp][16] m, [warp][16] l
+    float* mm = mo + 4 * 16 * HD;
+    float* ml = mm + 4 * 16;
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const int row = g + 8 * hh;
+#pragma unroll
+        for (int i = 0; i < NTO; ++i)
+            *reinterpret_cast<float2*>(mo + ((size_t)warp * 16 + row) * HD + i * 8 + 2 * t) =
+                make_float2(o[i][2 * hh], o[i][2 * hh + 1]);
+        if (t == 0) { mm[warp * 16 + row] = m_run[hh]; ml[warp * 16 + row] = l_run[hh]; }
+    }
+    __syncthreads();
+    // thread -> (row tile group, row, column pairs): RTW*16 rows x HD/2 pairs over 128 threads
+    for (int idx = threadIdx.x; idx < RTW * 16 * (HD / 2); idx += kAttnThreads) {
+        const int e = 2 * (idx % (HD / 2)), rr = idx / (HD / 2), tile = rr / 16, row = rr % 16;
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < KSW; ++k) m = fmaxf(m, mm[(k * RTW + tile) * 16 + row]);
+        float v0 = 0.f, v1 = 0.f, l = 0.f;
+#pragma unroll
+        for (int k = 0; k < KSW; ++k) {
+            const int w = k * RTW + tile;
+            const float ms = mm[w * 16 + row];
+            const float wgt = (ms == -INFINITY) ? 0.f : expf(ms - m);
+            const float2 ov = *reinterpret_cast<const float2*>(mo + ((size_t)w * 16 + row) * HD + e);
+            v0 += wgt * ov.x; v1 += wgt * ov.y;
+            l += wgt * ml[w * 16 + row];
+        }
+        emit(c.rho0 + tile * 16 + row, e, v0, v1, m, l, e == 0);
+    }
+}
+
+// grid (max_nsplit, n_kv_heads * row_groups, n_items), block 128.
 template <int HD>
 __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const float* __restrict__ q, PassMeta meta,
                                                                   const uint16_t* __restrict__ kv_pool,
                                                                   int layer, int n_pages, int page_size, int Hq,
-                                                                  int Hkv, float* __restrict__ o_part,
+                                                                  int Hkv, int q_tiles_smem,
+                                                                  float* __restrict__ o_part,
                                                                   float* __restrict__ m_part,
                                                                   float* __restrict__ l_part) {
     pdl_wait();
     pdl_launch_dependents();
-    constexpr int RG = kAttnThreads / HD;          // row groups in the P.V phase
-    constexpr int RPT = kMaxItemRows / RG;         // rows per thread in the P.V phase
-    const int item = blockIdx.z, h = blockIdx.y, sp = blockIdx.x;
+    extern __shared__ __align__(128) unsigned char smem[];
+    using SM = AttnSmem<HD>;
+    const int item = blockIdx.z, sp = blockIdx.x;
+    const int kvh = blockIdx.y % Hkv, rg = blockIdx.y / Hkv;
     const int nsplit = meta.it_nsplit[item];
     if (sp >= nsplit) return;
-    const int rows = meta.it_rows[item], row0 = meta.it_row0[item], base = meta.it_base[item];
-    const int total = base + rows, chunk = meta.it_chunk[item];
-    const int k0 = sp * chunk, k1 = min(k0 + chunk, total);
-    const int kvh = h / (Hq / Hkv);
-    const int32_t* bt = meta.block_tab + (size_t)meta.it_slot[item] * meta.max_pages;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = Hq / Hkv;
+    AttnCtx c;
+    c.rows = meta.it_rows[item];
+    c.R = G * c.rows;
+    c.rho0 = rg * (kAttnMaxRowTiles * 16);
+    if (c.rho0 >= c.R) return;
+    c.base = meta.it_base[item];
+    const int total = c.base + c.rows, chunk = meta.it_chunk[item];
+    c.k0 = sp * chunk;
+    c.k1 = min(c.k0 + chunk, total);
+    c.kv_pool = kv_pool;
+    c.bt = meta.block_tab + (size_t)meta.it_slot[item] * meta.max_pages;
+    c.layer = layer; c.n_pages = n_pages; c.page_size = page_size; c.Hkv = Hkv; c.kvh = kvh;
+    const int row0 = meta.it_row0[item];
+    int row_tiles = (c.R - c.rho0 + 15) / 16;
+    row_tiles = row_tiles > kAttnMaxRowTiles ? kAttnMaxRowTiles : row_tiles;
+    if (row_tiles > q_tiles_smem) return;   // cannot happen: the host sizes shared memory from the same rows
 
-    extern __shared__ float sm[];
-    float* Qs = sm;                                   // [32][HD]
-    float* Ss = Qs + kMaxItemRows * HD;               // [32][kAttnTile]
-    float* m_s = Ss + kMaxItemRows * kAttnTile;       // [32]
-    float* l_s = m_s + kMaxItemRows;
-    float* al_s = l_s + kMaxItemRows;
-    size_t* voff = reinterpret_cast<size_t*>(al_s + kMaxItemRows);  // [kAttnTile]
-
+    // ---- stage Q (scaled by 1/sqrt(hd)) as split-bf16 A fragments: [tile][k16 step][hi|lo][lane] uint4
     const float scale = rsqrtf((float)HD);
-    for (int i = tid; i < rows * HD; i += kAttnThreads) {
-        int r = i / HD, e = i % HD;
-        Qs[i] = q[((size_t)(row0 + r) * Hq + h) * HD + e] * scale;
+    uint4* qsm = reinterpret_cast<uint4*>(smem + SM::kRing);
+    for (int idx = threadIdx.x; idx < row_tiles * (HD / 16) * 32; idx += kAttnThreads) {
+        const int lane = idx & 31, ks = (idx >> 5) % (HD / 16), tile = idx / (32 * (HD / 16));
+        const int g = lane >> 2, t = lane & 3;
+        float v[8];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int rho = c.rho0 + tile * 16 + g + 8 * hh;
+            float2 a = make_float2(0.f, 0.f), b = make_float2(0.f, 0.f);
+            if (rho < c.R) {
+                const int gq = rho / c.rows, r = rho % c.rows;
+                const float* qp = q + ((size_t)(row0 + r) * Hq + kvh * G + gq) * HD + ks * 16 + 2 * t;
+                a = *reinterpret_cast<const float2*>(qp);
+                b = *reinterpret_cast<const float2*>(qp + 8);
+            }
+            v[2 * hh] = a.x * scale; v[2 * hh + 1] = a.y * scale;
+            v[4 + 2 * hh] = b.x * scale; v[4 + 2 * hh + 1] = b.y * scale;
+        }
+        uint16_t h[8], l[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) split_bf16(v[i], h[i], l[i]);
+        // A fragment order: (row g, k 2t..), (row g+8, k 2t..), (row g, k 2t+8..), (row g+8, k 2t+8..)
+        qsm[((tile * (HD / 16) + ks) * 2 + 0) * 32 + lane] =
+            make_uint4(pack2(h[0], h[1]), pack2(h[2], h[3]), pack2(h[4], h[5]), pack2(h[6], h[7]));
+        qsm[((tile * (HD / 16) + ks) * 2 + 1) * 32 + lane] =
+            make_uint4(pack2(l[0], l[1]), pack2(l[2], l[3]), pack2(l[4], l[5]), pack2(l[6], l[7]));
     }
-    if (tid < kMaxItemRows) { m_s[tid] = -INFINITY; l_s[tid] = 0.f; }
-    float o[RPT];
-#pragma unroll
-    for (int i = 0; i < RPT; ++i) o[i] = 0.f;
-    const int e_out = tid % HD, rg = tid / HD;
-    __syncthreads();
-
-    for (int j0 = k0; j0 < k1; j0 += kAttnTile) {
-        const int nkeys = min(kAttnTile, k1 - j0);
-        // phase 1: scores of key (j0 + tid) against every row
-        if (tid < nkeys) {
-            const int j = j0 + tid;
-            const int page = bt[j / page_size], slot = j % page_size;
-            const size_t koff = kv_index(layer, n_pages, page, 0, Hkv, kvh, page_size, slot, HD, 0);
-            voff[tid] = kv_index(layer, n_pages, page, 1, Hkv, kvh, page_size, slot, HD, 0);
-            uint4 kr[HD / 8];
-            const uint4* kp = reinterpret_cast<const uint4*>(kv_pool + koff);
-#pragma unroll
-            for (int i = 0; i < HD / 8; ++i) kr[i] = kp[i];
-            for (int r = 0; r < rows; ++r) {
-                const float4* qr = reinterpret_cast<const float4*>(Qs + r * HD);
-                float acc = 0.f;
-#pragma unroll
-                for (int i = 0; i < HD / 8; ++i) {
-                    float4 qa = qr[2 * i], qb = qr[2 * i + 1];
-                    uint4 kk = kr[i];
-                    acc += qa.x * __uint_as_float(kk.x << 16) + qa.y * __uint_as_float(kk.x & 0xffff0000u);
-                    acc += qa.z * __uint_as_float(kk.y << 16) + qa.w * __uint_as_float(kk.y & 0xffff0000u);
-                    acc += qb.x * __uint_as_float(kk.z << 16) + qb.y * __uint_as_float(kk.z & 0xffff0000u);
-                    acc += qb.z * __uint_as_float(kk.w << 16) + qb.w * __uint_as_float(kk.w & 0xffff0000u);
-                }
-                Ss[r * kAttnTile + tid] = (j <= base + r) ? acc : -INFINITY;   // causal inside the chunk
-            }
-        } else {
-            for (int r = 0; r < rows; ++r) Ss[r * kAttnTile + tid] = -INFINITY;
-        }
-        __syncthreads();
-        // phase 2: online softmax, one warp per row
-        for (int r = warp; r < rows; r += kAttnThreads / 32) {
-            float v[kAttnTile / 32];
-            float mx = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < kAttnTile / 32; ++i) { v[i] = Ss[r * kAttnTile + lane + 32 * i]; mx = fmaxf(mx, v[i]); }
-            mx = warp_max(mx);
-            const float m_old = m_s[r], m_new = fmaxf(m_old, mx);
-            float sum = 0.f;
-#pragma unroll
-            for (int i = 0; i < kAttnTile / 32; ++i) {
-                float p = (m_new == -INFINITY) ? 0.f : expf(v[i] - m_new);
-                Ss[r * kAttnTile + lane + 32 * i] = p;
-                sum += p;
-            }
-            sum = warp_sum(sum);
-            if (lane == 0) {
-                float al = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);
-                al_s[r] = al;
-                l_s[r] = l_s[r] * al + sum;
-                m_s[r] = m_new;
-            }
-        }
-        __syncthreads();
-        // phase 3: o[r][e] = o[r][e]*alpha[r] + sum_t P[r][t] V[t][e]
-#pragma unroll
-        for (int i = 0; i < RPT; ++i) {
-            int r = i * RG + rg;
-            if (r < rows) o[i] *= al_s[r];
-        }
-        for (int tk = 0; tk < nkeys; ++tk) {
-            const float v = bf16_bits_to_f32(kv_pool[voff[tk] + e_out]);
-#pragma unroll
-            for (int i = 0; i < RPT; ++i) {
-                int r = i * RG + rg;
-                if (r < rows) o[i] += Ss[r * kAttnTile + tk] * v;
-            }
-        }
-        __syncthreads();
-    }
+    // (the first __syncthreads of the tile loop orders these writes before any read)
     const int part0 = meta.it_part0[item];
-#pragma unroll
-    for (int i = 0; i < RPT; ++i) {
-        int r = i * RG + rg;
-        if (r < rows) {
-            size_t slot = (size_t)part0 + ((size_t)r * Hq + h) * nsplit + sp;
-            o_part[slot * HD + e_out] = o[i];
-            if (e_out == 0) { m_part[slot] = m_s[r]; l_part[slot] = l_s[r]; }
-        }
-    }
+    if (row_tiles == 1) attn_body<HD, 1>(c, smem, o_part, m_part, l_part, Hq, G, nsplit, sp, part0);
+    else if (row_tiles == 2) attn_body<HD, 2>(c, smem, o_part, m_part, l_part, Hq, G, nsplit, sp, part0);
+    else attn_body<HD, 4>(c, smem, o_part, m_part, l_part, Hq, G, nsplit, sp, part0);
 }
 
-static inline size_t attn_smem_bytes(int hd) {
-    return sizeof(float) * (kMaxItemRows * hd + kMaxItemRows * kAttnTile + 3 * kMaxItemRows) +
-           sizeof(size_t) * kAttnTile;
+static inline size_t attn_smem_bytes(int hd, int row_tiles) {
+    return hd == 128 ? AttnSmem<128>::bytes(row_tiles) : AttnSmem<64>::bytes(row_tiles);
 }
 
 // Merge the splits: out = sum_s e^{m_s - m} o_s / sum_s e^{m_s - m} l_s, stored as split-bf16 B fragments

@@ -321,7 +321,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     float* hu = reinterpret_cast<float*>(hm + ml.u);
     RejectItem* hr = reinterpret_cast<RejectItem*>(hm + ml.rej);
     // split policy: aim at two waves of CTAs over all (item, head, split) triples
-    int target = std::max(1, (2 * kWaveCtas + n_items * c.n_q_heads - 1) / (n_items * c.n_q_heads));
+    int target = std::max(1, (4 * 148 + n_items * c.n_kv_heads - 1) / (n_items * c.n_kv_heads));
     int row = 0, part0 = 0, max_nsplit = 1, u0 = 0;
     for (int i = 0; i < n_items; ++i) {
         const ItemDesc& it = items[i];
@@ -386,7 +386,12 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     }
     const float* part = nullptr;
     int S = 0;
-    const size_t asmem = attn_smem_bytes(hd);
+    int max_item_rows = 1;
+    for (auto& it : items) max_item_rows = std::max(max_item_rows, it.rows);
+    const int maxR = max_item_rows * (Hq / Hkv);                      // query rows that share one KV head
+    const int q_tiles = std::min(kAttnMaxRowTiles, (maxR + 15) / 16);
+    const int row_groups = (maxR + kAttnMaxRowTiles * 16 - 1) / (kAttnMaxRowTiles * 16);
+    const size_t asmem = attn_smem_bytes(hd, q_tiles);
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& lw = ctx->layers[l];
         CU(launch_pdl(add_norm_kernel, dim3(M), dim3(kNormThreads), 0, st, x, l == 0 ? (const uint16_t*)ctx->emb : no_emb,
@@ -395,13 +400,15 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         { int rc_ = launch_gemm(ctx, p, lw.qkv.packed, xf_h, partA, M, dv.Nqkv, d); if (rc_) return rc_; }
         CU(launch_pdl(rope_kv_kernel, dim3(M, Hq + 2 * Hkv), dim3(hd / 2), 0, st, (const float*)partA, p.S, M, Hq, Hkv, hd,
                       (const float*)cs, (const float*)sn, meta, qbuf, ctx->kv_pool, l, c.n_pages, c.page_size));
-        dim3 ag(max_nsplit, Hq, n_items);
+        dim3 ag(max_nsplit, Hkv * row_groups, n_items);
         if (hd == 128)
             CU(launch_pdl(attn_split_kernel<128>, ag, dim3(kAttnThreads), asmem, st, (const float*)qbuf, meta,
-                          (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, Hq, Hkv, o_part, m_part, l_part));
+                          (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, Hq, Hkv, q_tiles, o_part, m_part,
+                          l_part));
         else
             CU(launch_pdl(attn_split_kernel<64>, ag, dim3(kAttnThreads), asmem, st, (const float*)qbuf, meta,
-                          (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, Hq, Hkv, o_part, m_part, l_part));
+                          (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, Hq, Hkv, q_tiles, o_part, m_part,
+                          l_part));
         CU(launch_pdl(attn_combine_kernel, dim3(M, Hq), dim3(hd), 0, st, (const float*)o_part, (const float*)m_part,
                       (const float*)l_part, meta, M, Hq, hd, xf_attn));
         p = gemm_plan(M, d, dv.qd);
@@ -502,10 +509,10 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
     if ((e = gemm_init_attrs()) != cudaSuccess) return bail(PIPESD_E_CUDA);
     e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_smem_bytes(128));
+                             (int)attn_smem_bytes(128, kAttnMaxRowTiles));
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
     e = cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_smem_bytes(64));
+                             (int)attn_smem_bytes(64, kAttnMaxRowTiles));
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
 
     ctx->kv_pool = (uint16_t*)mem->kv;
