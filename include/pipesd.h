@@ -190,9 +190,10 @@ int32_t pipesd_profile_enable(pipesd_ctx *ctx, int32_t time_gemms);
 int32_t pipesd_profile_read(pipesd_ctx *ctx, pipesd_profile_info *out);
 
 /* Small-M weight-streaming GEMM on its own: y[M,N] = x[M,K] . W[N,K]^T with bf16 W, fp32 x and y.
- * pipesd_gemm_packed_bytes: size of the repacked copy of W (rows padded to a multiple of 128).  pipesd_gemm_pack: W (device, row-major
- * bf16 [N,K]) -> packed (device).  pipesd_gemm_run: x, y device; scratch device of
- * pipesd_gemm_scratch_bytes(M,N,K) bytes (split-K partial sums).  N, K multiples of 16. */
+ * pipesd_gemm_packed_bytes: size of the repacked copy of W (rows padded to a multiple of 128).
+ * pipesd_gemm_pack: W (device, row-major bf16 [N,K]) -> packed (device).  pipesd_gemm_run: x, y device;
+ * scratch device of pipesd_gemm_scratch_bytes(M,N,K) bytes (x split into bf16 hi/lo fragments; the K slices
+ * are summed inside the kernel over a thread-block cluster).  N, K multiples of 16. */
 uint64_t pipesd_gemm_packed_bytes(int32_t N, int32_t K);
 uint64_t pipesd_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K);
 int32_t pipesd_gemm_pack(const void *W, void *packed, int32_t N, int32_t K, void *cuda_stream);
@@ -209,7 +210,7 @@ int32_t pipesd_debug_gemm_force_split(int32_t S);
  * its input and output buffers and nothing else, a real-time or latency-critical loop that must not
  * take the allocator's lock or trigger an implicit device synchronisation, a process whose memory
  * budget was fixed at start-up and has no pool to draw from.  Such callers have nowhere to get the
- * split-K scratch that pipesd_gemm_run asks for.  Here the scratch is a fixed array of
+ * scratch that pipesd_gemm_run asks for (the activations split into bf16 fragments).  Here the scratch is a fixed array of
  * PIPESD_STATIC_SCRATCH_BYTES inside the library itself (every GPU that loads the library carries it
  * until the process ends); the call allocates and frees nothing, on the device or through any
  * library.  The caller still passes packed weights, x and y (device), exactly as for pipesd_gemm_run,
@@ -217,7 +218,7 @@ int32_t pipesd_debug_gemm_force_split(int32_t S);
  *
  * Limits and rules:
  *   - If pipesd_gemm_scratch_bytes(M, N, K) is larger than PIPESD_STATIC_SCRATCH_BYTES the call returns
- *     PIPESD_E_TOO_LARGE and launches nothing (8 MiB covers, e.g., M <= 16 rows against the 7B shapes).
+ *     PIPESD_E_TOO_LARGE and launches nothing (8 MiB covers M*K up to 2M elements, e.g. 190 rows at K=11008).
  *   - The first call on each device looks up the array's device address (with that device current)
  *     and sets kernel attributes; make that first call during set-up, before any stream capture.
  *   - All calls share the one array and it keeps whatever the last call left there.  Nothing needs

@@ -1,7 +1,11 @@
 // Multi-query decode attention over a paged bf16 KV cache: each request contributes a short chunk
 // of query rows (the pending token plus its k drafts) that attend to the cached prefix and, causally,
-// to each other.  The keys are cut into splits ("split-K"); every split produces an un-normalised
-// partial output with its running max and sum, and a second kernel merges the splits.
+// to each other.  The keys are cut into 8 splits ("split-K") handled by the 8 CTAs of a thread-block
+// cluster; every CTA produces an un-normalised partial output with its running max and sum in its own
+// shared memory, and after a cluster barrier the partials are merged over distributed shared memory and
+// written straight into the output projection's input format -- no partial results in global memory and
+// no separate merge kernel.  Tiles of keys that were cached before this pass do not depend on the
+// preceding QKV projection, so their copies are issued before the dependent-launch wait.
 //
 // One CTA (4 warps) = one KV head of one request x one split x up to 64 query rows, where the rows are
 // all (query head of the group, chunk row) pairs that share the KV head (GQA).  K and V tiles of 64 keys
@@ -81,10 +85,11 @@ __device__ __forceinline__ void attn_load_tile(const AttnCtx& c, uint32_t stage_
 }
 
 // Main loop for one CTA.  RTW = row-tile groups among the 4 warps (1, 2 or 4); 4/RTW = key strips.
+// On entry the copies of tiles 0 and 1 have been issued as two committed cp.async groups.  On exit the
+// CTA's partial result for its (up to 64) rows is in shared memory: Fo[row][HD], Fm[row], Fl[row].
 template <int HD, int RTW>
-__device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem, float* __restrict__ o_part,
-                                          float* __restrict__ m_part, float* __restrict__ l_part, int Hq, int G,
-                                          int nsplit, int sp, int part0) {
+__device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem, float* __restrict__ Fo,
+                                          float* __restrict__ Fm, float* __restrict__ Fl) {
     constexpr int KSW = 4 / RTW;               // key strips per tile
     constexpr int STRIP = kAttnTile / KSW;     // keys per warp per tile
     constexpr int NTS = STRIP / 8;             // score n-tiles per warp
@@ -112,11 +117,7 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
         horizon[hh] = rho < c.R ? c.base + rho % c.rows : -1;   // keys j <= horizon are visible; -1: padding row
     }
 
-    const int ntiles = (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile;
-    attn_load_tile<HD>(c, ring, c.k0);
-    cp_async_commit();
-    if (ntiles > 1) attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile);
-    cp_async_commit();
+    const int ntiles = c.k1 > c.k0 ? (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile : 0;
 
     for (int it = 0; it < ntiles; ++it) {
         cp_async_wait<1>();
@@ -224,26 +225,21 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
         l_run[hh] += __shfl_xor_sync(0xffffffffu, l_run[hh], 2);
     }
 
-    // ---- write the split's partial result: merge the key strips first when the warps split the keys
-    auto emit = [&](int rho, int e, float v0, float v1, float m, float l, bool write_ml) {
-        if (rho >= c.R) return;
-        const int gq = rho / c.rows, r = rho % c.rows;
-        const size_t slot = (size_t)part0 + ((size_t)r * Hq + c.kvh * G + gq) * nsplit + sp;
-        *reinterpret_cast<float2*>(o_part + slot * HD + e) = make_float2(v0, v1);
-        if (write_ml) { m_part[slot] = m; l_part[slot] = l; }
-    };
+    __syncthreads();                               // every warp is done with the ring: reuse it
+    // ---- leave the CTA's partial result in shared memory; merge the key strips first when the warps split the keys
     if (KSW == 1) {
-        if (!warp_active) return;
+        if (warp_active) {
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-            const int rho = c.rho0 + rtw * 16 + g + 8 * hh;
+            for (int hh = 0; hh < 2; ++hh) {
+                const int rl = rtw * 16 + g + 8 * hh;          // row within the CTA's row group
 #pragma unroll
-            for (int i = 0; i < NTO; ++i)
-                emit(rho, i * 8 + 2 * t, o[i][2 * hh], o[i][2 * hh + 1], m_run[hh], l_run[hh], i == 0 && t == 0);
+                for (int i = 0; i < NTO; ++i)
+                    *reinterpret_cast<float2*>(Fo + (size_t)rl * HD + i * 8 + 2 * t) = make_float2(o[i][2 * hh], o[i][2 * hh + 1]);
+                if (t == 0) { Fm[rl] = m_run[hh]; Fl[rl] = l_run[hh]; }
+            }
         }
         return;
     }
-    __syncthreads();                               // the ring is free: reuse it as the merge buffer
     float* mo = reinterpret_cast<float*>(smem);    // [warp][16 rows][HD] then [warp][16] m, [warp][16] l
     float* mm = mo + 4 * 16 * HD;
     float* ml = mm + 4 * 16;
@@ -273,44 +269,53 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
             v0 += wgt * ov.x; v1 += wgt * ov.y;
             l += wgt * ml[w * 16 + row];
         }
-        emit(c.rho0 + tile * 16 + row, e, v0, v1, m, l, e == 0);
+        *reinterpret_cast<float2*>(Fo + (size_t)rr * HD + e) = make_float2(v0, v1);
+        if (e == 0) { Fm[rr] = m; Fl[rr] = l; }
     }
 }
 
-// grid (max_nsplit, n_kv_heads * row_groups, n_items), block 128.
+constexpr int kAttnSplits = 8;   // = cluster size along x
+
+// grid (8, n_kv_heads * row_groups, n_items), cluster (8,1,1), block 128.
 template <int HD>
-__global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const float* __restrict__ q, PassMeta meta,
-                                                                  const uint16_t* __restrict__ kv_pool,
-                                                                  int layer, int n_pages, int page_size, int Hq,
-                                                                  int Hkv, int q_tiles_smem,
-                                                                  float* __restrict__ o_part,
-                                                                  float* __restrict__ m_part,
-                                                                  float* __restrict__ l_part) {
-    pdl_wait();
-    pdl_launch_dependents();
+__global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restrict__ q, PassMeta meta,
+                                                            const uint16_t* __restrict__ kv_pool, int layer,
+                                                            int n_pages, int page_size, int M, int Hq, int Hkv,
+                                                            int q_tiles_smem, uint16_t* __restrict__ xf_out) {
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = AttnSmem<HD>;
-    const int item = blockIdx.z, sp = blockIdx.x;
+    pdl_launch_dependents();
+    const int item = blockIdx.z, sp = blockIdx.x;                 // sp == rank in the cluster
     const int kvh = blockIdx.y % Hkv, rg = blockIdx.y / Hkv;
-    const int nsplit = meta.it_nsplit[item];
-    if (sp >= nsplit) return;
     const int G = Hq / Hkv;
     AttnCtx c;
     c.rows = meta.it_rows[item];
     c.R = G * c.rows;
     c.rho0 = rg * (kAttnMaxRowTiles * 16);
-    if (c.rho0 >= c.R) return;
+    int row_tiles = (c.R - c.rho0 + 15) / 16;
+    row_tiles = row_tiles > kAttnMaxRowTiles ? kAttnMaxRowTiles : row_tiles;
+    // the whole cluster shares (item, head, row group): these exits are taken by all 8 CTAs or by none
+    if (c.rho0 >= c.R || row_tiles > q_tiles_smem) return;
     c.base = meta.it_base[item];
     const int total = c.base + c.rows, chunk = meta.it_chunk[item];
-    c.k0 = sp * chunk;
+    c.k0 = min(sp * chunk, total);
     c.k1 = min(c.k0 + chunk, total);
     c.kv_pool = kv_pool;
     c.bt = meta.block_tab + (size_t)meta.it_slot[item] * meta.max_pages;
     c.layer = layer; c.n_pages = n_pages; c.page_size = page_size; c.Hkv = Hkv; c.kvh = kvh;
     const int row0 = meta.it_row0[item];
-    int row_tiles = (c.R - c.rho0 + 15) / 16;
-    row_tiles = row_tiles > kAttnMaxRowTiles ? kAttnMaxRowTiles : row_tiles;
-    if (row_tiles > q_tiles_smem) return;   // cannot happen: the host sizes shared memory from the same rows
+    const uint32_t ring = smem_u32(smem);
+
+    // Tiles made only of keys cached before this pass do not depend on the QKV projection that precedes this
+    // kernel: issue their copies now.  Group order is always [tile 0][tile 1].
+    const int ntiles = c.k1 > c.k0 ? (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile : 0;
+    const bool early0 = ntiles > 0 && min(c.k0 + kAttnTile, c.k1) <= c.base;
+    const bool early1 = ntiles > 1 && min(c.k0 + 2 * kAttnTile, c.k1) <= c.base;
+    if (early0) { attn_load_tile<HD>(c, ring, c.k0); cp_async_commit(); }
+    if (early1) { attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile); cp_async_commit(); }
+    pdl_wait();
+    if (!early0) { if (ntiles > 0) attn_load_tile<HD>(c, ring, c.k0); cp_async_commit(); }
+    if (!early1) { if (ntiles > 1) attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile); cp_async_commit(); }
 
     // ---- stage Q (scaled by 1/sqrt(hd)) as split-bf16 A fragments: [tile][k16 step][hi|lo][lane] uint4
     const float scale = rsqrtf((float)HD);
@@ -341,41 +346,57 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(const float* _
         qsm[((tile * (HD / 16) + ks) * 2 + 1) * 32 + lane] =
             make_uint4(pack2(l[0], l[1]), pack2(l[2], l[3]), pack2(l[4], l[5]), pack2(l[6], l[7]));
     }
-    // (the first __syncthreads of the tile loop orders these writes before any read)
-    const int part0 = meta.it_part0[item];
-    if (row_tiles == 1) attn_body<HD, 1>(c, smem, o_part, m_part, l_part, Hq, G, nsplit, sp, part0);
-    else if (row_tiles == 2) attn_body<HD, 2>(c, smem, o_part, m_part, l_part, Hq, G, nsplit, sp, part0);
-    else attn_body<HD, 4>(c, smem, o_part, m_part, l_part, Hq, G, nsplit, sp, part0);
+    __syncthreads();
+
+    // partial result of this CTA, placed behind the strip-merge buffer inside the (then idle) ring
+    float* Fo = reinterpret_cast<float*>(smem + (4 * 16 * HD + 256) * 4);   // [64][HD]
+    float* Fm = Fo + 64 * HD;                                                // [64]
+    float* Fl = Fm + 64;                                                     // [64]
+    if (ntiles == 0) {
+        cp_async_wait<0>();
+        for (int i = threadIdx.x; i < row_tiles * 16; i += kAttnThreads) { Fm[i] = -INFINITY; Fl[i] = 0.f; }
+    } else if (row_tiles == 1) attn_body<HD, 1>(c, smem, Fo, Fm, Fl);
+    else if (row_tiles == 2) attn_body<HD, 2>(c, smem, Fo, Fm, Fl);
+    else attn_body<HD, 4>(c, smem, Fo, Fm, Fl);
+
+    // ---- merge the 8 splits over distributed shared memory; rank r owns rows r, r+8, ... of the row group
+    cluster_sync_all();
+    const uint32_t fo_a = smem_u32(Fo), fm_a = smem_u32(Fm), fl_a = smem_u32(Fl);
+    const int n_rows = min(row_tiles * 16, c.R - c.rho0);
+    const int KSo = (Hq * HD) / 16, NTo = xf_nt(M);
+    for (int rl = sp; rl < n_rows; rl += kAttnSplits) {
+        float ms[kAttnSplits], ls[kAttnSplits];
+#pragma unroll
+        for (int r = 0; r < kAttnSplits; ++r) {
+            ms[r] = dsmem_ld_f32(dsmem_addr(fm_a + rl * 4, (uint32_t)r));
+            ls[r] = dsmem_ld_f32(dsmem_addr(fl_a + rl * 4, (uint32_t)r));
+        }
+        float m = -INFINITY;
+#pragma unroll
+        for (int r = 0; r < kAttnSplits; ++r) m = fmaxf(m, ms[r]);
+        float den = 0.f, w[kAttnSplits];
+#pragma unroll
+        for (int r = 0; r < kAttnSplits; ++r) {
+            w[r] = (ms[r] == -INFINITY) ? 0.f : expf(ms[r] - m);   // an empty split or one beyond the causal horizon
+            den += w[r] * ls[r];
+        }
+        const int rho = c.rho0 + rl, gq = rho / c.rows, r_in = rho % c.rows;
+        for (int e = threadIdx.x; e < HD; e += kAttnThreads) {
+            float ov[kAttnSplits];
+#pragma unroll
+            for (int r = 0; r < kAttnSplits; ++r)
+                ov[r] = w[r] != 0.f ? dsmem_ld_f32(dsmem_addr(fo_a + (uint32_t)(rl * HD + e) * 4, (uint32_t)r)) : 0.f;
+            float num = 0.f;
+#pragma unroll
+            for (int r = 0; r < kAttnSplits; ++r) num += w[r] * ov[r];
+            xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
+        }
+    }
+    cluster_sync_all();   // nobody leaves while its shared memory may still be read
 }
 
 static inline size_t attn_smem_bytes(int hd, int row_tiles) {
     return hd == 128 ? AttnSmem<128>::bytes(row_tiles) : AttnSmem<64>::bytes(row_tiles);
-}
-
-// Merge the splits: out = sum_s e^{m_s - m} o_s / sum_s e^{m_s - m} l_s, stored as split-bf16 B fragments
-// for the output projection (column index = head * hd + e).  grid (M, n_q_heads), block hd.
-__global__ void attn_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ m_part,
-                                    const float* __restrict__ l_part, PassMeta meta, int M, int Hq, int hd,
-                                    uint32_t* __restrict__ xf_out) {
-    pdl_wait();
-    pdl_launch_dependents();
-    const int row = blockIdx.x, h = blockIdx.y, e = threadIdx.x;
-    const int item = meta.row_item[row];
-    const int r = row - meta.it_row0[item], nsplit = meta.it_nsplit[item];
-    const size_t slot0 = (size_t)meta.it_part0[item] + ((size_t)r * Hq + h) * nsplit;
-    float m = -INFINITY;
-    for (int s = 0; s < nsplit; ++s) m = fmaxf(m, m_part[slot0 + s]);
-    float num = 0.f, den = 0.f;
-#pragma unroll 4
-    for (int s = 0; s < nsplit; ++s) {
-        const float ms = m_part[slot0 + s];
-        const float w = (ms == -INFINITY) ? 0.f : expf(ms - m);   // a split wholly beyond the causal horizon
-        num += w * o_part[(slot0 + s) * hd + e];
-        den += w * l_part[slot0 + s];
-    }
-    const float v = num / den;
-    const float v1 = __shfl_down_sync(0xffffffffu, v, 1);
-    if ((e & 1) == 0) xf_store_pair(xf_out, row, h * hd + e, v, v1, (Hq * hd) / 16, xf_nt(M));
 }
 
 }  // namespace pipesd

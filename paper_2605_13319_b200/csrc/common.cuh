@@ -128,6 +128,31 @@ static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 b
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// The same with a thread-block cluster of `cluster_x` consecutive CTAs along x (1: no cluster).
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                             cudaStream_t st, int cluster_x, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    int n = 1;
+    if (cluster_x > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)cluster_x;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        n = 2;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- split-bf16 activation arrays ("xf"): B fragments of mma.m16n8k16 in global memory ----------
 // Layout [token block][k16 step][n8 tile][lane] of uint4 = {hi.b0, hi.b1, lo.b0, lo.b1} where, for lane
 // = 4*g + t, b0 holds k = 2t, 2t+1 and b1 holds k = 2t+8, 2t+9 of token 8*tile + g.
@@ -142,6 +167,58 @@ __device__ __forceinline__ void xf_store_pair(uint32_t* xf, int tok, int k, floa
     xf[slot * 4 + half] = pack2(h0, h1);
     xf[slot * 4 + 2 + half] = pack2(l0, l1);
 }
+
+// 16-bit variant: stores one element (its hi and lo halves) of an xf array.
+__device__ __forceinline__ void xf_store_one(uint16_t* xf, int tok, int k, float v, int KS, int NT) {
+    const int tb = tok / (8 * NT), nt = (tok >> 3) % NT, g = tok & 7;
+    const int ks = k >> 4, kk = k & 15, t = (kk & 7) >> 1, half = kk >> 3;
+    const size_t slot = ((size_t)(tb * KS + ks) * NT + nt) * 32 + g * 4 + t;
+    uint16_t h, l;
+    split_bf16(v, h, l);
+    xf[slot * 8 + half * 2 + (kk & 1)] = h;
+    xf[slot * 8 + 4 + half * 2 + (kk & 1)] = l;
+}
+
+// ---- thread-block clusters: barrier and distributed shared memory --------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Every thread of every CTA of the cluster must execute this (hardware barrier, release/acquire).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float dsmem_ld_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void dsmem_st_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+// Per-pass metadata that lives in device memory (uploaded once per call).
+struct PassMeta {
+    const int32_t* row_item;   // [M] batch item of each row
+    const int32_t* row_pos;    // [M] absolute position of each row in its request
+    const int32_t* row_tok;    // [M] token id of each row
+    const int32_t* it_slot;    // [n_items] request slot (row of the block table)
+    const int32_t* it_row0;    // [n_items] first row of the item
+    const int32_t* it_rows;    // [n_items] rows of the item (k+1)
+    const int32_t* it_base;    // [n_items] cached positions before this pass
+    const int32_t* it_nsplit;  // [n_items] KV splits
+    const int32_t* it_chunk;   // [n_items] keys per split (multiple of the page size)
+    const int32_t* it_part0;   // [n_items] first slot of the item in the attention partial arrays
+    const int32_t* block_tab;  // [max_requests][max_pages] page ids, indexed by request slot
+    int max_pages;
+};
 
 // Offset (in elements) of K (kv=0) or V (kv=1) element (slot, e) of a head inside the paged pool:
 // layout [layer][page][kv][head][slot][e].

@@ -1,4 +1,5 @@
-// Small-M weight-streaming GEMM: y[M,N] = x[M,K] . W[N,K]^T, bf16 W (read once from HBM), fp32 x.
+// Small-M weight-streaming GEMM with fused epilogues: y[M,N] = x[M,K] . W[N,K]^T, bf16 W (read once
+// from HBM), fp32 x.
 //
 // The weight matrix is the wide operand: a 16-row x 16-column tile of W is the A fragment of a
 // warp-level m16n8k16 MMA and the (few) token rows are the narrow N dimension.  W is repacked once
@@ -7,35 +8,46 @@
 // One producer lane streams those runs into a shared-memory ring with bulk asynchronous copies
 // (cp.async.bulk + mbarrier transaction counts); four consumer warps, two row tiles each, read their
 // fragments back with conflict-free 16-byte loads and issue the MMAs.  The ring is the kernel's
-// memory-level parallelism: up to three CTAs x 3-4 stages x 16 KB are in flight per SM, and because
-// weights do not depend on the previous kernel, the ring is filled BEFORE the programmatic-dependent-
-// launch wait, so the weight stream of kernel n+1 starts while kernel n is still draining.
-// Activations stay fp32 in the residual stream; the kernels that produce a GEMM input store it
-// already split into bf16 hi + lo terms in B-fragment order ("xf" arrays), so the matching chunk of
-// activations rides in the same ring stage as its weights (two MMAs, one fp32 accumulator: 2^-17).
-// Work split: CTA = (128-row block of W, K slice, token block); partial sums of the K slices go to a
-// scratch array [S][M][N] that the consuming kernel adds up in fixed order (deterministic).
+// memory-level parallelism, and because weights do not depend on the previous kernel it is filled
+// BEFORE the programmatic-dependent-launch wait: the weight stream of kernel n+1 starts while kernel n
+// is still draining.
+// Activations stay fp32 in the residual stream; the kernel that produces a GEMM input stores it already
+// split into bf16 hi + lo terms in B-fragment order ("xf" arrays), so the matching chunk of activations
+// rides in the same ring stage as its weights (two MMAs, one fp32 accumulator: 2^-17 relative).
+// Split-K: the S CTAs that share a row block form a thread-block cluster.  Each leaves its partial tile
+// in its own shared memory; after a cluster barrier the tiles are summed over distributed shared memory
+// in rank order (deterministic) and the epilogue runs on the sums -- no partial sums in global memory.
+// Epilogues: plain fp32 output; RoPE + q store + bf16 K/V page append (QKV); residual add + next RMSNorm's
+// gain and sum of squares (O and down projections); SiLU(gate)*up (gate/up projection).  RMSNorm itself
+// never runs as a kernel: the producer stores x*gain and per-block sums of squares, the consumer scales
+// its result rows by rsqrt(mean(x^2)+eps), which commutes with the matrix product.
 #pragma once
 #include "common.cuh"
 
 namespace pipesd {
 
 constexpr int kGemmConsumerWarps = 4;                       // x 2 row tiles x 16 rows = 128 rows per CTA
-constexpr int kGemmThreads = (kGemmConsumerWarps + 1) * 32;  // + one producer warp
-constexpr int kGemmKC = 4;                                   // k16 steps per ring stage
-constexpr int kGemmWStage = kGemmKC * 4096;                  // weight bytes per stage
+constexpr int kGemmConsumers = kGemmConsumerWarps * 32;
+constexpr int kGemmThreads = kGemmConsumers + 32;           // + one producer warp
+constexpr int kGemmKC = 4;                                  // k16 steps per ring stage
+constexpr int kGemmWStage = kGemmKC * 4096;                 // weight bytes per stage
+constexpr int kGemmStages = 3;
 constexpr int kGemmCtasPerSm = 3;
 constexpr int kGemmWave = 148 * kGemmCtasPerSm;
+constexpr int kGemmMaxSplit = 8;                            // portable cluster size
 
-__host__ __device__ constexpr int gemm_stages(int NT) { return NT == 1 ? 4 : 3; }
+enum GemmMode { kPlain = 0, kQkvRope = 1, kResid = 2, kSwiglu = 3 };
+
 __host__ __device__ constexpr int gemm_stage_bytes(int NT) { return kGemmWStage + kGemmKC * NT * 512; }
-__host__ __device__ constexpr int gemm_smem_bytes(int NT) { return gemm_stages(NT) * gemm_stage_bytes(NT) + 128; }
+__host__ __device__ constexpr int gemm_ring_bytes(int NT) { return kGemmStages * gemm_stage_bytes(NT); }
+// ring | 2*stages barriers (64 B) | rstd[32] | tile sums of squares [8][32]
+__host__ __device__ constexpr int gemm_smem_bytes(int NT) { return gemm_ring_bytes(NT) + 64 + 128 + 1024; }
 
 struct GemmPlan {
     int NT;  // n8 token tiles per token block (1..4)
     int TB;  // token blocks
     int RB;  // 128-row blocks
-    int S;   // K slices
+    int S;   // K slices = cluster size
     int KS;  // k16 steps in K
 };
 
@@ -47,8 +59,8 @@ __host__ __device__ inline size_t xf_elems(int M, int K) { return (size_t)xf_tb(
 
 static int g_gemm_force_split = 0;   // 0: choose automatically (tuning hook)
 
-// Host: choose the K split.  CTAs are small and three fit on an SM, so what matters is a grid of a few
-// waves whose last wave is nearly full, against the partial-sum traffic every extra slice adds.
+// Host: choose the K split (cluster size).  What matters is enough CTAs to keep ~100 KB of copies in
+// flight per SM and a last wave that is nearly full.
 static inline GemmPlan gemm_plan(int M, int N, int K) {
     GemmPlan p;
     p.NT = xf_nt(M);
@@ -57,50 +69,70 @@ static inline GemmPlan gemm_plan(int M, int N, int K) {
     p.KS = K / 16;
     int best = 1;
     double best_score = -1e9;
-    const int mrows = M < p.NT * 8 ? M : p.NT * 8;
-    for (int s = 1; s <= 64 && s <= p.KS; ++s) {
+    for (int s = 1; s <= kGemmMaxSplit && s <= p.KS; ++s) {
         if (s > 1 && p.KS / s < 2 * kGemmKC) break;
         long ctas = (long)p.RB * s * p.TB;
         long waves = (ctas + kGemmWave - 1) / kGemmWave;
         double eff = (double)ctas / (double)(waves * kGemmWave);
-        double partial = s > 1 ? 4.0 * s * mrows / (double)K : 0.0;   // partial bytes (w+r) / weight bytes
-        double score = eff - 0.5 * partial;
+        if (ctas < kGemmWave) eff = 0.5 + 0.5 * eff;      // an under-full single wave still streams well
+        double score = eff - 0.004 * s;
         if (score > best_score) { best_score = score; best = s; }
     }
-    p.S = g_gemm_force_split > 0 && g_gemm_force_split <= p.KS ? g_gemm_force_split : best;
+    p.S = g_gemm_force_split > 0 && g_gemm_force_split <= kGemmMaxSplit && g_gemm_force_split <= p.KS
+              ? g_gemm_force_split : best;
     return p;
 }
 
 // Bytes of the packed copy of W[N][K] (row blocks padded to 128 rows).
 static inline size_t gemm_packed_bytes(int N, int K) { return (size_t)((N + 127) / 128) * 128 * K * 2; }
 
-// Repack row-major bf16 W rows [0, n_rows) into MMA A-fragment order, starting at packed row row0:
-// packed[((rb*KS + ks)*8 + tile)*32 + lane] = { W[r][c], W[r][c+1] | W[r+8][c], W[r+8][c+1] |
-//                                               W[r][c+8], W[r][c+9] | W[r+8][c+8], W[r+8][c+9] }
-// with r = (rb*8 + tile)*16 + lane/4 (in packed-row numbering), c = ks*16 + 2*(lane%4).
-// Rows beyond the source (padding of the last row block) are zero.  row0 and n_rows: multiples of 16.
-__global__ void gemm_pack_kernel(const uint16_t* __restrict__ W, uint4* __restrict__ packed, int row0, int n_rows,
-                                 int K, int pad_to) {
+// ---- packed-row <-> logical-row maps of the fused layouts ------------------------------------------
+// QKV: inside every head, tile tau holds dims 8*tau..8*tau+7 in rows 0..7 and their rotary partners
+// (+hd/2) in rows 8..15, so that one thread owns both elements of a rotation pair.
+__host__ __device__ inline int qkv_logical_row(int packed_row, int hd) {
+    const int head = packed_row / hd, within = packed_row % hd, tau = within >> 4, i = within & 15;
+    return head * hd + (i < 8 ? 8 * tau + i : hd / 2 + 8 * tau + (i - 8));
+}
+// gate/up: tile rows 0..7 are gate features f..f+7, rows 8..15 the matching up features.
+__host__ __device__ inline int gu_feature(int packed_row) { return (packed_row >> 4) * 8 + (packed_row & 7); }
+
+struct PackSrc {
+    const uint16_t* w[3];   // up to three row-major [rows_i][K] sources, concatenated along N
+    int rows[3];
+    int mode;               // GemmMode of the consumer (row permutation)
+    int hd;                 // head width (kQkvRope)
+};
+
+// Repack into MMA A-fragment order: packed[((rb*KS + ks)*8 + tile)*32 + lane] =
+//   { W[r][c], W[r][c+1] | W[r+8][c], W[r+8][c+1] | W[r][c+8], W[r][c+9] | W[r+8][c+8], W[r+8][c+9] }
+// with r = (rb*8 + tile)*16 + lane/4 in packed-row numbering, c = ks*16 + 2*(lane%4); packed rows map to
+// logical rows per `mode`; rows beyond the sources (padding of the last row block) are zero.
+__global__ void gemm_pack_kernel(PackSrc src, uint4* __restrict__ packed, int n_rows, int K) {
     const int KS = K / 16;
-    const int rt0 = row0 / 16, n_rt = (pad_to - row0) / 16;
+    const int n_rt = (n_rows + 127) / 128 * 8;
     const size_t total = (size_t)n_rt * KS * 32;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        int lane = (int)(i & 31);
-        size_t tile = i >> 5;
-        int ks = (int)(tile % KS);
-        int rt = rt0 + (int)(tile / KS);
-        int r = (rt - rt0) * 16 + (lane >> 2), c = ks * 16 + 2 * (lane & 3);
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (r < n_rows) {
-            const uint16_t* w0 = W + (size_t)r * K + c;
-            const uint16_t* w1 = W + (size_t)(r + 8) * K + c;
-            v.x = pack2(w0[0], w0[1]);
-            v.y = pack2(w1[0], w1[1]);
-            v.z = pack2(w0[8], w0[9]);
-            v.w = pack2(w1[8], w1[9]);
+    auto fetch = [&](int pr, int c, uint32_t& lo, uint32_t& hi) {
+        lo = hi = 0u;
+        if (pr >= n_rows) return;
+        int lr, which = 0;
+        if (src.mode == kSwiglu) { which = (pr & 15) < 8 ? 0 : 1; lr = gu_feature(pr); }
+        else {
+            lr = src.mode == kQkvRope ? qkv_logical_row(pr, src.hd) : pr;
+            while (which < 2 && lr >= src.rows[which]) { lr -= src.rows[which]; ++which; }
         }
-        int rb = rt >> 3, tl = rt & 7;
-        packed[(((size_t)rb * KS + ks) * 8 + tl) * 32 + lane] = v;
+        const uint16_t* w = src.w[which] + (size_t)lr * K + c;
+        lo = pack2(w[0], w[1]);
+        hi = pack2(w[8], w[9]);
+    };
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int lane = (int)(i & 31);
+        const size_t tile = i >> 5;
+        const int ks = (int)(tile % KS), rt = (int)(tile / KS);
+        const int r = rt * 16 + (lane >> 2), c = ks * 16 + 2 * (lane & 3);
+        uint4 v;
+        fetch(r, c, v.x, v.z);
+        fetch(r + 8, c, v.y, v.w);
+        packed[(((size_t)(rt >> 3) * KS + ks) * 8 + (rt & 7)) * 32 + lane] = v;
     }
 }
 
@@ -116,30 +148,53 @@ __global__ void xf_format_kernel(const float* __restrict__ x, uint32_t* __restri
 }
 
 struct GemmArgs {
-    const uint4* W;    // packed weights
-    const uint4* xf;   // activations, split-bf16 B fragments [tb][ks][nt][32]
-    float* out;        // [S][M][N] partial sums (S == 1: the result itself)
-    int* err;          // device error word (nullable): set when a bounded wait gives up
+    const uint4* W;     // packed weights
+    const uint4* xf;    // activations, split-bf16 B fragments [tb][ks][nt][32]
+    int* err;           // device error word (nullable): set when a bounded wait gives up
     int M, N, S, KS;
+    // input normalisation (nullable): ssq_in[b*M + tok], b < n_ssq, are sums of squares of the un-normalised
+    // input row; the result rows are scaled by rsqrt(sum / d_in + eps)
+    const float* ssq_in;
+    int n_ssq, d_in;
+    float eps;
+    // kPlain
+    float* out;         // [M][N]
+    // kQkvRope
+    float* q_out;       // [M][Hq*hd] rotated queries
+    uint16_t* kv_pool;
+    const float* cs;    // [M][hd/2] cos / sin of the row's position
+    const float* sn;
+    PassMeta meta;
+    int Hq, Hkv, hd, layer, n_pages, page_size;
+    // kResid
+    float* x;           // residual stream [M][N], updated in place
+    uint16_t* xf_out;   // x_new * gain_next as split-bf16 fragments (K of the consumer = N)
+    const float* gain_next;
+    float* ssq_out;     // [RB][M] sums of squares of x_new over the row block's columns
+    // kSwiglu
+    uint16_t* xf_act;   // silu(gate)*up as split-bf16 fragments, feature-major K = N/2
 };
 
-template <int NT>
-__global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_kernel(GemmArgs a) {
-    constexpr int kStages = gemm_stages(NT);
+template <int NT, int MODE>
+__global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_kernel(const GemmArgs a) {
     constexpr int kStageBytes = gemm_stage_bytes(NT);
     constexpr int kBStage = kGemmKC * NT * 512;
+    constexpr int MT = NT * 8;                        // tokens per token block
     extern __shared__ __align__(128) unsigned char smem[];
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);   // full[kStages], empty[kStages]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + gemm_ring_bytes(NT));   // full[3], empty[3]
+    float* rstd_s = reinterpret_cast<float*>(smem + gemm_ring_bytes(NT) + 64);  // [32]
+    float* tss_s = rstd_s + 32;                                                  // [8 tiles][32 tokens]
     const uint32_t smem_base = smem_u32(smem);
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kStages;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kGemmStages;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rb = blockIdx.x / a.S, s = blockIdx.x % a.S, tb = blockIdx.y;
+    const int rb = blockIdx.x / a.S, s = blockIdx.x % a.S, tb = blockIdx.y;   // s == rank in the cluster
     const int ks0 = (int)(((long)a.KS * s) / a.S), ks1 = (int)(((long)a.KS * (s + 1)) / a.S);
     const int nks = ks1 - ks0, nchunks = (nks + kGemmKC - 1) / kGemmKC;
+    const int tok0 = tb * MT;
 
     if (threadIdx.x == 0) {
 #pragma unroll
-        for (int i = 0; i < kStages; ++i) {
+        for (int i = 0; i < kGemmStages; ++i) {
             mbar_init(full0 + 8 * i, 1);
             mbar_init(empty0 + 8 * i, kGemmConsumerWarps);
         }
@@ -148,14 +203,15 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
     __syncthreads();
     pdl_launch_dependents();
 
+    bool ok = true;
     if (warp == kGemmConsumerWarps) {
-        // ---------------- producer: one lane streams (weights, activations) chunks into the ring
+        // ---------------- producer warp: lane 0 streams (weights, activations) chunks into the ring
         if (lane == 0) {
             const unsigned char* wsrc = reinterpret_cast<const unsigned char*>(a.W) + ((size_t)rb * a.KS + ks0) * 4096;
             const unsigned char* bsrc =
                 reinterpret_cast<const unsigned char*>(a.xf) + ((size_t)tb * a.KS + ks0) * (NT * 512);
             auto chunk_ks = [&](int c) { int r = nks - c * kGemmKC; return r < kGemmKC ? r : kGemmKC; };
-            const int pre = nchunks < kStages ? nchunks : kStages;
+            const int pre = nchunks < kGemmStages ? nchunks : kGemmStages;
             // weights do not depend on the previous kernel: start them before the dependency wait
             for (int c = 0; c < pre; ++c) {
                 const int kc = chunk_ks(c);
@@ -168,11 +224,10 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                 bulk_g2s(smem_base + c * kStageBytes + kGemmWStage, bsrc + (size_t)c * kBStage, (uint32_t)kc * NT * 512,
                          full0 + 8 * c);
             }
-            bool ok = true;
             int issued = pre;
-            for (int c = pre; c < nchunks && ok; ++c) {
-                const int st = c % kStages, kc = chunk_ks(c);
-                ok = mbar_wait(empty0 + 8 * st, ((c / kStages) - 1) & 1);
+            for (int c = pre; c < nchunks; ++c) {
+                const int st = c % kGemmStages, kc = chunk_ks(c);
+                ok = mbar_wait(empty0 + 8 * st, ((c / kGemmStages) - 1) & 1);
                 if (!ok) break;
                 mbar_expect_tx(full0 + 8 * st, (uint32_t)kc * (4096 + NT * 512));
                 bulk_g2s(smem_base + st * kStageBytes, wsrc + (size_t)c * kGemmWStage, (uint32_t)kc * 4096, full0 + 8 * st);
@@ -183,73 +238,173 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             if (!ok) {
                 if (a.err) atomicExch(a.err, 1);
                 // give up: let every copy already issued land before this CTA's shared memory is released
-                for (int c = issued > kStages ? issued - kStages : 0; c < issued; ++c)
-                    mbar_wait(full0 + 8 * (c % kStages), (c / kStages) & 1);
+                for (int c = issued > kGemmStages ? issued - kGemmStages : 0; c < issued; ++c)
+                    mbar_wait(full0 + 8 * (c % kGemmStages), (c / kGemmStages) & 1);
             }
-        }
-        return;
-    }
-
-    // ---------------- consumers: warp w owns row tiles 2w and 2w+1 of the block
-    float acc[2][NT][4];
+        } else if (a.ssq_in != nullptr) {
+            // lanes 1..31: the input's RMSNorm factor per token (off the critical path)
+            pdl_wait();
+            for (int tl = lane - 1; tl < MT; tl += 31) {
+                const int tok = tok0 + tl;
+                float ss = 0.f;
+                if (tok < a.M) {
+                    for (int b0 = 0; b0 < a.n_ssq; b0 += 32) {
+                        float part[32];
 #pragma unroll
-    for (int j = 0; j < 2; ++j)
+                        for (int b = 0; b < 32; ++b)     // all loads of a batch in flight together
+                            part[b] = b0 + b < a.n_ssq ? a.ssq_in[(size_t)(b0 + b) * a.M + tok] : 0.f;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[j][nt][e] = 0.f;
-
-    bool ok = true;
-    for (int c = 0; c < nchunks; ++c) {
-        const int st = c % kStages;
-        ok = mbar_wait(full0 + 8 * st, (c / kStages) & 1);
-        if (!ok) break;
-        const unsigned char* wst = smem + st * kStageBytes;
-        const unsigned char* bst = wst + kGemmWStage;
-        int kc = nks - c * kGemmKC;
-        kc = kc < kGemmKC ? kc : kGemmKC;
-#pragma unroll
-        for (int k = 0; k < kGemmKC; ++k) {
-            if (k < kc) {
-                const uint4 a0 = *reinterpret_cast<const uint4*>(wst + ((k * 8 + warp * 2) * 32 + lane) * 16);
-                const uint4 a1 = *reinterpret_cast<const uint4*>(wst + ((k * 8 + warp * 2 + 1) * 32 + lane) * 16);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const uint4 b = *reinterpret_cast<const uint4*>(bst + ((k * NT + nt) * 32 + lane) * 16);
-                    mma_bf16_16816(acc[0][nt], a0, b.x, b.y);
-                    mma_bf16_16816(acc[1][nt], a1, b.x, b.y);
-                    mma_bf16_16816(acc[0][nt], a0, b.z, b.w);
-                    mma_bf16_16816(acc[1][nt], a1, b.z, b.w);
+                        for (int b = 0; b < 32; ++b) ss += part[b];
+                    }
                 }
+                rstd_s[tl] = rsqrtf(ss / (float)a.d_in + a.eps);
             }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(empty0 + 8 * st);
-    }
-    if (!ok) {
-        if (a.err && lane == 0) atomicExch(a.err, 2);
-        return;
+    } else {
+        // ---------------- consumers: warp w owns row tiles 2w and 2w+1 of the block
+        float acc[2][NT][4];
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[j][nt][e] = 0.f;
+
+        for (int c = 0; c < nchunks; ++c) {
+            const int st = c % kGemmStages;
+            ok = mbar_wait(full0 + 8 * st, (c / kGemmStages) & 1);
+            if (!ok) break;
+            const unsigned char* wst = smem + st * kStageBytes;
+            const unsigned char* bst = wst + kGemmWStage;
+            int kc = nks - c * kGemmKC;
+            kc = kc < kGemmKC ? kc : kGemmKC;
+#pragma unroll
+            for (int k = 0; k < kGemmKC; ++k) {
+                if (k < kc) {
+                    const uint4 a0 = *reinterpret_cast<const uint4*>(wst + ((k * 8 + warp * 2) * 32 + lane) * 16);
+                    const uint4 a1 = *reinterpret_cast<const uint4*>(wst + ((k * 8 + warp * 2 + 1) * 32 + lane) * 16);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint4 b = *reinterpret_cast<const uint4*>(bst + ((k * NT + nt) * 32 + lane) * 16);
+                        mma_bf16_16816(acc[0][nt], a0, b.x, b.y);
+                        mma_bf16_16816(acc[1][nt], a1, b.x, b.y);
+                        mma_bf16_16816(acc[0][nt], a0, b.z, b.w);
+                        mma_bf16_16816(acc[1][nt], a1, b.z, b.w);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * st);
+        }
+        if (!ok && a.err && lane == 0) atomicExch(a.err, 2);
+        // All consumers are past their last ring read before the ring is reused for the partial tile.
+        asm volatile("bar.sync 1, %0;" ::"n"(kGemmConsumers) : "memory");
+        // partial tile P[tile 8][token MT][row 16] (fp32) at the start of the ring
+        float* P = reinterpret_cast<float*>(smem);
+        const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                float* pt = P + ((warp * 2 + j) * MT + nt * 8 + 2 * t) * 16;
+                pt[g] = acc[j][nt][0];
+                pt[16 + g] = acc[j][nt][1];
+                pt[g + 8] = acc[j][nt][2];
+                pt[16 + g + 8] = acc[j][nt][3];
+            }
     }
 
-    // C fragment: c0,c1 -> (row g, tokens 2t, 2t+1); c2,c3 -> (row g+8, same tokens).
-    const int g = lane >> 2, t = lane & 3;
-    float* outp = a.out + (size_t)s * a.M * a.N;
-    const int tok0 = tb * (NT * 8);
+    // ---------------- cluster reduction + epilogue (all 160 threads reach both barriers, also on errors)
+    if (a.S > 1) cluster_sync_all(); else __syncthreads();
+    pdl_wait();   // (long satisfied) every thread that touches the predecessors' global data has waited itself
+    if (warp < kGemmConsumerWarps) {
+        const int j = threadIdx.x, row = j & 15, tg = j >> 4;       // 16 lanes = the 16 rows of a tile
+        const uint32_t p_local = smem_base;
+        for (int tile = s; tile < 8; tile += a.S) {
+            const int pr = rb * 128 + tile * 16 + row;               // packed row
+            float ssq_acc = 0.f;
+            // gather the S partial values of this thread's NT elements first (independent loads, all in flight),
+            // then add them in rank order
+            float pv[NT][kGemmMaxSplit];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        const int r0 = ((rb * 8 + warp * 2 + j) * 16) + g;
-        if (r0 >= a.N) continue;      // padding rows of the last block (N is a multiple of 16)
+            for (int i = 0; i < NT; ++i) {
+                const uint32_t off = (uint32_t)(((tile * MT + tg + 8 * i) * 16 + row) * 4);
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const int tok = tok0 + nt * 8 + 2 * t;
-            if (tok < a.M) {
-                outp[(size_t)tok * a.N + r0] = acc[j][nt][0];
-                outp[(size_t)tok * a.N + r0 + 8] = acc[j][nt][2];
+                for (int r = 0; r < kGemmMaxSplit; ++r)
+                    pv[i][r] = r < a.S ? dsmem_ld_f32(dsmem_addr(p_local + off, (uint32_t)r)) : 0.f;
             }
-            if (tok + 1 < a.M) {
-                outp[(size_t)(tok + 1) * a.N + r0] = acc[j][nt][1];
-                outp[(size_t)(tok + 1) * a.N + r0 + 8] = acc[j][nt][3];
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+                const int tl = tg + 8 * i, tok = tok0 + tl;
+                float v = 0.f;
+#pragma unroll
+                for (int r = 0; r < kGemmMaxSplit; ++r) v += pv[i][r];
+                if (a.ssq_in != nullptr) v *= rstd_s[tl];
+                const bool live = tok < a.M && pr < a.N;
+                if (MODE == kPlain) {
+                    if (live) a.out[(size_t)tok * a.N + pr] = v;
+                } else if (MODE == kResid) {
+                    float xn = 0.f;
+                    if (live) {
+                        float* xp = a.x + (size_t)tok * a.N + pr;
+                        xn = *xp + v;
+                        *xp = xn;
+                        xf_store_one(a.xf_out, tok, pr, xn * a.gain_next[pr], a.N / 16, NT);
+                    }
+                    // sum of squares over the tile's 16 rows (lanes of a half-warp), fixed order
+                    float q = xn * xn;
+                    q += __shfl_xor_sync(0xffffffffu, q, 1);
+                    q += __shfl_xor_sync(0xffffffffu, q, 2);
+                    q += __shfl_xor_sync(0xffffffffu, q, 4);
+                    q += __shfl_xor_sync(0xffffffffu, q, 8);
+                    ssq_acc = q;
+                    if (row == 0) {
+                        // tile sums go to rank 0's shared memory, which adds the 8 tiles up after the barrier
+                        const uint32_t dst = smem_u32(tss_s + tile * 32 + tl);
+                        if (a.S > 1) dsmem_st_f32(dsmem_addr(dst, 0u), ssq_acc); else tss_s[tile * 32 + tl] = ssq_acc;
+                    }
+                } else {
+                    // both remaining modes pair row i (< 8) with row i + 8 of the tile
+                    const float partner = __shfl_xor_sync(0xffffffffu, v, 8);
+                    if (MODE == kSwiglu) {
+                        if (row < 8 && live) {
+                            const float act = v / (1.f + expf(-v)) * partner;      // own = gate, partner = up
+                            xf_store_one(a.xf_act, tok, gu_feature(pr), act, (a.N / 2) / 16, NT);
+                        }
+                    } else if (live) {                                           // kQkvRope
+                        const int lr = qkv_logical_row(pr, a.hd);                 // head * hd + dim
+                        const int head = lr / a.hd, dim = lr % a.hd, half = a.hd / 2;
+                        float val = v;
+                        if (head < a.Hq + a.Hkv) {                                // q and k heads are rotated
+                            const float c = a.cs[(size_t)tok * half + (dim % half)];
+                            const float sgn = a.sn[(size_t)tok * half + (dim % half)];
+                            val = row < 8 ? v * c - partner * sgn : v * c + partner * sgn;
+                        }
+                        if (head < a.Hq) {
+                            a.q_out[((size_t)tok * a.Hq + head) * a.hd + dim] = val;
+                        } else {
+                            const int item = a.meta.row_item[tok], pos = a.meta.row_pos[tok];
+                            const int page =
+                                a.meta.block_tab[(size_t)a.meta.it_slot[item] * a.meta.max_pages + pos / a.page_size];
+                            const int kv = head < a.Hq + a.Hkv ? 0 : 1;
+                            const int kvh = kv ? head - a.Hq - a.Hkv : head - a.Hq;
+                            a.kv_pool[kv_index(a.layer, a.n_pages, page, kv, a.Hkv, kvh, a.page_size, pos % a.page_size,
+                                               a.hd, dim)] = f32_to_bf16_bits(val);
+                        }
+                    }
+                }
             }
+        }
+    }
+    if (a.S > 1) cluster_sync_all(); else __syncthreads();
+    if (MODE == kResid && s == 0 && threadIdx.x < MT) {
+        const int tok = tok0 + threadIdx.x;
+        if (tok < a.M) {
+            float q = 0.f;
+#pragma unroll
+            for (int tile = 0; tile < 8; ++tile) q += tss_s[tile * 32 + threadIdx.x];
+            a.ssq_out[(size_t)rb * a.M + tok] = q;
         }
     }
 }
@@ -264,31 +419,49 @@ __global__ void reduce_partials_kernel(const float* __restrict__ part, float* __
     }
 }
 
-static inline cudaError_t gemm_launch(const GemmPlan& p, const uint4* W, const uint4* xf, float* out, int* err,
-                                      int M, int N, cudaStream_t st) {
-    GemmArgs a{W, xf, out, err, M, N, p.S, p.KS};
+template <int MODE>
+static inline cudaError_t gemm_launch_mode(const GemmPlan& p, const GemmArgs& a, cudaStream_t st) {
     dim3 grid(p.RB * p.S, p.TB);
     switch (p.NT) {
-        case 1: return launch_pdl(gemm_wstream_kernel<1>, grid, dim3(kGemmThreads), gemm_smem_bytes(1), st, a);
-        case 2: return launch_pdl(gemm_wstream_kernel<2>, grid, dim3(kGemmThreads), gemm_smem_bytes(2), st, a);
-        case 3: return launch_pdl(gemm_wstream_kernel<3>, grid, dim3(kGemmThreads), gemm_smem_bytes(3), st, a);
-        default: return launch_pdl(gemm_wstream_kernel<4>, grid, dim3(kGemmThreads), gemm_smem_bytes(4), st, a);
+        case 1: return launch_pdl_cluster(gemm_wstream_kernel<1, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(1), st, p.S, a);
+        case 2: return launch_pdl_cluster(gemm_wstream_kernel<2, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(2), st, p.S, a);
+        case 3: return launch_pdl_cluster(gemm_wstream_kernel<3, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(3), st, p.S, a);
+        default: return launch_pdl_cluster(gemm_wstream_kernel<4, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(4), st, p.S, a);
     }
 }
 
-template <typename K>
-static inline cudaError_t gemm_set_attr(K kernel, int NT) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(NT));
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+static inline cudaError_t gemm_launch(int mode, const GemmPlan& p, GemmArgs a, cudaStream_t st) {
+    a.S = p.S;
+    a.KS = p.KS;
+    switch (mode) {
+        case kQkvRope: return gemm_launch_mode<kQkvRope>(p, a, st);
+        case kResid: return gemm_launch_mode<kResid>(p, a, st);
+        case kSwiglu: return gemm_launch_mode<kSwiglu>(p, a, st);
+        default: return gemm_launch_mode<kPlain>(p, a, st);
+    }
 }
 
+template <int NT, int MODE>
+static inline cudaError_t gemm_set_attr() {
+    cudaError_t e = cudaFuncSetAttribute(gemm_wstream_kernel<NT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         gemm_smem_bytes(NT));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(gemm_wstream_kernel<NT, MODE>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+}
+template <int MODE>
+static inline cudaError_t gemm_set_attr_mode() {
+    cudaError_t e;
+    if ((e = gemm_set_attr<1, MODE>()) != cudaSuccess) return e;
+    if ((e = gemm_set_attr<2, MODE>()) != cudaSuccess) return e;
+    if ((e = gemm_set_attr<3, MODE>()) != cudaSuccess) return e;
+    return gemm_set_attr<4, MODE>();
+}
 static inline cudaError_t gemm_init_attrs() {
     cudaError_t e;
-    if ((e = gemm_set_attr(gemm_wstream_kernel<1>, 1)) != cudaSuccess) return e;
-    if ((e = gemm_set_attr(gemm_wstream_kernel<2>, 2)) != cudaSuccess) return e;
-    if ((e = gemm_set_attr(gemm_wstream_kernel<3>, 3)) != cudaSuccess) return e;
-    return gemm_set_attr(gemm_wstream_kernel<4>, 4);
+    if ((e = gemm_set_attr_mode<kPlain>()) != cudaSuccess) return e;
+    if ((e = gemm_set_attr_mode<kQkvRope>()) != cudaSuccess) return e;
+    if ((e = gemm_set_attr_mode<kResid>()) != cudaSuccess) return e;
+    return gemm_set_attr_mode<kSwiglu>();
 }
 
 }  // namespace pipesd

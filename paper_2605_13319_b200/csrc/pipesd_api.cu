@@ -68,7 +68,7 @@ MetaLayout meta_layout(int max_rows, int max_items) {
 
 struct Derived {
     int Nqkv, qd, kvd, max_pages, max_items;
-    size_t part_floats;  // largest split-K partial array over all GEMMs and row counts
+    size_t part_floats;  // floats in each of the two KV staging arrays
 };
 
 Derived derive(const pipesd_model_cfg& c) {
@@ -78,20 +78,14 @@ Derived derive(const pipesd_model_cfg& c) {
     d.Nqkv = d.qd + 2 * d.kvd;
     d.max_pages = (c.max_seq + c.page_size - 1) / c.page_size;
     d.max_items = std::min(c.max_requests, c.max_rows);
-    size_t best = 0;
-    const int shapes[5][2] = {{d.Nqkv, c.d_model}, {c.d_model, d.qd}, {2 * c.d_ffn, c.d_model},
-                              {c.d_model, c.d_ffn}, {c.vocab, c.d_model}};
-    for (int m = 1; m <= c.max_rows; ++m)
-        for (auto& s : shapes) {
-            GemmPlan p = gemm_plan(m, s[0], s[1]);
-            best = std::max(best, (size_t)p.S * m * s[0]);
-        }
+    // two staging arrays for pipesd_debug_read_kv / write_kv: 256 positions of K and of V per round
+    size_t best = (size_t)256 * d.kvd / 2 + 64;
     d.part_floats = best;
     return d;
 }
 
 struct WsLayout {
-    size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, o_part, m_part, l_part, cs, sn, stats, results, meta,
+    size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, cs, sn, stats, results, meta,
         block_tab, qstage, total;
 };
 
@@ -109,6 +103,9 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     w.logits = take(4 * M * c.vocab);
     w.partA = take(4 * d.part_floats);
     w.partB = take(4 * d.part_floats);
+    const size_t nssq = (c.d_model + 127) / 128;
+    w.ssqA = take(4 * nssq * M);
+    w.ssqB = take(4 * nssq * M);
     const size_t slots = M * c.n_q_heads * kMaxSplits;
     w.o_part = take(4 * slots * c.head_dim);
     w.m_part = take(4 * slots);
@@ -244,8 +241,9 @@ int cuda_fail(pipesd_ctx* c, cudaError_t e, const char* where) {
     } while (0)
 
 // Launch one weight-streaming GEMM with accounting (and event timing when profiling is on).
-int launch_gemm(pipesd_ctx* ctx, const GemmPlan& p, const uint4* W, const void* xf, float* out, int M, int N,
-                int K) {
+int launch_gemm(pipesd_ctx* ctx, int mode, GemmArgs a, int K) {
+    const GemmPlan p = gemm_plan(a.M, a.N, K);
+    a.err = ctx->err_word();
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (ctx->time_gemms) {
         if (ctx->prof_used + 2 > ctx->prof_ev.size()) {
@@ -260,11 +258,11 @@ int launch_gemm(pipesd_ctx* ctx, const GemmPlan& p, const uint4* W, const void* 
         ctx->prof_used += 2;
         CU(cudaEventRecord(e0, ctx->st));
     }
-    CU(gemm_launch(p, W, (const uint4*)xf, out, ctx->err_word(), M, N, ctx->st));
+    CU(gemm_launch(mode, p, a, ctx->st));
     if (e1) CU(cudaEventRecord(e1, ctx->st));
     ctx->n_launch += 1;
     ctx->n_gemm += 1;
-    ctx->gemm_bytes += 2.0 * N * K + 4.0 * M * K + 4.0 * M * N;
+    ctx->gemm_bytes += 2.0 * a.N * K + 4.0 * a.M * K + 4.0 * a.M * a.N;
     return PIPESD_OK;
 }
 
@@ -327,9 +325,8 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         const ItemDesc& it = items[i];
         const Request& r = ctx->reqs[it.slot];
         const int total = r.len + it.rows;
-        int chunk = (total + target - 1) / target;
-        chunk = std::max(chunk, 64);
-        chunk = std::max(chunk, (total + kMaxSplits - 1) / kMaxSplits);
+        // eight splits (one per CTA of the attention cluster), whole pages each
+        int chunk = (total + kAttnSplits - 1) / kAttnSplits;
         chunk = (chunk + c.page_size - 1) / c.page_size * c.page_size;
         int nsplit = (total + chunk - 1) / chunk;
         I(ml.it_slot)[i] = it.slot;
@@ -366,16 +363,15 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     float* qbuf = ctx->W<float>(ctx->ws.qbuf);
     uint32_t* xf_attn = ctx->W<uint32_t>(ctx->ws.xf_attn);
     uint32_t* xf_act = ctx->W<uint32_t>(ctx->ws.xf_act);
-    float* partA = ctx->W<float>(ctx->ws.partA);
-    float* partB = ctx->W<float>(ctx->ws.partB);
+    float* ssqA = ctx->W<float>(ctx->ws.ssqA);   // sums of squares of the attention-norm (and final-norm) input
+    float* ssqB = ctx->W<float>(ctx->ws.ssqB);   // ... of the FFN-norm input
     float* o_part = ctx->W<float>(ctx->ws.o_part);
     float* m_part = ctx->W<float>(ctx->ws.m_part);
     float* l_part = ctx->W<float>(ctx->ws.l_part);
     float* cs = ctx->W<float>(ctx->ws.cs);
     float* sn = ctx->W<float>(ctx->ws.sn);
     const int hd = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads, d = c.d_model, F = c.d_ffn;
-    const uint16_t* no_emb = nullptr;
-    const int32_t* no_tok = nullptr;
+    const int n_ssq = (d + 127) / 128;
 
     // Every kernel of the chain is launched with programmatic stream serialisation: it may start while its
     // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
@@ -383,64 +379,77 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         int n = M * hd / 2;
         CU(launch_pdl(rope_table_kernel, dim3((n + 127) / 128), dim3(128), 0, st, meta.row_pos, M, hd,
                       log((double)c.rope_base), cs, sn));
+        CU(launch_pdl(embed_kernel, dim3(M), dim3(kEmbedThreads), 0, st, x, (const uint16_t*)ctx->emb, meta.row_tok, M,
+                      (const float*)ctx->layers[0].n1, d, xf_h, ssqA, n_ssq));
+        ctx->n_launch += 2;
     }
-    const float* part = nullptr;
-    int S = 0;
     int max_item_rows = 1;
     for (auto& it : items) max_item_rows = std::max(max_item_rows, it.rows);
     const int maxR = max_item_rows * (Hq / Hkv);                      // query rows that share one KV head
     const int q_tiles = std::min(kAttnMaxRowTiles, (maxR + 15) / 16);
     const int row_groups = (maxR + kAttnMaxRowTiles * 16 - 1) / (kAttnMaxRowTiles * 16);
     const size_t asmem = attn_smem_bytes(hd, q_tiles);
+    GemmArgs base = {};
+    base.M = M;
+    base.eps = c.rms_eps;
+    base.d_in = d;
+    base.n_ssq = n_ssq;
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& lw = ctx->layers[l];
-        CU(launch_pdl(add_norm_kernel, dim3(M), dim3(kNormThreads), 0, st, x, l == 0 ? (const uint16_t*)ctx->emb : no_emb,
-                      meta.row_tok, part, S, M, (const float*)lw.n1, c.rms_eps, d, xf_h));
-        GemmPlan p = gemm_plan(M, dv.Nqkv, d);
-        { int rc_ = launch_gemm(ctx, p, lw.qkv.packed, xf_h, partA, M, dv.Nqkv, d); if (rc_) return rc_; }
-        CU(launch_pdl(rope_kv_kernel, dim3(M, Hq + 2 * Hkv), dim3(hd / 2), 0, st, (const float*)partA, p.S, M, Hq, Hkv, hd,
-                      (const float*)cs, (const float*)sn, meta, qbuf, ctx->kv_pool, l, c.n_pages, c.page_size));
-        dim3 ag(max_nsplit, Hkv * row_groups, n_items);
-        if (hd == 128)
-            CU(launch_pdl(attn_split_kernel<128>, ag, dim3(kAttnThreads), asmem, st, (const float*)qbuf, meta,
-                          (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, Hq, Hkv, q_tiles, o_part, m_part,
-                          l_part));
-        else
-            CU(launch_pdl(attn_split_kernel<64>, ag, dim3(kAttnThreads), asmem, st, (const float*)qbuf, meta,
-                          (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, Hq, Hkv, q_tiles, o_part, m_part,
-                          l_part));
-        CU(launch_pdl(attn_combine_kernel, dim3(M, Hq), dim3(hd), 0, st, (const float*)o_part, (const float*)m_part,
-                      (const float*)l_part, meta, M, Hq, hd, xf_attn));
-        p = gemm_plan(M, d, dv.qd);
-        { int rc_ = launch_gemm(ctx, p, lw.o.packed, xf_attn, partB, M, d, dv.qd); if (rc_) return rc_; }
-        CU(launch_pdl(add_norm_kernel, dim3(M), dim3(kNormThreads), 0, st, x, no_emb, no_tok, (const float*)partB, p.S, M,
-                      (const float*)lw.n2, c.rms_eps, d, xf_h));
-        p = gemm_plan(M, 2 * F, d);
-        { int rc_ = launch_gemm(ctx, p, lw.gu.packed, xf_h, partA, M, 2 * F, d); if (rc_) return rc_; }
-        {
-            size_t n = (size_t)M * (F / 2);
-            int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
-            CU(launch_pdl(silu_mul_kernel, dim3(blocks), dim3(256), 0, st, (const float*)partA, p.S, M, F, xf_act));
+        {   // q, k, v = W_qkv . norm(x); RoPE; K/V appended to the pages
+            GemmArgs a = base;
+            a.W = lw.qkv.packed; a.xf = (const uint4*)xf_h; a.N = dv.Nqkv; a.ssq_in = ssqA;
+            a.q_out = qbuf; a.kv_pool = ctx->kv_pool; a.cs = cs; a.sn = sn; a.meta = meta;
+            a.Hq = Hq; a.Hkv = Hkv; a.hd = hd; a.layer = l; a.n_pages = c.n_pages; a.page_size = c.page_size;
+            int rc_ = launch_gemm(ctx, kQkvRope, a, d);
+            if (rc_) return rc_;
         }
-        p = gemm_plan(M, d, F);
-        { int rc_ = launch_gemm(ctx, p, lw.dn.packed, xf_act, partB, M, d, F); if (rc_) return rc_; }
-        part = partB;
-        S = p.S;
-        ctx->n_launch += 6;   // add_norm x2, rope_kv, attn_split, attn_combine, silu_mul
+        dim3 ag(kAttnSplits, Hkv * row_groups, n_items);
+        if (hd == 128)
+            CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
+                                  meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
+                                  (uint16_t*)xf_attn));
+        else
+            CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
+                                  meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
+                                  (uint16_t*)xf_attn));
+        {   // x += W_o . attn; xf_h = x * ffn gain; ssqB
+            GemmArgs a = base;
+            a.W = lw.o.packed; a.xf = (const uint4*)xf_attn; a.N = d; a.ssq_in = nullptr;
+            a.x = x; a.xf_out = (uint16_t*)xf_h; a.gain_next = lw.n2; a.ssq_out = ssqB;
+            int rc_ = launch_gemm(ctx, kResid, a, dv.qd);
+            if (rc_) return rc_;
+        }
+        {   // act = silu(W_g . norm(x)) * (W_u . norm(x))
+            GemmArgs a = base;
+            a.W = lw.gu.packed; a.xf = (const uint4*)xf_h; a.N = 2 * F; a.ssq_in = ssqB;
+            a.xf_act = (uint16_t*)xf_act;
+            int rc_ = launch_gemm(ctx, kSwiglu, a, d);
+            if (rc_) return rc_;
+        }
+        {   // x += W_d . act; xf_h = x * (next layer's attention gain | final gain); ssqA
+            GemmArgs a = base;
+            a.W = lw.dn.packed; a.xf = (const uint4*)xf_act; a.N = d; a.ssq_in = nullptr;
+            a.x = x; a.xf_out = (uint16_t*)xf_h;
+            a.gain_next = l + 1 < c.n_layers ? ctx->layers[l + 1].n1 : ctx->final_norm;
+            a.ssq_out = ssqA;
+            int rc_ = launch_gemm(ctx, kResid, a, F);
+            if (rc_) return rc_;
+        }
+        ctx->n_launch += 1;   // attention
     }
-    ctx->n_launch += 1;       // rope_table
     if (want_logits) {
-        ctx->n_launch += 2 + (want_reject ? 1 : 0);   // add_norm, row_stats, accept_sample
+        ctx->n_launch += 1 + (want_reject ? 1 : 0);   // row_stats, accept_sample
         float* logits = ctx->W<float>(ctx->ws.logits);
         RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
-        CU(launch_pdl(add_norm_kernel, dim3(M), dim3(kNormThreads), 0, st, x, no_emb, no_tok, part, S, M,
-                      (const float*)ctx->final_norm, c.rms_eps, d, xf_h));
-        GemmPlan p = gemm_plan(M, c.vocab, d);
-        float* dst = p.S == 1 ? logits : partA;
-        { int rc_ = launch_gemm(ctx, p, ctx->lm.packed, xf_h, dst, M, c.vocab, d); if (rc_) return rc_; }
+        {
+            GemmArgs a = base;
+            a.W = ctx->lm.packed; a.xf = (const uint4*)xf_h; a.N = c.vocab; a.ssq_in = ssqA; a.out = logits;
+            int rc_ = launch_gemm(ctx, kPlain, a, d);
+            if (rc_) return rc_;
+        }
         // plain launches from here on: they start after the GEMM has fully completed
-        row_stats_kernel<<<dim3(M, kStatSplits), 256, 0, st>>>(p.S == 1 ? nullptr : partA, p.S, M, c.vocab, logits,
-                                                               stats);
+        row_stats_kernel<<<dim3(M, kStatSplits), 256, 0, st>>>(nullptr, 1, M, c.vocab, logits, stats);
         ctx->last_rows = M;
         if (want_reject) {
             accept_sample_kernel<<<n_items, kSampleThreads, 0, st>>>(
@@ -508,10 +517,10 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     cudaError_t e = cudaSetDevice(c.device);
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
     if ((e = gemm_init_attrs()) != cudaSuccess) return bail(PIPESD_E_CUDA);
-    e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)attn_smem_bytes(128, kAttnMaxRowTiles));
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
-    e = cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)attn_smem_bytes(64, kAttnMaxRowTiles));
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
 
@@ -531,20 +540,18 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     char* wp = (char*)mem->weights;
     size_t off = 0;
     auto take = [&](size_t bytes) { char* p = wp + off; off += align_up(bytes); return p; };
-    auto pack = [&](GemmW& g, int N, int K, std::initializer_list<std::pair<const void*, int>> srcs) {
+    auto pack = [&](GemmW& g, int N, int K, int mode, std::initializer_list<std::pair<const void*, int>> srcs) {
         g.packed = (uint4*)take(gemm_packed_bytes(N, K));
         g.N = N;
         g.K = K;
-        const int padded = (N + 127) / 128 * 128;
-        int r0 = 0;
-        size_t left = srcs.size();
-        for (auto& s : srcs) {
-            const int pad_to = --left == 0 ? padded : r0 + s.second;   // the last source also zero-fills the padding
-            size_t total = (size_t)((pad_to - r0) / 16) * (K / 16) * 32;
-            int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
-            gemm_pack_kernel<<<blocks, 256, 0, st>>>((const uint16_t*)s.first, g.packed, r0, s.second, K, pad_to);
-            r0 += s.second;
-        }
+        PackSrc ps = {};
+        ps.mode = mode;
+        ps.hd = c.head_dim;
+        int i = 0;
+        for (auto& s : srcs) { ps.w[i] = (const uint16_t*)s.first; ps.rows[i] = s.second; ++i; }
+        size_t total = (size_t)((N + 127) / 128 * 8) * (K / 16) * 32;
+        int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
+        gemm_pack_kernel<<<blocks, 256, 0, st>>>(ps, g.packed, N, K);
     };
     ctx->emb = (uint16_t*)take((size_t)c.vocab * c.d_model * 2);
     if (cudaMemcpyAsync(ctx->emb, w->tok_emb, (size_t)c.vocab * c.d_model * 2, cudaMemcpyDeviceToDevice, st) !=
@@ -556,16 +563,16 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         if (!s.wq || !s.wk || !s.wv || !s.wo || !s.wg || !s.wu || !s.wd || !s.attn_norm || !s.ffn_norm)
             return bail(PIPESD_E_INVALID);
         LayerW& lw = ctx->layers[l];
-        pack(lw.qkv, dv.Nqkv, c.d_model, {{s.wq, dv.qd}, {s.wk, dv.kvd}, {s.wv, dv.kvd}});
-        pack(lw.o, c.d_model, dv.qd, {{s.wo, c.d_model}});
-        pack(lw.gu, 2 * c.d_ffn, c.d_model, {{s.wg, c.d_ffn}, {s.wu, c.d_ffn}});
-        pack(lw.dn, c.d_model, c.d_ffn, {{s.wd, c.d_model}});
+        pack(lw.qkv, dv.Nqkv, c.d_model, kQkvRope, {{s.wq, dv.qd}, {s.wk, dv.kvd}, {s.wv, dv.kvd}});
+        pack(lw.o, c.d_model, dv.qd, kPlain, {{s.wo, c.d_model}});
+        pack(lw.gu, 2 * c.d_ffn, c.d_model, kSwiglu, {{s.wg, c.d_ffn}, {s.wu, c.d_ffn}});
+        pack(lw.dn, c.d_model, c.d_ffn, kPlain, {{s.wd, c.d_model}});
         lw.n1 = (float*)take(4 * (size_t)c.d_model);
         lw.n2 = (float*)take(4 * (size_t)c.d_model);
         cudaMemcpyAsync(lw.n1, s.attn_norm, 4 * (size_t)c.d_model, cudaMemcpyDeviceToDevice, st);
         cudaMemcpyAsync(lw.n2, s.ffn_norm, 4 * (size_t)c.d_model, cudaMemcpyDeviceToDevice, st);
     }
-    pack(ctx->lm, c.vocab, c.d_model, {{w->lm_head, c.vocab}});
+    pack(ctx->lm, c.vocab, c.d_model, kPlain, {{w->lm_head, c.vocab}});
     ctx->final_norm = (float*)take(4 * (size_t)c.d_model);
     cudaMemcpyAsync(ctx->final_norm, w->final_norm, 4 * (size_t)c.d_model, cudaMemcpyDeviceToDevice, st);
     if (cudaGetLastError() != cudaSuccess) return bail(PIPESD_E_CUDA);
@@ -909,37 +916,38 @@ static size_t gemm_xf_bytes(int M, int K) { return align_up(xf_elems(M, K) * 16)
 
 uint64_t pipesd_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K) {
     if (M < 1 || N < 16 || K < 16) return 0;
-    GemmPlan p = gemm_plan(M, N, K);
-    return gemm_xf_bytes(M, K) + (p.S > 1 ? (uint64_t)p.S * M * N * 4 : 0);
+    return gemm_xf_bytes(M, K);
 }
 
 int32_t pipesd_gemm_pack(const void* W, void* packed, int32_t N, int32_t K, void* cuda_stream) {
     if (!W || !packed || N < 16 || K < 16 || N % 16 || K % 16) return PIPESD_E_INVALID;
-    const int padded = (N + 127) / 128 * 128;
-    size_t total = (size_t)(padded / 16) * (K / 16) * 32;
+    PackSrc ps = {};
+    ps.mode = kPlain;
+    ps.w[0] = (const uint16_t*)W;
+    ps.rows[0] = N;
+    size_t total = (size_t)((N + 127) / 128 * 8) * (K / 16) * 32;
     int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
-    gemm_pack_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)W, (uint4*)packed, 0, N, K, padded);
+    gemm_pack_kernel<<<blocks, 256, 0, (cudaStream_t)cuda_stream>>>(ps, (uint4*)packed, N, K);
     return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
 }
 
-// x -> split-bf16 fragments, GEMM, fixed-order sum of the K slices.  scratch = [xf | partial sums].
+// x -> split-bf16 fragments (the scratch), then the GEMM; the K slices are summed inside the kernel.
 static int32_t gemm_run_with_scratch(const void* packed, const float* x, float* y, void* scratch, int M, int N, int K,
                                      cudaStream_t st) {
     const GemmPlan p = gemm_plan(M, N, K);
     uint32_t* xf = (uint32_t*)scratch;
-    float* part = (float*)((char*)scratch + gemm_xf_bytes(M, K));
     {
         size_t n = (size_t)M * (K / 2);
         int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
         xf_format_kernel<<<blocks, 256, 0, st>>>(x, xf, M, K);
     }
-    float* dst = p.S == 1 ? y : part;
-    if (gemm_launch(p, (const uint4*)packed, (const uint4*)xf, dst, nullptr, M, N, st) != cudaSuccess) return PIPESD_E_CUDA;
-    if (p.S > 1) {
-        size_t n = (size_t)M * N;
-        int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
-        reduce_partials_kernel<<<blocks, 256, 0, st>>>((const float*)part, y, n, p.S);
-    }
+    GemmArgs a = {};
+    a.W = (const uint4*)packed;
+    a.xf = (const uint4*)xf;
+    a.M = M;
+    a.N = N;
+    a.out = y;
+    if (gemm_launch(kPlain, p, a, st) != cudaSuccess) return PIPESD_E_CUDA;
     return cudaGetLastError() == cudaSuccess ? PIPESD_OK : PIPESD_E_CUDA;
 }
 
@@ -964,7 +972,7 @@ int32_t pipesd_debug_gemm_force_split(int32_t S) {
 extern "C" {
 
 // ---- GEMM without any caller- or library-side allocation ------------------------------------
-// Split-K partial sums of pipesd_gemm_run_static live in this fixed array.  It is part of the
+// The scratch of pipesd_gemm_run_static (activation fragments) lives in this fixed array.  It is part of the
 // library image: every GPU that loads the library keeps these bytes reserved until the process
 // exits, which is why the limit is modest.
 static __device__ __align__(256) unsigned char g_static_gemm_scratch[PIPESD_STATIC_SCRATCH_BYTES];
@@ -998,8 +1006,9 @@ int32_t pipesd_gemm_run_static(const void* packed, const float* x, float* y, int
     void* scratch = nullptr;
     int rc = static_scratch_for_current_device(&scratch);
     if (rc != PIPESD_OK) return rc;
-    // Nothing has to be cleared: the activation fragments and every partial sum the reduction reads are
-    // written by this same call first, so the previous call's contents never reach the output.
+    // Nothing has to be cleared: every activation fragment the GEMM reads is written by this same call
+    // first (padding tokens only feed output columns that are never stored), so the previous call's
+    // contents never reach the output.
     return gemm_run_with_scratch(packed, x, y, scratch, M, N, K, (cudaStream_t)cuda_stream);
 }
 

@@ -2,11 +2,11 @@
 
 Some users of the library run where cudaMalloc is not an option (a plugin that only gets its input and
 output buffers, a latency-critical loop that must not touch the allocator, a process with a memory budget
-fixed at start-up), so they cannot supply the split-K scratch that pipesd_gemm_run needs.  The static
-variant keeps that scratch in a fixed array inside the library.  This file checks, through the C ABI, that
-it returns what pipesd_gemm_run returns -- twice in a row with different inputs, because the array is
-shared by all calls and still holds the previous call's partial sums -- and that it refuses problems that
-do not fit the array.  It is named to be collected last, and it must pass alone in a fresh process too."""
+fixed at start-up), so they cannot supply the scratch that pipesd_gemm_run needs for the activations'
+split-bf16 fragments.  The static variant keeps that scratch in a fixed array inside the library.  This file
+checks, through the C ABI, that it returns what pipesd_gemm_run returns -- twice in a row with different
+inputs, because the array is shared by all calls and still holds the previous call's contents -- and that
+it refuses problems that do not fit the array.  It is named to be collected last, and it must pass alone in a fresh process too."""
 import numpy as np
 import pytest
 
@@ -14,7 +14,7 @@ from paper_2605_13319_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-# (M, N, K): several K slices (the scratch is used), a ragged row block, and a single-slice case
+# (M, N, K): several K slices, a ragged row block, and a single-slice case
 CASES = [(9, 4096, 4096), (5, 688, 2048), (16, 4096, 11008), (3, 128, 256)]
 
 
@@ -46,7 +46,7 @@ def test_static_scratch_gemm_rejects_what_does_not_fit():
     import torch
     from paper_2605_13319_b200 import binding
     dev = torch.device("cuda", 0)
-    M, N, K = 64, 22016, 4096
+    M, N, K = 256, 4096, 11008
     assert binding.lib().pipesd_gemm_scratch_bytes(M, N, K) > binding.STATIC_SCRATCH_BYTES
     # no weights are touched: the size check comes before any launch, so small stand-in buffers are enough
     stub = torch.zeros(1024, dtype=torch.uint8, device=dev)
