@@ -35,6 +35,7 @@ WORKLOADS = {
     "1b-k8": ("1b", 512, 8, 1.0),
     "8b-k16": ("8b", 8192, 16, 0.5),
     "tiny-k4": ("tiny", 64, 4, 1.0),
+    "7b2l-k8": ("7b2l", 2048, 8, 1.0),   # two layers of the 7b shape: small enough for counter captures
 }
 METRIC = "verified tokens/sec (verify-pass latency in ms_per_step), k=8, 7B shape, % of HBM roofline"
 NOMINAL_HBM_GBS = 8000.0
@@ -258,7 +259,7 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     sname, P, k, sigma = WORKLOADS[args.workload]
-    shape = synth.SHAPES[sname]
+    shape = synth.B7.scaled(name="7b2l", n_layers=2) if sname == "7b2l" else synth.SHAPES[sname]
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -55,36 +55,58 @@ struct AttnSmem {
 
 // Per-CTA constants shared by the mode-specialised bodies.
 struct AttnCtx {
-    const uint16_t* kv_pool;
+    const uint16_t* kbase;     // K row (slot 0) of page 0 for this layer and KV head
     const int32_t* bt;
-    int layer, n_pages, page_size, Hkv, kvh;
+    size_t page_stride;        // elements between consecutive pages of a layer
+    size_t v_off;              // elements from a K row to the V row of the same slot
+    int page_size;
     int k0, k1, base, rows, R, rho0;
 };
 
-// Issue the cp.async copies of one 64-key tile (K and V) into a ring stage.
+// Two values -> packed bf16x2 hi and lo terms (a = hi + lo up to 2^-17 |a|).
+__device__ __forceinline__ void split2_bf16(float a, float b, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    const float2 hf = __bfloat1622float2(h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(a - hf.x, b - hf.y);
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+// Issue the cp.async copies of one 64-key tile (K and V) into a ring stage.  Thread t copies chunk
+// t % (HD/8) of rows t / (HD/8) + i * (128 / (HD/8)); page and slot advance incrementally (no divisions
+// in the loop), the page table is read once per page change with all reads issued before the copies.
 template <int HD>
 __device__ __forceinline__ void attn_load_tile(const AttnCtx& c, uint32_t stage_addr, int j0) {
     constexpr int kChunks = HD / 8;                       // 16-byte chunks per row
     constexpr int kPerThread = kAttnTile * kChunks / kAttnThreads;
+    constexpr int kRowStep = kAttnThreads / kChunks;      // rows between a thread's consecutive copies
+    const int row0 = threadIdx.x / kChunks, ch = threadIdx.x % kChunks;
+    const int pidx0 = (j0 + row0) / c.page_size, slot0 = (j0 + row0) - pidx0 * c.page_size;
+    int page[kPerThread];
+    {
+        int pidx = pidx0, slot = slot0;
+#pragma unroll
+        for (int i = 0; i < kPerThread; ++i) {
+            page[i] = (j0 + row0 + i * kRowStep) < c.k1 ? c.bt[pidx] : 0;
+            slot += kRowStep;
+            while (slot >= c.page_size) { slot -= c.page_size; ++pidx; }
+        }
+    }
+    int slot = slot0;
 #pragma unroll
     for (int i = 0; i < kPerThread; ++i) {
-        const int idx = threadIdx.x + i * kAttnThreads;
-        const int row = idx / kChunks, ch = idx % kChunks;
-        const int j = j0 + row;
-        const bool valid = j < c.k1;
-        size_t ko = 0, vo = 0;
-        if (valid) {
-            const int page = c.bt[j / c.page_size], slot = j % c.page_size;
-            ko = kv_index(c.layer, c.n_pages, page, 0, c.Hkv, c.kvh, c.page_size, slot, HD, ch * 8);
-            vo = kv_index(c.layer, c.n_pages, page, 1, c.Hkv, c.kvh, c.page_size, slot, HD, ch * 8);
-        }
+        const int row = row0 + i * kRowStep;
+        const bool valid = j0 + row < c.k1;
+        const uint16_t* kp = c.kbase;
+        if (valid) kp += (size_t)page[i] * c.page_stride + (size_t)slot * HD + ch * 8;
         const uint32_t off = row * (HD * 2) + ((ch ^ (row & 7)) << 4);
-        cp_async16(stage_addr + off, c.kv_pool + ko, valid);
-        cp_async16(stage_addr + AttnSmem<HD>::kTileBytes + off, c.kv_pool + vo, valid);
+        cp_async16(stage_addr + off, kp, valid);
+        cp_async16(stage_addr + AttnSmem<HD>::kTileBytes + off, kp + (valid ? c.v_off : 0), valid);
+        slot += kRowStep;
+        while (slot >= c.page_size) slot -= c.page_size;
     }
 }
 
-// Main loop for one CTA.  RTW = row-tile groups among the 4 warps (1, 2 or 4); 4/RTW = key strips.
 // On entry the copies of tiles 0 and 1 have been issued as two committed cp.async groups.  On exit the
 // CTA's partial result for its (up to 64) rows is in shared memory: Fo[row][HD], Fm[row], Fl[row].
 template <int HD, int RTW>
@@ -131,11 +153,12 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
         const int j0 = c.k0 + it * kAttnTile + sk0;    // first key of this warp's strip
 
         // ---- S = Q K^T over the strip
-        float s[NTS][4];
+        constexpr bool kTwoChains = NTS <= 4;     // short strips: keep the hi and lo products in separate chains
+        float s[NTS][4], s2[kTwoChains ? NTS : 1][4];
 #pragma unroll
         for (int i = 0; i < NTS; ++i)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) s[i][e] = 0.f;
+            for (int e = 0; e < 4; ++e) { s[i][e] = 0.f; if (kTwoChains) s2[i][e] = 0.f; }
 #pragma unroll
         for (int kp = 0; kp < KSTEPS / 2; ++kp) {
             const uint4 qh0 = *reinterpret_cast<const uint4*>(qs + (((2 * kp) * 2 + 0) * 32 + lane) * 16);
@@ -149,10 +172,16 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
                 uint32_t b[4];
                 ldmatrix_x4(b, kst + row * (HD * 2) + ((ch ^ (row & 7)) << 4));
                 mma_bf16_16816(s[nt], qh0, b[0], b[1]);
-                mma_bf16_16816(s[nt], ql0, b[0], b[1]);
+                mma_bf16_16816(kTwoChains ? s2[nt] : s[nt], ql0, b[0], b[1]);
                 mma_bf16_16816(s[nt], qh1, b[2], b[3]);
-                mma_bf16_16816(s[nt], ql1, b[2], b[3]);
+                mma_bf16_16816(kTwoChains ? s2[nt] : s[nt], ql1, b[2], b[3]);
             }
+        }
+        if (kTwoChains) {
+#pragma unroll
+            for (int nt = 0; nt < NTS; ++nt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) s[nt][e] += s2[nt][e];
         }
         // ---- mask, online softmax (rows g and g+8 of the tile)
         float mx[2] = {-INFINITY, -INFINITY};
@@ -172,7 +201,7 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
             mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
             mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
             const float m_new = fmaxf(m_run[hh], mx[hh]);
-            alpha[hh] = (m_run[hh] == -INFINITY) ? 0.f : expf(m_run[hh] - m_new);
+            alpha[hh] = (m_run[hh] == -INFINITY) ? 0.f : exp2f(m_run[hh] - m_new);
             m_run[hh] = m_new;
             l_run[hh] *= alpha[hh];
         }
@@ -181,7 +210,7 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int hh = e >> 1;
-                const float p = (s[nt][e] == -INFINITY) ? 0.f : expf(s[nt][e] - m_run[hh]);
+                const float p = (s[nt][e] == -INFINITY) ? 0.f : exp2f(s[nt][e] - m_run[hh]);
                 s[nt][e] = p;
                 l_run[hh] += p;      // per-lane partial; the quad is summed once at the end
             }
@@ -194,17 +223,10 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
 #pragma unroll
         for (int kk = 0; kk < STRIP / 16; ++kk) {
             uint4 ph, pl;
-            {
-                uint16_t h0, l0, h1, l1;
-                split_bf16(s[2 * kk][0], h0, l0); split_bf16(s[2 * kk][1], h1, l1);
-                ph.x = pack2(h0, h1); pl.x = pack2(l0, l1);
-                split_bf16(s[2 * kk][2], h0, l0); split_bf16(s[2 * kk][3], h1, l1);
-                ph.y = pack2(h0, h1); pl.y = pack2(l0, l1);
-                split_bf16(s[2 * kk + 1][0], h0, l0); split_bf16(s[2 * kk + 1][1], h1, l1);
-                ph.z = pack2(h0, h1); pl.z = pack2(l0, l1);
-                split_bf16(s[2 * kk + 1][2], h0, l0); split_bf16(s[2 * kk + 1][3], h1, l1);
-                ph.w = pack2(h0, h1); pl.w = pack2(l0, l1);
-            }
+            split2_bf16(s[2 * kk][0], s[2 * kk][1], ph.x, pl.x);
+            split2_bf16(s[2 * kk][2], s[2 * kk][3], ph.y, pl.y);
+            split2_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1], ph.z, pl.z);
+            split2_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3], ph.w, pl.w);
 #pragma unroll
             for (int np = 0; np < NTO / 2; ++np) {
                 const int row = sk0 + kk * 16 + (lane & 7) + 8 * ((lane >> 3) & 1);
@@ -264,7 +286,7 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
         for (int k = 0; k < KSW; ++k) {
             const int w = k * RTW + tile;
             const float ms = mm[w * 16 + row];
-            const float wgt = (ms == -INFINITY) ? 0.f : expf(ms - m);
+            const float wgt = (ms == -INFINITY) ? 0.f : exp2f(ms - m);
             const float2 ov = *reinterpret_cast<const float2*>(mo + ((size_t)w * 16 + row) * HD + e);
             v0 += wgt * ov.x; v1 += wgt * ov.y;
             l += wgt * ml[w * 16 + row];
@@ -300,9 +322,11 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restr
     const int total = c.base + c.rows, chunk = meta.it_chunk[item];
     c.k0 = min(sp * chunk, total);
     c.k1 = min(c.k0 + chunk, total);
-    c.kv_pool = kv_pool;
+    c.kbase = kv_pool + kv_index(layer, n_pages, 0, 0, Hkv, kvh, page_size, 0, HD, 0);
+    c.page_stride = (size_t)2 * Hkv * page_size * HD;
+    c.v_off = (size_t)Hkv * page_size * HD;
+    c.page_size = page_size;
     c.bt = meta.block_tab + (size_t)meta.it_slot[item] * meta.max_pages;
-    c.layer = layer; c.n_pages = n_pages; c.page_size = page_size; c.Hkv = Hkv; c.kvh = kvh;
     const int row0 = meta.it_row0[item];
     const uint32_t ring = smem_u32(smem);
 
@@ -318,7 +342,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restr
     if (!early1) { if (ntiles > 1) attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile); cp_async_commit(); }
 
     // ---- stage Q (scaled by 1/sqrt(hd)) as split-bf16 A fragments: [tile][k16 step][hi|lo][lane] uint4
-    const float scale = rsqrtf((float)HD);
+    const float scale = rsqrtf((float)HD) * 1.4426950408889634f;   // scores in the log2 domain: p = 2^(s - m)
     uint4* qsm = reinterpret_cast<uint4*>(smem + SM::kRing);
     for (int idx = threadIdx.x; idx < row_tiles * (HD / 16) * 32; idx += kAttnThreads) {
         const int lane = idx & 31, ks = (idx >> 5) % (HD / 16), tile = idx / (32 * (HD / 16));
@@ -377,7 +401,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restr
         float den = 0.f, w[kAttnSplits];
 #pragma unroll
         for (int r = 0; r < kAttnSplits; ++r) {
-            w[r] = (ms[r] == -INFINITY) ? 0.f : expf(ms[r] - m);   // an empty split or one beyond the causal horizon
+            w[r] = (ms[r] == -INFINITY) ? 0.f : exp2f(ms[r] - m);   // an empty split or one beyond the causal horizon
             den += w[r] * ls[r];
         }
         const int rho = c.rho0 + rl, gq = rho / c.rows, r_in = rho % c.rows;
