@@ -31,17 +31,16 @@ constexpr int kGemmConsumers = kGemmConsumerWarps * 32;
 constexpr int kGemmThreads = kGemmConsumers + 32;           // + one producer warp
 constexpr int kGemmKC = 4;                                  // k16 steps per ring stage
 constexpr int kGemmWStage = kGemmKC * 4096;                 // weight bytes per stage
-constexpr int kGemmStages = 3;
+constexpr int kGemmMinStages = 3, kGemmMaxStages = 6;
 constexpr int kGemmCtasPerSm = 3;
 constexpr int kGemmWave = 148 * kGemmCtasPerSm;
 constexpr int kGemmMaxSplit = 8;                            // portable cluster size
+constexpr int kGemmSmemTail = 128 + 128 + 1024;             // barriers | rstd[32] | tile sums of squares [8][32]
 
 enum GemmMode { kPlain = 0, kQkvRope = 1, kResid = 2, kSwiglu = 3 };
 
 __host__ __device__ constexpr int gemm_stage_bytes(int NT) { return kGemmWStage + kGemmKC * NT * 512; }
-__host__ __device__ constexpr int gemm_ring_bytes(int NT) { return kGemmStages * gemm_stage_bytes(NT); }
-// ring | 2*stages barriers (64 B) | rstd[32] | tile sums of squares [8][32]
-__host__ __device__ constexpr int gemm_smem_bytes(int NT) { return gemm_ring_bytes(NT) + 64 + 128 + 1024; }
+__host__ __device__ constexpr int gemm_smem_bytes(int NT, int stages) { return stages * gemm_stage_bytes(NT) + kGemmSmemTail; }
 
 struct GemmPlan {
     int NT;  // n8 token tiles per token block (1..4)
@@ -49,6 +48,7 @@ struct GemmPlan {
     int RB;  // 128-row blocks
     int S;   // K slices = cluster size
     int KS;  // k16 steps in K
+    int stages;  // ring depth
 };
 
 // Tiles per token block / token blocks for M rows: shared by the GEMM and by the producers of xf arrays.
@@ -67,19 +67,22 @@ static inline GemmPlan gemm_plan(int M, int N, int K) {
     p.TB = xf_tb(M);
     p.RB = (N + 127) / 128;
     p.KS = K / 16;
+    // One resident wave if possible: every CTA streams from the first microsecond and the next kernel's
+    // CTAs find room to prefetch.  Largest K split that still fits the wave; no split when it cannot fit.
     int best = 1;
-    double best_score = -1e9;
     for (int s = 1; s <= kGemmMaxSplit && s <= p.KS; ++s) {
         if (s > 1 && p.KS / s < 2 * kGemmKC) break;
-        long ctas = (long)p.RB * s * p.TB;
-        long waves = (ctas + kGemmWave - 1) / kGemmWave;
-        double eff = (double)ctas / (double)(waves * kGemmWave);
-        if (ctas < kGemmWave) eff = 0.5 + 0.5 * eff;      // an under-full single wave still streams well
-        double score = eff - 0.004 * s;
-        if (score > best_score) { best_score = score; best = s; }
+        if ((long)p.RB * s * p.TB <= kGemmWave) best = s;
     }
     p.S = g_gemm_force_split > 0 && g_gemm_force_split <= kGemmMaxSplit && g_gemm_force_split <= p.KS
               ? g_gemm_force_split : best;
+    // ring depth: as deep as the shared memory of an SM allows for the number of CTAs it will hold
+    long ctas = (long)p.RB * p.S * p.TB;
+    int per_sm = (int)((ctas + 147) / 148);
+    per_sm = per_sm < 1 ? 1 : (per_sm > kGemmCtasPerSm ? kGemmCtasPerSm : per_sm);
+    int budget = (227 * 1024) / per_sm - 1024 - kGemmSmemTail;
+    p.stages = budget / gemm_stage_bytes(p.NT);
+    p.stages = p.stages < kGemmMinStages ? kGemmMinStages : (p.stages > kGemmMaxStages ? kGemmMaxStages : p.stages);
     return p;
 }
 
@@ -151,7 +154,7 @@ struct GemmArgs {
     const uint4* W;     // packed weights
     const uint4* xf;    // activations, split-bf16 B fragments [tb][ks][nt][32]
     int* err;           // device error word (nullable): set when a bounded wait gives up
-    int M, N, S, KS;
+    int M, N, S, KS, stages;
     // input normalisation (nullable): ssq_in[b*M + tok], b < n_ssq, are sums of squares of the un-normalised
     // input row; the result rows are scaled by rsqrt(sum / d_in + eps)
     const float* ssq_in;
@@ -164,7 +167,7 @@ struct GemmArgs {
     uint16_t* kv_pool;
     const float* cs;    // [M][hd/2] cos / sin of the row's position
     const float* sn;
-    PassMeta meta;
+    const long long* row_kvoff;   // [M] element offset of the row's K slot inside a layer (head 0)
     int Hq, Hkv, hd, layer, n_pages, page_size;
     // kResid
     float* x;           // residual stream [M][N], updated in place
@@ -181,11 +184,13 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
     constexpr int kBStage = kGemmKC * NT * 512;
     constexpr int MT = NT * 8;                        // tokens per token block
     extern __shared__ __align__(128) unsigned char smem[];
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + gemm_ring_bytes(NT));   // full[3], empty[3]
-    float* rstd_s = reinterpret_cast<float*>(smem + gemm_ring_bytes(NT) + 64);  // [32]
-    float* tss_s = rstd_s + 32;                                                  // [8 tiles][32 tokens]
+    const int stages = a.stages;
+    unsigned char* tail = smem + stages * kStageBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);              // full[stages], empty[stages]
+    float* rstd_s = reinterpret_cast<float*>(tail + 128);             // [32]
+    float* tss_s = rstd_s + 32;                                       // [8 tiles][32 tokens]
     const uint32_t smem_base = smem_u32(smem);
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kGemmStages;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kGemmMaxStages;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rb = blockIdx.x / a.S, s = blockIdx.x % a.S, tb = blockIdx.y;   // s == rank in the cluster
     const int ks0 = (int)(((long)a.KS * s) / a.S), ks1 = (int)(((long)a.KS * (s + 1)) / a.S);
@@ -193,8 +198,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
     const int tok0 = tb * MT;
 
     if (threadIdx.x == 0) {
-#pragma unroll
-        for (int i = 0; i < kGemmStages; ++i) {
+        for (int i = 0; i < stages; ++i) {
             mbar_init(full0 + 8 * i, 1);
             mbar_init(empty0 + 8 * i, kGemmConsumerWarps);
         }
@@ -202,6 +206,12 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
     }
     __syncthreads();
     pdl_launch_dependents();
+
+    // epilogue inputs that live in global memory are fetched right after the dependency wait, long before the
+    // epilogue needs them (only when a rank owns at most two tiles, i.e. S >= 4)
+    const bool prefetch = (8 + a.S - 1) / a.S <= 2;
+    float pf_a[2][NT], pf_b[2][NT], pf_g[2];
+    long long pf_kv[NT];
 
     bool ok = true;
     if (warp == kGemmConsumerWarps) {
@@ -211,7 +221,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             const unsigned char* bsrc =
                 reinterpret_cast<const unsigned char*>(a.xf) + ((size_t)tb * a.KS + ks0) * (NT * 512);
             auto chunk_ks = [&](int c) { int r = nks - c * kGemmKC; return r < kGemmKC ? r : kGemmKC; };
-            const int pre = nchunks < kGemmStages ? nchunks : kGemmStages;
+            const int pre = nchunks < stages ? nchunks : stages;
             // weights do not depend on the previous kernel: start them before the dependency wait
             for (int c = 0; c < pre; ++c) {
                 const int kc = chunk_ks(c);
@@ -224,22 +234,24 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                 bulk_g2s(smem_base + c * kStageBytes + kGemmWStage, bsrc + (size_t)c * kBStage, (uint32_t)kc * NT * 512,
                          full0 + 8 * c);
             }
-            int issued = pre;
+            int issued = pre, st = 0;
+            uint32_t ph = 0;                       // parity of the empty-barrier phase being waited for
             for (int c = pre; c < nchunks; ++c) {
-                const int st = c % kGemmStages, kc = chunk_ks(c);
-                ok = mbar_wait(empty0 + 8 * st, ((c / kGemmStages) - 1) & 1);
+                const int kc = chunk_ks(c);
+                ok = mbar_wait(empty0 + 8 * st, ph);
                 if (!ok) break;
                 mbar_expect_tx(full0 + 8 * st, (uint32_t)kc * (4096 + NT * 512));
                 bulk_g2s(smem_base + st * kStageBytes, wsrc + (size_t)c * kGemmWStage, (uint32_t)kc * 4096, full0 + 8 * st);
                 bulk_g2s(smem_base + st * kStageBytes + kGemmWStage, bsrc + (size_t)c * kBStage,
                          (uint32_t)kc * NT * 512, full0 + 8 * st);
                 issued = c + 1;
+                if (++st == stages) { st = 0; ph ^= 1u; }
             }
             if (!ok) {
                 if (a.err) atomicExch(a.err, 1);
                 // give up: let every copy already issued land before this CTA's shared memory is released
-                for (int c = issued > kGemmStages ? issued - kGemmStages : 0; c < issued; ++c)
-                    mbar_wait(full0 + 8 * (c % kGemmStages), (c / kGemmStages) & 1);
+                for (int c = issued > stages ? issued - stages : 0; c < issued; ++c)
+                    mbar_wait(full0 + 8 * (c % stages), (c / stages) & 1);
             }
         } else if (a.ssq_in != nullptr) {
             // lanes 1..31: the input's RMSNorm factor per token (off the critical path)
@@ -263,6 +275,37 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
         __syncwarp();
     } else {
         // ---------------- consumers: warp w owns row tiles 2w and 2w+1 of the block
+        if ((MODE == kResid || MODE == kQkvRope) && prefetch) {
+            pdl_wait();
+            const int row = threadIdx.x & 15, tg = threadIdx.x >> 4;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int tile = s + q * a.S, pr = rb * 128 + tile * 16 + row;
+                pf_g[q] = 0.f;
+#pragma unroll
+                for (int i = 0; i < NT; ++i) {
+                    const int tok = tok0 + tg + 8 * i;
+                    pf_a[q][i] = pf_b[q][i] = 0.f;
+                    if (tile < 8 && tok < a.M && pr < a.N) {
+                        if (MODE == kResid) {
+                            pf_a[q][i] = a.x[(size_t)tok * a.N + pr];
+                        } else {
+                            const int half = a.hd / 2, dim = qkv_logical_row(pr, a.hd) % a.hd;
+                            pf_a[q][i] = a.cs[(size_t)tok * half + (dim % half)];
+                            pf_b[q][i] = a.sn[(size_t)tok * half + (dim % half)];
+                        }
+                    }
+                }
+                if (MODE == kResid && tile < 8 && pr < a.N) pf_g[q] = a.gain_next[pr];
+            }
+            if (MODE == kQkvRope) {
+#pragma unroll
+                for (int i = 0; i < NT; ++i) {
+                    const int tok = tok0 + tg + 8 * i;
+                    pf_kv[i] = tok < a.M ? a.row_kvoff[tok] : 0;
+                }
+            }
+        }
         float acc[2][NT][4];
 #pragma unroll
         for (int j = 0; j < 2; ++j)
@@ -271,9 +314,10 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
 #pragma unroll
                 for (int e = 0; e < 4; ++e) acc[j][nt][e] = 0.f;
 
+        int st = 0;
+        uint32_t ph = 0;
         for (int c = 0; c < nchunks; ++c) {
-            const int st = c % kGemmStages;
-            ok = mbar_wait(full0 + 8 * st, (c / kGemmStages) & 1);
+            ok = mbar_wait(full0 + 8 * st, ph);
             if (!ok) break;
             const unsigned char* wst = smem + st * kStageBytes;
             const unsigned char* bst = wst + kGemmWStage;
@@ -296,6 +340,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8 * st);
+            if (++st == stages) { st = 0; ph ^= 1u; }
         }
         if (!ok && a.err && lane == 0) atomicExch(a.err, 2);
         // All consumers are past their last ring read before the ring is reused for the partial tile.
@@ -319,20 +364,21 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
     if (a.S > 1) cluster_sync_all(); else __syncthreads();
     pdl_wait();   // (long satisfied) every thread that touches the predecessors' global data has waited itself
     if (warp < kGemmConsumerWarps) {
-        const int j = threadIdx.x, row = j & 15, tg = j >> 4;       // 16 lanes = the 16 rows of a tile
+        const int row = threadIdx.x & 15, tg = threadIdx.x >> 4;   // 16 lanes = the 16 rows of a tile
         const uint32_t p_local = smem_base;
-        for (int tile = s; tile < 8; tile += a.S) {
+        // One tile of the row block: sum the S partial tiles in rank order, then the mode's epilogue.
+        // xin / gin / cin / sin_ : prefetched epilogue inputs of this tile, or null to load them here.
+        auto epi_tile = [&](int tile, const float* xin, const float* gin, const float* cin, const float* sin_) {
             const int pr = rb * 128 + tile * 16 + row;               // packed row
-            float ssq_acc = 0.f;
-            // gather the S partial values of this thread's NT elements first (independent loads, all in flight),
-            // then add them in rank order
             float pv[NT][kGemmMaxSplit];
 #pragma unroll
             for (int i = 0; i < NT; ++i) {
                 const uint32_t off = (uint32_t)(((tile * MT + tg + 8 * i) * 16 + row) * 4);
 #pragma unroll
-                for (int r = 0; r < kGemmMaxSplit; ++r)
-                    pv[i][r] = r < a.S ? dsmem_ld_f32(dsmem_addr(p_local + off, (uint32_t)r)) : 0.f;
+                for (int r = 0; r < kGemmMaxSplit; ++r)      // independent loads, all in flight
+                    pv[i][r] = r < a.S ? (a.S > 1 ? dsmem_ld_f32(dsmem_addr(p_local + off, (uint32_t)r))
+                                                  : *reinterpret_cast<const float*>(smem + off))
+                                       : 0.f;
             }
 #pragma unroll
             for (int i = 0; i < NT; ++i) {
@@ -348,9 +394,9 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                     float xn = 0.f;
                     if (live) {
                         float* xp = a.x + (size_t)tok * a.N + pr;
-                        xn = *xp + v;
+                        xn = (xin ? xin[i] : *xp) + v;
                         *xp = xn;
-                        xf_store_one(a.xf_out, tok, pr, xn * a.gain_next[pr], a.N / 16, NT);
+                        xf_store_one(a.xf_out, tok, pr, xn * (gin ? gin[0] : a.gain_next[pr]), a.N / 16, NT);
                     }
                     // sum of squares over the tile's 16 rows (lanes of a half-warp), fixed order
                     float q = xn * xn;
@@ -358,11 +404,10 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                     q += __shfl_xor_sync(0xffffffffu, q, 2);
                     q += __shfl_xor_sync(0xffffffffu, q, 4);
                     q += __shfl_xor_sync(0xffffffffu, q, 8);
-                    ssq_acc = q;
                     if (row == 0) {
                         // tile sums go to rank 0's shared memory, which adds the 8 tiles up after the barrier
                         const uint32_t dst = smem_u32(tss_s + tile * 32 + tl);
-                        if (a.S > 1) dsmem_st_f32(dsmem_addr(dst, 0u), ssq_acc); else tss_s[tile * 32 + tl] = ssq_acc;
+                        if (a.S > 1) dsmem_st_f32(dsmem_addr(dst, 0u), q); else tss_s[tile * 32 + tl] = q;
                     }
                 } else {
                     // both remaining modes pair row i (< 8) with row i + 8 of the tile
@@ -377,24 +422,33 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                         const int head = lr / a.hd, dim = lr % a.hd, half = a.hd / 2;
                         float val = v;
                         if (head < a.Hq + a.Hkv) {                                // q and k heads are rotated
-                            const float c = a.cs[(size_t)tok * half + (dim % half)];
-                            const float sgn = a.sn[(size_t)tok * half + (dim % half)];
+                            const float c = cin ? cin[i] : a.cs[(size_t)tok * half + (dim % half)];
+                            const float sgn = sin_ ? sin_[i] : a.sn[(size_t)tok * half + (dim % half)];
                             val = row < 8 ? v * c - partner * sgn : v * c + partner * sgn;
                         }
                         if (head < a.Hq) {
                             a.q_out[((size_t)tok * a.Hq + head) * a.hd + dim] = val;
                         } else {
-                            const int item = a.meta.row_item[tok], pos = a.meta.row_pos[tok];
-                            const int page =
-                                a.meta.block_tab[(size_t)a.meta.it_slot[item] * a.meta.max_pages + pos / a.page_size];
                             const int kv = head < a.Hq + a.Hkv ? 0 : 1;
                             const int kvh = kv ? head - a.Hq - a.Hkv : head - a.Hq;
-                            a.kv_pool[kv_index(a.layer, a.n_pages, page, kv, a.Hkv, kvh, a.page_size, pos % a.page_size,
-                                               a.hd, dim)] = f32_to_bf16_bits(val);
+                            const size_t per_head = (size_t)a.page_size * a.hd;
+                            const size_t off = (size_t)a.layer * a.n_pages * 2 * a.Hkv * per_head +
+                                               (size_t)(cin ? pf_kv[i] : a.row_kvoff[tok]) +
+                                               ((size_t)kv * a.Hkv + kvh) * per_head + dim;
+                            a.kv_pool[off] = f32_to_bf16_bits(val);
                         }
                     }
                 }
             }
+        };
+        if (prefetch) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int tile = s + q * a.S;
+                if (tile < 8) epi_tile(tile, pf_a[q], &pf_g[q], pf_a[q], pf_b[q]);
+            }
+        } else {
+            for (int tile = s; tile < 8; tile += a.S) epi_tile(tile, nullptr, nullptr, nullptr, nullptr);
         }
     }
     if (a.S > 1) cluster_sync_all(); else __syncthreads();
@@ -423,16 +477,17 @@ template <int MODE>
 static inline cudaError_t gemm_launch_mode(const GemmPlan& p, const GemmArgs& a, cudaStream_t st) {
     dim3 grid(p.RB * p.S, p.TB);
     switch (p.NT) {
-        case 1: return launch_pdl_cluster(gemm_wstream_kernel<1, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(1), st, p.S, a);
-        case 2: return launch_pdl_cluster(gemm_wstream_kernel<2, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(2), st, p.S, a);
-        case 3: return launch_pdl_cluster(gemm_wstream_kernel<3, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(3), st, p.S, a);
-        default: return launch_pdl_cluster(gemm_wstream_kernel<4, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(4), st, p.S, a);
+        case 1: return launch_pdl_cluster(gemm_wstream_kernel<1, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(1, p.stages), st, p.S, a);
+        case 2: return launch_pdl_cluster(gemm_wstream_kernel<2, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(2, p.stages), st, p.S, a);
+        case 3: return launch_pdl_cluster(gemm_wstream_kernel<3, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(3, p.stages), st, p.S, a);
+        default: return launch_pdl_cluster(gemm_wstream_kernel<4, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(4, p.stages), st, p.S, a);
     }
 }
 
 static inline cudaError_t gemm_launch(int mode, const GemmPlan& p, GemmArgs a, cudaStream_t st) {
     a.S = p.S;
     a.KS = p.KS;
+    a.stages = p.stages;
     switch (mode) {
         case kQkvRope: return gemm_launch_mode<kQkvRope>(p, a, st);
         case kResid: return gemm_launch_mode<kResid>(p, a, st);
@@ -444,7 +499,7 @@ static inline cudaError_t gemm_launch(int mode, const GemmPlan& p, GemmArgs a, c
 template <int NT, int MODE>
 static inline cudaError_t gemm_set_attr() {
     cudaError_t e = cudaFuncSetAttribute(gemm_wstream_kernel<NT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         gemm_smem_bytes(NT));
+                                         gemm_smem_bytes(NT, kGemmMaxStages));
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(gemm_wstream_kernel<NT, MODE>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
 }

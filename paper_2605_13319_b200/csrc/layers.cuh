@@ -51,17 +51,25 @@ __global__ void __launch_bounds__(kEmbedThreads) embed_kernel(float* __restrict_
 }
 
 // cos/sin of pos * base^(-2j/hd), evaluated in fp64 (positions reach 10^4, fp32 angles would lose
-// three digits), stored fp32 [M][hd/2].
-__global__ void rope_table_kernel(const int32_t* __restrict__ row_pos, int M, int hd, double log_base,
-                                  float* __restrict__ cs, float* __restrict__ sn) {
+// three digits), stored fp32 [M][hd/2]; and, per row, the element offset of its K slot (head 0) inside a
+// layer of the paged pool, so that the QKV epilogue appends K/V without walking the page table.
+__global__ void rope_table_kernel(PassMeta meta, int M, int hd, double log_base, float* __restrict__ cs,
+                                  float* __restrict__ sn, long long* __restrict__ row_kvoff, int n_pages, int Hkv,
+                                  int page_size) {
     pdl_wait();
     pdl_launch_dependents();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     int half = hd / 2;
     if (i >= M * half) return;
     int row = i / half, j = i % half;
+    const int pos = meta.row_pos[row];
+    if (j == 0) {
+        const int item = meta.row_item[row];
+        const int page = meta.block_tab[(size_t)meta.it_slot[item] * meta.max_pages + pos / page_size];
+        row_kvoff[row] = (long long)kv_index(0, n_pages, page, 0, Hkv, 0, page_size, pos % page_size, hd, 0);
+    }
     double theta = exp(-2.0 * (double)j / (double)hd * log_base);
-    double ang = (double)row_pos[row] * theta;
+    double ang = (double)pos * theta;
     double s, c;
     sincos(ang, &s, &c);
     cs[i] = (float)c;

@@ -85,7 +85,7 @@ Derived derive(const pipesd_model_cfg& c) {
 }
 
 struct WsLayout {
-    size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, cs, sn, stats, results, meta,
+    size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, cs, sn, kvoff, stats, results, meta,
         block_tab, qstage, total;
 };
 
@@ -112,6 +112,7 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     w.l_part = take(4 * slots);
     w.cs = take(4 * M * (c.head_dim / 2));
     w.sn = take(4 * M * (c.head_dim / 2));
+    w.kvoff = take(8 * M);
     w.stats = take(sizeof(RowStat) * M * kStatSplits);
     w.results = take(sizeof(RejectOut) * d.max_items + 16);   // + the device error word, read back with the results
     w.meta = take(meta_layout(c.max_rows, d.max_items).total);
@@ -377,8 +378,8 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
     {
         int n = M * hd / 2;
-        CU(launch_pdl(rope_table_kernel, dim3((n + 127) / 128), dim3(128), 0, st, meta.row_pos, M, hd,
-                      log((double)c.rope_base), cs, sn));
+        CU(launch_pdl(rope_table_kernel, dim3((n + 127) / 128), dim3(128), 0, st, meta, M, hd, log((double)c.rope_base),
+                      cs, sn, ctx->W<long long>(ctx->ws.kvoff), c.n_pages, Hkv, c.page_size));
         CU(launch_pdl(embed_kernel, dim3(M), dim3(kEmbedThreads), 0, st, x, (const uint16_t*)ctx->emb, meta.row_tok, M,
                       (const float*)ctx->layers[0].n1, d, xf_h, ssqA, n_ssq));
         ctx->n_launch += 2;
@@ -399,7 +400,8 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         {   // q, k, v = W_qkv . norm(x); RoPE; K/V appended to the pages
             GemmArgs a = base;
             a.W = lw.qkv.packed; a.xf = (const uint4*)xf_h; a.N = dv.Nqkv; a.ssq_in = ssqA;
-            a.q_out = qbuf; a.kv_pool = ctx->kv_pool; a.cs = cs; a.sn = sn; a.meta = meta;
+            a.q_out = qbuf; a.kv_pool = ctx->kv_pool; a.cs = cs; a.sn = sn;
+            a.row_kvoff = ctx->W<long long>(ctx->ws.kvoff);
             a.Hq = Hq; a.Hkv = Hkv; a.hd = hd; a.layer = l; a.n_pages = c.n_pages; a.page_size = c.page_size;
             int rc_ = launch_gemm(ctx, kQkvRope, a, d);
             if (rc_) return rc_;
