@@ -9,7 +9,7 @@
 //
 // One CTA (4 warps) = one KV head of one request x one split x up to 64 query rows, where the rows are
 // all (query head of the group, chunk row) pairs that share the KV head (GQA).  K and V tiles of 64 keys
-// travel global -> shared with 16-byte cp.async in a three-stage ring (page table resolved per key row,
+// travel global -> shared with 16-byte cp.async in a two-stage ring (page table resolved per key row,
 // rows XOR-swizzled so that ldmatrix is conflict-free).  QK^T and PV run on mma.sync m16n8k16 with fp32
 // accumulation; Q and the softmax probabilities are fp32 values split into bf16 hi + lo terms (two MMAs),
 // K and V are the cache's bf16.  How the 4 warps share a tile depends on the number of 16-row tiles:
@@ -23,7 +23,7 @@ namespace pipesd {
 
 constexpr int kAttnThreads = 128;
 constexpr int kAttnTile = 64;       // keys per tile
-constexpr int kAttnStages = 3;
+constexpr int kAttnStages = 2;
 constexpr int kAttnMaxRowTiles = 4; // 64 query rows per CTA
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
@@ -50,7 +50,8 @@ struct AttnSmem {
     static constexpr int kStageBytes = 2 * kTileBytes;                  // K then V
     static constexpr int kQTileBytes = (HD / 16) * 2 * 512;             // A fragments hi+lo of one 16-row tile
     static constexpr int kRing = kAttnStages * kStageBytes;
-    static size_t bytes(int row_tiles) { return (size_t)kRing + (size_t)row_tiles * kQTileBytes; }
+    // ring | Q fragments (reused for the CTA's partial result, which needs 128 B more per row tile)
+    static size_t bytes(int row_tiles) { return (size_t)kRing + (size_t)row_tiles * (kQTileBytes + 128); }
 };
 
 // Per-CTA constants shared by the mode-specialised bodies.
@@ -62,6 +63,12 @@ struct AttnCtx {
     int page_size;
     int k0, k1, base, rows, R, rho0;
 };
+
+__device__ __forceinline__ float fast_exp2(float x) {   // 2^x, relative error 2^-22; 2^-inf = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 // Two values -> packed bf16x2 hi and lo terms (a = hi + lo up to 2^-17 |a|).
 __device__ __forceinline__ void split2_bf16(float a, float b, uint32_t& hi, uint32_t& lo) {
@@ -136,17 +143,20 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
         const int rho = c.rho0 + rtw * 16 + g + 8 * hh;
-        horizon[hh] = rho < c.R ? c.base + rho % c.rows : -1;   // keys j <= horizon are visible; -1: padding row
+        horizon[hh] = rho < c.R ? c.base + rho % c.rows : -1;   // keys j <= horizon are visible (padding rows: results unused)
     }
 
     const int ntiles = c.k1 > c.k0 ? (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile : 0;
 
     for (int it = 0; it < ntiles; ++it) {
+        if (it > 0) {
+            __syncthreads();      // everyone is done with tile it-1: its stage can take tile it+1
+            if (it + 1 < ntiles)
+                attn_load_tile<HD>(c, ring + ((it + 1) % kAttnStages) * SM::kStageBytes, c.k0 + (it + 1) * kAttnTile);
+            cp_async_commit();
+        }
         cp_async_wait<1>();
-        __syncthreads();          // tile `it` has landed for everyone; everyone is done with tile it-1
-        if (it + 2 < ntiles)
-            attn_load_tile<HD>(c, ring + ((it + 2) % kAttnStages) * SM::kStageBytes, c.k0 + (it + 2) * kAttnTile);
-        cp_async_commit();
+        __syncthreads();          // tile `it` has landed for everyone
         if (!warp_active) continue;
         const uint32_t kst = ring + (it % kAttnStages) * SM::kStageBytes;
         const uint32_t vst = kst + SM::kTileBytes;
@@ -183,25 +193,28 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
 #pragma unroll
                 for (int e = 0; e < 4; ++e) s[nt][e] += s2[nt][e];
         }
-        // ---- mask, online softmax (rows g and g+8 of the tile)
+        // ---- mask (only strips that reach this pass's rows or the split's end), online softmax
+        const bool need_mask = j0 + STRIP - 1 > c.base || j0 + STRIP > c.k1;     // warp-uniform
         float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
         for (int nt = 0; nt < NTS; ++nt)
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int j = j0 + nt * 8 + 2 * t + (e & 1);
                 const int hh = e >> 1;
-                const float v = (j < c.k1 && j <= horizon[hh]) ? s[nt][e] : -INFINITY;
-                s[nt][e] = v;
-                mx[hh] = fmaxf(mx[hh], v);
+                if (need_mask) {
+                    const int j = j0 + nt * 8 + 2 * t + (e & 1);
+                    if (!(j < c.k1 && j <= horizon[hh])) s[nt][e] = -INFINITY;
+                }
+                mx[hh] = fmaxf(mx[hh], s[nt][e]);
             }
-        float alpha[2];
+        float alpha[2], m_use[2];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
             mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
             const float m_new = fmaxf(m_run[hh], mx[hh]);
-            alpha[hh] = (m_run[hh] == -INFINITY) ? 0.f : exp2f(m_run[hh] - m_new);
+            m_use[hh] = m_new == -INFINITY ? 0.f : m_new;       // keeps (-inf) - (-inf) out of the exponent
+            alpha[hh] = fast_exp2(m_run[hh] - m_use[hh]);       // 0 while nothing has been seen yet
             m_run[hh] = m_new;
             l_run[hh] *= alpha[hh];
         }
@@ -210,14 +223,16 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int hh = e >> 1;
-                const float p = (s[nt][e] == -INFINITY) ? 0.f : exp2f(s[nt][e] - m_run[hh]);
+                const float p = fast_exp2(s[nt][e] - m_use[hh]);  // masked: 2^-inf = 0
                 s[nt][e] = p;
                 l_run[hh] += p;      // per-lane partial; the quad is summed once at the end
             }
+        if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {   // the running max rarely moves
 #pragma unroll
-        for (int i = 0; i < NTO; ++i) {
-            o[i][0] *= alpha[0]; o[i][1] *= alpha[0];
-            o[i][2] *= alpha[1]; o[i][3] *= alpha[1];
+            for (int i = 0; i < NTO; ++i) {
+                o[i][0] *= alpha[0]; o[i][1] *= alpha[0];
+                o[i][2] *= alpha[1]; o[i][3] *= alpha[1];
+            }
         }
         // ---- O += P V over the strip's keys, P split into bf16 hi + lo
 #pragma unroll
@@ -372,10 +387,10 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restr
     }
     __syncthreads();
 
-    // partial result of this CTA, placed behind the strip-merge buffer inside the (then idle) ring
-    float* Fo = reinterpret_cast<float*>(smem + (4 * 16 * HD + 256) * 4);   // [64][HD]
-    float* Fm = Fo + 64 * HD;                                                // [64]
-    float* Fl = Fm + 64;                                                     // [64]
+    // partial result of this CTA: takes over the Q-fragment region once the tile loop is done
+    float* Fo = reinterpret_cast<float*>(smem + SM::kRing);     // [row_tiles*16][HD]
+    float* Fm = Fo + row_tiles * 16 * HD;                        // [row_tiles*16]
+    float* Fl = Fm + row_tiles * 16;                             // [row_tiles*16]
     if (ntiles == 0) {
         cp_async_wait<0>();
         for (int i = threadIdx.x; i < row_tiles * 16; i += kAttnThreads) { Fm[i] = -INFINITY; Fl[i] = 0.f; }
