@@ -315,7 +315,7 @@ constexpr int kAttnSplits = 8;   // = cluster size along x
 
 // grid (8, n_kv_heads * row_groups, n_items), cluster (8,1,1), block 128.
 template <int HD>
-__global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restrict__ q, PassMeta meta,
+__global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __restrict__ q, PassMeta meta,
                                                             const uint16_t* __restrict__ kv_pool, int layer,
                                                             int n_pages, int page_size, int M, int Hq, int Hkv,
                                                             int q_tiles_smem, uint16_t* __restrict__ xf_out) {
@@ -359,6 +359,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restr
     // ---- stage Q (scaled by 1/sqrt(hd)) as split-bf16 A fragments: [tile][k16 step][hi|lo][lane] uint4
     const float scale = rsqrtf((float)HD) * 1.4426950408889634f;   // scores in the log2 domain: p = 2^(s - m)
     uint4* qsm = reinterpret_cast<uint4*>(smem + SM::kRing);
+#pragma unroll 2
     for (int idx = threadIdx.x; idx < row_tiles * (HD / 16) * 32; idx += kAttnThreads) {
         const int lane = idx & 31, ks = (idx >> 5) % (HD / 16), tile = idx / (32 * (HD / 16));
         const int g = lane >> 2, t = lane & 3;
@@ -391,9 +392,10 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restr
     float* Fo = reinterpret_cast<float*>(smem + SM::kRing);     // [row_tiles*16][HD]
     float* Fm = Fo + row_tiles * 16 * HD;                        // [row_tiles*16]
     float* Fl = Fm + row_tiles * 16;                             // [row_tiles*16]
-    if (ntiles == 0) {
+    if (ntiles == 0) {   // empty split: contributes nothing (finite zeros, so the merge can read it unconditionally)
         cp_async_wait<0>();
         for (int i = threadIdx.x; i < row_tiles * 16; i += kAttnThreads) { Fm[i] = -INFINITY; Fl[i] = 0.f; }
+        for (int i = threadIdx.x; i < row_tiles * 16 * HD; i += kAttnThreads) Fo[i] = 0.f;
     } else if (row_tiles == 1) attn_body<HD, 1>(c, smem, Fo, Fm, Fl);
     else if (row_tiles == 2) attn_body<HD, 2>(c, smem, Fo, Fm, Fl);
     else attn_body<HD, 4>(c, smem, Fo, Fm, Fl);
@@ -403,12 +405,19 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restr
     const uint32_t fo_a = smem_u32(Fo), fm_a = smem_u32(Fm), fl_a = smem_u32(Fl);
     const int n_rows = min(row_tiles * 16, c.R - c.rho0);
     const int KSo = (Hq * HD) / 16, NTo = xf_nt(M);
+#pragma unroll 2
     for (int rl = sp; rl < n_rows; rl += kAttnSplits) {
-        float ms[kAttnSplits], ls[kAttnSplits];
+        // all remote reads of a row are issued together: 8 maxima, 8 sums, 8 output values per thread
+        float ms[kAttnSplits], ls[kAttnSplits], ov[HD / kAttnThreads > 0 ? HD / kAttnThreads : 1][kAttnSplits];
 #pragma unroll
         for (int r = 0; r < kAttnSplits; ++r) {
             ms[r] = dsmem_ld_f32(dsmem_addr(fm_a + rl * 4, (uint32_t)r));
             ls[r] = dsmem_ld_f32(dsmem_addr(fl_a + rl * 4, (uint32_t)r));
+#pragma unroll
+            for (int k = 0; k < (HD / kAttnThreads > 0 ? HD / kAttnThreads : 1); ++k) {
+                const int e = threadIdx.x + k * kAttnThreads;
+                ov[k][r] = e < HD ? dsmem_ld_f32(dsmem_addr(fo_a + (uint32_t)(rl * HD + e) * 4, (uint32_t)r)) : 0.f;
+            }
         }
         float m = -INFINITY;
 #pragma unroll
@@ -420,15 +429,15 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const float* __restr
             den += w[r] * ls[r];
         }
         const int rho = c.rho0 + rl, gq = rho / c.rows, r_in = rho % c.rows;
-        for (int e = threadIdx.x; e < HD; e += kAttnThreads) {
-            float ov[kAttnSplits];
 #pragma unroll
-            for (int r = 0; r < kAttnSplits; ++r)
-                ov[r] = w[r] != 0.f ? dsmem_ld_f32(dsmem_addr(fo_a + (uint32_t)(rl * HD + e) * 4, (uint32_t)r)) : 0.f;
-            float num = 0.f;
+        for (int k = 0; k < (HD / kAttnThreads > 0 ? HD / kAttnThreads : 1); ++k) {
+            const int e = threadIdx.x + k * kAttnThreads;
+            if (e < HD) {
+                float num = 0.f;
 #pragma unroll
-            for (int r = 0; r < kAttnSplits; ++r) num += w[r] * ov[r];
-            xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
+                for (int r = 0; r < kAttnSplits; ++r) num += w[r] * ov[k][r];
+                xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
+            }
         }
     }
     cluster_sync_all();   // nobody leaves while its shared memory may still be read

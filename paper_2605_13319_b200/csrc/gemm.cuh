@@ -68,11 +68,13 @@ static inline GemmPlan gemm_plan(int M, int N, int K) {
     p.RB = (N + 127) / 128;
     p.KS = K / 16;
     // One resident wave if possible: every CTA streams from the first microsecond and the next kernel's
-    // CTAs find room to prefetch.  Largest K split that still fits the wave; no split when it cannot fit.
+    // CTAs find room to prefetch.  Largest K split that still fits the wave of a single token block.  The
+    // split depends on (N, K) only, never on M: the order in which a result element is summed is then the
+    // same whether a request is verified alone or inside a batch (bit-identical decisions).
     int best = 1;
     for (int s = 1; s <= kGemmMaxSplit && s <= p.KS; ++s) {
         if (s > 1 && p.KS / s < 2 * kGemmKC) break;
-        if ((long)p.RB * s * p.TB <= kGemmWave) best = s;
+        if ((long)p.RB * s <= kGemmWave) best = s;
     }
     p.S = g_gemm_force_split > 0 && g_gemm_force_split <= kGemmMaxSplit && g_gemm_force_split <= p.KS
               ? g_gemm_force_split : best;
