@@ -368,7 +368,8 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "gemm_wstream_kernel", "achieved": gemm_gbs, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": gemm_gbs / peak,
                      "launches": int(gprof["gemm_launches"]), "share_of_step": gprof["gemm_ms"] / ms,
-                     "traffic": TRAFFIC_PER_LAUNCH},
+                     "algorithmic_bytes_per_launch": gprof["gemm_bytes"] / max(1, gprof["gemm_launches"]),
+                     "traffic": TRAFFIC_7B_K8 if args.workload == "7b-k8" else None},
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline:
@@ -416,9 +417,11 @@ def quick_run(args, ctx, shape, P, k, seed, torch):
     ctx.close()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from one ncu capture
-# (profiles/); None until captured for the current kernel.
-TRAFFIC_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (average over the 129 GEMM
+# launches of a 7b pass), from the ncu capture summarised in profiles/gemm_and_attention_7b_shape_counters.md:
+# taken on a two-layer model of the same shape (same per-layer kernels) and scaled by launch counts.
+# None for other workloads, and to be reset to None when the GEMM kernel changes.
+TRAFFIC_7B_K8 = 102.9e6
 
 
 if __name__ == "__main__":
