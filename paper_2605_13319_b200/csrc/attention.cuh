@@ -313,16 +313,25 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
 
 constexpr int kAttnSplits = 8;   // = cluster size along x
 
-// grid (8, n_kv_heads * row_groups, n_items), cluster (8,1,1), block 128.
+// grid (8 * max clusters per request, n_kv_heads * row_groups, n_items), cluster (8,1,1), block 128.
+// A request whose keys are shared by several clusters (long contexts) takes one more step: every cluster
+// writes its merged partial to global memory and the last cluster to arrive (atomic ticket, nobody waits)
+// merges those.
 template <int HD>
 __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __restrict__ q, PassMeta meta,
                                                             const uint16_t* __restrict__ kv_pool, int layer,
                                                             int n_pages, int page_size, int M, int Hq, int Hkv,
-                                                            int q_tiles_smem, uint16_t* __restrict__ xf_out) {
+                                                            int q_tiles_smem, int row_groups, float* __restrict__ o_part,
+                                                            float* __restrict__ m_part, float* __restrict__ l_part,
+                                                            int* __restrict__ tickets, uint16_t* __restrict__ xf_out) {
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = AttnSmem<HD>;
     pdl_launch_dependents();
-    const int item = blockIdx.z, sp = blockIdx.x;                 // sp == rank in the cluster
+    const int item = blockIdx.z;
+    const int cl = blockIdx.x / kAttnSplits, rank = blockIdx.x % kAttnSplits;   // cluster of this (request, head), rank in it
+    const int ncl = meta.it_nsplit[item];                          // clusters that share this request's keys
+    if (cl >= ncl) return;                                         // taken by a whole cluster or by none
+    const int sp = cl * kAttnSplits + rank;                        // key split of this CTA
     const int kvh = blockIdx.y % Hkv, rg = blockIdx.y / Hkv;
     const int G = Hq / Hkv;
     AttnCtx c;
@@ -400,21 +409,23 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     else if (row_tiles == 2) attn_body<HD, 2>(c, smem, Fo, Fm, Fl);
     else attn_body<HD, 4>(c, smem, Fo, Fm, Fl);
 
-    // ---- merge the 8 splits over distributed shared memory; rank r owns rows r, r+8, ... of the row group
+    // ---- merge the cluster's 8 splits over distributed shared memory; rank r owns rows r, r+8, ... of the group
     cluster_sync_all();
+    constexpr int EPT = HD / kAttnThreads > 0 ? HD / kAttnThreads : 1;   // output columns per thread
     const uint32_t fo_a = smem_u32(Fo), fm_a = smem_u32(Fm), fl_a = smem_u32(Fl);
     const int n_rows = min(row_tiles * 16, c.R - c.rho0);
     const int KSo = (Hq * HD) / 16, NTo = xf_nt(M);
+    const size_t slot0 = (size_t)meta.it_part0[item] + ((size_t)kvh * c.R + c.rho0) * ncl;   // + rl*ncl + cluster
 #pragma unroll 2
-    for (int rl = sp; rl < n_rows; rl += kAttnSplits) {
+    for (int rl = rank; rl < n_rows; rl += kAttnSplits) {
         // all remote reads of a row are issued together: 8 maxima, 8 sums, 8 output values per thread
-        float ms[kAttnSplits], ls[kAttnSplits], ov[HD / kAttnThreads > 0 ? HD / kAttnThreads : 1][kAttnSplits];
+        float ms[kAttnSplits], ls[kAttnSplits], ov[EPT][kAttnSplits];
 #pragma unroll
         for (int r = 0; r < kAttnSplits; ++r) {
             ms[r] = dsmem_ld_f32(dsmem_addr(fm_a + rl * 4, (uint32_t)r));
             ls[r] = dsmem_ld_f32(dsmem_addr(fl_a + rl * 4, (uint32_t)r));
 #pragma unroll
-            for (int k = 0; k < (HD / kAttnThreads > 0 ? HD / kAttnThreads : 1); ++k) {
+            for (int k = 0; k < EPT; ++k) {
                 const int e = threadIdx.x + k * kAttnThreads;
                 ov[k][r] = e < HD ? dsmem_ld_f32(dsmem_addr(fo_a + (uint32_t)(rl * HD + e) * 4, (uint32_t)r)) : 0.f;
             }
@@ -430,17 +441,72 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
         }
         const int rho = c.rho0 + rl, gq = rho / c.rows, r_in = rho % c.rows;
 #pragma unroll
-        for (int k = 0; k < (HD / kAttnThreads > 0 ? HD / kAttnThreads : 1); ++k) {
+        for (int k = 0; k < EPT; ++k) {
             const int e = threadIdx.x + k * kAttnThreads;
             if (e < HD) {
                 float num = 0.f;
 #pragma unroll
                 for (int r = 0; r < kAttnSplits; ++r) num += w[r] * ov[k][r];
+                if (ncl == 1) xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
+                else o_part[(slot0 + (size_t)rl * ncl + cl) * HD + e] = num;     // un-normalised, with (m, den)
+            }
+        }
+        if (ncl > 1 && threadIdx.x == 0) {
+            m_part[slot0 + (size_t)rl * ncl + cl] = m;
+            l_part[slot0 + (size_t)rl * ncl + cl] = den;
+        }
+    }
+    __shared__ int s_last;
+    if (ncl > 1) __threadfence();
+    cluster_sync_all();   // nobody leaves while its shared memory may still be read; partials are published
+    if (ncl == 1) return;
+    // ---- several clusters share the keys: the last one to arrive merges their partials
+    if (rank == 0 && threadIdx.x == 0) {
+        int* ticket = tickets + ((size_t)item * Hkv + kvh) * row_groups + rg;
+        const int t = atomicAdd(ticket, 1);
+        const int last = (t == ncl - 1);
+        if (last) *ticket = 0;                                   // self-cleaning: ready for the next launch
+        const uint32_t fa = smem_u32(&s_last);
+        for (int r = 0; r < kAttnSplits; ++r) dsmem_st_f32(dsmem_addr(fa, (uint32_t)r), __int_as_float(last));
+    }
+    cluster_sync_all();
+    if (!s_last) return;
+    __threadfence();
+    for (int rl = rank; rl < n_rows; rl += kAttnSplits) {
+        float ms[kMaxSplits / kAttnSplits], ls[kMaxSplits / kAttnSplits], ov[EPT][kMaxSplits / kAttnSplits];
+#pragma unroll
+        for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) {
+            const bool on = j < ncl;
+            const size_t sl = slot0 + (size_t)rl * ncl + j;
+            ms[j] = on ? __ldcg(m_part + sl) : -INFINITY;
+            ls[j] = on ? __ldcg(l_part + sl) : 0.f;
+#pragma unroll
+            for (int k = 0; k < EPT; ++k) {
+                const int e = threadIdx.x + k * kAttnThreads;
+                ov[k][j] = (on && e < HD) ? __ldcg(o_part + sl * HD + e) : 0.f;
+            }
+        }
+        float m = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) m = fmaxf(m, ms[j]);
+        float den = 0.f, w[kMaxSplits / kAttnSplits];
+#pragma unroll
+        for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) {
+            w[j] = (ms[j] == -INFINITY) ? 0.f : exp2f(ms[j] - m);
+            den += w[j] * ls[j];
+        }
+        const int rho = c.rho0 + rl, gq = rho / c.rows, r_in = rho % c.rows;
+#pragma unroll
+        for (int k = 0; k < EPT; ++k) {
+            const int e = threadIdx.x + k * kAttnThreads;
+            if (e < HD) {
+                float num = 0.f;
+#pragma unroll
+                for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) num += w[j] * ov[k][j];
                 xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
             }
         }
     }
-    cluster_sync_all();   // nobody leaves while its shared memory may still be read
 }
 
 static inline size_t attn_smem_bytes(int hd, int row_tiles) {

@@ -85,7 +85,7 @@ Derived derive(const pipesd_model_cfg& c) {
 }
 
 struct WsLayout {
-    size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, cs, sn, kvoff, stats, results, meta,
+    size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, tickets, cs, sn, kvoff, stats, results, meta,
         block_tab, qstage, total;
 };
 
@@ -106,10 +106,11 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     const size_t nssq = (c.d_model + 127) / 128;
     w.ssqA = take(4 * nssq * M);
     w.ssqB = take(4 * nssq * M);
-    const size_t slots = M * c.n_q_heads * kMaxSplits;
+    const size_t slots = M * c.n_q_heads * (kMaxSplits / kAttnSplits);   // one per (row, head, cluster)
     w.o_part = take(4 * slots * c.head_dim);
     w.m_part = take(4 * slots);
     w.l_part = take(4 * slots);
+    w.tickets = take(4 * M * c.n_q_heads);   // one per (item, KV head, row group); zero between launches
     w.cs = take(4 * M * (c.head_dim / 2));
     w.sn = take(4 * M * (c.head_dim / 2));
     w.kvoff = take(8 * M);
@@ -319,17 +320,18 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     auto I = [&](size_t off) { return reinterpret_cast<int32_t*>(hm + off); };
     float* hu = reinterpret_cast<float*>(hm + ml.u);
     RejectItem* hr = reinterpret_cast<RejectItem*>(hm + ml.rej);
-    // split policy: aim at two waves of CTAs over all (item, head, split) triples
-    int target = std::max(1, (4 * 148 + n_items * c.n_kv_heads - 1) / (n_items * c.n_kv_heads));
     int row = 0, part0 = 0, max_nsplit = 1, u0 = 0;
     for (int i = 0; i < n_items; ++i) {
         const ItemDesc& it = items[i];
         const Request& r = ctx->reqs[it.slot];
         const int total = r.len + it.rows;
-        // eight splits (one per CTA of the attention cluster), whole pages each
-        int chunk = (total + kAttnSplits - 1) / kAttnSplits;
+        // one cluster of eight key splits per (request, KV head, row group); a long context gets one more
+        // cluster per 2048 keys (up to four).  The count depends on the request alone, never on what else
+        // is in the batch, so that a request's summation order is the same in every batch.
+        const int ncl = std::max(1, std::min(kMaxSplits / kAttnSplits, total / 2048));
+        int chunk = (total + kAttnSplits * ncl - 1) / (kAttnSplits * ncl);
         chunk = (chunk + c.page_size - 1) / c.page_size * c.page_size;
-        int nsplit = (total + chunk - 1) / chunk;
+        int nsplit = ncl;   // stored per item: clusters sharing its keys
         I(ml.it_slot)[i] = it.slot;
         I(ml.it_row0)[i] = row;
         I(ml.it_rows)[i] = it.rows;
@@ -406,15 +408,16 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             int rc_ = launch_gemm(ctx, kQkvRope, a, d);
             if (rc_) return rc_;
         }
-        dim3 ag(kAttnSplits, Hkv * row_groups, n_items);
+        dim3 ag(kAttnSplits * max_nsplit, Hkv * row_groups, n_items);
+        int* tickets = ctx->W<int>(ctx->ws.tickets);
         if (hd == 128)
             CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  (uint16_t*)xf_attn));
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn));
         else
             CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  (uint16_t*)xf_attn));
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn));
         {   // x += W_o . attn; xf_h = x * ffn gain; ssqB
             GemmArgs a = base;
             a.W = lw.o.packed; a.xf = (const uint4*)xf_attn; a.N = d; a.ssq_in = nullptr;
@@ -537,8 +540,13 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     if (cudaHostAlloc((void**)&ctx->h_results, sizeof(RejectOut) * dv.max_items + 16, cudaHostAllocDefault) != cudaSuccess)
         return bail(PIPESD_E_CUDA);
 
-    // ---- repack the weights into the library's own layout
     cudaStream_t st = ctx->st;
+    // the device error word and the attention tickets start at zero (the tickets reset themselves after use)
+    if (cudaMemsetAsync(ctx->err_word(), 0, 4, st) != cudaSuccess) return bail(PIPESD_E_CUDA);
+    if (cudaMemsetAsync(ctx->wsp + ctx->ws.tickets, 0, 4 * (size_t)c.max_rows * c.n_q_heads, st) != cudaSuccess)
+        return bail(PIPESD_E_CUDA);
+
+    // ---- repack the weights into the library's own layout
     char* wp = (char*)mem->weights;
     size_t off = 0;
     auto take = [&](size_t bytes) { char* p = wp + off; off += align_up(bytes); return p; };
@@ -609,6 +617,7 @@ int32_t pipesd_ctx_sync(pipesd_ctx* ctx) {
             ctx->pend_dst = nullptr;
             ctx->pend_n = 0;
             cudaMemsetAsync(ctx->err_word(), 0, 4, ctx->st);
+            cudaMemsetAsync(ctx->wsp + ctx->ws.tickets, 0, 4 * (size_t)ctx->cfg.max_rows * ctx->cfg.n_q_heads, ctx->st);
             return fail(ctx, PIPESD_E_CUDA, "a device-side wait timed out (kernel error word set)");
         }
         for (int i = 0; i < ctx->pend_n; ++i) {
