@@ -81,6 +81,7 @@ _SIGNATURES = {
     "pipesd_debug_write_kv": (i32, [vp, i32, i32, i32, i32, vp, vp]),
     "pipesd_reject_from_logits": (i32, [vp, i32, i32, vp, vp, vp, vp, ctypes.POINTER(VerifyResult)]),
     "pipesd_debug_set_len": (i32, [vp, i32, i32]),
+    "pipesd_debug_set_engine": (i32, [vp, i32]),
     "pipesd_profile_enable": (i32, [vp, i32]),
     "pipesd_profile_read": (i32, [vp, ctypes.POINTER(ProfileInfo)]),
     "pipesd_gemm_packed_bytes": (u64, [i32, i32]),
@@ -274,6 +275,10 @@ class Context:
         v = np.ascontiguousarray(v_bf16, np.uint16)
         self._check(lib().pipesd_debug_write_kv(self._h, req, layer, pos0, k.shape[0], _np_ptr(k), _np_ptr(v)),
                     "pipesd_debug_write_kv")
+
+    def debug_set_engine(self, engine: int):
+        """0: persistent kernel for passes of <= 32 rows (default); 1: tiled kernels for every pass."""
+        self._check(lib().pipesd_debug_set_engine(self._h, engine), "pipesd_debug_set_engine")
 
     def debug_set_len(self, req: int, new_len: int):
         self._check(lib().pipesd_debug_set_len(self._h, req, new_len), "pipesd_debug_set_len")

@@ -16,6 +16,7 @@
 #include "common.cuh"
 #include "gemm.cuh"
 #include "layers.cuh"
+#include "mega.cuh"
 #include "reject.cuh"
 
 using namespace pipesd;
@@ -86,7 +87,8 @@ Derived derive(const pipesd_model_cfg& c) {
 
 struct WsLayout {
     size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, tickets, cs, sn, kvoff, stats, results, meta,
-        block_tab, qstage, total;
+        block_tab, qstage, mega_phases, mega_ctr, mega_scratch, total;
+    size_t mega_ctr_ints;
 };
 
 WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
@@ -119,6 +121,15 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     w.meta = take(meta_layout(c.max_rows, d.max_items).total);
     w.block_tab = take(4 * (size_t)c.max_requests * d.max_pages);
     w.qstage = take(4 * M * c.vocab);
+    // persistent layer-stack kernel: phase table, counters (finished units per phase | started CTAs per launch |
+    // one ticket per 256-row unit), accumulator fragments of units shared by several CTAs
+    const size_t n_phases = 4 * (size_t)c.n_layers + 1;
+    auto units = [](size_t N) { return ((N + 127) / 128 + 1) / 2; };
+    const size_t n_tickets = (size_t)c.n_layers * (units(d.Nqkv) + 2 * units(c.d_model) + units(2 * (size_t)c.d_ffn)) + units(c.vocab);
+    w.mega_phases = take(sizeof(MegaPhase) * n_phases);
+    w.mega_ctr_ints = n_phases + (size_t)c.n_layers + 2 + n_tickets;
+    w.mega_ctr = take(4 * w.mega_ctr_ints);
+    w.mega_scratch = take((size_t)kMegaMaxCtas * 2 * 8 * kMegaConsumers * sizeof(float4));
     w.total = o;
     return w;
 }
@@ -193,7 +204,11 @@ struct pipesd_ctx {
     RejectOut* h_results = nullptr;
     pipesd_verify_result* pend_dst = nullptr;
     int pend_n = 0;
+    bool pend_check = false;   // a prefill is in flight whose device error word has not been looked at yet
     int last_rows = 0;
+    int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
+    int engine = 1;         // 0: persistent kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only
+    std::vector<MegaPhase> phases;
     std::string err;
     // launch accounting
     int64_t n_launch = 0, n_gemm = 0;
@@ -376,6 +391,10 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     const int hd = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads, d = c.d_model, F = c.d_ffn;
     const int n_ssq = (d + 127) / 128;
 
+    // Passes of at most 32 rows (one token block) run their GEMMs in the persistent kernel, whose counters
+    // start every pass at zero.
+    const bool use_mega = ctx->engine == 0 && M <= 32;
+    if (use_mega) CU(cudaMemsetAsync(ctx->wsp + ctx->ws.mega_ctr, 0, 4 * ctx->ws.mega_ctr_ints, st));
     // Every kernel of the chain is launched with programmatic stream serialisation: it may start while its
     // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
     {
@@ -397,6 +416,73 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     base.eps = c.rms_eps;
     base.d_in = d;
     base.n_ssq = n_ssq;
+    auto launch_attn = [&](int l) -> int {
+        dim3 ag(kAttnSplits * max_nsplit, Hkv * row_groups, n_items);
+        int* tickets = ctx->W<int>(ctx->ws.tickets);
+        if (hd == 128)
+            CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
+                                  meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn));
+        else
+            CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
+                                  meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn));
+        ctx->n_launch += 1;
+        return PIPESD_OK;
+    };
+    if (use_mega) {
+        // Persistent kernel: [QKV 0] attn [O, gate/up, down, QKV 1] attn ... [O, gate/up, down, LM head]
+        MegaArgs ma = {};
+        ma.phases = ctx->W<MegaPhase>(ctx->ws.mega_phases);
+        ma.M = M;
+        int* ctr = ctx->W<int>(ctx->ws.mega_ctr);
+        const int n_phases = (int)ctx->phases.size();
+        ma.done = ctr;
+        ma.tickets = ctr + n_phases + c.n_layers + 2;
+        ma.scratch = ctx->W<float4>(ctx->ws.mega_scratch);
+        ma.err = ctx->err_word();
+        ma.eps = c.rms_eps;
+        ma.d_in = d;
+        ma.q_out = qbuf; ma.kv_pool = ctx->kv_pool; ma.cs = cs; ma.sn = sn;
+        ma.row_kvoff = ctx->W<long long>(ctx->ws.kvoff);
+        ma.Hq = Hq; ma.Hkv = Hkv; ma.hd = hd; ma.n_pages = c.n_pages; ma.page_size = c.page_size;
+        const int NT = xf_nt(M);
+        auto launch_mega = [&](int launch_idx, int p0, int p1) -> int {
+            MegaArgs a = ma;
+            a.p0 = p0; a.p1 = p1;
+            a.launch_idx = launch_idx;
+            a.arrived = ctr + n_phases + launch_idx;
+            cudaEvent_t e1 = nullptr;
+            if (ctx->time_gemms) {
+                if (ctx->prof_used + 2 > ctx->prof_ev.size())
+                    for (int i = 0; i < 2; ++i) {
+                        cudaEvent_t e;
+                        CU(cudaEventCreate(&e));
+                        ctx->prof_ev.push_back(e);
+                    }
+                CU(cudaEventRecord(ctx->prof_ev[ctx->prof_used], st));
+                e1 = ctx->prof_ev[ctx->prof_used + 1];
+                ctx->prof_used += 2;
+            }
+            CU(mega_launch(NT, a, ctx->mega_grid, st));
+            if (e1) CU(cudaEventRecord(e1, st));
+            ctx->n_launch += 1;
+            ctx->n_gemm += 1;
+            for (int p = p0; p < p1; ++p) {
+                const MegaPhase& ph = ctx->phases[p];
+                ctx->gemm_bytes += 2.0 * ph.N * ph.KS * 16 + 4.0 * M * ph.KS * 16 + 4.0 * M * ph.N;
+            }
+            return PIPESD_OK;
+        };
+        int rc_ = launch_mega(0, 0, 1);
+        if (rc_) return rc_;
+        for (int l = 0; l < c.n_layers; ++l) {
+            if ((rc_ = launch_attn(l))) return rc_;
+            const bool last = l + 1 == c.n_layers;
+            const int p1 = last ? (want_logits ? 4 * l + 5 : 4 * l + 4) : 4 * l + 5;
+            if ((rc_ = launch_mega(l + 1, 4 * l + 1, p1))) return rc_;
+        }
+    } else
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& lw = ctx->layers[l];
         {   // q, k, v = W_qkv . norm(x); RoPE; K/V appended to the pages
@@ -408,16 +494,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             int rc_ = launch_gemm(ctx, kQkvRope, a, d);
             if (rc_) return rc_;
         }
-        dim3 ag(kAttnSplits * max_nsplit, Hkv * row_groups, n_items);
-        int* tickets = ctx->W<int>(ctx->ws.tickets);
-        if (hd == 128)
-            CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
-                                  meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn));
-        else
-            CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
-                                  meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn));
+        { int rc_ = launch_attn(l); if (rc_) return rc_; }
         {   // x += W_o . attn; xf_h = x * ffn gain; ssqB
             GemmArgs a = base;
             a.W = lw.o.packed; a.xf = (const uint4*)xf_attn; a.N = d; a.ssq_in = nullptr;
@@ -441,13 +518,12 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             int rc_ = launch_gemm(ctx, kResid, a, F);
             if (rc_) return rc_;
         }
-        ctx->n_launch += 1;   // attention
     }
     if (want_logits) {
         ctx->n_launch += 1 + (want_reject ? 1 : 0);   // row_stats, accept_sample
         float* logits = ctx->W<float>(ctx->ws.logits);
         RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
-        {
+        if (!use_mega) {
             GemmArgs a = base;
             a.W = ctx->lm.packed; a.xf = (const uint4*)xf_h; a.N = c.vocab; a.ssq_in = ssqA; a.out = logits;
             int rc_ = launch_gemm(ctx, kPlain, a, d);
@@ -587,6 +663,65 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     cudaMemcpyAsync(ctx->final_norm, w->final_norm, 4 * (size_t)c.d_model, cudaMemcpyDeviceToDevice, st);
     if (cudaGetLastError() != cudaSuccess) return bail(PIPESD_E_CUDA);
 
+    // ---- phase table of the persistent kernel: QKV(0) | O, gate/up, down, QKV(l+1) per layer | ... | LM head
+    {
+        int n_sm = 0;
+        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, c.device) != cudaSuccess || n_sm < 1)
+            return bail(PIPESD_E_CUDA);
+        ctx->mega_grid = std::min(n_sm, kMegaMaxCtas);
+        if (mega_init_attrs() != cudaSuccess) return bail(PIPESD_E_CUDA);
+        const int d = c.d_model, F = c.d_ffn;
+        const int n_ssq = ((d + 127) / 128 + 1) / 2;      // 256-row units of the residual stream
+        uint32_t* xf_h = ctx->W<uint32_t>(ctx->ws.xf_h);
+        uint32_t* xf_attn = ctx->W<uint32_t>(ctx->ws.xf_attn);
+        uint32_t* xf_act = ctx->W<uint32_t>(ctx->ws.xf_act);
+        float* ssqA = ctx->W<float>(ctx->ws.ssqA);
+        float* ssqB = ctx->W<float>(ctx->ws.ssqB);
+        float* x = ctx->W<float>(ctx->ws.x);
+        int ticket0 = 0;
+        auto add = [&](const GemmW& g, int mode, const uint32_t* xf) -> MegaPhase& {
+            MegaPhase ph = {};
+            ph.W = g.packed;
+            ph.xf = (const uint4*)xf;
+            ph.mode = mode;
+            mega_phase_geometry(ph, g.N, g.K);
+            ph.ticket0 = ticket0;
+            ticket0 += ph.UB;
+            ctx->phases.push_back(ph);
+            return ctx->phases.back();
+        };
+        for (int l = 0; l < c.n_layers; ++l) {
+            const LayerW& lw = ctx->layers[l];
+            {
+                MegaPhase& ph = add(lw.qkv, kQkvRope, xf_h);
+                ph.ssq_in = ssqA; ph.n_ssq = n_ssq; ph.layer = l;
+            }
+            {
+                MegaPhase& ph = add(lw.o, kResid, xf_attn);
+                ph.x = x; ph.xf_out = (uint16_t*)xf_h; ph.gain_next = lw.n2; ph.ssq_out = ssqB;
+            }
+            {
+                MegaPhase& ph = add(lw.gu, kSwiglu, xf_h);
+                ph.ssq_in = ssqB; ph.n_ssq = n_ssq; ph.xf_out = (uint16_t*)xf_act;
+            }
+            {
+                MegaPhase& ph = add(lw.dn, kResid, xf_act);
+                ph.x = x; ph.xf_out = (uint16_t*)xf_h;
+                ph.gain_next = l + 1 < c.n_layers ? ctx->layers[l + 1].n1 : ctx->final_norm;
+                ph.ssq_out = ssqA;
+            }
+        }
+        {
+            MegaPhase& ph = add(ctx->lm, kPlain, xf_h);
+            ph.ssq_in = ssqA; ph.n_ssq = n_ssq; ph.out = ctx->W<float>(ctx->ws.logits);
+        }
+        if ((size_t)ticket0 + ctx->phases.size() + c.n_layers + 2 > ctx->ws.mega_ctr_ints) return bail(PIPESD_E_INVALID);
+        if (cudaMemcpyAsync(ctx->wsp + ctx->ws.mega_phases, ctx->phases.data(), sizeof(MegaPhase) * ctx->phases.size(),
+                            cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return bail(PIPESD_E_CUDA);
+        if (cudaStreamSynchronize(st) != cudaSuccess) return bail(PIPESD_E_CUDA);   // the table is read from pageable memory
+    }
+
     ctx->reqs.resize(c.max_requests);
     ctx->free_pages.resize(c.n_pages);
     for (int i = 0; i < c.n_pages; ++i) ctx->free_pages[i] = c.n_pages - 1 - i;
@@ -610,7 +745,8 @@ int32_t pipesd_ctx_destroy(pipesd_ctx* ctx) {
 int32_t pipesd_ctx_sync(pipesd_ctx* ctx) {
     if (!ctx) return PIPESD_E_INVALID;
     CU(cudaStreamSynchronize(ctx->st));
-    if (ctx->pend_dst) {
+    if (ctx->pend_dst || ctx->pend_check) {
+        ctx->pend_check = false;
         const int dev_err = *reinterpret_cast<const int*>(ctx->h_results + ctx->dv.max_items);
         if (dev_err) {   // a bounded device-side wait gave up: the results of this call are void
             for (int i = 0; i < ctx->pend_n; ++i) ctx->pend_dst[i].status = PIPESD_E_CUDA;
@@ -618,7 +754,9 @@ int32_t pipesd_ctx_sync(pipesd_ctx* ctx) {
             ctx->pend_n = 0;
             cudaMemsetAsync(ctx->err_word(), 0, 4, ctx->st);
             cudaMemsetAsync(ctx->wsp + ctx->ws.tickets, 0, 4 * (size_t)ctx->cfg.max_rows * ctx->cfg.n_q_heads, ctx->st);
-            return fail(ctx, PIPESD_E_CUDA, "a device-side wait timed out (kernel error word set)");
+            char msg[96];
+            snprintf(msg, sizeof msg, "a device-side wait timed out (kernel error word %d)", dev_err);
+            return fail(ctx, PIPESD_E_CUDA, msg);
         }
         for (int i = 0; i < ctx->pend_n; ++i) {
             ctx->pend_dst[i].n_accepted = ctx->h_results[i].n_accepted;
@@ -682,10 +820,16 @@ int32_t pipesd_prefill(pipesd_ctx* ctx, int32_t req, const int32_t* tokens, int3
         rc = run_pass(ctx, items, last && last_logits, false);
         if (rc != PIPESD_OK) return rc;
         r.len += rows;
+        if (last) {   // the device error word travels back with the (unused) result slots; pipesd_ctx_sync reads it
+            CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results),
+                               sizeof(RejectOut) * ctx->dv.max_items + 4, cudaMemcpyDeviceToHost, ctx->st));
+            ctx->pend_check = true;
+        }
         if (last && last_logits) {
             CU(cudaMemcpyAsync(last_logits, ctx->W<float>(ctx->ws.logits) + (size_t)(rows - 1) * ctx->cfg.vocab,
                                4 * (size_t)ctx->cfg.vocab, cudaMemcpyDeviceToHost, ctx->st));
-            CU(cudaStreamSynchronize(ctx->st));
+            rc = pipesd_ctx_sync(ctx);
+            if (rc != PIPESD_OK) return rc;
         }
     }
     return PIPESD_OK;
@@ -696,7 +840,7 @@ int32_t pipesd_verify(pipesd_ctx* ctx, int32_t n_req, const pipesd_verify_item* 
     if (!ctx || !items_in || !results || n_req < 1 || n_req > ctx->dv.max_items)
         return fail(ctx, PIPESD_E_INVALID, "pipesd_verify: arguments");
     const pipesd_model_cfg& c = ctx->cfg;
-    if (ctx->pend_dst) {  // deliver the previous call's results before their staging is reused
+    if (ctx->pend_dst || ctx->pend_check) {  // deliver the previous call's results before their staging is reused
         int rc = pipesd_ctx_sync(ctx);
         if (rc != PIPESD_OK) return rc;
     }
@@ -886,6 +1030,18 @@ int32_t pipesd_debug_set_len(pipesd_ctx* ctx, int32_t req, int32_t new_len) {
     if (new_len < 0 || new_len > r.len) return fail(ctx, PIPESD_E_RANGE, "set_len can only truncate");
     r.len = new_len;
     shrink_pages(ctx, r, r.len);
+    return PIPESD_OK;
+}
+
+#ifdef PIPESD_MEGA_TRACE
+int32_t pipesd_debug_mega_trace(unsigned long long* dst, int32_t n) {
+    return cudaMemcpyFromSymbol(dst, g_mega_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
+}
+#endif
+
+int32_t pipesd_debug_set_engine(pipesd_ctx* ctx, int32_t engine) {
+    if (!ctx || engine < 0 || engine > 1) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine");
+    ctx->engine = engine;
     return PIPESD_OK;
 }
 
