@@ -323,7 +323,8 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
                                                             int n_pages, int page_size, int M, int Hq, int Hkv,
                                                             int q_tiles_smem, int row_groups, float* __restrict__ o_part,
                                                             float* __restrict__ m_part, float* __restrict__ l_part,
-                                                            int* __restrict__ tickets, uint16_t* __restrict__ xf_out) {
+                                                            int* __restrict__ tickets, uint16_t* __restrict__ xf_out,
+                                                            int xu_layout) {
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = AttnSmem<HD>;
     pdl_launch_dependents();
@@ -447,7 +448,10 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
                 float num = 0.f;
 #pragma unroll
                 for (int r = 0; r < kAttnSplits; ++r) num += w[r] * ov[k][r];
-                if (ncl == 1) xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
+                if (ncl == 1) {
+                    if (xu_layout) xu_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, NTo);
+                    else xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
+                }
                 else o_part[(slot0 + (size_t)rl * ncl + cl) * HD + e] = num;     // un-normalised, with (m, den)
             }
         }
@@ -503,7 +507,8 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
                 float num = 0.f;
 #pragma unroll
                 for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) num += w[j] * ov[k][j];
-                xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
+                if (xu_layout) xu_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, NTo);
+                else xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
             }
         }
     }

@@ -179,6 +179,23 @@ __device__ __forceinline__ void xf_store_one(uint16_t* xf, int tok, int k, float
     xf[slot * 8 + 4 + half * 2 + (kk & 1)] = l;
 }
 
+// ---- "xu" activation arrays: the token-major B operand of tcgen05.mma, in global memory ------------------
+// One token block of at most 32 tokens (NT = tiles of 8 tokens).  Per k16 step NT*512 bytes, cut into 16-byte
+// pieces = 8 consecutive tokens of one k: piece (k half kg, token group ng, k row) at ((kg*2NT + ng)*8 + row)*16,
+// token groups 0..NT-1 hold the bf16 hi terms, NT..2NT-1 the lo terms.  A chunk of consecutive k16 steps is one
+// contiguous run, copied into shared memory as it is.
+__host__ __device__ __forceinline__ size_t xu_piece_offset(int k, int ng, int NT) {
+    return (size_t)(k >> 4) * NT * 512 + (size_t)(((((k >> 3) & 1) * 2 * NT + ng) * 8 + (k & 7)) * 16);
+}
+// Stores one element (its hi and lo terms) of an xu array.
+__device__ __forceinline__ void xu_store_one(uint16_t* xu, int tok, int k, float v, int NT) {
+    uint16_t h, l;
+    split_bf16(v, h, l);
+    unsigned char* b = reinterpret_cast<unsigned char*>(xu);
+    *reinterpret_cast<uint16_t*>(b + xu_piece_offset(k, tok >> 3, NT) + (tok & 7) * 2) = h;
+    *reinterpret_cast<uint16_t*>(b + xu_piece_offset(k, NT + (tok >> 3), NT) + (tok & 7) * 2) = l;
+}
+
 // ---- thread-block clusters: barrier and distributed shared memory --------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;

@@ -16,7 +16,7 @@
 #include "common.cuh"
 #include "gemm.cuh"
 #include "layers.cuh"
-#include "mega.cuh"
+#include "mega_tc.cuh"
 #include "reject.cuh"
 
 using namespace pipesd;
@@ -33,7 +33,8 @@ struct Request {
 };
 
 struct GemmW {
-    uint4* packed = nullptr;
+    uint4* packed = nullptr;     // MMA-fragment order (tiled kernels; only packed when max_rows > 32)
+    uint4* packed_u = nullptr;   // tensor-core operand order (persistent kernel)
     int N = 0, K = 0;
 };
 
@@ -129,19 +130,24 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     w.mega_phases = take(sizeof(MegaPhase) * n_phases);
     w.mega_ctr_ints = n_phases + (size_t)c.n_layers + 2 + n_tickets;
     w.mega_ctr = take(4 * w.mega_ctr_ints);
-    w.mega_scratch = take((size_t)kMegaMaxCtas * 2 * 8 * kMegaConsumers * sizeof(float4));
+    w.mega_scratch = take((size_t)kMegaMaxCtas * 8 * kMegaEpiThreads * sizeof(float4));
     w.total = o;
     return w;
 }
 
 size_t packed_bytes(int N, int K) { return align_up(gemm_packed_bytes(N, K)); }
 
+// Passes of more than 32 rows run on the tiled kernels, which read the weights in MMA-fragment order; a context
+// that admits such passes keeps a second copy of the matrices in that order.
+bool needs_tiled(const pipesd_model_cfg& c) { return c.max_rows > 32; }
+
 size_t weights_bytes(const pipesd_model_cfg& c, const Derived& d) {
-    size_t per_layer = packed_bytes(d.Nqkv, c.d_model) + packed_bytes(c.d_model, d.qd) +
-                       packed_bytes(2 * c.d_ffn, c.d_model) + packed_bytes(c.d_model, c.d_ffn) +
+    const size_t copies = needs_tiled(c) ? 2 : 1;
+    size_t per_layer = copies * (packed_bytes(d.Nqkv, c.d_model) + packed_bytes(c.d_model, d.qd) +
+                                 packed_bytes(2 * c.d_ffn, c.d_model) + packed_bytes(c.d_model, c.d_ffn)) +
                        2 * align_up(4 * (size_t)c.d_model);
     return (size_t)c.n_layers * per_layer + align_up((size_t)c.vocab * c.d_model * 2) +
-           packed_bytes(c.vocab, c.d_model) + align_up(4 * (size_t)c.d_model);
+           copies * packed_bytes(c.vocab, c.d_model) + align_up(4 * (size_t)c.d_model);
 }
 
 size_t kv_bytes(const pipesd_model_cfg& c) {
@@ -207,7 +213,7 @@ struct pipesd_ctx {
     bool pend_check = false;   // a prefill is in flight whose device error word has not been looked at yet
     int last_rows = 0;
     int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
-    int engine = 1;         // 0: persistent kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only
+    int engine = 0;         // 0: persistent kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only
     std::vector<MegaPhase> phases;
     std::string err;
     // launch accounting
@@ -393,7 +399,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
 
     // Passes of at most 32 rows (one token block) run their GEMMs in the persistent kernel, whose counters
     // start every pass at zero.
-    const bool use_mega = ctx->engine == 0 && M <= 32;
+    const bool use_mega = (ctx->engine == 0 && M <= 32) || !needs_tiled(c);
     if (use_mega) CU(cudaMemsetAsync(ctx->wsp + ctx->ws.mega_ctr, 0, 4 * ctx->ws.mega_ctr_ints, st));
     // Every kernel of the chain is launched with programmatic stream serialisation: it may start while its
     // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
@@ -402,7 +408,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         CU(launch_pdl(rope_table_kernel, dim3((n + 127) / 128), dim3(128), 0, st, meta, M, hd, log((double)c.rope_base),
                       cs, sn, ctx->W<long long>(ctx->ws.kvoff), c.n_pages, Hkv, c.page_size));
         CU(launch_pdl(embed_kernel, dim3(M), dim3(kEmbedThreads), 0, st, x, (const uint16_t*)ctx->emb, meta.row_tok, M,
-                      (const float*)ctx->layers[0].n1, d, xf_h, ssqA, n_ssq));
+                      (const float*)ctx->layers[0].n1, d, xf_h, ssqA, n_ssq, use_mega ? 1 : 0));
         ctx->n_launch += 2;
     }
     int max_item_rows = 1;
@@ -422,11 +428,11 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         if (hd == 128)
             CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn));
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0));
         else
             CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn));
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0));
         ctx->n_launch += 1;
         return PIPESD_OK;
     };
@@ -626,8 +632,8 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     char* wp = (char*)mem->weights;
     size_t off = 0;
     auto take = [&](size_t bytes) { char* p = wp + off; off += align_up(bytes); return p; };
+    const bool tiled = needs_tiled(c);
     auto pack = [&](GemmW& g, int N, int K, int mode, std::initializer_list<std::pair<const void*, int>> srcs) {
-        g.packed = (uint4*)take(gemm_packed_bytes(N, K));
         g.N = N;
         g.K = K;
         PackSrc ps = {};
@@ -637,7 +643,12 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         for (auto& s : srcs) { ps.w[i] = (const uint16_t*)s.first; ps.rows[i] = s.second; ++i; }
         size_t total = (size_t)((N + 127) / 128 * 8) * (K / 16) * 32;
         int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
-        gemm_pack_kernel<<<blocks, 256, 0, st>>>(ps, g.packed, N, K);
+        g.packed_u = (uint4*)take(gemm_packed_bytes(N, K));
+        gemm_pack_umma_kernel<<<blocks, 256, 0, st>>>(ps, g.packed_u, N, K);
+        if (tiled) {
+            g.packed = (uint4*)take(gemm_packed_bytes(N, K));
+            gemm_pack_kernel<<<blocks, 256, 0, st>>>(ps, g.packed, N, K);
+        }
     };
     ctx->emb = (uint16_t*)take((size_t)c.vocab * c.d_model * 2);
     if (cudaMemcpyAsync(ctx->emb, w->tok_emb, (size_t)c.vocab * c.d_model * 2, cudaMemcpyDeviceToDevice, st) !=
@@ -681,7 +692,7 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         int ticket0 = 0;
         auto add = [&](const GemmW& g, int mode, const uint32_t* xf) -> MegaPhase& {
             MegaPhase ph = {};
-            ph.W = g.packed;
+            ph.W = g.packed_u;
             ph.xf = (const uint4*)xf;
             ph.mode = mode;
             mega_phase_geometry(ph, g.N, g.K);
@@ -1041,6 +1052,8 @@ int32_t pipesd_debug_mega_trace(unsigned long long* dst, int32_t n) {
 
 int32_t pipesd_debug_set_engine(pipesd_ctx* ctx, int32_t engine) {
     if (!ctx || engine < 0 || engine > 1) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine");
+    if (engine == 1 && !needs_tiled(ctx->cfg))
+        return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine: the tiled kernels need a context with max_rows > 32");
     ctx->engine = engine;
     return PIPESD_OK;
 }
