@@ -53,7 +53,7 @@ typedef struct pipesd_model_cfg {
     int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
     float rms_eps;
     float rope_base;
-    int32_t page_size;    /* tokens per KV page (16)                                           */
+    int32_t page_size;    /* tokens per KV page: a multiple of 8 (16)                          */
     int32_t n_pages;      /* pages in the pool; one page holds page_size positions of ALL layers */
     int32_t max_requests; /* request slots                                                     */
     int32_t max_draft;    /* largest k accepted by pipesd_verify (<= 31)                       */

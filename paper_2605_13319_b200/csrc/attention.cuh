@@ -10,7 +10,7 @@
 // One CTA (4 warps) = one KV head of one request x one split x up to 64 query rows, where the rows are
 // all (query head of the group, chunk row) pairs that share the KV head (GQA).  K and V tiles of 64 keys
 // travel global -> shared with 16-byte cp.async in a two-stage ring (page table resolved per key row,
-// rows XOR-swizzled so that ldmatrix is conflict-free).  QK^T and PV run on mma.sync m16n8k16 with fp32
+// the pool stores every row with its 16-byte chunks XOR-permuted, so that ldmatrix is conflict-free).  QK^T and PV run on mma.sync m16n8k16 with fp32
 // accumulation; Q and the softmax probabilities are fp32 values split into bf16 hi + lo terms (two MMAs),
 // K and V are the cache's bf16.  How the 4 warps share a tile depends on the number of 16-row tiles:
 // 1 tile -> 4 key strips of 16, 2 tiles -> 2 x 2 strips of 32, 3-4 tiles -> one tile each over all 64 keys;
@@ -106,7 +106,7 @@ __device__ __forceinline__ void attn_load_tile(const AttnCtx& c, uint32_t stage_
         const bool valid = j0 + row < c.k1;
         const uint16_t* kp = c.kbase;
         if (valid) kp += (size_t)page[i] * c.page_stride + (size_t)slot * HD + ch * 8;
-        const uint32_t off = row * (HD * 2) + ((ch ^ (row & 7)) << 4);
+        const uint32_t off = row * (HD * 2) + (ch << 4);   // the pool's rows are stored chunk-permuted already
         cp_async16(stage_addr + off, kp, valid);
         cp_async16(stage_addr + AttnSmem<HD>::kTileBytes + off, kp + (valid ? c.v_off : 0), valid);
         slot += kRowStep;

@@ -238,10 +238,15 @@ struct PassMeta {
 };
 
 // Offset (in elements) of K (kv=0) or V (kv=1) element (slot, e) of a head inside the paged pool:
-// layout [layer][page][kv][head][slot][e].
+// layout [layer][page][kv][head][slot][e'], where the 16-byte chunks of a row are XOR-permuted by the slot's low
+// three bits (e' = kv_swizzle(e, slot)): a tile of rows copied to shared memory as it is can then be read with
+// ldmatrix without bank conflicts.  The page size is a multiple of 8, so a row's permutation is also that of
+// its index in any 8-aligned tile.
+__device__ __host__ __forceinline__ int kv_swizzle(int e, int slot) { return ((((e >> 3) ^ (slot & 7)) << 3) | (e & 7)); }
 __device__ __host__ __forceinline__ size_t kv_index(int layer, int n_pages, int page, int kv, int n_kv_heads,
                                                     int head, int page_size, int slot, int hd, int e) {
-    return (((((size_t)layer * n_pages + page) * 2 + kv) * n_kv_heads + head) * page_size + slot) * (size_t)hd + e;
+    return (((((size_t)layer * n_pages + page) * 2 + kv) * n_kv_heads + head) * page_size + slot) * (size_t)hd +
+           kv_swizzle(e, slot);
 }
 
 }  // namespace pipesd

@@ -434,9 +434,9 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                             const int kv = head < a.Hq + a.Hkv ? 0 : 1;
                             const int kvh = kv ? head - a.Hq - a.Hkv : head - a.Hq;
                             const size_t per_head = (size_t)a.page_size * a.hd;
-                            const size_t off = (size_t)a.layer * a.n_pages * 2 * a.Hkv * per_head +
-                                               (size_t)(cin ? pf_kv[i] : a.row_kvoff[tok]) +
-                                               ((size_t)kv * a.Hkv + kvh) * per_head + dim;
+                            const long long rk = cin ? pf_kv[i] : a.row_kvoff[tok];   // row offset | slot & 7
+                            const size_t off = (size_t)a.layer * a.n_pages * 2 * a.Hkv * per_head + (size_t)(rk & ~7ll) +
+                                               ((size_t)kv * a.Hkv + kvh) * per_head + kv_swizzle(dim, (int)(rk & 7));
                             a.kv_pool[off] = f32_to_bf16_bits(val);
                         }
                     }

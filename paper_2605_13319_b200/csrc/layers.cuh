@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(kEmbedThreads) embed_kernel(float* __restrict_
 
 // cos/sin of pos * base^(-2j/hd), evaluated in fp64 (positions reach 10^4, fp32 angles would lose
 // three digits), stored fp32 [M][hd/2]; and, per row, the element offset of its K slot (head 0) inside a
-// layer of the paged pool, so that the QKV epilogue appends K/V without walking the page table.
+// layer of the paged pool (with the slot's chunk permutation in the low bits), so that the QKV epilogue appends K/V without walking the page table.
 __global__ void rope_table_kernel(PassMeta meta, int M, int hd, double log_base, float* __restrict__ cs,
                                   float* __restrict__ sn, long long* __restrict__ row_kvoff, int n_pages, int Hkv,
                                   int page_size) {
@@ -74,7 +74,10 @@ __global__ void rope_table_kernel(PassMeta meta, int M, int hd, double log_base,
     if (j == 0) {
         const int item = meta.row_item[row];
         const int page = meta.block_tab[(size_t)meta.it_slot[item] * meta.max_pages + pos / page_size];
-        row_kvoff[row] = (long long)kv_index(0, n_pages, page, 0, Hkv, 0, page_size, pos % page_size, hd, 0);
+        // element offset of the row inside a layer (head 0, K); its low three bits carry slot & 7, the row's
+        // chunk permutation (the offset itself is a multiple of the head width)
+        const int slot = pos % page_size;
+        row_kvoff[row] = (long long)(kv_index(0, n_pages, page, 0, Hkv, 0, page_size, 0, hd, 0) + (size_t)slot * hd) | (slot & 7);
     }
     double theta = exp(-2.0 * (double)j / (double)hd * log_base);
     double ang = (double)pos * theta;

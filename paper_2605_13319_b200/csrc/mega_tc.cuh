@@ -37,20 +37,37 @@ constexpr int kMegaWHalf = kMegaKC * 4096;                 // one 128-row block 
 constexpr int kMegaWStage = 2 * kMegaWHalf;                // 256 rows
 constexpr int kMegaMaxStages = 6;
 constexpr int kMegaTail = 2048;                            // barriers | tmem base | rstd[32] | ssq exchange [8][32]
+constexpr int kMegaQArea = 8192;                           // attention phases: the head's queries as MMA A fragments (hi | lo)
+constexpr int kPhaseAttn = 4;                              // MegaPhase::mode of an attention phase (the GEMM modes are 0..3)
+constexpr int kAttTile = 64;                               // keys per attention chunk: K tile + V tile fill a ring stage
 constexpr int kMegaMaxCtas = 160;
 constexpr int kMegaSmemMax = 227 * 1024;
 constexpr int kMegaTmemCols = 256;                         // 2 accumulators x 2 blocks x up to 64 columns
-constexpr int kMegaL2Ahead = 8;                            // chunks a blocked weight producer pulls into L2
+#ifndef PIPESD_MEGA_L2AHEAD
+#define PIPESD_MEGA_L2AHEAD 8
+#endif
+constexpr int kMegaL2Ahead = PIPESD_MEGA_L2AHEAD;                           // chunks a blocked weight producer pulls into L2
+#ifndef PIPESD_MEGA_INFLIGHT
+#define PIPESD_MEGA_INFLIGHT 3
+#endif
+constexpr int kMegaMaxInFlight = PIPESD_MEGA_INFLIGHT;                     // weight chunks one CTA has outstanding at a time (see below)
+#ifndef PIPESD_MEGA_PACE
+#define PIPESD_MEGA_PACE 1400
+#endif
+constexpr int kMegaL2PaceClk = PIPESD_MEGA_PACE;                       // SM clocks between two L2 prefetches (32 KB at an SM's fair share of HBM)
 constexpr unsigned long long kMegaWaitNs = 1000000000ull;  // bound of every wait
 
 __host__ __device__ constexpr int mega_stage_bytes(int NT) { return kMegaWStage + kMegaKC * NT * 512; }
 __host__ __device__ constexpr int mega_stages(int NT) {
-    return (kMegaSmemMax - kMegaTail) / mega_stage_bytes(NT) > kMegaMaxStages ? kMegaMaxStages
-                                                                               : (kMegaSmemMax - kMegaTail) / mega_stage_bytes(NT);
+    return (kMegaSmemMax - kMegaTail - kMegaQArea) / mega_stage_bytes(NT) > kMegaMaxStages
+               ? kMegaMaxStages
+               : (kMegaSmemMax - kMegaTail - kMegaQArea) / mega_stage_bytes(NT);
 }
-__host__ __device__ constexpr int mega_smem_bytes(int NT) { return mega_stages(NT) * mega_stage_bytes(NT) + kMegaTail; }
+__host__ __device__ constexpr int mega_smem_bytes(int NT) { return mega_stages(NT) * mega_stage_bytes(NT) + kMegaTail + kMegaQArea; }
 
-// One GEMM of the chain.  Built once per context; lives in device memory.
+// One GEMM of the chain, or one attention phase (mode == kPhaseAttn: UB = KV heads, layer and xf_out set; the
+// number of key tiles per head changes from pass to pass and comes with the launch arguments).  Built once per
+// context; lives in device memory.
 struct MegaPhase {
     const uint4* W;        // weights in tensor-core operand order (see gemm_pack_umma_kernel)
     const uint4* xf;       // input activations of one token block, "xu" layout (see xu_piece_offset)
@@ -87,6 +104,10 @@ struct MegaArgs {
     const float* sn;
     const long long* row_kvoff;
     int Hq, Hkv, hd, n_pages, page_size;
+    // attention phases (one request per pass): keys [0, att_base) are cached, [att_base, att_base + att_rows) are
+    // this pass's rows; att_cpr = tiles of 64 keys per head
+    int att_base, att_rows, att_cpr;
+    const int32_t* att_bt;   // the request's block table row
 };
 
 // ---- weights in tensor-core operand order -----------------------------------------------------------------
@@ -168,6 +189,14 @@ __device__ __forceinline__ int ld_relaxed(const int* p) {
 __device__ __forceinline__ void red_release_add(int* p, int v) {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ void st_release_cta(int* smem_p, int v) {
+    asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(smem_p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_cta(const int* smem_p) {
+    int v;
+    asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(smem_p)) : "memory");
+    return v;
+}
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 #ifdef PIPESD_MEGA_TRACE
@@ -222,17 +251,36 @@ __device__ __forceinline__ bool poll_counter(const int* ctr, int target, const i
 __device__ __forceinline__ int mega_owner(int c, int T, int G) { return (int)((((unsigned)c + 1u) * (unsigned)G - 1u) / (unsigned)T); }
 __device__ __forceinline__ int mega_begin(int i, int T, int G) { return (int)(((unsigned)T * (unsigned)i) / (unsigned)G); }
 
-// Cursor over one CTA's weight chunks through the phases of a launch.
+// Weights are read once per pass: their lines are marked evict-first in L2, so that the 400 MB a layer streams
+// do not push out the few megabytes every phase boundary depends on (residual stream, activations, partial sums,
+// rotary tables), which would otherwise come back from HBM behind the weight stream's own queue.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+                 : "memory");
+}
+__device__ __forceinline__ int phase_cpr(const MegaArgs& a, const MegaPhase& ph) { return ph.mode == kPhaseAttn ? a.att_cpr : ph.CPR; }
+__device__ __forceinline__ int phase_chunks(const MegaArgs& a, const MegaPhase& ph) {
+    return ph.mode == kPhaseAttn ? a.att_cpr * ph.UB : ph.T;
+}
+
+// Cursor over one CTA's chunks (weights, or K/V tiles of an attention phase) through the phases of a launch.
 struct MegaWalk {
-    int p, p1, c, ce, u, cc, KS, CPR, RB;
+    int p, p1, c, ce, u, cc, KS, CPR, RB, mode, layer;
     const unsigned char* W;
     __device__ __forceinline__ void load_phase(const MegaArgs& a, int cta, int G) {
         for (; p < p1; ++p) {
             const MegaPhase& ph = a.phases[p];
-            c = mega_begin(cta, ph.T, G);
-            ce = mega_begin(cta + 1, ph.T, G);
+            const int T = phase_chunks(a, ph);
+            c = mega_begin(cta, T, G);
+            ce = mega_begin(cta + 1, T, G);
             if (c < ce) {
-                KS = ph.KS; CPR = ph.CPR; RB = ph.RB;
+                KS = ph.KS; CPR = phase_cpr(a, ph); RB = ph.RB; mode = ph.mode; layer = ph.layer;
                 W = reinterpret_cast<const unsigned char*>(ph.W);
                 u = c / CPR;
                 cc = c - u * CPR;
@@ -252,12 +300,48 @@ struct MegaWalk {
     __device__ __forceinline__ const unsigned char* src(int half) const {
         return W + ((size_t)(2 * u + half) * KS + cc * kMegaKC) * 4096;
     }
-    __device__ __forceinline__ void prefetch_l2() const {
+    __device__ __forceinline__ void prefetch_l2(uint64_t pol) const {
+        if (mode == kPhaseAttn) return;
         const uint32_t bytes = (uint32_t)kc() * 4096u;
+#ifdef PIPESD_MEGA_PF_NORMAL
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src(0)), "r"(bytes) : "memory");
         if (two()) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src(1)), "r"(bytes) : "memory");
+        return;
+#endif
+        asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src(0)), "r"(bytes), "l"(pol) : "memory");
+        if (two())
+            asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src(1)), "r"(bytes), "l"(pol) : "memory");
     }
 };
+
+// Attention chunk (KV head `kvh`, key tile `tile`): copies the pages of the tile into a stage -- K rows at the
+// stage's start, V rows 64 rows further -- and returns the bytes to expect.  `fresh` selects which pages: false
+// = pages made only of keys cached before this pass (they depend on nothing: the weight producer's share), true
+// = pages that hold rows of this pass (the activation producer's share, after the QKV phase has finished).
+// Pages hold 16 positions (the host admits nothing else to these phases).
+__device__ __forceinline__ uint32_t att_issue_pages(const MegaArgs& a, int layer, int kvh, int tile, bool fresh, int4 pages,
+                                                    uint32_t stage_addr, uint32_t bar, bool dry) {
+    const int total = a.att_base + a.att_rows;
+    const uint32_t blk = 16u * (uint32_t)a.hd * 2u;                 // one page of one head: K or V
+    const int pg[4] = {pages.x, pages.y, pages.z, pages.w};
+    uint32_t bytes = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int pos0 = tile * kAttTile + 16 * q;
+        if (pos0 >= total) continue;
+        const bool is_fresh = pos0 + 16 > a.att_base;
+        if (is_fresh != fresh) continue;
+        bytes += 2 * blk;
+        if (dry) continue;
+        const uint16_t* k = a.kv_pool + kv_index(layer, a.n_pages, pg[q], 0, a.Hkv, kvh, 16, 0, a.hd, 0);
+        bulk_g2s(stage_addr + q * blk, k, blk, bar);
+        bulk_g2s(stage_addr + 4 * blk + q * blk, k + (size_t)a.Hkv * 16 * a.hd, blk, bar);
+    }
+    return bytes;
+}
+__device__ __forceinline__ int4 att_tile_pages(const MegaArgs& a, int tile) {
+    return __ldcg(reinterpret_cast<const int4*>(a.att_bt) + tile);      // 4 pages of 16 positions per 64-key tile
+}
 
 // 8 fp32 values -> 8 bf16 hi terms and 8 bf16 lo terms, each one 16-byte word.
 __device__ __forceinline__ void split8(const float* v, uint4& hi, uint4& lo) {
@@ -295,7 +379,7 @@ __device__ __forceinline__ float warp_token_sums(float (&s)[MTP], int lane, int&
 // its value for every token.  The fused layouts put a rotary pair / a (gate, up) pair in rows i and i + 8 of a
 // 16-row tile: lanes l and l ^ 8.
 template <int NT, int MODE>
-__device__ __forceinline__ void mega_epilogue(const MegaArgs& a, const MegaPhase& ph, int u, int warp, int lane,
+__device__ __forceinline__ void mega_epilogue(const MegaArgs& a, const MegaPhase& ph, int p, int cta, int u, int warp, int lane,
                                               float (&v)[NT * 8], const float* rstd_s, float* ssq_w) {
     constexpr int MT = NT * 8;
     const int N = ph.N, M = a.M;
@@ -389,24 +473,355 @@ __device__ __forceinline__ void mega_epilogue(const MegaArgs& a, const MegaPhase
         const int kv = head < a.Hq + a.Hkv ? 0 : 1;
         const int kvh = kv ? head - a.Hq - a.Hkv : head - a.Hq;
         const size_t per_head = (size_t)a.page_size * hd;
-        const size_t kv_base = (size_t)ph.layer * a.n_pages * 2 * a.Hkv * per_head + ((size_t)kv * a.Hkv + kvh) * per_head + dim;
+        const size_t kv_base = (size_t)ph.layer * a.n_pages * 2 * a.Hkv * per_head + ((size_t)kv * a.Hkv + kvh) * per_head;
+        // every global load first (rotary factors, K/V slots), then the arithmetic and the stores
+        float cv[MT], sv[MT];
+        long long ko[MT];
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+            const bool on = row_live && t < M;
+            cv[t] = (on && rot) ? a.cs[(size_t)t * half + dlow] : 1.f;
+            sv[t] = (on && rot) ? a.sn[(size_t)t * half + dlow] : 0.f;
+            ko[t] = (on && head >= a.Hq) ? a.row_kvoff[t] : 0;
+        }
 #pragma unroll
         for (int t = 0; t < MT; ++t) {
             const float other = __shfl_xor_sync(0xffffffffu, v[t], 8);
-            float o = v[t];
-            if (rot && row_live && t < M) {
-                const float c = a.cs[(size_t)t * half + dlow], s = a.sn[(size_t)t * half + dlow];
-                o = upper ? v[t] * c + other * s : v[t] * c - other * s;
-            }
+            const float o = upper ? v[t] * cv[t] + other * sv[t] : v[t] * cv[t] - other * sv[t];
             // K/V: neighbouring dims of one token travel as one 4-byte store
             const uint32_t mine = f32_to_bf16_bits(o);
             const uint32_t nb = __shfl_xor_sync(0xffffffffu, mine, 1);
             if (row_live && t < M) {
                 if (head < a.Hq) a.q_out[((size_t)t * a.Hq + head) * hd + dim] = o;
                 else if ((lane & 1) == 0)
-                    *reinterpret_cast<uint32_t*>(a.kv_pool + (size_t)a.row_kvoff[t] + kv_base) = mine | (nb << 16);
+                    *reinterpret_cast<uint32_t*>(a.kv_pool + (size_t)(ko[t] & ~7ll) + kv_base + kv_swizzle(dim, (int)(ko[t] & 7))) =
+                        mine | (nb << 16);
             }
         }
+    }
+}
+
+// ---- attention phase: one segment = one KV head x a run of 64-key tiles, consumed by the eight epilogue warps --
+__device__ __forceinline__ void mma_bf16_1688(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(b0));
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ float ex2_approx(float x) {   // 2^x, relative error 2^-22; 2^-inf = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t& lo) {   // packed bf16x2 hi and lo terms
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    const float2 hf = __bfloat1622float2(h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(a - hf.x, b - hf.y);
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+// The (at most 16) query rows that share KV head `kvh` -- every (query head of the group, chunk row) pair --
+// attend to the keys of tiles [tile0, tile1).  A tile is 64 keys: K rows at the start of a ring stage, V rows
+// behind them, rows chunk-permuted as in the pool.  Warp w takes keys 8w..8w+7 of every tile: Q K^T on
+// m16n8k16 (Q split into bf16 hi + lo), online softmax in the log2 domain, P V on m16n8k8 (P split likewise).
+// At the end the eight warps' running (max, sum, output) are merged through the last stage's shared memory in a
+// fixed order; heads whose tiles are spread over several CTAs are merged through global memory by the CTA that
+// owns the head's first tile, exactly as the GEMM units are, and the normalised output goes to the output
+// projection's input array.  Every named barrier below is reached by all 256 threads, also after a failed wait.
+template <int HD>
+__device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& ph, int cta, int G, int kvh, int tile0, int tile1,
+                                            int ub, int T, int CPR, int NT, int kStages, int kStage, unsigned char* smem,
+                                            uint32_t fullW0, uint32_t fullX0, uint32_t empty0, int& n, int& st, bool& ok,
+                                            unsigned char* qarea, float* xch, int pseg, int* pub_seq) {
+    constexpr int KSTEPS = HD / 16, NTO = HD / 8, ROWB = HD * 2;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int Gq = a.Hq / a.Hkv, rows = a.att_rows, R = Gq * rows, base = a.att_base, total = base + rows;
+    const uint32_t smem_base = smem_u32(smem);
+    // ---- the queries come from the QKV phase: the activation producer's first arrival says it has finished
+    if (ok) {
+        ok = mbar_wait_err(fullX0 + 8 * st, (uint32_t)(n / kStages) & 1u, a.err);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok && lane == 0) atomicCAS(a.err, 0, 17);
+    }
+    uint4* qsm = reinterpret_cast<uint4*>(qarea);      // [k16 step][hi | lo][lane] A fragments of the 16 rows
+    const float scale = rsqrtf((float)HD) * 1.4426950408889634f;   // scores in the log2 domain: p = 2^(s - m)
+    for (int idx = threadIdx.x; idx < KSTEPS * 32; idx += kMegaEpiThreads) {
+        const int ln = idx & 31, ks = idx >> 5, gg = ln >> 2, tt = ln & 3;
+        float v[8];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int rho = gg + 8 * hh;
+            float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
+            if (rho < R && ok) {
+                const int gq = rho / rows, r = rho - gq * rows;
+                const float* qp = a.q_out + ((size_t)r * a.Hq + kvh * Gq + gq) * HD + ks * 16 + 2 * tt;
+                x0 = __ldcg(reinterpret_cast<const float2*>(qp));
+                x1 = __ldcg(reinterpret_cast<const float2*>(qp + 8));
+            }
+            v[2 * hh] = x0.x * scale; v[2 * hh + 1] = x0.y * scale;
+            v[4 + 2 * hh] = x1.x * scale; v[4 + 2 * hh + 1] = x1.y * scale;
+        }
+        uint16_t h[8], l[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) split_bf16(v[i], h[i], l[i]);
+        qsm[(ks * 2 + 0) * 32 + ln] = make_uint4(pack2(h[0], h[1]), pack2(h[2], h[3]), pack2(h[4], h[5]), pack2(h[6], h[7]));
+        qsm[(ks * 2 + 1) * 32 + ln] = make_uint4(pack2(l[0], l[1]), pack2(l[2], l[3]), pack2(l[4], l[5]), pack2(l[6], l[7]));
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+
+    float o[NTO][4];
+#pragma unroll
+    for (int i = 0; i < NTO; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[i][e] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    int horizon[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const int rho = g + 8 * hh;
+        horizon[hh] = rho < R ? base + rho % rows : -1;     // keys j <= horizon are visible (padding rows: unused)
+    }
+    int last_st = st;
+    for (int tile = tile0; tile < tile1; ++tile, ++n) {
+        if (ok) {
+            const uint32_t par = (uint32_t)(n / kStages) & 1u;
+            ok = mbar_wait_err(fullW0 + 8 * st, par, a.err) && mbar_wait_err(fullX0 + 8 * st, par, a.err);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok && lane == 0) atomicCAS(a.err, 0, 18);
+        }
+        const int j0 = tile * kAttTile + 8 * warp;           // first key of this warp's strip
+        if (ok && j0 < total) {
+            const uint32_t kst = smem_base + st * kStage, vst = kst + kAttTile * ROWB;
+            const int row = 8 * warp + (lane & 7);
+            if (j0 + 8 > total) {
+                // rows beyond the keys hold whatever the pool or the stage held before: their probabilities are
+                // exactly zero, but 0 x NaN is not, so their V rows are cleared (this warp's strip only)
+                for (int i = lane; i < 8 * (ROWB / 16); i += 32) {
+                    const int r = i / (ROWB / 16), cpos = i % (ROWB / 16);
+                    if (j0 + r >= total)
+                        *reinterpret_cast<uint4*>(smem + st * kStage + kAttTile * ROWB + (8 * warp + r) * ROWB + cpos * 16) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                }
+                __syncwarp();
+            }
+            float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int kp = 0; kp < KSTEPS / 2; ++kp) {
+                const uint4 qh0 = qsm[((2 * kp) * 2 + 0) * 32 + lane], ql0 = qsm[((2 * kp) * 2 + 1) * 32 + lane];
+                const uint4 qh1 = qsm[((2 * kp + 1) * 2 + 0) * 32 + lane], ql1 = qsm[((2 * kp + 1) * 2 + 1) * 32 + lane];
+                const int ch = kp * 4 + (lane >> 3);
+                uint32_t b[4];
+                ldsm_x4(b, kst + row * ROWB + ((ch ^ (row & 7)) << 4));
+                mma_bf16_16816(s, qh0, b[0], b[1]);
+                mma_bf16_16816(s2, ql0, b[0], b[1]);
+                mma_bf16_16816(s, qh1, b[2], b[3]);
+                mma_bf16_16816(s2, ql1, b[2], b[3]);
+            }
+            float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int hh = e >> 1, j = j0 + 2 * t + (e & 1);
+                s[e] += s2[e];
+                if (!(j < total && j <= horizon[hh])) s[e] = -INFINITY;
+                mx[hh] = fmaxf(mx[hh], s[e]);
+            }
+            float alpha[2], m_use[2];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
+                mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
+                const float m_new = fmaxf(m_run[hh], mx[hh]);
+                m_use[hh] = m_new == -INFINITY ? 0.f : m_new;      // keeps (-inf) - (-inf) out of the exponent
+                alpha[hh] = ex2_approx(m_run[hh] - m_use[hh]);     // 0 while nothing has been seen yet
+                m_run[hh] = m_new;
+                l_run[hh] *= alpha[hh];
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                s[e] = ex2_approx(s[e] - m_use[e >> 1]);           // masked: 2^-inf = 0
+                l_run[e >> 1] += s[e];                             // per-lane partial; the quad is summed at the end
+            }
+            if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+#pragma unroll
+                for (int i = 0; i < NTO; ++i) {
+                    o[i][0] *= alpha[0]; o[i][1] *= alpha[0];
+                    o[i][2] *= alpha[1]; o[i][3] *= alpha[1];
+                }
+            }
+            uint32_t ph0, pl0, ph1, pl1;
+            split2(s[0], s[1], ph0, pl0);
+            split2(s[2], s[3], ph1, pl1);
+#pragma unroll
+            for (int np = 0; np < NTO / 4; ++np) {
+                const int ch = np * 4 + (lane >> 3);
+                uint32_t b[4];
+                ldsm_x4_trans(b, vst + row * ROWB + ((ch ^ (row & 7)) << 4));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    mma_bf16_1688(o[4 * np + i], ph0, ph1, b[i]);
+                    mma_bf16_1688(o[4 * np + i], pl0, pl1, b[i]);
+                }
+            }
+        }
+        last_st = st;
+        if (tile + 1 < tile1) {      // the last tile's stage is kept: it is the merge's scratch
+            asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+            if (threadIdx.x == 0 && ok) mbar_arrive(empty0 + 8 * st);
+        }
+        if (++st == kStages) st = 0;
+    }
+    // ---- merge the eight warps: common maximum, rescaled sums, outputs added in the order
+    // ((w0 + w4) + (w1 + w5)) + (w2 + w6) + (w3 + w7)
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        l_run[hh] += __shfl_xor_sync(0xffffffffu, l_run[hh], 1);
+        l_run[hh] += __shfl_xor_sync(0xffffffffu, l_run[hh], 2);
+    }
+    float* ms = xch;            // [8 warps][16 rows] running maxima
+    float* ls = xch + 128;      // [8 warps][16 rows] running sums
+    if (t == 0) {
+        ms[warp * 16 + g] = m_run[0]; ms[warp * 16 + g + 8] = m_run[1];
+        ls[warp * 16 + g] = l_run[0]; ls[warp * 16 + g + 8] = l_run[1];
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+    float m_tot[2], l_tot[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const int row = g + 8 * hh;
+        float m = -INFINITY, l = 0.f;
+#pragma unroll
+        for (int w = 0; w < kMegaEpiWarps; ++w) m = fmaxf(m, ms[w * 16 + row]);
+#pragma unroll
+        for (int w = 0; w < kMegaEpiWarps; ++w) {
+            const float mw = ms[w * 16 + row];
+            l += (mw == -INFINITY ? 0.f : exp2f(mw - m)) * ls[w * 16 + row];
+        }
+        const float sc = m_run[hh] == -INFINITY ? 0.f : exp2f(m_run[hh] - m);
+#pragma unroll
+        for (int i = 0; i < NTO; ++i) { o[i][2 * hh] *= sc; o[i][2 * hh + 1] *= sc; }
+        m_tot[hh] = m;
+        l_tot[hh] = l;
+    }
+    float* mo = reinterpret_cast<float*>(smem + last_st * kStage);      // [4][16 rows][HD]
+    auto put = [&](int slot) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+            for (int i = 0; i < NTO; ++i)
+                *reinterpret_cast<float2*>(mo + ((size_t)slot * 16 + g + 8 * hh) * HD + i * 8 + 2 * t) =
+                    make_float2(o[i][2 * hh], o[i][2 * hh + 1]);
+    };
+    auto add = [&](int slot) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+            for (int i = 0; i < NTO; ++i) {
+                const float2 v = *reinterpret_cast<const float2*>(mo + ((size_t)slot * 16 + g + 8 * hh) * HD + i * 8 + 2 * t);
+                o[i][2 * hh] += v.x;
+                o[i][2 * hh + 1] += v.y;
+            }
+    };
+    if (warp >= 4) put(warp - 4);
+    asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+    if (warp < 4) add(warp);
+    asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+    if (warp >= 1 && warp < 4) put(warp);
+    asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+    if (warp == 0) { add(1); add(2); add(3); }
+    // warp 0 now holds the CTA's un-normalised output for the head, relative to m_tot, with the sum l_tot
+    const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
+    constexpr int kSlotFloats = 8 * kMegaEpiThreads * 4;       // one CTA's slot of the exchange array
+    if (i0 != i1 && cta != i0) {
+        // contributor: output rows, maxima and sums to this CTA's slot; the publisher counts it in
+        if (warp == 0) {
+            float* dst = reinterpret_cast<float*>(a.scratch) + (size_t)cta * kSlotFloats;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                for (int i = 0; i < NTO; ++i)
+                    *reinterpret_cast<float2*>(dst + (size_t)(g + 8 * hh) * HD + i * 8 + 2 * t) = make_float2(o[i][2 * hh], o[i][2 * hh + 1]);
+                if (t == 0) { dst[16 * HD + g + 8 * hh] = m_tot[hh]; dst[16 * HD + 16 + g + 8 * hh] = l_tot[hh]; }
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+        if (threadIdx.x == 0) {
+            if (ok) mbar_arrive(empty0 + 8 * last_st);
+            st_release_cta(pub_seq, pseg);
+        }
+        return;
+    }
+    // collector (or alone on the head): own partial to shared memory, then all 256 threads finish the head
+    if (warp == 0) {
+        put(0);          // slot 0 of the scratch was last read by this warp itself
+        if (t == 0) {
+            ms[g] = m_tot[0]; ms[g + 8] = m_tot[1];
+            ls[g] = l_tot[0]; ls[g + 8] = l_tot[1];
+        }
+    }
+    if (i0 != i1 && threadIdx.x == 0) {
+        const int n_contrib = T >= G ? i1 - i0 + 1 : CPR;
+        if (!poll_counter(a.tickets + ph.ticket0 + kvh, n_contrib - 1, a.err)) atomicCAS(a.err, 0, 19);
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+    {
+        constexpr int CPT = HD / 16;                            // output columns per thread
+        const int row = threadIdx.x >> 4, c0 = (threadIdx.x & 15) * CPT;
+        float num[CPT];
+#pragma unroll
+        for (int k = 0; k < CPT; ++k) num[k] = mo[(size_t)row * HD + c0 + k];
+        float m = ms[row], den = ls[row];
+        if (i0 != i1) {
+            // contributions are fetched four CTAs at a time (all loads in flight) and merged in CTA order
+            for (int ib = i0 + 1; ib <= i1; ib += 4) {
+                float4 ov[4][CPT / 4];
+                float mc[4], lc[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int i = ib + q;
+                    const bool on = i <= i1 && (T >= G || mega_begin(i, T, G) != mega_begin(i + 1, T, G));
+                    const float* src = reinterpret_cast<const float*>(a.scratch) + (size_t)i * kSlotFloats;
+#pragma unroll
+                    for (int k = 0; k < CPT / 4; ++k)
+                        ov[q][k] = on ? __ldcg(reinterpret_cast<const float4*>(src + (size_t)row * HD + c0) + k)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                    mc[q] = on ? __ldcg(src + 16 * HD + row) : -INFINITY;
+                    lc[q] = on ? __ldcg(src + 16 * HD + 16 + row) : 0.f;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float mn = fmaxf(m, mc[q]);
+                    const float wa = m == -INFINITY ? 0.f : exp2f(m - mn), wb = mc[q] == -INFINITY ? 0.f : exp2f(mc[q] - mn);
+#pragma unroll
+                    for (int k = 0; k < CPT / 4; ++k) {
+                        num[4 * k] = num[4 * k] * wa + ov[q][k].x * wb;
+                        num[4 * k + 1] = num[4 * k + 1] * wa + ov[q][k].y * wb;
+                        num[4 * k + 2] = num[4 * k + 2] * wa + ov[q][k].z * wb;
+                        num[4 * k + 3] = num[4 * k + 3] * wa + ov[q][k].w * wb;
+                    }
+                    den = den * wa + lc[q] * wb;
+                    m = mn;
+                }
+            }
+        }
+        if (row < R && ok) {
+            const int gq = row / rows, r = row - gq * rows;
+            const float inv = 1.f / den;
+#pragma unroll
+            for (int k = 0; k < CPT; ++k) xu_store_one(ph.xf_out, r, (kvh * Gq + gq) * HD + c0 + k, num[k] * inv, NT);
+        }
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
+    if (threadIdx.x == 0) {
+        if (ok) mbar_arrive(empty0 + 8 * last_st);
+        st_release_cta(pub_seq, pseg);
     }
 }
 
@@ -422,6 +837,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
     unsigned char* tail = smem + kStages * kStage;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);          // fullW[8] | fullX[8] | empty[8] | accfull[2] | accempty[2] | drain | rstd
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256);
+    int* pub_seq = reinterpret_cast<int*>(tail + 320);            // segments whose stores are complete (epilogue -> publisher)
     float* rstd_s = reinterpret_cast<float*>(tail + 384);        // [32]
     float* ssq_w = reinterpret_cast<float*>(tail + 512);         // [8][32]
     const uint32_t smem_base = smem_u32(smem);
@@ -442,6 +858,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
         }
         mbar_init(drain0, 1);
         mbar_init(rstd0, 1);
+        *pub_seq = 0;
         fence_mbar_init();
         red_release_add(a.arrived, 1);
     }
@@ -464,15 +881,27 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
             pf = ring;
             int n = 0, st = 0, n_pf = 0;
             bool ok = true;
+            long long t_pf = clock64();
+            const uint64_t pol = l2_evict_first_policy();
+            int4 att_pages = make_int4(0, 0, 0, 0);
+            int att_tile = -1, att_phase = -1;   // chunk index and phase whose page ids att_pages holds
             while (ring.valid()) {
-                if (n >= kStages) {
+                // At most kMegaMaxInFlight chunks are outstanding: enough to keep HBM busy (148 SMs x 96 KB is
+                // twice the bandwidth-latency product), while every byte beyond that only queues in front of
+                // the small latency-critical accesses of the phase boundaries (counters, partial sums, x).
+                if (ok && n >= kMegaMaxInFlight) {
+                    const int m = n - kMegaMaxInFlight;
+                    ok = mbar_wait_err(fullW0 + 8 * (m % kStages), (uint32_t)(m / kStages) & 1u, a.err);
+                }
+                if (ok && n >= kStages) {
                     // Ring full: the MMAs are held up (usually at a phase boundary).  HBM must not go idle
-                    // meanwhile: pull the chunks after the ring's into L2, up to kMegaL2Ahead chunks ahead.
+                    // meanwhile: pull the chunks after the ring's into L2, up to kMegaL2Ahead chunks ahead, paced
+                    // at the SM's fair share of the bandwidth so that the queues stay short.
                     const uint32_t bar = empty0 + 8 * st, par = (uint32_t)((n / kStages) - 1) & 1u;
                     uint64_t t0 = 0;
                     for (uint32_t it = 0; !mbar_try(bar, par); ++it) {
-                        if (n_pf < n + kMegaL2Ahead && pf.valid()) {
-                            if (n_pf >= n) pf.prefetch_l2();
+                        if (n_pf < n + kMegaL2Ahead && pf.valid() && clock64() - t_pf >= kMegaL2PaceClk) {
+                            if (n_pf >= n) { pf.prefetch_l2(pol); t_pf = clock64(); }
                             pf.next(a, cta, G);
                             ++n_pf;
                             continue;
@@ -484,13 +913,27 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                             else if (now - t0 > kMegaWaitNs) { ok = false; break; }
                         }
                     }
-                    if (!ok) break;
                 }
-                const uint32_t bytes = (uint32_t)ring.kc() * 4096u;
-                const bool two = ring.two();
-                mbar_expect_tx(fullW0 + 8 * st, two ? 2 * bytes : bytes);
-                bulk_g2s(smem_base + st * kStage, ring.src(0), bytes, fullW0 + 8 * st);
-                if (two) bulk_g2s(smem_base + st * kStage + kMegaWHalf, ring.src(1), bytes, fullW0 + 8 * st);
+                if (!ok) break;
+                if (ring.mode == kPhaseAttn) {
+                    // K/V tile of an attention phase: the pages cached before this pass (the others are the
+                    // activation producer's); the next tile's page ids are fetched one chunk ahead
+                    if (att_tile != ring.c || att_phase != ring.p) att_pages = att_tile_pages(a, ring.cc);
+                    att_phase = ring.p;
+                    const uint32_t bytes = att_issue_pages(a, ring.layer, ring.u, ring.cc, false, att_pages, 0, 0, true);
+                    mbar_expect_tx(fullW0 + 8 * st, bytes);
+                    att_issue_pages(a, ring.layer, ring.u, ring.cc, false, att_pages, smem_base + st * kStage, fullW0 + 8 * st, false);
+                    if (ring.c + 1 < ring.ce) {
+                        att_pages = att_tile_pages(a, ring.cc + 1 == ring.CPR ? 0 : ring.cc + 1);
+                        att_tile = ring.c + 1;
+                    }
+                } else {
+                    const uint32_t bytes = (uint32_t)ring.kc() * 4096u;
+                    const bool two = ring.two();
+                    mbar_expect_tx(fullW0 + 8 * st, two ? 2 * bytes : bytes);
+                    bulk_g2s_hint(smem_base + st * kStage, ring.src(0), bytes, fullW0 + 8 * st, pol);
+                    if (two) bulk_g2s_hint(smem_base + st * kStage + kMegaWHalf, ring.src(1), bytes, fullW0 + 8 * st, pol);
+                }
                 if (++st == kStages) st = 0;
                 ring.next(a, cta, G);
                 ++n;
@@ -500,6 +943,37 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 // let every copy already issued land before the CTA's shared memory can be released
                 for (int i = n > kStages ? n - kStages : 0; i < n; ++i)
                     mbar_wait(fullW0 + 8 * (i % kStages), (uint32_t)(i / kStages) & 1u);
+            }
+        } else if (lane == 1) {
+            // ---------------------------------------- publisher: walks the same schedule as the epilogue warps
+            // and, whenever they have finished a segment (pub_seq), makes it known to the other CTAs: a
+            // contribution counted in, or a unit counted as done.  The release (a fence over all the CTA's
+            // earlier stores) costs a microsecond that no epilogue warp has to spend waiting.
+            int seg = 0;
+            bool ok = true;
+            for (int p = a.p0; p < a.p1 && ok; ++p) {
+                const MegaPhase& ph = a.phases[p];
+                const int T = phase_chunks(a, ph), CPR = phase_cpr(a, ph);
+                const int cb = mega_begin(cta, T, G), ce = mega_begin(cta + 1, T, G);
+                int c = cb;
+                while (c < ce) {
+                    const int u = c / CPR, ub = u * CPR;
+                    c = ce < ub + CPR ? ce : ub + CPR;
+                    ++seg;
+                    uint64_t t0 = 0;
+                    for (uint32_t it = 0; ld_acquire_cta(pub_seq) < seg; ++it) {
+                        if ((it & 63u) == 63u) {
+                            if (ld_relaxed(a.err) != 0) { ok = false; break; }
+                            const uint64_t now = global_ns();
+                            if (t0 == 0) t0 = now;
+                            else if (now - t0 > 4 * kMegaWaitNs) { ok = false; break; }
+                        }
+                    }
+                    if (!ok) break;
+                    const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
+                    if (i0 != i1 && cta != i0) red_release_add(a.tickets + ph.ticket0 + u, 1);
+                    else red_release_add(a.done + p, 1);
+                }
             }
         }
     } else if (warp == kMegaWarpX) {
@@ -525,25 +999,39 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 if (!ok) break;
                 pdl_launch_dependents();
             }
-            const int T = ph.T, CPR = ph.CPR, KS = ph.KS;
+            const int T = phase_chunks(a, ph), CPR = phase_cpr(a, ph), KS = ph.KS;
             const int cb = mega_begin(cta, T, G), ce = mega_begin(cta + 1, T, G);
             if (cb == ce) continue;
             if (lane == 0) {
                 fence_proxy_async_all();          // activations were written with ordinary stores by other SMs
                 const unsigned char* X = reinterpret_cast<const unsigned char*>(ph.xf);
-                int cc = cb % CPR;
+                int cc = cb % CPR, u = cb / CPR;
                 for (int c = cb; c < ce; ++c, ++n) {
                     if (n >= kStages) {
                         ok = mbar_wait_err(empty0 + 8 * st, (uint32_t)((n / kStages) - 1) & 1u, a.err);
                         if (!ok) break;
                     }
-                    const int ks = cc * kMegaKC;
-                    const int kc = KS - ks < kMegaKC ? KS - ks : kMegaKC;
-                    const uint32_t bytes = (uint32_t)kc * NT * 512u;
-                    mbar_expect_tx(fullX0 + 8 * st, bytes);
-                    bulk_g2s(smem_base + st * kStage + kMegaWStage, X + (size_t)ks * NT * 512, bytes, fullX0 + 8 * st);
+                    if (ph.mode == kPhaseAttn) {
+                        // the pages of the tile that hold rows of this pass (written by the QKV phase); a tile
+                        // without such pages still gets its arrival: the queries, too, come from that phase
+                        uint32_t bytes = 0;
+                        if ((cc + 1) * kAttTile > a.att_base) {
+                            const int4 pages = att_tile_pages(a, cc);
+                            bytes = att_issue_pages(a, ph.layer, u, cc, true, pages, 0, 0, true);
+                            mbar_expect_tx(fullX0 + 8 * st, bytes);
+                            att_issue_pages(a, ph.layer, u, cc, true, pages, smem_base + st * kStage, fullX0 + 8 * st, false);
+                        } else {
+                            mbar_expect_tx(fullX0 + 8 * st, 0u);
+                        }
+                    } else {
+                        const int ks = cc * kMegaKC;
+                        const int kc = KS - ks < kMegaKC ? KS - ks : kMegaKC;
+                        const uint32_t bytes = (uint32_t)kc * NT * 512u;
+                        mbar_expect_tx(fullX0 + 8 * st, bytes);
+                        bulk_g2s(smem_base + st * kStage + kMegaWStage, X + (size_t)ks * NT * 512, bytes, fullX0 + 8 * st);
+                    }
                     if (++st == kStages) st = 0;
-                    if (++cc == CPR) cc = 0;
+                    if (++cc == CPR) { cc = 0; ++u; }
                 }
             } else {
                 // lanes 1..31: the input rows' RMSNorm factors, needed only by the epilogue, computed while
@@ -581,9 +1069,14 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
             bool ok = true;
             for (int p = a.p0; p < a.p1; ++p) {
                 const MegaPhase& ph = a.phases[p];
-                const int T = ph.T, CPR = ph.CPR, KS = ph.KS, RB = ph.RB;
+                const int T = phase_chunks(a, ph), CPR = phase_cpr(a, ph), KS = ph.KS, RB = ph.RB;
                 const int cb = mega_begin(cta, T, G), ce = mega_begin(cta + 1, T, G);
                 int c = cb;
+                if (ph.mode == kPhaseAttn) {      // the attention chunks are consumed by the epilogue warps
+                    n += ce - cb;
+                    st = (st + (ce - cb)) % kStages;
+                    continue;
+                }
                 while (c < ce) {
                     const int u = c / CPR, ub = u * CPR;
                     const int se = ce < ub + CPR ? ce : ub + CPR;
@@ -614,6 +1107,8 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                                 accumulate = 1;
                             }
                             umma_commit(empty0 + 8 * st);      // the stage is free when these MMAs have read it
+                            if (c == cb) MEGA_TRACE(1);
+                            if (c == ce - 1) MEGA_TRACE(6);
                         }
                         if (++st == kStages) st = 0;
                     }
@@ -630,13 +1125,32 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
         // ------------------------------------------------ epilogue warps
         pdl_wait();      // epilogues read what earlier kernels wrote (rotary tables, K/V offsets, residual stream)
         int seg = 0, n_norm = 0;      // n_norm: phases so far whose input is normalised and in which this CTA has work
+        int pseg = 0;                 // segments finished (GEMM units and attention heads): what the publisher counts
+        int n = 0, st = 0;            // chunk counter / ring stage: followed for the attention phases
         bool ok = true;
         const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * kCols);
         for (int p = a.p0; p < a.p1; ++p) {
             const MegaPhase& ph = a.phases[p];
-            const int T = ph.T, CPR = ph.CPR, mode = ph.mode;
+            const int T = phase_chunks(a, ph), CPR = phase_cpr(a, ph), mode = ph.mode;
             const int cb = mega_begin(cta, T, G), ce = mega_begin(cta + 1, T, G);
             int c = cb;
+            if (mode == kPhaseAttn) {
+                while (c < ce) {
+                    const int u = c / CPR, ub = u * CPR;
+                    const int se = ce < ub + CPR ? ce : ub + CPR;
+                    ++pseg;
+                    if (a.hd == 128)
+                        att_segment<128>(a, ph, cta, G, u, c - ub, se - ub, ub, T, CPR, NT, kStages, kStage, smem, fullW0, fullX0,
+                                         empty0, n, st, ok, tail + kMegaTail, ssq_w, pseg, pub_seq);
+                    else
+                        att_segment<64>(a, ph, cta, G, u, c - ub, se - ub, ub, T, CPR, NT, kStages, kStage, smem, fullW0, fullX0,
+                                        empty0, n, st, ok, tail + kMegaTail, ssq_w, pseg, pub_seq);
+                    c = se;
+                }
+                continue;
+            }
+            n += ce - cb;
+            st = (st + (ce - cb)) % kStages;
             if (cb < ce && ph.ssq_in != nullptr) {
                 // the activation producer has derived this phase's RMSNorm factors
                 if (ok) {
@@ -680,6 +1194,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     for (int t = 0; t < MT; ++t) v[t] = 0.f;
                 }
                 ++seg;
+                ++pseg;
                 if (threadIdx.x == 0) MEGA_TRACE(2);
                 // ---- the CTA's part of unit u is summed.  Alone on the unit: epilogue.  Otherwise the CTA that
                 // owns the unit's first chunk collects (the unit is the last thing that CTA does in the phase,
@@ -693,10 +1208,10 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
 #pragma unroll
                         for (int q = 0; q < 2 * NT; ++q)
                             mine[(size_t)q * kMegaEpiThreads] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-                        // all stores of the CTA happen before thread 0's release (ordered by the named barrier)
+                        // all stores of the CTA happen before thread 0's signal to the publisher thread (ordered by
+                        // the named barrier), which counts the CTA in with a release
                         asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
-                        if (threadIdx.x == 0) red_release_add(a.tickets + ph.ticket0 + u, 1);
-                        if (threadIdx.x == 0) MEGA_TRACE(3);
+                        if (threadIdx.x == 0) { st_release_cta(pub_seq, pseg); MEGA_TRACE(3); }
                         continue;
                     }
                     if (threadIdx.x == 0) {
@@ -707,40 +1222,41 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     }
                     asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
                     if (threadIdx.x == 0) MEGA_TRACE(3);
-                    // contributions are fetched kBatch at a time (all loads of a batch in flight)
-                    constexpr int kBatch = NT == 1 ? 8 : (NT == 2 ? 4 : 2);
-                    for (int ib = i0 + 1; ib <= i1; ib += kBatch) {
-                        float4 w[kBatch][2 * NT];
+                    // contributions are fetched eight CTAs at a time, two 16-byte words each (16 loads in flight),
+                    // and added in CTA order
+                    for (int q0 = 0; q0 < 2 * NT; q0 += 2) {
+                        for (int ib = i0 + 1; ib <= i1; ib += 8) {
+                            float4 w[8][2];
 #pragma unroll
-                        for (int k = 0; k < kBatch; ++k) {
-                            const int i = ib + k;
-                            const bool on = i <= i1 && (T >= G || mega_begin(i, T, G) != mega_begin(i + 1, T, G));
-                            const float4* src = a.scratch + ((size_t)i * (2 * NT)) * kMegaEpiThreads + threadIdx.x;
-#pragma unroll
-                            for (int q = 0; q < 2 * NT; ++q)
-                                w[k][q] = on ? __ldcg(src + (size_t)q * kMegaEpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-#pragma unroll
-                        for (int k = 0; k < kBatch; ++k)
-#pragma unroll
-                            for (int q = 0; q < 2 * NT; ++q) {
-                                v[4 * q] += w[k][q].x;
-                                v[4 * q + 1] += w[k][q].y;
-                                v[4 * q + 2] += w[k][q].z;
-                                v[4 * q + 3] += w[k][q].w;
+                            for (int k = 0; k < 8; ++k) {
+                                const int i = ib + k;
+                                const bool on = i <= i1 && (T >= G || mega_begin(i, T, G) != mega_begin(i + 1, T, G));
+                                const float4* src = a.scratch + ((size_t)i * (2 * NT) + q0) * kMegaEpiThreads + threadIdx.x;
+                                w[k][0] = on ? __ldcg(src) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                w[k][1] = on ? __ldcg(src + kMegaEpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
                             }
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    v[4 * (q0 + h)] += w[k][h].x;
+                                    v[4 * (q0 + h) + 1] += w[k][h].y;
+                                    v[4 * (q0 + h) + 2] += w[k][h].z;
+                                    v[4 * (q0 + h) + 3] += w[k][h].w;
+                                }
+                        }
                     }
                 }
                 if (threadIdx.x == 0) MEGA_TRACE(4);
-                if (mode == kPlain) mega_epilogue<NT, kPlain>(a, ph, u, warp, lane, v, rstd_s, ssq_w);
-                else if (mode == kQkvRope) mega_epilogue<NT, kQkvRope>(a, ph, u, warp, lane, v, rstd_s, ssq_w);
-                else if (mode == kResid) mega_epilogue<NT, kResid>(a, ph, u, warp, lane, v, rstd_s, ssq_w);
-                else mega_epilogue<NT, kSwiglu>(a, ph, u, warp, lane, v, rstd_s, ssq_w);
-                // publish: the named barrier orders every thread's stores before thread 0's release; readers
-                // acquire the counter (and fence the asynchronous proxy before their bulk copies)
+                if (mode == kPlain) mega_epilogue<NT, kPlain>(a, ph, p, cta, u, warp, lane, v, rstd_s, ssq_w);
+                else if (mode == kQkvRope) mega_epilogue<NT, kQkvRope>(a, ph, p, cta, u, warp, lane, v, rstd_s, ssq_w);
+                else if (mode == kResid) mega_epilogue<NT, kResid>(a, ph, p, cta, u, warp, lane, v, rstd_s, ssq_w);
+                else mega_epilogue<NT, kSwiglu>(a, ph, p, cta, u, warp, lane, v, rstd_s, ssq_w);
+                // publish: the named barrier orders every thread's stores before thread 0's signal; the publisher
+                // thread counts the unit as done with a release, so that no epilogue warp waits for the fence;
+                // readers acquire the counter (and fence the asynchronous proxy before their bulk copies)
                 asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
-                if (threadIdx.x == 0) MEGA_TRACE(5);
-                if (threadIdx.x == 0) red_release_add(a.done + p, 1);
+                if (threadIdx.x == 0) { st_release_cta(pub_seq, pseg); MEGA_TRACE(5); }
             }
         }
     }

@@ -78,7 +78,9 @@ Derived derive(const pipesd_model_cfg& c) {
     d.qd = c.n_q_heads * c.head_dim;
     d.kvd = c.n_kv_heads * c.head_dim;
     d.Nqkv = d.qd + 2 * d.kvd;
-    d.max_pages = (c.max_seq + c.page_size - 1) / c.page_size;
+    // block-table rows are read four entries at a time (one 64-key tile of 16-position pages): padded to a
+    // multiple of four entries with one spare group
+    d.max_pages = ((c.max_seq + c.page_size - 1) / c.page_size + 3) / 4 * 4 + 4;
     d.max_items = std::min(c.max_requests, c.max_rows);
     // two staging arrays for pipesd_debug_read_kv / write_kv: 256 positions of K and of V per round
     size_t best = (size_t)256 * d.kvd / 2 + 64;
@@ -88,7 +90,7 @@ Derived derive(const pipesd_model_cfg& c) {
 
 struct WsLayout {
     size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, tickets, cs, sn, kvoff, stats, results, meta,
-        block_tab, qstage, mega_phases, mega_ctr, mega_scratch, total;
+        block_tab, qstage, mega_phases, mega_phases_att, mega_ctr, mega_scratch, total;
     size_t mega_ctr_ints;
 };
 
@@ -124,10 +126,12 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     w.qstage = take(4 * M * c.vocab);
     // persistent layer-stack kernel: phase table, counters (finished units per phase | started CTAs per launch |
     // one ticket per 256-row unit), accumulator fragments of units shared by several CTAs
-    const size_t n_phases = 4 * (size_t)c.n_layers + 1;
+    const size_t n_phases = 5 * (size_t)c.n_layers + 1;      // with the attention phases
     auto units = [](size_t N) { return ((N + 127) / 128 + 1) / 2; };
-    const size_t n_tickets = (size_t)c.n_layers * (units(d.Nqkv) + 2 * units(c.d_model) + units(2 * (size_t)c.d_ffn)) + units(c.vocab);
+    const size_t n_tickets = (size_t)c.n_layers * (units(d.Nqkv) + 2 * units(c.d_model) + units(2 * (size_t)c.d_ffn) + c.n_kv_heads) +
+                             units(c.vocab);
     w.mega_phases = take(sizeof(MegaPhase) * n_phases);
+    w.mega_phases_att = take(sizeof(MegaPhase) * n_phases);
     w.mega_ctr_ints = n_phases + (size_t)c.n_layers + 2 + n_tickets;
     w.mega_ctr = take(4 * w.mega_ctr_ints);
     w.mega_scratch = take((size_t)kMegaMaxCtas * 8 * kMegaEpiThreads * sizeof(float4));
@@ -162,7 +166,8 @@ int check_cfg(const pipesd_model_cfg* c) {
     if (c->head_dim != 64 && c->head_dim != 128) return PIPESD_E_INVALID;
     if (c->d_model % 16 || c->d_ffn % 16 || c->vocab % 16 || c->d_model > 8192) return PIPESD_E_INVALID;
     if (c->n_q_heads % c->n_kv_heads) return PIPESD_E_INVALID;
-    if (c->page_size < 1 || c->page_size > 256 || c->n_pages < 1 || c->max_requests < 1) return PIPESD_E_INVALID;
+    if (c->page_size < 8 || c->page_size > 256 || c->page_size % 8 || c->n_pages < 1 || c->max_requests < 1)
+        return PIPESD_E_INVALID;
     if (c->max_draft < 1 || c->max_draft > kMaxItemRows - 1) return PIPESD_E_INVALID;
     if (c->max_rows < c->max_draft + 1 || c->max_rows > 4096 || c->max_seq < 1) return PIPESD_E_INVALID;
     if (!(c->rms_eps >= 0.f) || !(c->rope_base > 1.f)) return PIPESD_E_INVALID;
@@ -214,7 +219,8 @@ struct pipesd_ctx {
     int last_rows = 0;
     int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
     int engine = 0;         // 0: persistent kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only
-    std::vector<MegaPhase> phases;
+    std::vector<MegaPhase> phases;       // GEMM phases only: attention runs as its own kernel between launches
+    std::vector<MegaPhase> phases_att;   // with one attention phase per layer: the whole pass is one launch
     std::string err;
     // launch accounting
     int64_t n_launch = 0, n_gemm = 0;
@@ -689,6 +695,8 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         float* ssqA = ctx->W<float>(ctx->ws.ssqA);
         float* ssqB = ctx->W<float>(ctx->ws.ssqB);
         float* x = ctx->W<float>(ctx->ws.x);
+        for (int with_att = 0; with_att < 2; ++with_att) {
+        std::vector<MegaPhase>& table = with_att ? ctx->phases_att : ctx->phases;
         int ticket0 = 0;
         auto add = [&](const GemmW& g, int mode, const uint32_t* xf) -> MegaPhase& {
             MegaPhase ph = {};
@@ -698,14 +706,24 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
             mega_phase_geometry(ph, g.N, g.K);
             ph.ticket0 = ticket0;
             ticket0 += ph.UB;
-            ctx->phases.push_back(ph);
-            return ctx->phases.back();
+            table.push_back(ph);
+            return table.back();
         };
         for (int l = 0; l < c.n_layers; ++l) {
             const LayerW& lw = ctx->layers[l];
             {
                 MegaPhase& ph = add(lw.qkv, kQkvRope, xf_h);
                 ph.ssq_in = ssqA; ph.n_ssq = n_ssq; ph.layer = l;
+            }
+            if (with_att) {
+                MegaPhase ph = {};
+                ph.mode = kPhaseAttn;
+                ph.UB = c.n_kv_heads;          // one unit per KV head; tiles per head come with each launch
+                ph.layer = l;
+                ph.xf_out = (uint16_t*)xf_attn;
+                ph.ticket0 = ticket0;
+                ticket0 += ph.UB;
+                table.push_back(ph);
             }
             {
                 MegaPhase& ph = add(lw.o, kResid, xf_attn);
@@ -726,10 +744,11 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
             MegaPhase& ph = add(ctx->lm, kPlain, xf_h);
             ph.ssq_in = ssqA; ph.n_ssq = n_ssq; ph.out = ctx->W<float>(ctx->ws.logits);
         }
-        if ((size_t)ticket0 + ctx->phases.size() + c.n_layers + 2 > ctx->ws.mega_ctr_ints) return bail(PIPESD_E_INVALID);
-        if (cudaMemcpyAsync(ctx->wsp + ctx->ws.mega_phases, ctx->phases.data(), sizeof(MegaPhase) * ctx->phases.size(),
-                            cudaMemcpyHostToDevice, st) != cudaSuccess)
+        if ((size_t)ticket0 + table.size() + c.n_layers + 2 > ctx->ws.mega_ctr_ints) return bail(PIPESD_E_INVALID);
+        if (cudaMemcpyAsync(ctx->wsp + (with_att ? ctx->ws.mega_phases_att : ctx->ws.mega_phases), table.data(),
+                            sizeof(MegaPhase) * table.size(), cudaMemcpyHostToDevice, st) != cudaSuccess)
             return bail(PIPESD_E_CUDA);
+        }
         if (cudaStreamSynchronize(st) != cudaSuccess) return bail(PIPESD_E_CUDA);   // the table is read from pageable memory
     }
 
