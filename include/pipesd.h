@@ -177,12 +177,14 @@ int32_t pipesd_reject_from_logits(pipesd_ctx *ctx, int32_t k, int32_t mode, cons
  * pool).  Lets a harness replay rounds from a recorded point; the serving path uses pipesd_kv_rollback. */
 int32_t pipesd_debug_set_len(pipesd_ctx *ctx, int32_t req, int32_t new_len);
 
-/* Which kernels run the GEMM chain.  0 (default): passes of at most 32 rows use the persistent layer-stack
+/* Which kernels run the layer stack.  0 (default): passes of at most 32 rows use the persistent layer-stack
  * kernel (one CTA per SM streams the weights of consecutive projections through the tcgen05 tensor cores
- * without a kernel boundary), larger passes the tiled per-projection kernels.  1: the tiled kernels for every
- * pass; needs a context created with max_rows > 32 (only such a context keeps the weights in the tiled
- * kernels' order as well), PIPESD_E_INVALID otherwise.  Both compute the same forward; their summation
- * orders differ, so results agree to rounding, not bit for bit. */
+ * without a kernel boundary); when the pass is a single request whose query rows per KV head fit one 16-row
+ * tile, attention is a phase of the same kernel and the whole pass is one launch.  Larger passes use the
+ * tiled per-projection kernels.  1: the tiled kernels for every pass; needs a context created with
+ * max_rows > 32 (only such a context keeps the weights in the tiled kernels' order as well), PIPESD_E_INVALID
+ * otherwise.  2: as 0, but attention always runs as its own kernel between persistent launches.  All compute
+ * the same forward; their summation orders differ, so results agree to rounding, not bit for bit. */
 int32_t pipesd_debug_set_engine(pipesd_ctx *ctx, int32_t engine);
 
 /* Launch accounting.  While enabled, every kernel launch of the context is counted and every

@@ -30,8 +30,8 @@ namespace pipesd {
 
 constexpr int kMegaEpiWarps = 8;                           // warp w: 128-row block w >> 2, TMEM lane quarter w & 3
 constexpr int kMegaEpiThreads = kMegaEpiWarps * 32;
-constexpr int kMegaWarpW = 8, kMegaWarpX = 9, kMegaWarpMma = 10;
-constexpr int kMegaThreads = 11 * 32;
+constexpr int kMegaWarpW = 8, kMegaWarpX = 9, kMegaWarpMma = 10, kMegaWarpPub = 11;
+constexpr int kMegaThreads = 12 * 32;
 constexpr int kMegaKC = 4;                                 // k16 steps per chunk
 constexpr int kMegaWHalf = kMegaKC * 4096;                 // one 128-row block of a chunk
 constexpr int kMegaWStage = 2 * kMegaWHalf;                // 256 rows
@@ -207,8 +207,11 @@ __device__ unsigned long long g_mega_trace[64 * 4 * kMegaMaxCtas * 8];
         if (a.launch_idx < 64)                                                                                  \
             g_mega_trace[(((size_t)a.launch_idx * 4 + (p - a.p0)) * kMegaMaxCtas + cta) * 8 + (k)] = global_ns(); \
     } while (0)
+__device__ int g_mega_dbg[kMegaMaxCtas * 8];
+#define MEGA_DBG(slot, val) (g_mega_dbg[blockIdx.x * 8 + (slot)] = (val))
 #else
 #define MEGA_TRACE(k) do { } while (0)
+#define MEGA_DBG(slot, val) do { } while (0)
 #endif
 
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
@@ -549,7 +552,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     if (ok) {
         ok = mbar_wait_err(fullX0 + 8 * st, (uint32_t)(n / kStages) & 1u, a.err);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok && lane == 0) atomicCAS(a.err, 0, 17);
+        if (!ok && lane == 0) atomicCAS(a.err, 0, 17000 + ph.layer);
     }
     uint4* qsm = reinterpret_cast<uint4*>(qarea);      // [k16 step][hi | lo][lane] A fragments of the 16 rows
     const float scale = rsqrtf((float)HD) * 1.4426950408889634f;   // scores in the log2 domain: p = 2^(s - m)
@@ -591,11 +594,12 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     }
     int last_st = st;
     for (int tile = tile0; tile < tile1; ++tile, ++n) {
+        if (threadIdx.x == 0 && ok) { MEGA_DBG(3, n); MEGA_DBG(4, kvh * 1000 + tile); }
         if (ok) {
             const uint32_t par = (uint32_t)(n / kStages) & 1u;
             ok = mbar_wait_err(fullW0 + 8 * st, par, a.err) && mbar_wait_err(fullX0 + 8 * st, par, a.err);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok && lane == 0) atomicCAS(a.err, 0, 18);
+            if (!ok && lane == 0) atomicCAS(a.err, 0, 18000 + ph.layer);
         }
         const int j0 = tile * kAttTile + 8 * warp;           // first key of this warp's strip
         if (ok && j0 < total) {
@@ -737,6 +741,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
     if (warp == 0) { add(1); add(2); add(3); }
     // warp 0 now holds the CTA's un-normalised output for the head, relative to m_tot, with the sum l_tot
+    if (threadIdx.x == 0 && ok) MEGA_DBG(5, 100000 + kvh);
     const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
     constexpr int kSlotFloats = 8 * kMegaEpiThreads * 4;       // one CTA's slot of the exchange array
     if (i0 != i1 && cta != i0) {
@@ -753,6 +758,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
         if (threadIdx.x == 0) {
+            fence_proxy_async_all();      // the stage served as scratch: ordinary stores before the next bulk copy into it
             if (ok) mbar_arrive(empty0 + 8 * last_st);
             st_release_cta(pub_seq, pseg);
         }
@@ -768,7 +774,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     }
     if (i0 != i1 && threadIdx.x == 0) {
         const int n_contrib = T >= G ? i1 - i0 + 1 : CPR;
-        if (!poll_counter(a.tickets + ph.ticket0 + kvh, n_contrib - 1, a.err)) atomicCAS(a.err, 0, 19);
+        if (!poll_counter(a.tickets + ph.ticket0 + kvh, n_contrib - 1, a.err)) atomicCAS(a.err, 0, 19000 + kvh);
     }
     asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
     {
@@ -820,6 +826,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     }
     asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
     if (threadIdx.x == 0) {
+        fence_proxy_async_all();
         if (ok) mbar_arrive(empty0 + 8 * last_st);
         st_release_cta(pub_seq, pseg);
     }
@@ -937,6 +944,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 if (++st == kStages) st = 0;
                 ring.next(a, cta, G);
                 ++n;
+                MEGA_DBG(0, n);
             }
             if (!ok) {
                 atomicCAS(a.err, 0, 11);
@@ -944,7 +952,9 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 for (int i = n > kStages ? n - kStages : 0; i < n; ++i)
                     mbar_wait(fullW0 + 8 * (i % kStages), (uint32_t)(i / kStages) & 1u);
             }
-        } else if (lane == 1) {
+        }
+    } else if (warp == kMegaWarpPub) {
+        if (lane == 0) {
             // ---------------------------------------- publisher: walks the same schedule as the epilogue warps
             // and, whenever they have finished a segment (pub_seq), makes it known to the other CTAs: a
             // contribution counted in, or a unit counted as done.  The release (a fence over all the CTA's
@@ -962,6 +972,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     ++seg;
                     uint64_t t0 = 0;
                     for (uint32_t it = 0; ld_acquire_cta(pub_seq) < seg; ++it) {
+                        __nanosleep(40);
                         if ((it & 63u) == 63u) {
                             if (ld_relaxed(a.err) != 0) { ok = false; break; }
                             const uint64_t now = global_ns();
@@ -973,6 +984,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
                     if (i0 != i1 && cta != i0) red_release_add(a.tickets + ph.ticket0 + u, 1);
                     else red_release_add(a.done + p, 1);
+                    MEGA_DBG(6, seg);
                 }
             }
         }
@@ -985,7 +997,10 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
             if (p == a.p0) {
                 pdl_wait();                       // the kernels launched before this one have completed
             } else {
-                if (lane == 0) ok = poll_counter(a.done + (p - 1), a.phases[p - 1].UB, a.err);
+                if (lane == 0) {
+                    ok = poll_counter(a.done + (p - 1), a.phases[p - 1].UB, a.err);
+                    if (!ok) atomicCAS(a.err, 0, 12000 + p);
+                }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
             }
             if (!ok) break;
@@ -1008,8 +1023,10 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 int cc = cb % CPR, u = cb / CPR;
                 for (int c = cb; c < ce; ++c, ++n) {
                     if (n >= kStages) {
+                        MEGA_DBG(7, 1000 + n);
                         ok = mbar_wait_err(empty0 + 8 * st, (uint32_t)((n / kStages) - 1) & 1u, a.err);
                         if (!ok) break;
+                        MEGA_DBG(7, 2000 + n);
                     }
                     if (ph.mode == kPhaseAttn) {
                         // the pages of the tile that hold rows of this pass (written by the QKV phase); a tile
@@ -1032,7 +1049,9 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     }
                     if (++st == kStages) st = 0;
                     if (++cc == CPR) { cc = 0; ++u; }
+                    MEGA_DBG(1, n + 1);
                 }
+                MEGA_DBG(2, p);
             } else {
                 // lanes 1..31: the input rows' RMSNorm factors, needed only by the epilogue, computed while
                 // lane 0's copies are in flight and handed to the epilogue warps through their own barrier
@@ -1072,9 +1091,18 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 const int T = phase_chunks(a, ph), CPR = phase_cpr(a, ph), KS = ph.KS, RB = ph.RB;
                 const int cb = mega_begin(cta, T, G), ce = mega_begin(cta + 1, T, G);
                 int c = cb;
-                if (ph.mode == kPhaseAttn) {      // the attention chunks are consumed by the epilogue warps
-                    n += ce - cb;
-                    st = (st + (ce - cb)) % kStages;
+                if (ph.mode == kPhaseAttn) {
+                    // The attention chunks are consumed by the epilogue warps.  This thread still follows them
+                    // one by one: a parity wait only tells the current barrier phase from the previous one, so
+                    // a thread that skipped ahead by two uses of a stage would take an old phase for its own.
+                    for (; c < ce; ++c, ++n) {
+                        if (ok) {
+                            const uint32_t par = (uint32_t)(n / kStages) & 1u;
+                            ok = mbar_wait_err(fullW0 + 8 * st, par, a.err) && mbar_wait_err(fullX0 + 8 * st, par, a.err);
+                            if (!ok) atomicCAS(a.err, 0, 13000 + p);
+                        }
+                        if (++st == kStages) st = 0;
+                    }
                     continue;
                 }
                 while (c < ce) {
@@ -1091,7 +1119,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                         if (ok) {
                             const uint32_t par = (uint32_t)(n / kStages) & 1u;
                             ok = mbar_wait_err(fullW0 + 8 * st, par, a.err) && mbar_wait_err(fullX0 + 8 * st, par, a.err);
-                            if (!ok) atomicCAS(a.err, 0, 13);
+                            if (!ok) atomicCAS(a.err, 0, 13000 + p);
                         }
                         if (ok) {
                             tc_fence_after();
@@ -1170,7 +1198,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 if (ok) {
                     ok = mbar_wait_err(accfull0 + 8 * buf, (uint32_t)(seg >> 1) & 1u, a.err);
                     ok = __all_sync(0xffffffffu, ok);
-                    if (!ok && lane == 0) atomicCAS(a.err, 0, 15);
+                    if (!ok && lane == 0) atomicCAS(a.err, 0, 15000 + p);
                 }
                 float v[MT];
                 if (ok) {
@@ -1218,7 +1246,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                         // contributors: every CTA from i0 to i1 when each CTA owns at least one chunk; otherwise
                         // (fewer chunks than CTAs) every chunk of the unit belongs to a different CTA
                         const int n_contrib = T >= G ? i1 - i0 + 1 : CPR;
-                        if (!poll_counter(a.tickets + ph.ticket0 + u, n_contrib - 1, a.err)) atomicCAS(a.err, 0, 14);
+                        if (!poll_counter(a.tickets + ph.ticket0 + u, n_contrib - 1, a.err)) atomicCAS(a.err, 0, 14000 + p);
                     }
                     asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
                     if (threadIdx.x == 0) MEGA_TRACE(3);

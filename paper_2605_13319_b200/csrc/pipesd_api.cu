@@ -218,7 +218,8 @@ struct pipesd_ctx {
     bool pend_check = false;   // a prefill is in flight whose device error word has not been looked at yet
     int last_rows = 0;
     int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
-    int engine = 0;         // 0: persistent kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only
+    int engine = 0;         // 0: persistent kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only;
+                            // 2: as 0, but attention always as its own kernel between the persistent launches
     std::vector<MegaPhase> phases;       // GEMM phases only: attention runs as its own kernel between launches
     std::vector<MegaPhase> phases_att;   // with one attention phase per layer: the whole pass is one launch
     std::string err;
@@ -405,7 +406,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
 
     // Passes of at most 32 rows (one token block) run their GEMMs in the persistent kernel, whose counters
     // start every pass at zero.
-    const bool use_mega = (ctx->engine == 0 && M <= 32) || !needs_tiled(c);
+    const bool use_mega = (ctx->engine != 1 && M <= 32) || !needs_tiled(c);
     if (use_mega) CU(cudaMemsetAsync(ctx->wsp + ctx->ws.mega_ctr, 0, 4 * ctx->ws.mega_ctr_ints, st));
     // Every kernel of the chain is launched with programmatic stream serialisation: it may start while its
     // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
@@ -444,11 +445,22 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     };
     if (use_mega) {
         // Persistent kernel: [QKV 0] attn [O, gate/up, down, QKV 1] attn ... [O, gate/up, down, LM head]
+        // One request whose query rows per KV head fit one 16-row MMA tile (and 16-position pages): attention
+        // runs as a phase of the same launch, and the whole pass is ONE persistent kernel.
+        const bool one_launch = ctx->engine == 0 && n_items == 1 && (Hq / Hkv) * items[0].rows <= 16 && c.page_size == 16;
+        const std::vector<MegaPhase>& table = one_launch ? ctx->phases_att : ctx->phases;
         MegaArgs ma = {};
-        ma.phases = ctx->W<MegaPhase>(ctx->ws.mega_phases);
+        ma.phases = ctx->W<MegaPhase>(one_launch ? ctx->ws.mega_phases_att : ctx->ws.mega_phases);
         ma.M = M;
         int* ctr = ctx->W<int>(ctx->ws.mega_ctr);
-        const int n_phases = (int)ctx->phases.size();
+        const int n_phases = 5 * c.n_layers + 1;      // counters are laid out for the longer table
+        if (one_launch) {
+            const Request& r = ctx->reqs[items[0].slot];
+            ma.att_base = r.len;
+            ma.att_rows = items[0].rows;
+            ma.att_cpr = (r.len + items[0].rows + kAttTile - 1) / kAttTile;
+            ma.att_bt = ctx->W<int32_t>(ctx->ws.block_tab) + (size_t)items[0].slot * dv.max_pages;
+        }
         ma.done = ctr;
         ma.tickets = ctr + n_phases + c.n_layers + 2;
         ma.scratch = ctx->W<float4>(ctx->ws.mega_scratch);
@@ -481,18 +493,25 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             ctx->n_launch += 1;
             ctx->n_gemm += 1;
             for (int p = p0; p < p1; ++p) {
-                const MegaPhase& ph = ctx->phases[p];
-                ctx->gemm_bytes += 2.0 * ph.N * ph.KS * 16 + 4.0 * M * ph.KS * 16 + 4.0 * M * ph.N;
+                const MegaPhase& ph = table[p];
+                if (ph.mode == kPhaseAttn)   // K and V of every key once
+                    ctx->gemm_bytes += 2.0 * (ma.att_base + ma.att_rows) * Hkv * hd * 2.0;
+                else
+                    ctx->gemm_bytes += 2.0 * ph.N * ph.KS * 16 + 4.0 * M * ph.KS * 16 + 4.0 * M * ph.N;
             }
             return PIPESD_OK;
         };
-        int rc_ = launch_mega(0, 0, 1);
-        if (rc_) return rc_;
+        int rc_;
+        if (one_launch) {
+            if ((rc_ = launch_mega(0, 0, want_logits ? 5 * c.n_layers + 1 : 5 * c.n_layers))) return rc_;
+        } else {
+        if ((rc_ = launch_mega(0, 0, 1))) return rc_;
         for (int l = 0; l < c.n_layers; ++l) {
             if ((rc_ = launch_attn(l))) return rc_;
             const bool last = l + 1 == c.n_layers;
             const int p1 = last ? (want_logits ? 4 * l + 5 : 4 * l + 4) : 4 * l + 5;
             if ((rc_ = launch_mega(l + 1, 4 * l + 1, p1))) return rc_;
+        }
         }
     } else
     for (int l = 0; l < c.n_layers; ++l) {
@@ -1064,13 +1083,16 @@ int32_t pipesd_debug_set_len(pipesd_ctx* ctx, int32_t req, int32_t new_len) {
 }
 
 #ifdef PIPESD_MEGA_TRACE
+int32_t pipesd_debug_mega_dbg(int* dst, int32_t n) {
+    return cudaMemcpyFromSymbol(dst, g_mega_dbg, sizeof(int) * (size_t)n) == cudaSuccess ? 0 : -6;
+}
 int32_t pipesd_debug_mega_trace(unsigned long long* dst, int32_t n) {
     return cudaMemcpyFromSymbol(dst, g_mega_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
 }
 #endif
 
 int32_t pipesd_debug_set_engine(pipesd_ctx* ctx, int32_t engine) {
-    if (!ctx || engine < 0 || engine > 1) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine");
+    if (!ctx || engine < 0 || engine > 2) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine");
     if (engine == 1 && !needs_tiled(ctx->cfg))
         return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine: the tiled kernels need a context with max_rows > 32");
     ctx->engine = engine;
