@@ -44,7 +44,7 @@ constexpr int kMegaMaxCtas = 160;
 constexpr int kMegaSmemMax = 227 * 1024;
 constexpr int kMegaTmemCols = 256;                         // 2 accumulators x 2 blocks x up to 64 columns
 #ifndef PIPESD_MEGA_L2AHEAD
-#define PIPESD_MEGA_L2AHEAD 8
+#define PIPESD_MEGA_L2AHEAD 0
 #endif
 constexpr int kMegaL2Ahead = PIPESD_MEGA_L2AHEAD;                           // chunks a blocked weight producer pulls into L2
 #ifndef PIPESD_MEGA_INFLIGHT
@@ -383,7 +383,8 @@ __device__ __forceinline__ float warp_token_sums(float (&s)[MTP], int lane, int&
 // 16-row tile: lanes l and l ^ 8.
 template <int NT, int MODE>
 __device__ __forceinline__ void mega_epilogue(const MegaArgs& a, const MegaPhase& ph, int p, int cta, int u, int warp, int lane,
-                                              float (&v)[NT * 8], const float* rstd_s, float* ssq_w) {
+                                              float (&v)[NT * 8], const float (&pa)[NT * 8], const float (&pb)[NT * 8],
+                                              const float* rstd_s, float* ssq_w, const long long* kvoff_s) {
     constexpr int MT = NT * 8;
     const int N = ph.N, M = a.M;
     const int pr = u * 256 + warp * 32 + lane;
@@ -402,20 +403,22 @@ __device__ __forceinline__ void mega_epilogue(const MegaArgs& a, const MegaPhase
     }
     if (MODE == kResid) {
         constexpr int MTP = MT <= 8 ? 8 : (MT <= 16 ? 16 : 32);
-        float xv[MT], sq[MTP];
-#pragma unroll
-        for (int t = 0; t < MT; ++t) xv[t] = (row_live && t < M) ? __ldcg(ph.x + (size_t)t * N + pr) : 0.f;
-        const float gain = row_live ? ph.gain_next[pr] : 0.f;
+        float sq[MTP];
+        const float gain = pb[0];                    // pa: the row's residual values, fetched when the unit started
 #pragma unroll
         for (int t = 0; t < MTP; ++t) sq[t] = 0.f;
 #pragma unroll
         for (int t = 0; t < MT; ++t) {
-            const float xn = xv[t] + v[t];
-            if (row_live && t < M) {
-                ph.x[(size_t)t * N + pr] = xn;
-                sq[t] = xn * xn;
+            if (t < M) {                              // uniform: rows of padding tokens cost nothing
+                const float xn = pa[t] + v[t];
+                if (row_live) {
+                    ph.x[(size_t)t * N + pr] = xn;
+                    sq[t] = xn * xn;
+                }
+                v[t] = xn * gain;
+            } else {
+                v[t] = 0.f;
             }
-            v[t] = (t < M) ? xn * gain : 0.f;
         }
         if (row_live) {
             // this row is k index pr of the next projection: one 16-byte piece per 8 tokens, hi and lo
@@ -450,9 +453,13 @@ __device__ __forceinline__ void mega_epilogue(const MegaArgs& a, const MegaPhase
         // lane stores the hi pieces and the up lane the lo pieces
 #pragma unroll
         for (int t = 0; t < MT; ++t) {
-            const float other = __shfl_xor_sync(0xffffffffu, v[t], 8);
-            const float gt = upper ? other : v[t], up = upper ? v[t] : other;
-            v[t] = (t < M) ? gt / (1.f + expf(-gt)) * up : 0.f;
+            if (t < M) {                              // uniform
+                const float other = __shfl_xor_sync(0xffffffffu, v[t], 8);
+                const float gt = upper ? other : v[t], up = upper ? v[t] : other;
+                v[t] = gt / (1.f + expf(-gt)) * up;
+            } else {
+                v[t] = 0.f;
+            }
         }
         if ((pr | 8) < N) {
             const int f = (pr >> 4) * 8 + (lane & 7);
@@ -477,29 +484,50 @@ __device__ __forceinline__ void mega_epilogue(const MegaArgs& a, const MegaPhase
         const int kvh = kv ? head - a.Hq - a.Hkv : head - a.Hq;
         const size_t per_head = (size_t)a.page_size * hd;
         const size_t kv_base = (size_t)ph.layer * a.n_pages * 2 * a.Hkv * per_head + ((size_t)kv * a.Hkv + kvh) * per_head;
-        // every global load first (rotary factors, K/V slots), then the arithmetic and the stores
-        float cv[MT], sv[MT];
-        long long ko[MT];
+        // pa / pb: the rotary factors of this row's dim for every token, fetched when the unit started
 #pragma unroll
         for (int t = 0; t < MT; ++t) {
-            const bool on = row_live && t < M;
-            cv[t] = (on && rot) ? a.cs[(size_t)t * half + dlow] : 1.f;
-            sv[t] = (on && rot) ? a.sn[(size_t)t * half + dlow] : 0.f;
-            ko[t] = (on && head >= a.Hq) ? a.row_kvoff[t] : 0;
-        }
-#pragma unroll
-        for (int t = 0; t < MT; ++t) {
+            if (t >= M) break;                        // uniform
             const float other = __shfl_xor_sync(0xffffffffu, v[t], 8);
-            const float o = upper ? v[t] * cv[t] + other * sv[t] : v[t] * cv[t] - other * sv[t];
+            const float o = rot ? (upper ? v[t] * pa[t] + other * pb[t] : v[t] * pa[t] - other * pb[t]) : v[t];
             // K/V: neighbouring dims of one token travel as one 4-byte store
             const uint32_t mine = f32_to_bf16_bits(o);
             const uint32_t nb = __shfl_xor_sync(0xffffffffu, mine, 1);
-            if (row_live && t < M) {
+            if (row_live) {
                 if (head < a.Hq) a.q_out[((size_t)t * a.Hq + head) * hd + dim] = o;
-                else if ((lane & 1) == 0)
-                    *reinterpret_cast<uint32_t*>(a.kv_pool + (size_t)(ko[t] & ~7ll) + kv_base + kv_swizzle(dim, (int)(ko[t] & 7))) =
+                else if ((lane & 1) == 0) {
+                    const long long ko = kvoff_s[t];
+                    *reinterpret_cast<uint32_t*>(a.kv_pool + (size_t)(ko & ~7ll) + kv_base + kv_swizzle(dim, (int)(ko & 7))) =
                         mine | (nb << 16);
+                }
             }
+        }
+    }
+}
+
+// What the epilogue of unit u will read from global memory besides the accumulators, fetched before the
+// accumulators are waited for (none of it depends on the phase in progress): kResid -- the row's residual values
+// (pa) and the next norm's gain (pb[0]); kQkvRope -- cos (pa) and sin (pb) of the row's dim for every token.
+template <int NT>
+__device__ __forceinline__ void mega_preload(const MegaArgs& a, const MegaPhase& ph, int u, int warp, int lane,
+                                             float (&pa)[NT * 8], float (&pb)[NT * 8]) {
+    constexpr int MT = NT * 8;
+    const int N = ph.N, M = a.M;
+    const int pr = u * 256 + warp * 32 + lane;
+    const bool row_live = pr < N;
+    if (ph.mode == kResid) {
+#pragma unroll
+        for (int t = 0; t < MT; ++t) pa[t] = (row_live && t < M) ? __ldcg(ph.x + (size_t)t * N + pr) : 0.f;
+        pb[0] = row_live ? ph.gain_next[pr] : 0.f;
+    } else if (ph.mode == kQkvRope) {
+        const int hd = a.hd, half = hd / 2;
+        const int head = pr / hd, within = pr - head * hd;
+        const int dlow = 8 * (within >> 4) + (lane & 7);
+        const bool rot = row_live && head < a.Hq + a.Hkv;
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+            pa[t] = (rot && t < M) ? a.cs[(size_t)t * half + dlow] : 1.f;
+            pb[t] = (rot && t < M) ? a.sn[(size_t)t * half + dlow] : 0.f;
         }
     }
 }
@@ -540,7 +568,7 @@ __device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t&
 // owns the head's first tile, exactly as the GEMM units are, and the normalised output goes to the output
 // projection's input array.  Every named barrier below is reached by all 256 threads, also after a failed wait.
 template <int HD>
-__device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& ph, int cta, int G, int kvh, int tile0, int tile1,
+__device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& ph, int p, int cta, int G, int kvh, int tile0, int tile1,
                                             int ub, int T, int CPR, int NT, int kStages, int kStage, unsigned char* smem,
                                             uint32_t fullW0, uint32_t fullX0, uint32_t empty0, int& n, int& st, bool& ok,
                                             unsigned char* qarea, float* xch, int pseg, int* pub_seq) {
@@ -595,6 +623,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     int last_st = st;
     for (int tile = tile0; tile < tile1; ++tile, ++n) {
         if (threadIdx.x == 0 && ok) { MEGA_DBG(3, n); MEGA_DBG(4, kvh * 1000 + tile); }
+        if (threadIdx.x == 0 && tile == tile0) MEGA_TRACE(1);
         if (ok) {
             const uint32_t par = (uint32_t)(n / kStages) & 1u;
             ok = mbar_wait_err(fullW0 + 8 * st, par, a.err) && mbar_wait_err(fullX0 + 8 * st, par, a.err);
@@ -682,6 +711,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
         }
         if (++st == kStages) st = 0;
     }
+    if (threadIdx.x == 0) MEGA_TRACE(6);
     // ---- merge the eight warps: common maximum, rescaled sums, outputs added in the order
     // ((w0 + w4) + (w1 + w5)) + (w2 + w6) + (w3 + w7)
 #pragma unroll
@@ -742,6 +772,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     if (warp == 0) { add(1); add(2); add(3); }
     // warp 0 now holds the CTA's un-normalised output for the head, relative to m_tot, with the sum l_tot
     if (threadIdx.x == 0 && ok) MEGA_DBG(5, 100000 + kvh);
+    if (threadIdx.x == 0) MEGA_TRACE(2);
     const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
     constexpr int kSlotFloats = 8 * kMegaEpiThreads * 4;       // one CTA's slot of the exchange array
     if (i0 != i1 && cta != i0) {
@@ -761,6 +792,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
             fence_proxy_async_all();      // the stage served as scratch: ordinary stores before the next bulk copy into it
             if (ok) mbar_arrive(empty0 + 8 * last_st);
             st_release_cta(pub_seq, pseg);
+            MEGA_TRACE(3);
         }
         return;
     }
@@ -829,6 +861,7 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
         fence_proxy_async_all();
         if (ok) mbar_arrive(empty0 + 8 * last_st);
         st_release_cta(pub_seq, pseg);
+        MEGA_TRACE(5);
     }
 }
 
@@ -844,6 +877,9 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
     unsigned char* tail = smem + kStages * kStage;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);          // fullW[8] | fullX[8] | empty[8] | accfull[2] | accempty[2] | drain | rstd
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256);
+    long long* kvoff_s = reinterpret_cast<long long*>(tail + 1536);   // [32] K/V slot offsets of the pass's rows
+    int4* att_pg_s = reinterpret_cast<int4*>(tail + 1792);        // page ids of sixteen attention tiles (weight producer's)
+    int* dep_seq = reinterpret_cast<int*>(tail + 328);            // 1 + last phase whose input is complete (activation producer -> epilogue)
     int* pub_seq = reinterpret_cast<int*>(tail + 320);            // segments whose stores are complete (epilogue -> publisher)
     float* rstd_s = reinterpret_cast<float*>(tail + 384);        // [32]
     float* ssq_w = reinterpret_cast<float*>(tail + 512);         // [8][32]
@@ -866,6 +902,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
         mbar_init(drain0, 1);
         mbar_init(rstd0, 1);
         *pub_seq = 0;
+        *dep_seq = 0;
         fence_mbar_init();
         red_release_add(a.arrived, 1);
     }
@@ -890,8 +927,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
             bool ok = true;
             long long t_pf = clock64();
             const uint64_t pol = l2_evict_first_policy();
-            int4 att_pages = make_int4(0, 0, 0, 0);
-            int att_tile = -1, att_phase = -1;   // chunk index and phase whose page ids att_pages holds
+            int att_phase = -1, att_c0 = 0;      // phase and first chunk whose page ids att_pg_s holds
             while (ring.valid()) {
                 // At most kMegaMaxInFlight chunks are outstanding: enough to keep HBM busy (148 SMs x 96 KB is
                 // twice the bandwidth-latency product), while every byte beyond that only queues in front of
@@ -924,16 +960,22 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 if (!ok) break;
                 if (ring.mode == kPhaseAttn) {
                     // K/V tile of an attention phase: the pages cached before this pass (the others are the
-                    // activation producer's); the next tile's page ids are fetched one chunk ahead
-                    if (att_tile != ring.c || att_phase != ring.p) att_pages = att_tile_pages(a, ring.cc);
-                    att_phase = ring.p;
+                    // activation producer's).  Page ids are fetched sixteen tiles at a time (one memory latency
+                    // per sixteen chunks instead of one per chunk) and kept in shared memory.
+                    if (att_phase != ring.p || ring.c < att_c0 || ring.c >= att_c0 + 16) {
+                        int4 tmp[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            tmp[i] = ring.c + i < ring.ce ? att_tile_pages(a, (ring.cc + i) % ring.CPR) : make_int4(0, 0, 0, 0);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) att_pg_s[i] = tmp[i];
+                        att_phase = ring.p;
+                        att_c0 = ring.c;
+                    }
+                    const int4 att_pages = att_pg_s[ring.c - att_c0];
                     const uint32_t bytes = att_issue_pages(a, ring.layer, ring.u, ring.cc, false, att_pages, 0, 0, true);
                     mbar_expect_tx(fullW0 + 8 * st, bytes);
                     att_issue_pages(a, ring.layer, ring.u, ring.cc, false, att_pages, smem_base + st * kStage, fullW0 + 8 * st, false);
-                    if (ring.c + 1 < ring.ce) {
-                        att_pages = att_tile_pages(a, ring.cc + 1 == ring.CPR ? 0 : ring.cc + 1);
-                        att_tile = ring.c + 1;
-                    }
                 } else {
                     const uint32_t bytes = (uint32_t)ring.kc() * 4096u;
                     const bool two = ring.two();
@@ -1004,7 +1046,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 ok = __shfl_sync(0xffffffffu, ok, 0);
             }
             if (!ok) break;
-            if (lane == 0) MEGA_TRACE(0);
+            if (lane == 0) { st_release_cta(dep_seq, p + 1); MEGA_TRACE(0); }
             if (p == a.p1 - 1) {
                 // Successor kernels may be scheduled from here on -- but only once every CTA of this grid
                 // is resident: a successor that took the place of a CTA still to come would wait for this
@@ -1152,6 +1194,8 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
     } else {
         // ------------------------------------------------ epilogue warps
         pdl_wait();      // epilogues read what earlier kernels wrote (rotary tables, K/V offsets, residual stream)
+        if (threadIdx.x < 32) kvoff_s[threadIdx.x] = threadIdx.x < a.M ? a.row_kvoff[threadIdx.x] : 0;
+        asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
         int seg = 0, n_norm = 0;      // n_norm: phases so far whose input is normalised and in which this CTA has work
         int pseg = 0;                 // segments finished (GEMM units and attention heads): what the publisher counts
         int n = 0, st = 0;            // chunk counter / ring stage: followed for the attention phases
@@ -1168,17 +1212,15 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     const int se = ce < ub + CPR ? ce : ub + CPR;
                     ++pseg;
                     if (a.hd == 128)
-                        att_segment<128>(a, ph, cta, G, u, c - ub, se - ub, ub, T, CPR, NT, kStages, kStage, smem, fullW0, fullX0,
+                        att_segment<128>(a, ph, p, cta, G, u, c - ub, se - ub, ub, T, CPR, NT, kStages, kStage, smem, fullW0, fullX0,
                                          empty0, n, st, ok, tail + kMegaTail, ssq_w, pseg, pub_seq);
                     else
-                        att_segment<64>(a, ph, cta, G, u, c - ub, se - ub, ub, T, CPR, NT, kStages, kStage, smem, fullW0, fullX0,
+                        att_segment<64>(a, ph, p, cta, G, u, c - ub, se - ub, ub, T, CPR, NT, kStages, kStage, smem, fullW0, fullX0,
                                         empty0, n, st, ok, tail + kMegaTail, ssq_w, pseg, pub_seq);
                     c = se;
                 }
                 continue;
             }
-            n += ce - cb;
-            st = (st + (ce - cb)) % kStages;
             if (cb < ce && ph.ssq_in != nullptr) {
                 // the activation producer has derived this phase's RMSNorm factors
                 if (ok) {
@@ -1191,8 +1233,29 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
             while (c < ce) {
                 const int u = c / CPR, ub = u * CPR;
                 const int se = ce < ub + CPR ? ce : ub + CPR;
-                c = se;
                 const int buf = seg & 1;
+                const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
+                float pa[MT], pb[MT];
+                if (i0 == i1 || cta == i0) {      // this CTA runs the unit's epilogue: fetch its inputs now
+                    // the residual stream is final once the phase's input is complete (it was written two phases
+                    // back): the activation producer notes in dep_seq which phases' inputs it has seen complete
+                    if (ok && mode == kResid) {
+                        uint64_t t0 = 0;
+                        for (uint32_t it = 0; ld_acquire_cta(dep_seq) <= p; ++it) {
+                            if ((it & 63u) == 63u) {
+                                const uint64_t now = global_ns();
+                                if (t0 == 0) t0 = now;
+                                else if (ld_relaxed(a.err) != 0 || now - t0 > kMegaWaitNs) { ok = false; break; }
+                            }
+                        }
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok && lane == 0) atomicCAS(a.err, 0, 20000 + p);
+                    }
+                    mega_preload<NT>(a, ph, u, warp, lane, pa, pb);
+                }
+                n += se - c;
+                st = (st + (se - c)) % kStages;
+                c = se;
                 // A wait that gave up is not an exit: the warp keeps walking the schedule (without waiting) so
                 // that it still meets the other epilogue warps at every named barrier below.
                 if (ok) {
@@ -1229,13 +1292,13 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 // so it waits for little): the others leave their rows in global memory and count themselves
                 // in; the collector waits for that count, adds the contributions to its own in CTA order (a
                 // fixed order), and runs the epilogue.  Contributors never wait.
-                const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
+                const int nq = (a.M + 3) / 4;           // 16-byte words of a row that hold real tokens
                 if (i0 != i1) {
                     if (cta != i0) {
                         float4* mine = a.scratch + ((size_t)cta * (2 * NT)) * kMegaEpiThreads + threadIdx.x;
 #pragma unroll
                         for (int q = 0; q < 2 * NT; ++q)
-                            mine[(size_t)q * kMegaEpiThreads] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                            if (q < nq) mine[(size_t)q * kMegaEpiThreads] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
                         // all stores of the CTA happen before thread 0's signal to the publisher thread (ordered by
                         // the named barrier), which counts the CTA in with a release
                         asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
@@ -1253,6 +1316,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     // contributions are fetched eight CTAs at a time, two 16-byte words each (16 loads in flight),
                     // and added in CTA order
                     for (int q0 = 0; q0 < 2 * NT; q0 += 2) {
+                        if (q0 >= nq) break;
                         for (int ib = i0 + 1; ib <= i1; ib += 8) {
                             float4 w[8][2];
 #pragma unroll
@@ -1261,7 +1325,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                                 const bool on = i <= i1 && (T >= G || mega_begin(i, T, G) != mega_begin(i + 1, T, G));
                                 const float4* src = a.scratch + ((size_t)i * (2 * NT) + q0) * kMegaEpiThreads + threadIdx.x;
                                 w[k][0] = on ? __ldcg(src) : make_float4(0.f, 0.f, 0.f, 0.f);
-                                w[k][1] = on ? __ldcg(src + kMegaEpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                w[k][1] = (on && q0 + 1 < nq) ? __ldcg(src + kMegaEpiThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
                             }
 #pragma unroll
                             for (int k = 0; k < 8; ++k)
@@ -1276,10 +1340,10 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     }
                 }
                 if (threadIdx.x == 0) MEGA_TRACE(4);
-                if (mode == kPlain) mega_epilogue<NT, kPlain>(a, ph, p, cta, u, warp, lane, v, rstd_s, ssq_w);
-                else if (mode == kQkvRope) mega_epilogue<NT, kQkvRope>(a, ph, p, cta, u, warp, lane, v, rstd_s, ssq_w);
-                else if (mode == kResid) mega_epilogue<NT, kResid>(a, ph, p, cta, u, warp, lane, v, rstd_s, ssq_w);
-                else mega_epilogue<NT, kSwiglu>(a, ph, p, cta, u, warp, lane, v, rstd_s, ssq_w);
+                if (mode == kPlain) mega_epilogue<NT, kPlain>(a, ph, p, cta, u, warp, lane, v, pa, pb, rstd_s, ssq_w, kvoff_s);
+                else if (mode == kQkvRope) mega_epilogue<NT, kQkvRope>(a, ph, p, cta, u, warp, lane, v, pa, pb, rstd_s, ssq_w, kvoff_s);
+                else if (mode == kResid) mega_epilogue<NT, kResid>(a, ph, p, cta, u, warp, lane, v, pa, pb, rstd_s, ssq_w, kvoff_s);
+                else mega_epilogue<NT, kSwiglu>(a, ph, p, cta, u, warp, lane, v, pa, pb, rstd_s, ssq_w, kvoff_s);
                 // publish: the named barrier orders every thread's stores before thread 0's signal; the publisher
                 // thread counts the unit as done with a release, so that no epilogue warp waits for the fence;
                 // readers acquire the counter (and fence the asynchronous proxy before their bulk copies)
