@@ -253,6 +253,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b-k8", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--engine", default="tiled", choices=["tiled", "persistent"],
+                    help="which kernels run the layer stack (the headline is the faster one on this workload: tiled)")
+    ap.add_argument("--no-other-engine", action="store_true", help="skip the short timing of the other engine")
     ap.add_argument("--quick-inputs", action="store_true",
                     help="profiler runs: seeded synthetic K/V prefix and random drafts instead of a recorded "
                          "trajectory, one timed region only, so that few launches precede the captured ones")
@@ -282,7 +285,7 @@ def main():
     max_seq = P + n_rounds * (k + 1) + 64
     weights = synth.make_weights(shape, seed)
     ctx = binding.Context(shape, weights, n_pages=max_seq // 16 + 4, max_seq=max_seq, max_draft=max(k, 16),
-                          device=local)
+                          device=local, engine=args.engine)
     prefix = synth.make_prefix(shape, P, seed + rank)
     if args.quick_inputs:
         quick_run(args, ctx, shape, P, k, seed, torch)
@@ -330,8 +333,26 @@ def main():
     replay(ctx, req, rounds[args.warmup:], False, torch)
     gprof = ctx.profile_read()
     ctx.profile_enable(False)
-    clocks = sampler.stop()
     ctx.req_close(req)
+    # -- the other engine on the same recorded rounds (device-resident inputs only), for comparison
+    other = None
+    if world == 1 and not args.no_other_engine:
+        ctx.close()
+        oname = "persistent" if args.engine == "tiled" else "tiled"
+        ctx = binding.Context(shape, weights, n_pages=max_seq // 16 + 4, max_seq=max_seq, max_draft=max(k, 16),
+                              device=local, engine=oname)
+        req = ctx.req_open()
+        ctx.prefill(req, prefix)
+        replay(ctx, req, rounds[:args.warmup], False, torch, timed=False)
+        ctx.profile_enable(False)
+        ctx.profile_read()
+        ms_o, tokens_o, mism_o = replay(ctx, req, rounds[args.warmup:], False, torch)
+        prof_o = ctx.profile_read()
+        other = {"engine": oname, "ms_per_step": ms_o / args.steps, "value": tokens_o / (ms_o * 1e-3), "unit": "tokens/s",
+                 "gpu_launches": int(prof_o["kernel_launches"]),
+                 "decisions_differing_from_recording": int(mism_o)}
+        ctx.req_close(req)
+    clocks = sampler.stop()
 
     # -- reduce over ranks: max time, summed tokens
     if world > 1:
@@ -355,7 +376,7 @@ def main():
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 weights x split-bf16 activations, fp32 accumulate", "data": "synthetic",
-        "config": {"workload": args.workload, "shape": shape.name, "prefix": P, "k": k, "sigma": sigma,
+        "config": {"workload": args.workload, "shape": shape.name, "prefix": P, "k": k, "sigma": sigma, "engine": args.engine,
                    "rounds": steps, "l2": "inputs larger than L2 (weights streamed once per pass)",
                    "accepted_per_step": tokens / world / steps - 1.0, "replay_mismatches": int(mism + mism2)},
         "pass": {"bytes": bytes_pass, "gbs": bytes_pass / (ms_step * 1e-3) / 1e9,
@@ -365,13 +386,15 @@ def main():
                 "h2d_bytes_per_step": int(4 * k * shape.vocab + 4 * (k + 1) * 2),
                 "d2h_bytes_per_step": 16},
         "gpu_launches": int(prof["kernel_launches"]),
-        "roofline": {"bound": "hbm", "kernel": "gemm_wstream_kernel", "achieved": gemm_gbs, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "gemm_wstream_kernel" if args.engine == "tiled" else "mega_kernel", "achieved": gemm_gbs, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": gemm_gbs / peak,
                      "launches": int(gprof["gemm_launches"]), "share_of_step": gprof["gemm_ms"] / ms,
                      "algorithmic_bytes_per_launch": gprof["gemm_bytes"] / max(1, gprof["gemm_launches"]),
-                     "traffic": TRAFFIC_7B_K8 if args.workload == "7b-k8" else None},
+                     "traffic": TRAFFIC_7B_K8.get(args.engine) if args.workload == "7b-k8" else None},
         "clocks": clocks,
     }
+    if other is not None:
+        line["other_engine"] = other
     if world == 1 and not args.no_cpu_baseline:
         dt, toks_o, _ = oracle_sample(shape, weights, P, k, sigma, seed)
         line["cpu_baseline"] = {"value": toks_o / dt, "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle",
@@ -417,11 +440,11 @@ def quick_run(args, ctx, shape, P, k, seed, torch):
     ctx.close()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (average over the 129 GEMM
-# launches of a 7b pass), from the ncu capture summarised in profiles/gemm_and_attention_7b_shape_counters.md:
-# taken on a two-layer model of the same shape (same per-layer kernels) and scaled by launch counts.
-# None for other workloads, and to be reset to None when the GEMM kernel changes.
-TRAFFIC_7B_K8 = 102.9e6
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
+# under profiles/ (taken on a two-layer model of the same shape -- same per-layer work -- and scaled to a full
+# launch by the layers it covers).  None until a capture of the current kernel exists, and to be reset to None
+# whenever that kernel changes.
+TRAFFIC_7B_K8 = {"tiled": None, "persistent": None}
 
 
 if __name__ == "__main__":

@@ -19,6 +19,9 @@ OK, E_INVALID, E_FULL, E_OOM_PAGES, E_STATE, E_RANGE, E_CUDA, E_NOMEM = 0, -1, -
 E_TOO_LARGE = -8
 STATIC_SCRATCH_BYTES = 8 << 20
 MODE_STOCHASTIC, MODE_GREEDY = 0, 1
+ENGINE_TILED, ENGINE_PERSISTENT = 0, 1
+ENGINES = {"tiled": ENGINE_TILED, "persistent": ENGINE_PERSISTENT}
+DEFAULT_ENGINE = "tiled"
 Q_HOST = 1
 
 i32, u32, u64, f32, vp = ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float, ctypes.c_void_p
@@ -27,7 +30,7 @@ i32, u32, u64, f32, vp = ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctype
 class ModelCfg(ctypes.Structure):
     _fields_ = [(n, i32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab")] \
         + [("rms_eps", f32), ("rope_base", f32)] \
-        + [(n, i32) for n in ("page_size", "n_pages", "max_requests", "max_draft", "max_rows", "max_seq", "device")]
+        + [(n, i32) for n in ("page_size", "n_pages", "max_requests", "max_draft", "max_rows", "max_seq", "device", "engine")]
 
 
 class LayerWeights(ctypes.Structure):
@@ -126,7 +129,7 @@ class Context:
 
     def __init__(self, shape, weights: dict, *, n_pages: int, max_requests: int = 1, max_draft: int = 16,
                  max_rows: int | None = None, max_seq: int = 4096, page_size: int = 16, device: int = 0,
-                 stream=None):
+                 stream=None, engine: str | None = None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: the verify pass has no CPU path")
@@ -139,7 +142,8 @@ class Context:
             max_rows = max(max_draft + 1, 32)
         self.cfg = ModelCfg(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                             shape.d_ffn, shape.vocab, shape.rms_eps, shape.rope_base, page_size, n_pages,
-                            max_requests, max_draft, max_rows, max_seq, device)
+                            max_requests, max_draft, max_rows, max_seq, device, ENGINES[engine or DEFAULT_ENGINE])
+        self.engine = engine or DEFAULT_ENGINE
         L = lib()
         sz = Sizes()
         rc = L.pipesd_query_sizes(ctypes.byref(self.cfg), ctypes.byref(sz))

@@ -106,6 +106,19 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uin
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// Weights are read once per pass: their lines are marked evict-first in L2, so that the 400 MB a layer streams
+// do not push out the few megabytes every phase boundary depends on (residual stream, activations, partial sums,
+// rotary tables), which would otherwise come back from HBM behind the weight stream's own queue.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+                 : "memory");
+}
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
 // while its predecessor drains; pdl_wait() blocks until the predecessor has completed and its writes
 // are visible, pdl_launch_dependents() lets the successor start early.

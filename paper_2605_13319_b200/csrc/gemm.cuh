@@ -224,11 +224,12 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                 reinterpret_cast<const unsigned char*>(a.xf) + ((size_t)tb * a.KS + ks0) * (NT * 512);
             auto chunk_ks = [&](int c) { int r = nks - c * kGemmKC; return r < kGemmKC ? r : kGemmKC; };
             const int pre = nchunks < stages ? nchunks : stages;
+            const uint64_t pol = l2_evict_first_policy();   // weights are read once: they must not push the activations out of L2
             // weights do not depend on the previous kernel: start them before the dependency wait
             for (int c = 0; c < pre; ++c) {
                 const int kc = chunk_ks(c);
                 mbar_expect_tx(full0 + 8 * c, (uint32_t)kc * (4096 + NT * 512));
-                bulk_g2s(smem_base + c * kStageBytes, wsrc + (size_t)c * kGemmWStage, (uint32_t)kc * 4096, full0 + 8 * c);
+                bulk_g2s_hint(smem_base + c * kStageBytes, wsrc + (size_t)c * kGemmWStage, (uint32_t)kc * 4096, full0 + 8 * c, pol);
             }
             pdl_wait();
             for (int c = 0; c < pre; ++c) {
@@ -243,7 +244,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                 ok = mbar_wait(empty0 + 8 * st, ph);
                 if (!ok) break;
                 mbar_expect_tx(full0 + 8 * st, (uint32_t)kc * (4096 + NT * 512));
-                bulk_g2s(smem_base + st * kStageBytes, wsrc + (size_t)c * kGemmWStage, (uint32_t)kc * 4096, full0 + 8 * st);
+                bulk_g2s_hint(smem_base + st * kStageBytes, wsrc + (size_t)c * kGemmWStage, (uint32_t)kc * 4096, full0 + 8 * st, pol);
                 bulk_g2s(smem_base + st * kStageBytes + kGemmWStage, bsrc + (size_t)c * kBStage,
                          (uint32_t)kc * NT * 512, full0 + 8 * st);
                 issued = c + 1;

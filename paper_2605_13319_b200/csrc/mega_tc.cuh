@@ -254,19 +254,6 @@ __device__ __forceinline__ bool poll_counter(const int* ctr, int target, const i
 __device__ __forceinline__ int mega_owner(int c, int T, int G) { return (int)((((unsigned)c + 1u) * (unsigned)G - 1u) / (unsigned)T); }
 __device__ __forceinline__ int mega_begin(int i, int T, int G) { return (int)(((unsigned)T * (unsigned)i) / (unsigned)G); }
 
-// Weights are read once per pass: their lines are marked evict-first in L2, so that the 400 MB a layer streams
-// do not push out the few megabytes every phase boundary depends on (residual stream, activations, partial sums,
-// rotary tables), which would otherwise come back from HBM behind the weight stream's own queue.
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst_smem),
-                 "l"(src), "r"(bytes), "r"(bar), "l"(pol)
-                 : "memory");
-}
 __device__ __forceinline__ int phase_cpr(const MegaArgs& a, const MegaPhase& ph) { return ph.mode == kPhaseAttn ? a.att_cpr : ph.CPR; }
 __device__ __forceinline__ int phase_chunks(const MegaArgs& a, const MegaPhase& ph) {
     return ph.mode == kPhaseAttn ? a.att_cpr * ph.UB : ph.T;
@@ -645,7 +632,8 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
                 }
                 __syncwarp();
             }
-            float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+            // four independent accumulation chains (hi / lo terms x even / odd k16 steps), summed in a fixed order
+            float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f}, s3[4] = {0.f, 0.f, 0.f, 0.f}, s4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int kp = 0; kp < KSTEPS / 2; ++kp) {
                 const uint4 qh0 = qsm[((2 * kp) * 2 + 0) * 32 + lane], ql0 = qsm[((2 * kp) * 2 + 1) * 32 + lane];
@@ -655,14 +643,14 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
                 ldsm_x4(b, kst + row * ROWB + ((ch ^ (row & 7)) << 4));
                 mma_bf16_16816(s, qh0, b[0], b[1]);
                 mma_bf16_16816(s2, ql0, b[0], b[1]);
-                mma_bf16_16816(s, qh1, b[2], b[3]);
-                mma_bf16_16816(s2, ql1, b[2], b[3]);
+                mma_bf16_16816(s3, qh1, b[2], b[3]);
+                mma_bf16_16816(s4, ql1, b[2], b[3]);
             }
             float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int hh = e >> 1, j = j0 + 2 * t + (e & 1);
-                s[e] += s2[e];
+                s[e] = (s[e] + s3[e]) + (s2[e] + s4[e]);
                 if (!(j < total && j <= horizon[hh])) s[e] = -INFINITY;
                 mx[hh] = fmaxf(mx[hh], s[e]);
             }

@@ -141,12 +141,14 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
 
 size_t packed_bytes(int N, int K) { return align_up(gemm_packed_bytes(N, K)); }
 
-// Passes of more than 32 rows run on the tiled kernels, which read the weights in MMA-fragment order; a context
-// that admits such passes keeps a second copy of the matrices in that order.
-bool needs_tiled(const pipesd_model_cfg& c) { return c.max_rows > 32; }
+// Two sets of kernels run the layer stack and each reads the weights in its own order.  The tiled per-projection
+// kernels (cfg.engine == PIPESD_ENGINE_TILED) take any pass.  The persistent kernel (PIPESD_ENGINE_PERSISTENT) takes
+// passes of at most 32 rows; a context that selects it and admits larger passes keeps both copies of the matrices.
+bool has_mega(const pipesd_model_cfg& c) { return c.engine == PIPESD_ENGINE_PERSISTENT; }
+bool needs_tiled(const pipesd_model_cfg& c) { return !has_mega(c) || c.max_rows > 32; }
 
 size_t weights_bytes(const pipesd_model_cfg& c, const Derived& d) {
-    const size_t copies = needs_tiled(c) ? 2 : 1;
+    const size_t copies = (needs_tiled(c) ? 1 : 0) + (has_mega(c) ? 1 : 0);
     size_t per_layer = copies * (packed_bytes(d.Nqkv, c.d_model) + packed_bytes(c.d_model, d.qd) +
                                  packed_bytes(2 * c.d_ffn, c.d_model) + packed_bytes(c.d_model, c.d_ffn)) +
                        2 * align_up(4 * (size_t)c.d_model);
@@ -171,6 +173,7 @@ int check_cfg(const pipesd_model_cfg* c) {
     if (c->max_draft < 1 || c->max_draft > kMaxItemRows - 1) return PIPESD_E_INVALID;
     if (c->max_rows < c->max_draft + 1 || c->max_rows > 4096 || c->max_seq < 1) return PIPESD_E_INVALID;
     if (!(c->rms_eps >= 0.f) || !(c->rope_base > 1.f)) return PIPESD_E_INVALID;
+    if (c->engine != PIPESD_ENGINE_TILED && c->engine != PIPESD_ENGINE_PERSISTENT) return PIPESD_E_INVALID;
     return PIPESD_OK;
 }
 
@@ -218,8 +221,9 @@ struct pipesd_ctx {
     bool pend_check = false;   // a prefill is in flight whose device error word has not been looked at yet
     int last_rows = 0;
     int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
-    int engine = 0;         // 0: persistent kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only;
-                            // 2: as 0, but attention always as its own kernel between the persistent launches
+    int engine = 0;         // run-time switch (pipesd_debug_set_engine) inside a context of the persistent engine: 0: persistent
+                            // kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only; 2: as 0, but attention
+                            // always as its own kernel between the persistent launches
     std::vector<MegaPhase> phases;       // GEMM phases only: attention runs as its own kernel between launches
     std::vector<MegaPhase> phases_att;   // with one attention phase per layer: the whole pass is one launch
     std::string err;
@@ -406,7 +410,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
 
     // Passes of at most 32 rows (one token block) run their GEMMs in the persistent kernel, whose counters
     // start every pass at zero.
-    const bool use_mega = (ctx->engine != 1 && M <= 32) || !needs_tiled(c);
+    const bool use_mega = has_mega(c) && ((ctx->engine != 1 && M <= 32) || !needs_tiled(c));
     if (use_mega) CU(cudaMemsetAsync(ctx->wsp + ctx->ws.mega_ctr, 0, 4 * ctx->ws.mega_ctr_ints, st));
     // Every kernel of the chain is launched with programmatic stream serialisation: it may start while its
     // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
@@ -668,8 +672,10 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         for (auto& s : srcs) { ps.w[i] = (const uint16_t*)s.first; ps.rows[i] = s.second; ++i; }
         size_t total = (size_t)((N + 127) / 128 * 8) * (K / 16) * 32;
         int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
-        g.packed_u = (uint4*)take(gemm_packed_bytes(N, K));
-        gemm_pack_umma_kernel<<<blocks, 256, 0, st>>>(ps, g.packed_u, N, K);
+        if (has_mega(c)) {
+            g.packed_u = (uint4*)take(gemm_packed_bytes(N, K));
+            gemm_pack_umma_kernel<<<blocks, 256, 0, st>>>(ps, g.packed_u, N, K);
+        }
         if (tiled) {
             g.packed = (uint4*)take(gemm_packed_bytes(N, K));
             gemm_pack_kernel<<<blocks, 256, 0, st>>>(ps, g.packed, N, K);
@@ -700,7 +706,7 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     if (cudaGetLastError() != cudaSuccess) return bail(PIPESD_E_CUDA);
 
     // ---- phase table of the persistent kernel: QKV(0) | O, gate/up, down, QKV(l+1) per layer | ... | LM head
-    {
+    if (has_mega(c)) {
         int n_sm = 0;
         if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, c.device) != cudaSuccess || n_sm < 1)
             return bail(PIPESD_E_CUDA);
@@ -1094,7 +1100,8 @@ int32_t pipesd_debug_mega_trace(unsigned long long* dst, int32_t n) {
 int32_t pipesd_debug_set_engine(pipesd_ctx* ctx, int32_t engine) {
     if (!ctx || engine < 0 || engine > 2) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine");
     if (engine == 1 && !needs_tiled(ctx->cfg))
-        return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine: the tiled kernels need a context with max_rows > 32");
+        return fail(ctx, PIPESD_E_INVALID,
+                    "pipesd_debug_set_engine: this context keeps no weights in the tiled kernels' order (persistent engine, max_rows <= 32)");
     ctx->engine = engine;
     return PIPESD_OK;
 }

@@ -29,12 +29,13 @@ def _load_synthetic_prefix(ctx, orc, shape, req, P, seed, request=0):
     assert ctx.req_len(req) == P
 
 
-def test_1b_shape_real_prefill_sigma_sweep():
+@pytest.mark.parametrize("engine", ["tiled", "persistent"])
+def test_1b_shape_real_prefill_sigma_sweep(engine):
     """16 layers, d 2048, 32/8 heads x 64, FFN 8192, vocab 32000; P=512, k=8, sigma in {0.3, 1, 3}."""
     from paper_2605_13319_b200 import binding
     shape, P, k = synth.B1, 512, 8
     w = synth.make_weights(shape, 0)
-    ctx = binding.Context(shape, w, n_pages=P // 16 + 8, max_seq=P + 64)
+    ctx = binding.Context(shape, w, n_pages=P // 16 + 8, max_seq=P + 64, engine=engine)
     orc = oracle.Oracle(shape, w, P + 64)
     prefix = synth.make_prefix(shape, P, 0)
     t0 = time.time()
@@ -71,8 +72,10 @@ def seven_b():
     w = synth.make_weights(shape, 0)
     lens, ks, sig = synth.ragged_requests(0, 32)
     pages = int(sum((int(l) + 17 + 15) // 16 for l in lens)) + (2048 + 512) // 16 + 64
+    # persistent engine with room for the 300-row batch: the context keeps the weights in both orders, single
+    # requests run on the persistent kernel, the batch (and whatever debug_set_engine(1) asks for) on the tiled ones
     ctx = binding.Context(shape, w, n_pages=pages, max_seq=4096 + 32, max_requests=34,
-                          max_rows=int(ks.sum()) + 32, max_draft=16)
+                          max_rows=int(ks.sum()) + 32, max_draft=16, engine="persistent")
     print(f"\n7b weights + context: {time.time() - t0:.1f} s")
     yield shape, w, ctx, (lens, ks, sig)
     ctx.close()
@@ -94,14 +97,17 @@ def test_7b_shape_k_4_8_16_and_lockstep_rounds(seven_b):
         ref = orc.verify(toks, q, u)
         dt = time.time() - t0
         orc.truncate(P)
-        (got,) = ctx.verify([dict(req=req, tokens=toks, q=q, u=u)], flags=binding.Q_HOST)
-        err = logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max()
-        print(f"k={k}: oracle verify {dt:.1f} s, n_accepted {ref['n_accepted']}, gpu {got}, rel logit err {err:.2e}")
-        assert err < LOGIT_TOL
-        tally.max_logit_err = max(tally.max_logit_err, err)
-        tally.check(got, ref, ref["logits"], q, u, where=f"k={k}")
-        ctx.kv_rollback([req], [0])
-        ctx.debug_set_len(req, P)
+        for eng, name in ((0, "persistent"), (1, "tiled")):      # both sets of kernels against the same reference
+            ctx.debug_set_engine(eng)
+            (got,) = ctx.verify([dict(req=req, tokens=toks, q=q, u=u)], flags=binding.Q_HOST)
+            err = logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max()
+            print(f"k={k} {name}: oracle verify {dt:.1f} s, n_accepted {ref['n_accepted']}, gpu {got}, rel logit err {err:.2e}")
+            assert err < LOGIT_TOL
+            tally.max_logit_err = max(tally.max_logit_err, err)
+            tally.check(got, ref, ref["logits"], q, u, where=f"k={k} {name}")
+            ctx.kv_rollback([req], [0])
+            ctx.debug_set_len(req, P)
+        ctx.debug_set_engine(0)
     pending = synth.make_pending(shape, 7)
     for r in range(64 if FULL else 3):
         k = 8
@@ -178,13 +184,15 @@ def test_7b_ragged_batch_of_32_requests(seven_b):
         ctx.req_close(it["req"])
 
 
-def test_8b_shape_long_context_large_vocab():
+@pytest.mark.parametrize("engine", ["tiled", "persistent"])
+def test_8b_shape_long_context_large_vocab(engine):
     """32 layers, d 4096, 32/8 heads x 128, FFN 14336, vocab 128256, rope base 5e5; 8192-row prefix, k=16,
-    sigma 0.5: long-context split-K attention and the 128k-vocabulary rejection kernel."""
+    sigma 0.5: long-context split-K attention and the 128k-vocabulary rejection kernel.  (68 query rows per KV
+    head: under the persistent engine attention stays its own kernel between the persistent launches.)"""
     from paper_2605_13319_b200 import binding
     shape, P, k = synth.B8, 8192, 16
     w = synth.make_weights(shape, 0)
-    ctx = binding.Context(shape, w, n_pages=P // 16 + 8, max_seq=P + 64)
+    ctx = binding.Context(shape, w, n_pages=P // 16 + 8, max_seq=P + 64, engine=engine)
     orc = oracle.Oracle(shape, w, P + 64)
     req = ctx.req_open()
     _load_synthetic_prefix(ctx, orc, shape, req, P, seed=3)

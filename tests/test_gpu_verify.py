@@ -7,6 +7,7 @@ from paper_2605_13319_b200 import synth
 from harness import LOGIT_TOL, Tally, draft_inputs, logit_rel_err
 
 pytestmark = pytest.mark.gpu
+ENGINES = pytest.mark.parametrize("engine", ["tiled", "persistent"])
 
 
 def _mk(shape, seed, P, n_pages=None, **kw):
@@ -19,11 +20,13 @@ def _mk(shape, seed, P, n_pages=None, **kw):
     return w, ctx, orc
 
 
-def test_tiny_config_many_seeds():
-    """2 layers, d 256, 4 heads x 64, FFN 688, vocab 1024; P=64, k=4, sigma=1; stochastic and greedy."""
+@ENGINES
+def test_tiny_config_many_seeds(engine):
+    """2 layers, d 256, 4 heads x 64, FFN 688, vocab 1024; P=64, k=4, sigma=1; stochastic and greedy.
+    With the persistent engine every verify here is ONE launch (attention inside the kernel)."""
     from paper_2605_13319_b200 import binding
     shape, P, k = synth.TINY, 64, 4
-    w, ctx, orc = _mk(shape, 0, P)
+    w, ctx, orc = _mk(shape, 0, P, engine=engine)
     tally, gt = Tally(), Tally()
     prefix = synth.make_prefix(shape, P, 0)
     orc.prefill(prefix)
@@ -70,13 +73,16 @@ def test_tiny_config_many_seeds():
     ctx.close()
 
 
-def test_multi_round_verify_rollback_lockstep():
+@ENGINES
+def test_multi_round_verify_rollback_lockstep(engine):
     """Rounds of verify + rollback: the cache grows by n_accepted+1 and is truncated each round; the checker
-    leads (its decision is committed on both sides) so a counted near-tie cannot desynchronise later rounds."""
+    leads (its decision is committed on both sides) so a counted near-tie cannot desynchronise later rounds.
+    Two query heads per KV head and k up to 8: with the persistent engine the rounds alternate between attention
+    inside the kernel (at most 16 query rows per KV head) and attention as its own kernel."""
     from paper_2605_13319_b200 import binding
     shape = synth.TINY.scaled(name="tiny-gqa", n_kv_heads=2)
     P, rounds = 37, 24                       # prefix not a multiple of the page size
-    w, ctx, orc = _mk(shape, 1, P, max_seq=P + rounds * 9 + 16)
+    w, ctx, orc = _mk(shape, 1, P, max_seq=P + rounds * 9 + 16, engine=engine)
     prefix = synth.make_prefix(shape, P, 1)
     orc.prefill(prefix)
     req = ctx.req_open()
@@ -102,15 +108,19 @@ def test_multi_round_verify_rollback_lockstep():
     ctx.close()
 
 
-def test_batched_ragged_verify_and_batch_invariance():
-    """Several requests with different prefix lengths and draft counts in ONE call == each alone == checker."""
+@ENGINES
+def test_batched_ragged_verify_and_batch_invariance(engine):
+    """Several requests with different prefix lengths and draft counts in ONE call == each alone == checker.
+    The bit-for-bit comparison holds on one set of kernels: the batch (more than 32 rows) runs on the tiled ones,
+    so under the persistent engine the single requests are switched to them as well."""
     from paper_2605_13319_b200 import binding
     shape = synth.TINY.scaled(name="tiny-gqa", n_kv_heads=2)
     n_req = 6
     lens, ks, sig = synth.ragged_requests(3, n_req, 5, 150, 1, 16)
     w = synth.make_weights(shape, 2)
     ctx = binding.Context(shape, w, n_pages=(200 // 16 + 2) * n_req * 2, max_seq=200, max_requests=2 * n_req,
-                          max_rows=int(ks.sum() + n_req), max_draft=16)
+                          max_rows=max(33, int(ks.sum() + n_req)), max_draft=16, engine=engine)
+    assert int(ks.sum() + n_req) > 32
     tally = Tally()
     items, refs, solo = [], [], []
     for i in range(n_req):
@@ -125,6 +135,7 @@ def test_batched_ragged_verify_and_batch_invariance():
             bank.append(dict(req=req, tokens=toks, q=q, u=u))
     got = ctx.verify(items, flags=binding.Q_HOST)
     logits = ctx.debug_get_logits(int(ks.sum() + n_req))
+    ctx.debug_set_engine(1)
     row = 0
     for i in range(n_req):
         ref, q, u = refs[i]
