@@ -444,7 +444,7 @@ def quick_run(args, ctx, shape, P, k, seed, torch):
 # under profiles/ (taken on a two-layer model of the same shape -- same per-layer work -- and scaled to a full
 # launch by the layers it covers).  None until a capture of the current kernel exists, and to be reset to None
 # whenever that kernel changes.
-TRAFFIC_7B_K8 = {"tiled": None, "persistent": None}
+TRAFFIC_7B_K8 = {"tiled": 103.0e6, "persistent": 14.37e9}
 
 
 if __name__ == "__main__":
