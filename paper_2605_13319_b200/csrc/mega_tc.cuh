@@ -5,9 +5,9 @@
 // (unit, chunk) list is dealt out in equal contiguous ranges to the CTAs ("stream-K"), so that every SM streams
 // the same number of weight bytes whatever the matrix shape.  Warp roles inside a CTA:
 //   - weight producer (1 thread): walks the CTA's chunk list of ALL phases and keeps a 5-6 stage shared-memory
-//     ring (32 KB of packed weights per stage) full with bulk asynchronous copies.  Weights depend on nothing,
-//     so the stream runs ahead across phase boundaries; while the ring is full it pulls the chunks after the
-//     ring's into L2, so that HBM keeps streaming while the SM waits at a boundary.
+//     ring (32 KB of packed weights per stage) full with bulk asynchronous copies, at most three outstanding
+//     (more only queues in front of the boundaries' small latency-critical accesses).  Weights depend on
+//     nothing, so the stream runs ahead across phase boundaries.  The copies carry an L2 evict-first hint.
 //   - activation producer (1 warp): waits until the phase that produces the input has finished everywhere (a
 //     counter in global memory, released by the epilogues), then adds the matching activation chunk to each
 //     stage and, where the phase normalises its input, derives the rows' RMSNorm factors.
@@ -17,11 +17,15 @@
 //     stage back to the producers, and a finished accumulator (one of two) to the epilogue warps.
 //   - eight epilogue warps: tcgen05.ld (thread = weight row, registers = tokens), hi + lo columns added, then
 //     the fused epilogue (RoPE + K/V append | residual + next norm's gain and sum of squares | SwiGLU | plain).
+//   - publisher (1 thread): tells the other CTAs that a segment of this CTA is finished (a release on a global
+//     counter, i.e. a fence over the CTA's stores), so that no epilogue warp spends that microsecond.
 // A unit whose chunks are spread over several CTAs is summed through global memory: contributors store their
 // rows and count themselves in; the CTA that owns the unit's first chunk (for which the unit comes last in
-// the phase) waits for the count and adds the contributions in CTA order -- a fixed order.  Every wait is
-// bounded; a wait that gives up raises the device error word, which every other wait polls, so the kernel
-// always terminates, and tensor memory is released on every path.
+// the phase) waits for the count and adds the contributions in CTA order -- a fixed order.
+// An attention phase (single-request passes) runs in the same ring: its chunks are 64-key tiles of one KV head
+// (K rows + V rows = one stage, fetched page by page), consumed by the eight epilogue warps (att_segment).
+// Every wait is bounded; a wait that gives up raises the device error word, which every other wait polls, so the
+// kernel always terminates, and tensor memory is released on every path.
 #pragma once
 #include "common.cuh"
 #include "gemm.cuh"
@@ -43,18 +47,7 @@ constexpr int kAttTile = 64;                               // keys per attention
 constexpr int kMegaMaxCtas = 160;
 constexpr int kMegaSmemMax = 227 * 1024;
 constexpr int kMegaTmemCols = 256;                         // 2 accumulators x 2 blocks x up to 64 columns
-#ifndef PIPESD_MEGA_L2AHEAD
-#define PIPESD_MEGA_L2AHEAD 0
-#endif
-constexpr int kMegaL2Ahead = PIPESD_MEGA_L2AHEAD;                           // chunks a blocked weight producer pulls into L2
-#ifndef PIPESD_MEGA_INFLIGHT
-#define PIPESD_MEGA_INFLIGHT 3
-#endif
-constexpr int kMegaMaxInFlight = PIPESD_MEGA_INFLIGHT;                     // weight chunks one CTA has outstanding at a time (see below)
-#ifndef PIPESD_MEGA_PACE
-#define PIPESD_MEGA_PACE 1400
-#endif
-constexpr int kMegaL2PaceClk = PIPESD_MEGA_PACE;                       // SM clocks between two L2 prefetches (32 KB at an SM's fair share of HBM)
+constexpr int kMegaMaxInFlight = 3;                        // weight chunks one CTA has outstanding at a time (see the weight producer)
 constexpr unsigned long long kMegaWaitNs = 1000000000ull;  // bound of every wait
 
 __host__ __device__ constexpr int mega_stage_bytes(int NT) { return kMegaWStage + kMegaKC * NT * 512; }
@@ -207,11 +200,8 @@ __device__ unsigned long long g_mega_trace[64 * 4 * kMegaMaxCtas * 8];
         if (a.launch_idx < 64)                                                                                  \
             g_mega_trace[(((size_t)a.launch_idx * 4 + (p - a.p0)) * kMegaMaxCtas + cta) * 8 + (k)] = global_ns(); \
     } while (0)
-__device__ int g_mega_dbg[kMegaMaxCtas * 8];
-#define MEGA_DBG(slot, val) (g_mega_dbg[blockIdx.x * 8 + (slot)] = (val))
 #else
 #define MEGA_TRACE(k) do { } while (0)
-#define MEGA_DBG(slot, val) do { } while (0)
 #endif
 
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
@@ -289,18 +279,6 @@ struct MegaWalk {
     __device__ __forceinline__ bool two() const { return 2 * u + 1 < RB; }
     __device__ __forceinline__ const unsigned char* src(int half) const {
         return W + ((size_t)(2 * u + half) * KS + cc * kMegaKC) * 4096;
-    }
-    __device__ __forceinline__ void prefetch_l2(uint64_t pol) const {
-        if (mode == kPhaseAttn) return;
-        const uint32_t bytes = (uint32_t)kc() * 4096u;
-#ifdef PIPESD_MEGA_PF_NORMAL
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src(0)), "r"(bytes) : "memory");
-        if (two()) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src(1)), "r"(bytes) : "memory");
-        return;
-#endif
-        asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src(0)), "r"(bytes), "l"(pol) : "memory");
-        if (two())
-            asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src(1)), "r"(bytes), "l"(pol) : "memory");
     }
 };
 
@@ -609,7 +587,6 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     }
     int last_st = st;
     for (int tile = tile0; tile < tile1; ++tile, ++n) {
-        if (threadIdx.x == 0 && ok) { MEGA_DBG(3, n); MEGA_DBG(4, kvh * 1000 + tile); }
         if (threadIdx.x == 0 && tile == tile0) MEGA_TRACE(1);
         if (ok) {
             const uint32_t par = (uint32_t)(n / kStages) & 1u;
@@ -759,7 +736,6 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
     if (warp == 0) { add(1); add(2); add(3); }
     // warp 0 now holds the CTA's un-normalised output for the head, relative to m_tot, with the sum l_tot
-    if (threadIdx.x == 0 && ok) MEGA_DBG(5, 100000 + kvh);
     if (threadIdx.x == 0) MEGA_TRACE(2);
     const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
     constexpr int kSlotFloats = 8 * kMegaEpiThreads * 4;       // one CTA's slot of the exchange array
@@ -908,12 +884,10 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
     if (warp == kMegaWarpW) {
         // ------------------------------------------------ weight producer: runs ahead of everything
         if (lane == 0) {
-            MegaWalk ring, pf;               // next chunk for the ring / next chunk to prefetch into L2
+            MegaWalk ring;
             ring.start(a, cta, G);
-            pf = ring;
-            int n = 0, st = 0, n_pf = 0;
+            int n = 0, st = 0;
             bool ok = true;
-            long long t_pf = clock64();
             const uint64_t pol = l2_evict_first_policy();
             int att_phase = -1, att_c0 = 0;      // phase and first chunk whose page ids att_pg_s holds
             while (ring.valid()) {
@@ -924,27 +898,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     const int m = n - kMegaMaxInFlight;
                     ok = mbar_wait_err(fullW0 + 8 * (m % kStages), (uint32_t)(m / kStages) & 1u, a.err);
                 }
-                if (ok && n >= kStages) {
-                    // Ring full: the MMAs are held up (usually at a phase boundary).  HBM must not go idle
-                    // meanwhile: pull the chunks after the ring's into L2, up to kMegaL2Ahead chunks ahead, paced
-                    // at the SM's fair share of the bandwidth so that the queues stay short.
-                    const uint32_t bar = empty0 + 8 * st, par = (uint32_t)((n / kStages) - 1) & 1u;
-                    uint64_t t0 = 0;
-                    for (uint32_t it = 0; !mbar_try(bar, par); ++it) {
-                        if (n_pf < n + kMegaL2Ahead && pf.valid() && clock64() - t_pf >= kMegaL2PaceClk) {
-                            if (n_pf >= n) { pf.prefetch_l2(pol); t_pf = clock64(); }
-                            pf.next(a, cta, G);
-                            ++n_pf;
-                            continue;
-                        }
-                        if ((it & 255u) == 255u) {
-                            if (ld_relaxed(a.err) != 0) { ok = false; break; }
-                            const uint64_t now = global_ns();
-                            if (t0 == 0) t0 = now;
-                            else if (now - t0 > kMegaWaitNs) { ok = false; break; }
-                        }
-                    }
-                }
+                if (ok && n >= kStages) ok = mbar_wait_err(empty0 + 8 * st, (uint32_t)((n / kStages) - 1) & 1u, a.err);
                 if (!ok) break;
                 if (ring.mode == kPhaseAttn) {
                     // K/V tile of an attention phase: the pages cached before this pass (the others are the
@@ -974,7 +928,6 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 if (++st == kStages) st = 0;
                 ring.next(a, cta, G);
                 ++n;
-                MEGA_DBG(0, n);
             }
             if (!ok) {
                 atomicCAS(a.err, 0, 11);
@@ -1014,7 +967,6 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
                     if (i0 != i1 && cta != i0) red_release_add(a.tickets + ph.ticket0 + u, 1);
                     else red_release_add(a.done + p, 1);
-                    MEGA_DBG(6, seg);
                 }
             }
         }
@@ -1053,10 +1005,8 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 int cc = cb % CPR, u = cb / CPR;
                 for (int c = cb; c < ce; ++c, ++n) {
                     if (n >= kStages) {
-                        MEGA_DBG(7, 1000 + n);
                         ok = mbar_wait_err(empty0 + 8 * st, (uint32_t)((n / kStages) - 1) & 1u, a.err);
                         if (!ok) break;
-                        MEGA_DBG(7, 2000 + n);
                     }
                     if (ph.mode == kPhaseAttn) {
                         // the pages of the tile that hold rows of this pass (written by the QKV phase); a tile
@@ -1079,9 +1029,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                     }
                     if (++st == kStages) st = 0;
                     if (++cc == CPR) { cc = 0; ++u; }
-                    MEGA_DBG(1, n + 1);
                 }
-                MEGA_DBG(2, p);
             } else {
                 // lanes 1..31: the input rows' RMSNorm factors, needed only by the epilogue, computed while
                 // lane 0's copies are in flight and handed to the epilogue warps through their own barrier

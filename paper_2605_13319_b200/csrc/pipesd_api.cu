@@ -712,7 +712,7 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
             return bail(PIPESD_E_CUDA);
         ctx->mega_grid = std::min(n_sm, kMegaMaxCtas);
         if (mega_init_attrs() != cudaSuccess) return bail(PIPESD_E_CUDA);
-        const int d = c.d_model, F = c.d_ffn;
+        const int d = c.d_model;
         const int n_ssq = ((d + 127) / 128 + 1) / 2;      // 256-row units of the residual stream
         uint32_t* xf_h = ctx->W<uint32_t>(ctx->ws.xf_h);
         uint32_t* xf_attn = ctx->W<uint32_t>(ctx->ws.xf_attn);
@@ -1089,9 +1089,6 @@ int32_t pipesd_debug_set_len(pipesd_ctx* ctx, int32_t req, int32_t new_len) {
 }
 
 #ifdef PIPESD_MEGA_TRACE
-int32_t pipesd_debug_mega_dbg(int* dst, int32_t n) {
-    return cudaMemcpyFromSymbol(dst, g_mega_dbg, sizeof(int) * (size_t)n) == cudaSuccess ? 0 : -6;
-}
 int32_t pipesd_debug_mega_trace(unsigned long long* dst, int32_t n) {
     return cudaMemcpyFromSymbol(dst, g_mega_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
 }
