@@ -356,12 +356,8 @@ def main():
 
     # -- reduce over ranks: max time, summed tokens
     if world > 1:
-        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
-        n = torch.tensor([tokens, tokens_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(n, op=dist.ReduceOp.SUM)
-        tokens, tokens_e2e = float(n[0]), float(n[1])
+        from paper_2605_13319_b200 import replicas
+        (ms, ms_e2e), (tokens, tokens_e2e) = replicas.reduce_replicas([ms, ms_e2e], [tokens, tokens_e2e], device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
