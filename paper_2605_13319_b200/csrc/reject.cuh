@@ -81,6 +81,14 @@ struct RejectItem {
 struct RejectOut { int n_accepted, next_token, status, reserved; };
 
 // One CTA per request: combine the row statistics, run the accept chain, make the final draw.
+//
+// Accept chain: the k ratio tests are independent of each other (only "stop at the first failure" is sequential),
+// so thread i evaluates test i and thread 0 takes the first failure.
+// Final draw, inverse CDF in token-id order: warp w owns the contiguous ids [w*R, (w+1)*R) (R a multiple of 32)
+// and walks them 32 at a time, lane = id, so that every load is coalesced.  Pass 1 adds each lane's terms in walk
+// order and the lanes in butterfly order (fixed); the warp totals are scanned in warp order.  Pass 2 runs only in
+// the warp whose range holds the target: an inclusive shuffle scan per 32 ids on top of the running prefix, the
+// first id whose prefix exceeds u * total wins.
 __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const float* __restrict__ logits, int V,
                                                                        const RowStat* __restrict__ stats,
                                                                        const RejectItem* __restrict__ items,
@@ -90,12 +98,14 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
     const RejectItem it = items[blockIdx.x];
     if (it.mode == 2) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kWarps = kSampleThreads / 32;
     __shared__ double s_m[kMaxItemRows], s_z[kMaxItemRows];
     __shared__ int s_arg[kMaxItemRows];
-    __shared__ int s_nacc, s_tok, s_owner;
-    __shared__ double s_warp[32];
+    __shared__ int s_ok[kMaxItemRows];
+    __shared__ int s_nacc, s_tok;
+    __shared__ double s_warp[kWarps];      // warp totals, then their exclusive prefixes
+    __shared__ double s_incl[kWarps];      // inclusive prefixes of the warp totals
     __shared__ double s_total;
-    __shared__ double s_incl[kSampleThreads];
 
     if (tid <= it.k) {   // rows 0..k: merge the column splits
         const RowStat* st = stats + (size_t)(it.row0 + tid) * kStatSplits;
@@ -109,25 +119,25 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
         s_m[tid] = (double)m; s_z[tid] = z; s_arg[tid] = arg;
     }
     __syncthreads();
+    if (tid < it.k) {    // test i: draft i+1 against row i
+        const int x = row_tok[it.row0 + tid + 1];
+        bool ok;
+        if (it.mode == 1) {
+            ok = (x == s_arg[tid]);
+        } else {
+            const double p = exp((double)logits[(size_t)(it.row0 + tid) * V + x] - s_m[tid]) / s_z[tid];
+            const double qx = (double)it.q[(size_t)tid * V + x];
+            const double ratio = qx > 0.0 ? p / qx : (p > 0.0 ? INFINITY : 0.0);
+            ok = (double)u_all[it.u0 + tid] < fmin(ratio, 1.0);
+        }
+        s_ok[tid] = ok ? 1 : 0;
+    }
+    __syncthreads();
     if (tid == 0) {
         int n = 0;
-        for (int i = 0; i < it.k; ++i) {
-            const int x = row_tok[it.row0 + i + 1];
-            bool ok;
-            if (it.mode == 1) {
-                ok = (x == s_arg[i]);
-            } else {
-                const double p = exp((double)logits[(size_t)(it.row0 + i) * V + x] - s_m[i]) / s_z[i];
-                const double qx = (double)it.q[(size_t)i * V + x];
-                double ratio = qx > 0.0 ? p / qx : (p > 0.0 ? INFINITY : 0.0);
-                ok = (double)u_all[it.u0 + i] < fmin(ratio, 1.0);
-            }
-            if (!ok) break;
-            ++n;
-        }
+        while (n < it.k && s_ok[n]) ++n;
         s_nacc = n;
         s_tok = -1;
-        s_owner = 0x7fffffff;
     }
     __syncthreads();
     const int n_acc = s_nacc;
@@ -139,25 +149,21 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
     const float* lr = logits + (size_t)(it.row0 + n_acc) * V;
     const double m = s_m[n_acc], inv_z = 1.0 / s_z[n_acc];
     const double uk = (double)u_all[it.u0 + it.k];
-    const int per = (V + kSampleThreads - 1) / kSampleThreads;
-    const int j0 = min(V, tid * per), j1 = min(V, j0 + per);
+    const int R = ((V + kWarps - 1) / kWarps + 31) / 32 * 32;     // ids per warp
+    const int j0 = min(V, warp * R), j1 = min(V, j0 + R);
     bool use_q = n_acc < it.k;
     const float* qr = use_q ? it.q + (size_t)n_acc * V : nullptr;
+    auto term = [&](int j) -> double {
+        if (j >= j1) return 0.0;
+        double r = exp((double)lr[j] - m) * inv_z;
+        if (use_q) r = fmax(0.0, r - (double)qr[j]);
+        return r;
+    };
     for (int attempt = 0; attempt < 2; ++attempt) {
         double loc = 0.0;
-        for (int j = j0; j < j1; ++j) {
-            double r = exp((double)lr[j] - m) * inv_z;
-            if (use_q) r = fmax(0.0, r - (double)qr[j]);
-            loc += r;
-        }
-        // inclusive scan over threads in index order: warp scan, then scan of warp totals
-        double inc = loc;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            double t = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += t;
-        }
-        if (lane == 31) s_warp[warp] = inc;
+        for (int j = j0 + lane; j < j1; j += 32) loc += term(j);
+        const double wsum = warp_sum_d(loc);
+        if (lane == 0) s_warp[warp] = wsum;
         __syncthreads();
         if (warp == 0) {
             double w = s_warp[lane], winc = w;
@@ -166,7 +172,10 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
                 double t = __shfl_up_sync(0xffffffffu, winc, o);
                 if (lane >= o) winc += t;
             }
-            s_warp[lane] = winc - w;     // exclusive prefix of the warp totals
+            double excl = __shfl_up_sync(0xffffffffu, winc, 1);
+            if (lane == 0) excl = 0.0;
+            s_warp[lane] = excl;         // exclusive prefix of the warp totals = the previous warp's inclusive one, exactly
+            s_incl[lane] = winc;
             if (lane == 31) s_total = winc;
         }
         __syncthreads();
@@ -176,28 +185,31 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
             __syncthreads();
             continue;
         }
-        const double incl = inc + s_warp[warp];
-        s_incl[tid] = incl;
         const double target = uk * total;
-        // the owner is the first thread whose inclusive prefix exceeds the target
-        if (incl > target) atomicMin(&s_owner, tid);
-        __syncthreads();
-        const int owner = s_owner;
-        const double excl = tid ? s_incl[tid - 1] : 0.0;
-        if (owner == tid) {
-            double run = excl;
-            int tok = -1;
-            for (int j = j0; j < j1; ++j) {
-                double r = exp((double)lr[j] - m) * inv_z;
-                if (use_q) r = fmax(0.0, r - (double)qr[j]);
-                run += r;
-                if (run > target) { tok = j; break; }
+        // the owner is the first warp whose inclusive prefix exceeds the target (warp-uniform test)
+        const double before = s_warp[warp];
+        const bool mine = s_incl[warp] > target && !(before > target);     // exactly one warp: prefixes are monotone
+        if (mine) {
+            double run = before;
+            int tok = -1, last_mass = -1;
+            for (int c = j0; c < j1 && tok < 0; c += 32) {
+                double inc = term(c + lane);
+                const unsigned mass = __ballot_sync(0xffffffffu, inc > 0.0);
+                if (mass) last_mass = c + 31 - __clz(mass);
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    double t = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc += t;
+                }
+                const unsigned hit = __ballot_sync(0xffffffffu, run + inc > target && c + lane < j1);
+                if (hit) tok = c + __ffs(hit) - 1;
+                run += __shfl_sync(0xffffffffu, inc, 31);
             }
-            if (tok < 0) tok = j1 - 1;   // rounding at the range's upper edge
-            s_tok = tok;
+            if (tok < 0) tok = last_mass;    // the walk's rounding fell short of the range's total: its last id with mass
+            if (lane == 0) s_tok = tok;
         }
         __syncthreads();
-        if (owner == 0x7fffffff && tid == 0) {
+        if (s_tok < 0 && tid == 0) {
             // target >= every prefix (rounding at the top of the CDF): last token with mass
             int tok = V - 1;
             for (int j = V - 1; j >= 0; --j) {
