@@ -152,6 +152,40 @@ def test_batched_ragged_verify_and_batch_invariance(engine):
     ctx.close()
 
 
+@ENGINES
+def test_draft_lengths_across_token_tile_counts(engine):
+    """k = 1, 7, 8, 15, 16, 31 (the maximum): 2, 8, 9, 16, 17 and 32 rows per pass, i.e. one to four 8-token
+    tiles in the GEMMs and, with the persistent engine, both sides of the 16-query-row limit up to which
+    attention runs inside the kernel.  Prefix lengths straddle page and 64-key tile boundaries."""
+    from paper_2605_13319_b200 import binding
+    shape = synth.TINY
+    w = synth.make_weights(shape, 5)
+    tally = Tally()
+    for n, (k, P) in enumerate(((1, 1), (7, 63), (8, 64), (15, 65), (16, 127), (31, 130))):
+        ctx = binding.Context(shape, w, n_pages=16, max_seq=200, max_draft=31, engine=engine)
+        orc = oracle.Oracle(shape, w, 200)
+        prefix = synth.make_prefix(shape, P, 5, request=n)
+        orc.prefill(prefix)
+        req = ctx.req_open()
+        ctx.prefill(req, prefix)
+        for greedy in (False, True):
+            toks, q, u, _ = draft_inputs(orc, shape, k, 0.7, 50 + n)
+            ref = orc.verify(toks, q, u, greedy=greedy)
+            item = dict(req=req, tokens=toks, q=None if greedy else q, u=u,
+                        mode=binding.MODE_GREEDY if greedy else binding.MODE_STOCHASTIC)
+            (got,) = ctx.verify([item], flags=binding.Q_HOST)
+            err = logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max()
+            assert err < LOGIT_TOL, (k, P, err)
+            tally.max_logit_err = max(tally.max_logit_err, err)
+            tally.check(got, ref, ref["logits"], q, u, greedy=greedy, where=f"k={k} P={P}")
+            orc.truncate(P)
+            ctx.kv_rollback([req], [0])
+            ctx.debug_set_len(req, P)
+        ctx.close()
+    print("\n" + tally.report())
+    assert tally.max_logit_err < 1e-3
+
+
 def test_host_side_errors_and_page_accounting():
     from paper_2605_13319_b200 import binding
     shape = synth.TINY
