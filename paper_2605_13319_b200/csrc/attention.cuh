@@ -25,6 +25,7 @@ constexpr int kAttnThreads = 128;
 constexpr int kAttnTile = 64;       // keys per tile
 constexpr int kAttnStages = 2;
 constexpr int kAttnMaxRowTiles = 4; // 64 query rows per CTA
+constexpr int kAttnPagesSmem = 512; // page ids of a CTA's key range kept in shared memory (longer ranges read the table)
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
     const int sz = valid ? 16 : 0;   // size 0: the 16 destination bytes are zero-filled
@@ -57,7 +58,8 @@ struct AttnSmem {
 // Per-CTA constants shared by the mode-specialised bodies.
 struct AttnCtx {
     const uint16_t* kbase;     // K row (slot 0) of page 0 for this layer and KV head
-    const int32_t* bt;
+    const int32_t* bt;         // page ids of the request, indexed from bt_first: shared-memory copy of the CTA's range, or the table
+    int bt_first;
     size_t page_stride;        // elements between consecutive pages of a layer
     size_t v_off;              // elements from a K row to the V row of the same slot
     int page_size;
@@ -94,7 +96,7 @@ __device__ __forceinline__ void attn_load_tile(const AttnCtx& c, uint32_t stage_
         int pidx = pidx0, slot = slot0;
 #pragma unroll
         for (int i = 0; i < kPerThread; ++i) {
-            page[i] = (j0 + row0 + i * kRowStep) < c.k1 ? c.bt[pidx] : 0;
+            page[i] = (j0 + row0 + i * kRowStep) < c.k1 ? c.bt[pidx - c.bt_first] : 0;
             slot += kRowStep;
             while (slot >= c.page_size) { slot -= c.page_size; ++pidx; }
         }
@@ -313,6 +315,18 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
 
 constexpr int kAttnSplits = 8;   // = cluster size along x
 
+#ifdef PIPESD_GEMM_TRACE
+// Development build only: per (layer, CTA) timestamps of the attention kernel's anatomy.
+__device__ unsigned long long g_attn_trace[64 * 512 * 8];
+#define ATTN_TRACE(k)                                                                                               \
+    do {                                                                                                             \
+        if (threadIdx.x == 0 && layer < 64 && blockIdx.z == 0)                                                       \
+            g_attn_trace[((size_t)layer * 512 + blockIdx.y * gridDim.x + blockIdx.x) * 8 + (k)] = global_ns();       \
+    } while (0)
+#else
+#define ATTN_TRACE(k) do { } while (0)
+#endif
+
 // grid (8 * max clusters per request, n_kv_heads * row_groups, n_items), cluster (8,1,1), block 128.
 // A request whose keys are shared by several clusters (long contexts) takes one more step: every cluster
 // writes its merged partial to global memory and the last cluster to arrive (atomic ticket, nobody waits)
@@ -328,6 +342,7 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = AttnSmem<HD>;
     pdl_launch_dependents();
+    ATTN_TRACE(0);
     const int item = blockIdx.z;
     const int cl = blockIdx.x / kAttnSplits, rank = blockIdx.x % kAttnSplits;   // cluster of this (request, head), rank in it
     const int ncl = meta.it_nsplit[item];                          // clusters that share this request's keys
@@ -352,6 +367,19 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     c.v_off = (size_t)Hkv * page_size * HD;
     c.page_size = page_size;
     c.bt = meta.block_tab + (size_t)meta.it_slot[item] * meta.max_pages;
+    c.bt_first = 0;
+    // The page ids of this CTA's key range go to shared memory once: a tile's copies then start without a trip to
+    // the block table first (that lookup, ahead of every tile's loads, cost about a microsecond per tile).
+    __shared__ int s_pages[kAttnPagesSmem];
+    if (c.k1 > c.k0) {
+        const int p_first = c.k0 / page_size, n_pg = (c.k1 - 1) / page_size - p_first + 1;
+        if (n_pg <= kAttnPagesSmem) {                              // uniform over the CTA
+            for (int i = threadIdx.x; i < n_pg; i += kAttnThreads) s_pages[i] = c.bt[p_first + i];
+            __syncthreads();
+            c.bt = s_pages;
+            c.bt_first = p_first;
+        }
+    }
     const int row0 = meta.it_row0[item];
     const uint32_t ring = smem_u32(smem);
 
@@ -363,6 +391,7 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     if (early0) { attn_load_tile<HD>(c, ring, c.k0); cp_async_commit(); }
     if (early1) { attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile); cp_async_commit(); }
     pdl_wait();
+    ATTN_TRACE(1);
     if (!early0) { if (ntiles > 0) attn_load_tile<HD>(c, ring, c.k0); cp_async_commit(); }
     if (!early1) { if (ntiles > 1) attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile); cp_async_commit(); }
 
@@ -397,6 +426,7 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
             make_uint4(pack2(l[0], l[1]), pack2(l[2], l[3]), pack2(l[4], l[5]), pack2(l[6], l[7]));
     }
     __syncthreads();
+    ATTN_TRACE(2);
 
     // partial result of this CTA: takes over the Q-fragment region once the tile loop is done
     float* Fo = reinterpret_cast<float*>(smem + SM::kRing);     // [row_tiles*16][HD]
@@ -410,8 +440,10 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     else if (row_tiles == 2) attn_body<HD, 2>(c, smem, Fo, Fm, Fl);
     else attn_body<HD, 4>(c, smem, Fo, Fm, Fl);
 
+    ATTN_TRACE(3);
     // ---- merge the cluster's 8 splits over distributed shared memory; rank r owns rows r, r+8, ... of the group
     cluster_sync_all();
+    ATTN_TRACE(4);
     constexpr int EPT = HD / kAttnThreads > 0 ? HD / kAttnThreads : 1;   // output columns per thread
     const uint32_t fo_a = smem_u32(Fo), fm_a = smem_u32(Fm), fl_a = smem_u32(Fl);
     const int n_rows = min(row_tiles * 16, c.R - c.rho0);
@@ -461,8 +493,10 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
         }
     }
     __shared__ int s_last;
+    ATTN_TRACE(5);
     if (ncl > 1) __threadfence();
     cluster_sync_all();   // nobody leaves while its shared memory may still be read; partials are published
+    ATTN_TRACE(6);
     if (ncl == 1) return;
     // ---- several clusters share the keys: the last one to arrive merges their partials
     if (rank == 0 && threadIdx.x == 0) {

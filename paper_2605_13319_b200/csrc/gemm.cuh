@@ -39,6 +39,18 @@ constexpr int kGemmSmemTail = 128 + 128 + 1024;             // barriers | rstd[3
 
 enum GemmMode { kPlain = 0, kQkvRope = 1, kResid = 2, kSwiglu = 3 };
 
+#ifdef PIPESD_GEMM_TRACE
+// Development build only: per (launch, CTA) timestamps of the kernel's anatomy.
+__device__ unsigned long long g_gemm_trace[512 * 512 * 8];
+#define GEMM_TRACE(k)                                                                                              \
+    do {                                                                                                            \
+        if (a.trace_idx >= 0 && a.trace_idx < 512 && blockIdx.x < 512 && blockIdx.y == 0)                           \
+            g_gemm_trace[((size_t)a.trace_idx * 512 + blockIdx.x) * 8 + (k)] = global_ns();                         \
+    } while (0)
+#else
+#define GEMM_TRACE(k) do { } while (0)
+#endif
+
 __host__ __device__ constexpr int gemm_stage_bytes(int NT) { return kGemmWStage + kGemmKC * NT * 512; }
 __host__ __device__ constexpr int gemm_smem_bytes(int NT, int stages) { return stages * gemm_stage_bytes(NT) + kGemmSmemTail; }
 
@@ -156,6 +168,7 @@ struct GemmArgs {
     const uint4* W;     // packed weights
     const uint4* xf;    // activations, split-bf16 B fragments [tb][ks][nt][32]
     int* err;           // device error word (nullable): set when a bounded wait gives up
+    int trace_idx;      // development build: slot of this launch in the trace array
     int M, N, S, KS, stages;
     // input normalisation (nullable): ssq_in[b*M + tok], b < n_ssq, are sums of squares of the un-normalised
     // input row; the result rows are scaled by rsqrt(sum / d_in + eps)
@@ -200,6 +213,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
     const int tok0 = tb * MT;
 
     if (threadIdx.x == 0) {
+        GEMM_TRACE(0);
         for (int i = 0; i < stages; ++i) {
             mbar_init(full0 + 8 * i, 1);
             mbar_init(empty0 + 8 * i, kGemmConsumerWarps);
@@ -232,6 +246,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                 bulk_g2s_hint(smem_base + c * kStageBytes, wsrc + (size_t)c * kGemmWStage, (uint32_t)kc * 4096, full0 + 8 * c, pol);
             }
             pdl_wait();
+            GEMM_TRACE(1);
             for (int c = 0; c < pre; ++c) {
                 const int kc = chunk_ks(c);
                 bulk_g2s(smem_base + c * kStageBytes + kGemmWStage, bsrc + (size_t)c * kBStage, (uint32_t)kc * NT * 512,
@@ -322,6 +337,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
         for (int c = 0; c < nchunks; ++c) {
             ok = mbar_wait(full0 + 8 * st, ph);
             if (!ok) break;
+            if (c == 0 && threadIdx.x == 0) GEMM_TRACE(2);
             const unsigned char* wst = smem + st * kStageBytes;
             const unsigned char* bst = wst + kGemmWStage;
             int kc = nks - c * kGemmKC;
@@ -346,6 +362,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             if (++st == stages) { st = 0; ph ^= 1u; }
         }
         if (!ok && a.err && lane == 0) atomicExch(a.err, 2);
+        if (threadIdx.x == 0) GEMM_TRACE(3);
         // All consumers are past their last ring read before the ring is reused for the partial tile.
         asm volatile("bar.sync 1, %0;" ::"n"(kGemmConsumers) : "memory");
         // partial tile P[tile 8][token MT][row 16] (fp32) at the start of the ring
@@ -365,6 +382,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
 
     // ---------------- cluster reduction + epilogue (all 160 threads reach both barriers, also on errors)
     if (a.S > 1) cluster_sync_all(); else __syncthreads();
+    if (threadIdx.x == 0) GEMM_TRACE(4);
     pdl_wait();   // (long satisfied) every thread that touches the predecessors' global data has waited itself
     if (warp < kGemmConsumerWarps) {
         const int row = threadIdx.x & 15, tg = threadIdx.x >> 4;   // 16 lanes = the 16 rows of a tile
@@ -454,7 +472,9 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             for (int tile = s; tile < 8; tile += a.S) epi_tile(tile, nullptr, nullptr, nullptr, nullptr);
         }
     }
+    if (threadIdx.x == 0) GEMM_TRACE(5);
     if (a.S > 1) cluster_sync_all(); else __syncthreads();
+    if (threadIdx.x == 0) GEMM_TRACE(6);
     if (MODE == kResid && s == 0 && threadIdx.x < MT) {
         const int tok = tok0 + threadIdx.x;
         if (tok < a.M) {

@@ -229,6 +229,7 @@ struct pipesd_ctx {
     std::string err;
     // launch accounting
     int64_t n_launch = 0, n_gemm = 0;
+    int n_gemm_in_pass = 0;   // position of the next GEMM launch in the current pass (development traces)
     double gemm_bytes = 0.0;
     bool time_gemms = false;
     std::vector<cudaEvent_t> prof_ev;   // start/stop pairs
@@ -278,6 +279,7 @@ int cuda_fail(pipesd_ctx* c, cudaError_t e, const char* where) {
 int launch_gemm(pipesd_ctx* ctx, int mode, GemmArgs a, int K) {
     const GemmPlan p = gemm_plan(a.M, a.N, K);
     a.err = ctx->err_word();
+    a.trace_idx = (int)(ctx->n_gemm_in_pass++);
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (ctx->time_gemms) {
         if (ctx->prof_used + 2 > ctx->prof_ev.size()) {
@@ -391,6 +393,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     CU(cudaEventRecord(ctx->ev_meta[sidx], ctx->st));
 
     // ---- layer stack
+    ctx->n_gemm_in_pass = 0;
     const PassMeta meta = ctx->pass_meta();
     cudaStream_t st = ctx->st;
     float* x = ctx->W<float>(ctx->ws.x);
@@ -1088,6 +1091,14 @@ int32_t pipesd_debug_set_len(pipesd_ctx* ctx, int32_t req, int32_t new_len) {
     return PIPESD_OK;
 }
 
+#ifdef PIPESD_GEMM_TRACE
+int32_t pipesd_debug_attn_trace(unsigned long long* dst, int32_t n) {
+    return cudaMemcpyFromSymbol(dst, g_attn_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
+}
+int32_t pipesd_debug_gemm_trace(unsigned long long* dst, int32_t n) {
+    return cudaMemcpyFromSymbol(dst, g_gemm_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
+}
+#endif
 #ifdef PIPESD_MEGA_TRACE
 int32_t pipesd_debug_mega_trace(unsigned long long* dst, int32_t n) {
     return cudaMemcpyFromSymbol(dst, g_mega_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
