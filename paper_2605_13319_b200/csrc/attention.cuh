@@ -313,7 +313,9 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
     }
 }
 
-constexpr int kAttnSplits = 8;   // = cluster size along x
+constexpr int kAttnSplits = 8;        // key splits per cluster of a request whose keys several clusters share
+constexpr int kAttnMaxCluster = 10;   // largest cluster along x (above 8: the non-portable sizes, opted into by the host;
+                                      // a B200 keeps 41 clusters of 10 of this kernel resident but only 31 of 11 or 12)
 
 #ifdef PIPESD_GEMM_TRACE
 // Development build only: per (layer, CTA) timestamps of the attention kernel's anatomy.
@@ -327,7 +329,9 @@ __device__ unsigned long long g_attn_trace[64 * 512 * 8];
 #define ATTN_TRACE(k) do { } while (0)
 #endif
 
-// grid (8 * max clusters per request, n_kv_heads * row_groups, n_items), cluster (8,1,1), block 128.
+// grid (cs * max clusters per request, n_kv_heads * row_groups, n_items), cluster (cs,1,1), 8 <= cs <= 10, block 128.
+// A request uses the first it_cs <= cs CTAs of its cluster; the others hold an empty split (exact zeros in the
+// merge), so a request's result does not depend on the cluster size its batch was launched with.
 // A request whose keys are shared by several clusters (long contexts) takes one more step: every cluster
 // writes its merged partial to global memory and the last cluster to arrive (atomic ticket, nobody waits)
 // merges those.
@@ -344,10 +348,12 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     pdl_launch_dependents();
     ATTN_TRACE(0);
     const int item = blockIdx.z;
-    const int cl = blockIdx.x / kAttnSplits, rank = blockIdx.x % kAttnSplits;   // cluster of this (request, head), rank in it
+    const int cs = (int)cluster_nctaid_x();
+    const int cl = blockIdx.x / cs, rank = blockIdx.x % cs;        // cluster of this (request, head), rank in it
     const int ncl = meta.it_nsplit[item];                          // clusters that share this request's keys
     if (cl >= ncl) return;                                         // taken by a whole cluster or by none
-    const int sp = cl * kAttnSplits + rank;                        // key split of this CTA
+    const int S = meta.it_cs[item];                                // key splits per cluster of this request (<= cs)
+    const int sp = cl * S + rank;                                  // key split of this CTA (rank < S)
     const int kvh = blockIdx.y % Hkv, rg = blockIdx.y / Hkv;
     const int G = Hq / Hkv;
     AttnCtx c;
@@ -356,11 +362,11 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     c.rho0 = rg * (kAttnMaxRowTiles * 16);
     int row_tiles = (c.R - c.rho0 + 15) / 16;
     row_tiles = row_tiles > kAttnMaxRowTiles ? kAttnMaxRowTiles : row_tiles;
-    // the whole cluster shares (item, head, row group): these exits are taken by all 8 CTAs or by none
+    // the whole cluster shares (item, head, row group): these exits are taken by all CTAs of the cluster or by none
     if (c.rho0 >= c.R || row_tiles > q_tiles_smem) return;
     c.base = meta.it_base[item];
     const int total = c.base + c.rows, chunk = meta.it_chunk[item];
-    c.k0 = min(sp * chunk, total);
+    c.k0 = rank < S ? min(sp * chunk, total) : total;
     c.k1 = min(c.k0 + chunk, total);
     c.kbase = kv_pool + kv_index(layer, n_pages, 0, 0, Hkv, kvh, page_size, 0, HD, 0);
     c.page_stride = (size_t)2 * Hkv * page_size * HD;
@@ -441,7 +447,7 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     else attn_body<HD, 4>(c, smem, Fo, Fm, Fl);
 
     ATTN_TRACE(3);
-    // ---- merge the cluster's 8 splits over distributed shared memory; rank r owns rows r, r+8, ... of the group
+    // ---- merge the cluster's splits over distributed shared memory; rank r owns rows r, r+cs, ... of the group
     cluster_sync_all();
     ATTN_TRACE(4);
     constexpr int EPT = HD / kAttnThreads > 0 ? HD / kAttnThreads : 1;   // output columns per thread
@@ -450,11 +456,17 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     const int KSo = (Hq * HD) / 16, NTo = xf_nt(M);
     const size_t slot0 = (size_t)meta.it_part0[item] + ((size_t)kvh * c.R + c.rho0) * ncl;   // + rl*ncl + cluster
 #pragma unroll 2
-    for (int rl = rank; rl < n_rows; rl += kAttnSplits) {
-        // all remote reads of a row are issued together: 8 maxima, 8 sums, 8 output values per thread
-        float ms[kAttnSplits], ls[kAttnSplits], ov[EPT][kAttnSplits];
+    for (int rl = rank; rl < n_rows; rl += cs) {
+        // all remote reads of a row are issued together: cs maxima, cs sums, cs output values per thread
+        float ms[kAttnMaxCluster], ls[kAttnMaxCluster], ov[EPT][kAttnMaxCluster];
 #pragma unroll
-        for (int r = 0; r < kAttnSplits; ++r) {
+        for (int r = 0; r < kAttnMaxCluster; ++r) {
+            if (r >= cs) {                       // beyond this launch's cluster: an empty split
+                ms[r] = -INFINITY; ls[r] = 0.f;
+#pragma unroll
+                for (int k = 0; k < EPT; ++k) ov[k][r] = 0.f;
+                continue;
+            }
             ms[r] = dsmem_ld_f32(dsmem_addr(fm_a + rl * 4, (uint32_t)r));
             ls[r] = dsmem_ld_f32(dsmem_addr(fl_a + rl * 4, (uint32_t)r));
 #pragma unroll
@@ -465,10 +477,10 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
         }
         float m = -INFINITY;
 #pragma unroll
-        for (int r = 0; r < kAttnSplits; ++r) m = fmaxf(m, ms[r]);
-        float den = 0.f, w[kAttnSplits];
+        for (int r = 0; r < kAttnMaxCluster; ++r) m = fmaxf(m, ms[r]);
+        float den = 0.f, w[kAttnMaxCluster];
 #pragma unroll
-        for (int r = 0; r < kAttnSplits; ++r) {
+        for (int r = 0; r < kAttnMaxCluster; ++r) {
             w[r] = (ms[r] == -INFINITY) ? 0.f : exp2f(ms[r] - m);   // an empty split or one beyond the causal horizon
             den += w[r] * ls[r];
         }
@@ -479,7 +491,7 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
             if (e < HD) {
                 float num = 0.f;
 #pragma unroll
-                for (int r = 0; r < kAttnSplits; ++r) num += w[r] * ov[k][r];
+                for (int r = 0; r < kAttnMaxCluster; ++r) num += w[r] * ov[k][r];
                 if (ncl == 1) {
                     if (xu_layout) xu_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, NTo);
                     else xf_store_one(xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
@@ -505,12 +517,12 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
         const int last = (t == ncl - 1);
         if (last) *ticket = 0;                                   // self-cleaning: ready for the next launch
         const uint32_t fa = smem_u32(&s_last);
-        for (int r = 0; r < kAttnSplits; ++r) dsmem_st_f32(dsmem_addr(fa, (uint32_t)r), __int_as_float(last));
+        for (int r = 0; r < cs; ++r) dsmem_st_f32(dsmem_addr(fa, (uint32_t)r), __int_as_float(last));
     }
     cluster_sync_all();
     if (!s_last) return;
     __threadfence();
-    for (int rl = rank; rl < n_rows; rl += kAttnSplits) {
+    for (int rl = rank; rl < n_rows; rl += cs) {
         float ms[kMaxSplits / kAttnSplits], ls[kMaxSplits / kAttnSplits], ov[EPT][kMaxSplits / kAttnSplits];
 #pragma unroll
         for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) {

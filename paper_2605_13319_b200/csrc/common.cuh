@@ -215,6 +215,11 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
+__device__ __forceinline__ uint32_t cluster_nctaid_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctaid.x;" : "=r"(r));
+    return r;
+}
 // Every thread of every CTA of the cluster must execute this (hardware barrier, release/acquire).
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -245,6 +250,7 @@ struct PassMeta {
     const int32_t* it_base;    // [n_items] cached positions before this pass
     const int32_t* it_nsplit;  // [n_items] KV splits
     const int32_t* it_chunk;   // [n_items] keys per split (multiple of the page size)
+    const int32_t* it_cs;      // [n_items] key splits per cluster (the request's own: 8..10)
     const int32_t* it_part0;   // [n_items] first slot of the item in the attention partial arrays
     const int32_t* block_tab;  // [max_requests][max_pages] page ids, indexed by request slot
     int max_pages;

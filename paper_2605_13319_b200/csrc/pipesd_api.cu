@@ -45,7 +45,7 @@ struct LayerW {
 
 // Fixed offsets of the per-call metadata block (same layout in pinned host staging and on device).
 struct MetaLayout {
-    size_t row_item, row_pos, row_tok, it_slot, it_row0, it_rows, it_base, it_nsplit, it_chunk, it_part0, u, rej, total;
+    size_t row_item, row_pos, row_tok, it_slot, it_row0, it_rows, it_base, it_nsplit, it_chunk, it_cs, it_part0, u, rej, total;
 };
 
 MetaLayout meta_layout(int max_rows, int max_items) {
@@ -61,6 +61,7 @@ MetaLayout meta_layout(int max_rows, int max_items) {
     m.it_base = take(4 * (size_t)max_items);
     m.it_nsplit = take(4 * (size_t)max_items);
     m.it_chunk = take(4 * (size_t)max_items);
+    m.it_cs = take(4 * (size_t)max_items);
     m.it_part0 = take(4 * (size_t)max_items);
     m.u = take(4 * (size_t)max_rows);
     m.rej = take(sizeof(RejectItem) * (size_t)max_items);
@@ -220,6 +221,7 @@ struct pipesd_ctx {
     int pend_n = 0;
     bool pend_check = false;   // a prefill is in flight whose device error word has not been looked at yet
     int last_rows = 0;
+    int attn_max_cs = kAttnSplits;   // largest attention cluster this device schedules (8, or 12 where the larger sizes are available)
     int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
     int engine = 0;         // run-time switch (pipesd_debug_set_engine) inside a context of the persistent engine: 0: persistent
                             // kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only; 2: as 0, but attention
@@ -250,6 +252,7 @@ struct pipesd_ctx {
         m.it_base = (const int32_t*)(b + ml.it_base);
         m.it_nsplit = (const int32_t*)(b + ml.it_nsplit);
         m.it_chunk = (const int32_t*)(b + ml.it_chunk);
+        m.it_cs = (const int32_t*)(b + ml.it_cs);
         m.it_part0 = (const int32_t*)(b + ml.it_part0);
         m.block_tab = W<int32_t>(ws.block_tab);
         m.max_pages = dv.max_pages;
@@ -354,7 +357,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     auto I = [&](size_t off) { return reinterpret_cast<int32_t*>(hm + off); };
     float* hu = reinterpret_cast<float*>(hm + ml.u);
     RejectItem* hr = reinterpret_cast<RejectItem*>(hm + ml.rej);
-    int row = 0, part0 = 0, max_nsplit = 1, u0 = 0;
+    int row = 0, part0 = 0, max_nsplit = 1, u0 = 0, max_cs = kAttnSplits;
     for (int i = 0; i < n_items; ++i) {
         const ItemDesc& it = items[i];
         const Request& r = ctx->reqs[it.slot];
@@ -363,8 +366,18 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         // cluster per 2048 keys (up to four).  The count depends on the request alone, never on what else
         // is in the batch, so that a request's summation order is the same in every batch.
         const int ncl = std::max(1, std::min(kMaxSplits / kAttnSplits, total / 2048));
-        int chunk = (total + kAttnSplits * ncl - 1) / (kAttnSplits * ncl);
-        chunk = (chunk + c.page_size - 1) / c.page_size * c.page_size;
+        // A single cluster may be wider than eight: the width (8..10) that leaves each CTA the fewest 64-key tiles,
+        // the smallest such.  (2057 keys: 8 splits of 272 keys are five tiles each, 9 splits of 240 are four.)
+        int cs_i = kAttnSplits;
+        auto chunk_of = [&](int splits) {
+            const int ch = (total + splits - 1) / splits;
+            return (ch + c.page_size - 1) / c.page_size * c.page_size;
+        };
+        if (ncl == 1)
+            for (int s = kAttnSplits + 1; s <= ctx->attn_max_cs; ++s)
+                if ((chunk_of(s) + kAttnTile - 1) / kAttnTile < (chunk_of(cs_i) + kAttnTile - 1) / kAttnTile) cs_i = s;
+        const int chunk = chunk_of(cs_i * ncl);
+        max_cs = std::max(max_cs, cs_i);
         int nsplit = ncl;   // stored per item: clusters sharing its keys
         I(ml.it_slot)[i] = it.slot;
         I(ml.it_row0)[i] = row;
@@ -372,6 +385,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         I(ml.it_base)[i] = r.len;
         I(ml.it_nsplit)[i] = nsplit;
         I(ml.it_chunk)[i] = chunk;
+        I(ml.it_cs)[i] = cs_i;
         I(ml.it_part0)[i] = part0;
         max_nsplit = std::max(max_nsplit, nsplit);
         part0 += it.rows * c.n_q_heads * nsplit;
@@ -437,14 +451,14 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     base.d_in = d;
     base.n_ssq = n_ssq;
     auto launch_attn = [&](int l) -> int {
-        dim3 ag(kAttnSplits * max_nsplit, Hkv * row_groups, n_items);
+        dim3 ag(max_cs * max_nsplit, Hkv * row_groups, n_items);   // cluster = the widest any request of the batch asks for
         int* tickets = ctx->W<int>(ctx->ws.tickets);
         if (hd == 128)
-            CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
+            CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, max_cs, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
                                   row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0));
         else
-            CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, kAttnSplits, (const float*)qbuf,
+            CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, max_cs, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
                                   row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0));
         ctx->n_launch += 1;
@@ -643,6 +657,25 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
                              (int)attn_smem_bytes(64, kAttnMaxRowTiles));
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
 
+    {   // clusters of 9 or 10 CTAs are non-portable sizes: opt in, and use them only if the device says it can
+        // keep one request's worth of such clusters resident at once (otherwise every cluster stays at eight)
+        const bool hd128 = c.head_dim == 128;
+        const void* fn = hd128 ? (const void*)attn_kernel<128> : (const void*)attn_kernel<64>;
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchConfig_t lc = {};
+            lc.gridDim = dim3(kAttnMaxCluster, 1, 1);
+            lc.blockDim = dim3(kAttnThreads);
+            lc.dynamicSmemBytes = attn_smem_bytes(c.head_dim, 1);     // a draft of up to 15 tokens per query head
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = kAttnMaxCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            lc.attrs = at; lc.numAttrs = 1;
+            int n_clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) == cudaSuccess && n_clusters >= c.n_kv_heads)   // one request's clusters in one wave
+                ctx->attn_max_cs = kAttnMaxCluster;
+        }
+        (void)cudaGetLastError();
+    }
     ctx->kv_pool = (uint16_t*)mem->kv;
     ctx->wsp = (char*)mem->workspace;
     for (int i = 0; i < pipesd_ctx::kStages; ++i) {
