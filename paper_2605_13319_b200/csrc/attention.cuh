@@ -27,13 +27,20 @@ constexpr int kAttnStages = 2;
 constexpr int kAttnMaxRowTiles = 4; // 64 query rows per CTA
 constexpr int kAttnPagesSmem = 512; // page ids of a CTA's key range kept in shared memory (longer ranges read the table)
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-    const int sz = valid ? 16 : 0;   // size 0: the 16 destination bytes are zero-filled
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+// Wait for a stage barrier.  Bounded by a try count (each try suspends for a hardware-chosen time; 2^22 of them take
+// seconds), so that a protocol error cannot hang the GPU: the caller raises the error word and carries on.
+__device__ __forceinline__ bool attn_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -81,46 +88,31 @@ __device__ __forceinline__ void split2_bf16(float a, float b, uint32_t& hi, uint
     lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-// Issue the cp.async copies of one 64-key tile (K and V) into a ring stage.  Thread t copies chunk
-// t % (HD/8) of rows t / (HD/8) + i * (128 / (HD/8)); page and slot advance incrementally (no divisions
-// in the loop), the page table is read once per page change with all reads issued before the copies.
+// Issue (one thread) the copies of one 64-key tile into a ring stage: the rows of a page that belong to one KV head
+// are contiguous in the pool (already chunk-permuted), so every page the tile touches is one bulk copy of K rows
+// and one of V rows, counted in bytes on the stage's barrier.  Rows at or beyond k1 are not copied.
 template <int HD>
-__device__ __forceinline__ void attn_load_tile(const AttnCtx& c, uint32_t stage_addr, int j0) {
-    constexpr int kChunks = HD / 8;                       // 16-byte chunks per row
-    constexpr int kPerThread = kAttnTile * kChunks / kAttnThreads;
-    constexpr int kRowStep = kAttnThreads / kChunks;      // rows between a thread's consecutive copies
-    const int row0 = threadIdx.x / kChunks, ch = threadIdx.x % kChunks;
-    const int pidx0 = (j0 + row0) / c.page_size, slot0 = (j0 + row0) - pidx0 * c.page_size;
-    int page[kPerThread];
-    {
-        int pidx = pidx0, slot = slot0;
-#pragma unroll
-        for (int i = 0; i < kPerThread; ++i) {
-            page[i] = (j0 + row0 + i * kRowStep) < c.k1 ? c.bt[pidx - c.bt_first] : 0;
-            slot += kRowStep;
-            while (slot >= c.page_size) { slot -= c.page_size; ++pidx; }
-        }
-    }
-    int slot = slot0;
-#pragma unroll
-    for (int i = 0; i < kPerThread; ++i) {
-        const int row = row0 + i * kRowStep;
-        const bool valid = j0 + row < c.k1;
-        const uint16_t* kp = c.kbase;
-        if (valid) kp += (size_t)page[i] * c.page_stride + (size_t)slot * HD + ch * 8;
-        const uint32_t off = row * (HD * 2) + (ch << 4);   // the pool's rows are stored chunk-permuted already
-        cp_async16(stage_addr + off, kp, valid);
-        cp_async16(stage_addr + AttnSmem<HD>::kTileBytes + off, kp + (valid ? c.v_off : 0), valid);
-        slot += kRowStep;
-        while (slot >= c.page_size) slot -= c.page_size;
+__device__ __forceinline__ void attn_issue_tile(const AttnCtx& c, uint32_t stage_addr, uint32_t bar, int j0) {
+    const int j1 = min(j0 + kAttnTile, c.k1);
+    mbar_expect_tx(bar, (uint32_t)(j1 - j0) * (HD * 2) * 2);
+    int pidx = j0 / c.page_size, slot = j0 - pidx * c.page_size;
+    for (int j = j0; j < j1;) {
+        const int n = min(c.page_size - slot, j1 - j);
+        const uint16_t* kp = c.kbase + (size_t)c.bt[pidx - c.bt_first] * c.page_stride + (size_t)slot * HD;
+        const uint32_t dst = stage_addr + (uint32_t)(j - j0) * (HD * 2);
+        bulk_g2s(dst, kp, (uint32_t)n * (HD * 2), bar);
+        bulk_g2s(dst + AttnSmem<HD>::kTileBytes, kp + c.v_off, (uint32_t)n * (HD * 2), bar);
+        j += n;
+        slot = 0;
+        ++pidx;
     }
 }
 
-// On entry the copies of tiles 0 and 1 have been issued as two committed cp.async groups.  On exit the
+// On entry the copies of tiles 0 and 1 have been issued on the two stage barriers.  On exit the
 // CTA's partial result for its (up to 64) rows is in shared memory: Fo[row][HD], Fm[row], Fl[row].
 template <int HD, int RTW>
-__device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem, float* __restrict__ Fo,
-                                          float* __restrict__ Fm, float* __restrict__ Fl) {
+__device__ __forceinline__ void attn_body(const AttnCtx& c, const AttnCtx* c_issue, unsigned char* smem, uint32_t bars, int* err,
+                                          float* __restrict__ Fo, float* __restrict__ Fm, float* __restrict__ Fl) {
     constexpr int KSW = 4 / RTW;               // key strips per tile
     constexpr int STRIP = kAttnTile / KSW;     // keys per warp per tile
     constexpr int NTS = STRIP / 8;             // score n-tiles per warp
@@ -151,16 +143,29 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
     const int ntiles = c.k1 > c.k0 ? (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile : 0;
 
     for (int it = 0; it < ntiles; ++it) {
+        const int stg = it % kAttnStages;
         if (it > 0) {
             __syncthreads();      // everyone is done with tile it-1: its stage can take tile it+1
-            if (it + 1 < ntiles)
-                attn_load_tile<HD>(c, ring + ((it + 1) % kAttnStages) * SM::kStageBytes, c.k0 + (it + 1) * kAttnTile);
-            cp_async_commit();
+            if (it + 1 < ntiles && threadIdx.x == 0) {
+                fence_proxy_async_smem();      // the stage was read with ordinary loads; the copy engine writes it next
+                attn_issue_tile<HD>(*c_issue, ring + ((it + 1) % kAttnStages) * SM::kStageBytes,
+                                    bars + 8 * ((it + 1) % kAttnStages), c.k0 + (it + 1) * kAttnTile);
+            }
         }
-        cp_async_wait<1>();
-        __syncthreads();          // tile `it` has landed for everyone
+        // a ragged last tile: its rows at and beyond k1 are not copied; V there must be finite (P is 0, but 0 * NaN
+        // is not), so those rows are cleared, by everyone, in the part of the stage the copy does not touch
+        const int n_valid = min(kAttnTile, c.k1 - (c.k0 + it * kAttnTile));
+        if (n_valid < kAttnTile) {
+            unsigned char* sp = smem + stg * SM::kStageBytes;
+            for (int i = n_valid * (HD / 8) + threadIdx.x; i < kAttnTile * (HD / 8); i += kAttnThreads) {
+                *reinterpret_cast<uint4*>(sp + (size_t)i * 16) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(sp + SM::kTileBytes + (size_t)i * 16) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        if (!attn_wait(bars + 8 * stg, (uint32_t)(it / kAttnStages) & 1u) && err) atomicExch(err, 3);   // tile `it` has landed
+        if (n_valid < kAttnTile) __syncthreads();
         if (!warp_active) continue;
-        const uint32_t kst = ring + (it % kAttnStages) * SM::kStageBytes;
+        const uint32_t kst = ring + stg * SM::kStageBytes;
         const uint32_t vst = kst + SM::kTileBytes;
         const int j0 = c.k0 + it * kAttnTile + sk0;    // first key of this warp's strip
 
@@ -257,7 +262,6 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, unsigned char* smem,
             }
         }
     }
-    cp_async_wait<0>();
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
         l_run[hh] += __shfl_xor_sync(0xffffffffu, l_run[hh], 1);
@@ -342,7 +346,7 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
                                                             int q_tiles_smem, int row_groups, float* __restrict__ o_part,
                                                             float* __restrict__ m_part, float* __restrict__ l_part,
                                                             int* __restrict__ tickets, uint16_t* __restrict__ xf_out,
-                                                            int xu_layout) {
+                                                            int xu_layout, int* __restrict__ err) {
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = AttnSmem<HD>;
     pdl_launch_dependents();
@@ -390,16 +394,26 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     const uint32_t ring = smem_u32(smem);
 
     // Tiles made only of keys cached before this pass do not depend on the QKV projection that precedes this
-    // kernel: issue their copies now.  Group order is always [tile 0][tile 1].
+    // kernel: their copies are issued now, the others after the dependency has resolved.
+    __shared__ AttnCtx s_ctx;      // thread 0's copy: what issuing a tile needs stays out of everyone's registers
+    __shared__ __align__(8) unsigned long long s_bars[kAttnStages];
+    const uint32_t bars = smem_u32(s_bars);
     const int ntiles = c.k1 > c.k0 ? (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile : 0;
     const bool early0 = ntiles > 0 && min(c.k0 + kAttnTile, c.k1) <= c.base;
     const bool early1 = ntiles > 1 && min(c.k0 + 2 * kAttnTile, c.k1) <= c.base;
-    if (early0) { attn_load_tile<HD>(c, ring, c.k0); cp_async_commit(); }
-    if (early1) { attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile); cp_async_commit(); }
+    if (threadIdx.x == 0) {
+        s_ctx = c;
+        for (int i = 0; i < kAttnStages; ++i) mbar_init(bars + 8 * i, 1);
+        fence_mbar_init();
+        if (early0) attn_issue_tile<HD>(s_ctx, ring, bars, c.k0);
+        if (early1) attn_issue_tile<HD>(s_ctx, ring + SM::kStageBytes, bars + 8, c.k0 + kAttnTile);
+    }
     pdl_wait();
     ATTN_TRACE(1);
-    if (!early0) { if (ntiles > 0) attn_load_tile<HD>(c, ring, c.k0); cp_async_commit(); }
-    if (!early1) { if (ntiles > 1) attn_load_tile<HD>(c, ring + SM::kStageBytes, c.k0 + kAttnTile); cp_async_commit(); }
+    if (threadIdx.x == 0) {
+        if (!early0 && ntiles > 0) attn_issue_tile<HD>(s_ctx, ring, bars, c.k0);
+        if (!early1 && ntiles > 1) attn_issue_tile<HD>(s_ctx, ring + SM::kStageBytes, bars + 8, c.k0 + kAttnTile);
+    }
 
     // ---- stage Q (scaled by 1/sqrt(hd)) as split-bf16 A fragments: [tile][k16 step][hi|lo][lane] uint4
     const float scale = rsqrtf((float)HD) * 1.4426950408889634f;   // scores in the log2 domain: p = 2^(s - m)
@@ -439,12 +453,11 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     float* Fm = Fo + row_tiles * 16 * HD;                        // [row_tiles*16]
     float* Fl = Fm + row_tiles * 16;                             // [row_tiles*16]
     if (ntiles == 0) {   // empty split: contributes nothing (finite zeros, so the merge can read it unconditionally)
-        cp_async_wait<0>();
         for (int i = threadIdx.x; i < row_tiles * 16; i += kAttnThreads) { Fm[i] = -INFINITY; Fl[i] = 0.f; }
         for (int i = threadIdx.x; i < row_tiles * 16 * HD; i += kAttnThreads) Fo[i] = 0.f;
-    } else if (row_tiles == 1) attn_body<HD, 1>(c, smem, Fo, Fm, Fl);
-    else if (row_tiles == 2) attn_body<HD, 2>(c, smem, Fo, Fm, Fl);
-    else attn_body<HD, 4>(c, smem, Fo, Fm, Fl);
+    } else if (row_tiles == 1) attn_body<HD, 1>(c, &s_ctx, smem, bars, err, Fo, Fm, Fl);
+    else if (row_tiles == 2) attn_body<HD, 2>(c, &s_ctx, smem, bars, err, Fo, Fm, Fl);
+    else attn_body<HD, 4>(c, &s_ctx, smem, bars, err, Fo, Fm, Fl);
 
     ATTN_TRACE(3);
     // ---- merge the cluster's splits over distributed shared memory; rank r owns rows r, r+cs, ... of the group

@@ -456,11 +456,11 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         if (hd == 128)
             CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, max_cs, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0));
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0, ctx->err_word()));
         else
             CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, max_cs, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0));
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0, ctx->err_word()));
         ctx->n_launch += 1;
         return PIPESD_OK;
     };
