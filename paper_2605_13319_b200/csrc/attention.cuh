@@ -283,37 +283,52 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, const AttnCtx* c_iss
         }
         return;
     }
-    float* mo = reinterpret_cast<float*>(smem);    // [warp][16 rows][HD] then [warp][16] m, [warp][16] l
-    float* mm = mo + 4 * 16 * HD;
+    constexpr int MOS = HD + 8;                    // padded row: a warp's float2 stores of one n-tile fall on distinct banks
+    float* mo = reinterpret_cast<float*>(smem);    // [warp][16 rows][MOS] then [warp][16] m, [warp][16] l, [warp][16] weight
+    float* mm = mo + 4 * 16 * MOS;
     float* ml = mm + 4 * 16;
+    float* mw = ml + 4 * 16;
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
         const int row = g + 8 * hh;
 #pragma unroll
         for (int i = 0; i < NTO; ++i)
-            *reinterpret_cast<float2*>(mo + ((size_t)warp * 16 + row) * HD + i * 8 + 2 * t) =
+            *reinterpret_cast<float2*>(mo + ((size_t)warp * 16 + row) * MOS + i * 8 + 2 * t) =
                 make_float2(o[i][2 * hh], o[i][2 * hh + 1]);
         if (t == 0) { mm[warp * 16 + row] = m_run[hh]; ml[warp * 16 + row] = l_run[hh]; }
     }
     __syncthreads();
-    // thread -> (row tile group, row, column pairs): RTW*16 rows x HD/2 pairs over 128 threads
-    for (int idx = threadIdx.x; idx < RTW * 16 * (HD / 2); idx += kAttnThreads) {
-        const int e = 2 * (idx % (HD / 2)), rr = idx / (HD / 2), tile = rr / 16, row = rr % 16;
+    // per row: the merged maximum, every strip's weight 2^(m_strip - m) and the merged sum, once (not per column)
+    if (threadIdx.x < RTW * 16) {
+        const int tile = threadIdx.x / 16, row = threadIdx.x % 16;
         float m = -INFINITY;
 #pragma unroll
         for (int k = 0; k < KSW; ++k) m = fmaxf(m, mm[(k * RTW + tile) * 16 + row]);
-        float v0 = 0.f, v1 = 0.f, l = 0.f;
+        float l = 0.f;
 #pragma unroll
         for (int k = 0; k < KSW; ++k) {
             const int w = k * RTW + tile;
             const float ms = mm[w * 16 + row];
             const float wgt = (ms == -INFINITY) ? 0.f : exp2f(ms - m);
-            const float2 ov = *reinterpret_cast<const float2*>(mo + ((size_t)w * 16 + row) * HD + e);
-            v0 += wgt * ov.x; v1 += wgt * ov.y;
+            mw[w * 16 + row] = wgt;
             l += wgt * ml[w * 16 + row];
         }
+        Fm[threadIdx.x] = m;
+        Fl[threadIdx.x] = l;
+    }
+    __syncthreads();
+    // thread -> (row tile group, row, column pairs): RTW*16 rows x HD/2 pairs over 128 threads
+    for (int idx = threadIdx.x; idx < RTW * 16 * (HD / 2); idx += kAttnThreads) {
+        const int e = 2 * (idx % (HD / 2)), rr = idx / (HD / 2), tile = rr / 16, row = rr % 16;
+        float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+        for (int k = 0; k < KSW; ++k) {
+            const int w = k * RTW + tile;
+            const float wgt = mw[w * 16 + row];
+            const float2 ov = *reinterpret_cast<const float2*>(mo + ((size_t)w * 16 + row) * MOS + e);
+            v0 += wgt * ov.x; v1 += wgt * ov.y;
+        }
         *reinterpret_cast<float2*>(Fo + (size_t)rr * HD + e) = make_float2(v0, v1);
-        if (e == 0) { Fm[rr] = m; Fl[rr] = l; }
     }
 }
 
