@@ -186,6 +186,41 @@ def test_draft_lengths_across_token_tile_counts(engine):
     assert tally.max_logit_err < 1e-3
 
 
+@ENGINES
+def test_page_sizes_other_than_16(engine):
+    """Pages of 8, 24, 32, 64 and 128 positions: a 64-key attention tile then covers eight pages, straddles pages
+    unevenly, covers two, one, or half of one; the appended rows land across page boundaries.  (The persistent
+    engine runs attention inside its kernel only for 16-position pages: here it uses the separate kernel.)"""
+    from paper_2605_13319_b200 import binding
+    shape = synth.TINY
+    w = synth.make_weights(shape, 6)
+    tally = Tally()
+    for n, (ps, P, k) in enumerate(((8, 150, 5), (24, 101, 8), (32, 193, 3), (64, 130, 8), (128, 200, 12))):
+        ctx = binding.Context(shape, w, n_pages=(P + 48) // ps + 3, max_seq=P + 40, max_draft=16, page_size=ps,
+                              engine=engine)
+        orc = oracle.Oracle(shape, w, P + 40)
+        prefix = synth.make_prefix(shape, P, 6, request=n)
+        orc.prefill(prefix)
+        req = ctx.req_open()
+        ctx.prefill(req, prefix)
+        pending = None
+        for r in range(3):              # the cache grows across a page boundary and is truncated again
+            toks, q, u, _ = draft_inputs(orc, shape, k, 0.8, 60 + n, round_=r, pending=pending)
+            ref = orc.verify(toks, q, u)
+            (got,) = ctx.verify([dict(req=req, tokens=toks, q=q, u=u)], flags=binding.Q_HOST)
+            err = logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max()
+            assert err < LOGIT_TOL, (ps, P, r, err)
+            tally.max_logit_err = max(tally.max_logit_err, err)
+            tally.check(got, ref, ref["logits"], q, u, where=f"page_size={ps} round {r}")
+            orc.rollback(ref["base_len"], ref["n_accepted"])
+            ctx.kv_rollback([req], [ref["n_accepted"]])
+            assert ctx.req_len(req) == orc.len
+            pending = ref["next_token"]
+        ctx.close()
+    print("\n" + tally.report())
+    assert tally.max_logit_err < 1e-3
+
+
 def test_host_side_errors_and_page_accounting():
     from paper_2605_13319_b200 import binding
     shape = synth.TINY
