@@ -221,7 +221,8 @@ struct pipesd_ctx {
     int pend_n = 0;
     bool pend_check = false;   // a prefill is in flight whose device error word has not been looked at yet
     int last_rows = 0;
-    int attn_max_cs = kAttnSplits;   // largest attention cluster this device schedules (8, or 12 where the larger sizes are available)
+    int attn_occ[kAttnMaxCluster + 1][kAttnMaxRowTiles + 1] = {};   // [cluster width 9..][query row tiles]: clusters of the
+                                                                     // attention kernel the device keeps resident at once (0: width unavailable)
     int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
     int engine = 0;         // run-time switch (pipesd_debug_set_engine) inside a context of the persistent engine: 0: persistent
                             // kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only; 2: as 0, but attention
@@ -367,15 +368,21 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         // is in the batch, so that a request's summation order is the same in every batch.
         const int ncl = std::max(1, std::min(kMaxSplits / kAttnSplits, total / 2048));
         // A single cluster may be wider than eight: the width (8..10) that leaves each CTA the fewest 64-key tiles,
-        // the smallest such.  (2057 keys: 8 splits of 272 keys are five tiles each, 9 splits of 240 are four.)
+        // the smallest such, provided the request's clusters still fit the device in one wave at that width.  (2057 keys: 8 splits of 272 keys are five tiles each, 9 splits of 240 are four.)
         int cs_i = kAttnSplits;
         auto chunk_of = [&](int splits) {
             const int ch = (total + splits - 1) / splits;
             return (ch + c.page_size - 1) / c.page_size * c.page_size;
         };
-        if (ncl == 1)
-            for (int s = kAttnSplits + 1; s <= ctx->attn_max_cs; ++s)
-                if ((chunk_of(s) + kAttnTile - 1) / kAttnTile < (chunk_of(cs_i) + kAttnTile - 1) / kAttnTile) cs_i = s;
+        if (ncl == 1) {
+            const int R_i = it.rows * (c.n_q_heads / c.n_kv_heads);                  // the request's own footprint: query
+            const int qt_i = std::min(kAttnMaxRowTiles, (R_i + 15) / 16);            // row tiles and row groups per KV head
+            const int rg_i = (R_i + kAttnMaxRowTiles * 16 - 1) / (kAttnMaxRowTiles * 16);
+            for (int s = kAttnSplits + 1; s <= kAttnMaxCluster; ++s)
+                if (ctx->attn_occ[s][qt_i] >= c.n_kv_heads * rg_i &&
+                    (chunk_of(s) + kAttnTile - 1) / kAttnTile < (chunk_of(cs_i) + kAttnTile - 1) / kAttnTile)
+                    cs_i = s;
+        }
         const int chunk = chunk_of(cs_i * ncl);
         max_cs = std::max(max_cs, cs_i);
         int nsplit = ncl;   // stored per item: clusters sharing its keys
@@ -657,22 +664,25 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
                              (int)attn_smem_bytes(64, kAttnMaxRowTiles));
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
 
-    {   // clusters of 9 or 10 CTAs are non-portable sizes: opt in, and use them only if the device says it can
-        // keep one request's worth of such clusters resident at once (otherwise every cluster stays at eight)
+    {   // clusters of 9 or 10 CTAs are non-portable sizes: opt in and ask how many such clusters the device keeps
+        // resident for each shared-memory footprint (query row tiles); run_pass widens a request's cluster only if
+        // all of the request's clusters then still run in one wave
         const bool hd128 = c.head_dim == 128;
         const void* fn = hd128 ? (const void*)attn_kernel<128> : (const void*)attn_kernel<64>;
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
-            cudaLaunchConfig_t lc = {};
-            lc.gridDim = dim3(kAttnMaxCluster, 1, 1);
-            lc.blockDim = dim3(kAttnThreads);
-            lc.dynamicSmemBytes = attn_smem_bytes(c.head_dim, 1);     // a draft of up to 15 tokens per query head
-            cudaLaunchAttribute at[1];
-            at[0].id = cudaLaunchAttributeClusterDimension;
-            at[0].val.clusterDim.x = kAttnMaxCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-            lc.attrs = at; lc.numAttrs = 1;
-            int n_clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) == cudaSuccess && n_clusters >= c.n_kv_heads)   // one request's clusters in one wave
-                ctx->attn_max_cs = kAttnMaxCluster;
+            for (int w = kAttnSplits + 1; w <= kAttnMaxCluster; ++w)
+                for (int qt = 1; qt <= kAttnMaxRowTiles; ++qt) {
+                    cudaLaunchConfig_t lc = {};
+                    lc.gridDim = dim3(w, 1, 1);
+                    lc.blockDim = dim3(kAttnThreads);
+                    lc.dynamicSmemBytes = attn_smem_bytes(c.head_dim, qt);
+                    cudaLaunchAttribute at[1];
+                    at[0].id = cudaLaunchAttributeClusterDimension;
+                    at[0].val.clusterDim.x = w; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                    lc.attrs = at; lc.numAttrs = 1;
+                    int n_clusters = 0;
+                    if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) == cudaSuccess) ctx->attn_occ[w][qt] = n_clusters;
+                }
         }
         (void)cudaGetLastError();
     }
