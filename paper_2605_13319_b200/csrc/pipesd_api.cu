@@ -592,10 +592,11 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         row_stats_kernel<<<dim3(M, kStatSplits), 256, 0, st>>>(nullptr, 1, M, c.vocab, logits, stats);
         ctx->last_rows = M;
         if (want_reject) {
-            accept_sample_kernel<<<n_items, kSampleThreads, 0, st>>>(
-                logits, c.vocab, stats, reinterpret_cast<const RejectItem*>(ctx->wsp + ctx->ws.meta + ml.rej),
-                meta.row_tok, reinterpret_cast<const float*>(ctx->wsp + ctx->ws.meta + ml.u),
-                ctx->W<RejectOut>(ctx->ws.results));
+            CU(launch_pdl_cluster(accept_sample_kernel, dim3(kSampleCluster, n_items), dim3(kSampleThreads), 0, st,
+                                  kSampleCluster, (const float*)logits, c.vocab, (const RowStat*)stats,
+                                  reinterpret_cast<const RejectItem*>(ctx->wsp + ctx->ws.meta + ml.rej), meta.row_tok,
+                                  reinterpret_cast<const float*>(ctx->wsp + ctx->ws.meta + ml.u),
+                                  ctx->W<RejectOut>(ctx->ws.results)));
         }
     }
     CU(cudaGetLastError());
@@ -1109,11 +1110,13 @@ int32_t pipesd_reject_from_logits(pipesd_ctx* ctx, int32_t k, int32_t mode, cons
     if (mode == PIPESD_MODE_STOCHASTIC) CU(cudaMemcpyAsync(dq, q, 4 * (size_t)k * V, cudaMemcpyHostToDevice, st));
     RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
     row_stats_kernel<<<dim3(k + 1, kStatSplits), 256, 0, st>>>(nullptr, 1, k + 1, V, dl, stats);
-    accept_sample_kernel<<<1, kSampleThreads, 0, st>>>(
-        dl, V, stats, reinterpret_cast<const RejectItem*>(ctx->wsp + ctx->ws.meta + ml.rej),
-        reinterpret_cast<const int32_t*>(ctx->wsp + ctx->ws.meta + ml.row_tok),
-        reinterpret_cast<const float*>(ctx->wsp + ctx->ws.meta + ml.u), ctx->W<RejectOut>(ctx->ws.results));
     CU(cudaGetLastError());
+    CU(launch_pdl_cluster(accept_sample_kernel, dim3(kSampleCluster, 1), dim3(kSampleThreads), 0, st, kSampleCluster,
+                          (const float*)dl, V, (const RowStat*)stats,
+                          reinterpret_cast<const RejectItem*>(ctx->wsp + ctx->ws.meta + ml.rej),
+                          reinterpret_cast<const int32_t*>(ctx->wsp + ctx->ws.meta + ml.row_tok),
+                          reinterpret_cast<const float*>(ctx->wsp + ctx->ws.meta + ml.u),
+                          ctx->W<RejectOut>(ctx->ws.results)));
     CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     result->n_accepted = ctx->h_results[0].n_accepted;

@@ -84,28 +84,39 @@ struct RejectOut { int n_accepted, next_token, status, reserved; };
 //
 // Accept chain: the k ratio tests are independent of each other (only "stop at the first failure" is sequential),
 // so thread i evaluates test i and thread 0 takes the first failure.
-// Final draw, inverse CDF in token-id order: warp w owns the contiguous ids [w*R, (w+1)*R) (R a multiple of 32)
-// and walks them 32 at a time, lane = id, so that every load is coalesced.  Pass 1 adds each lane's terms in walk
-// order and the lanes in butterfly order (fixed); the warp totals are scanned in warp order.  Pass 2 runs only in
-// the warp whose range holds the target: an inclusive shuffle scan per 32 ids on top of the running prefix, the
-// first id whose prefix exceeds u * total wins.
+// Final draw, inverse CDF in token-id order, by a cluster of kSampleCluster CTAs per request: warp w of CTA r owns
+// the contiguous ids [(r * warps + w) * R, ... + R) (R a multiple of 32) and walks them 32 at a time, lane = id, so
+// that every load is coalesced and the fp64 exponentials of a vocabulary-wide row are spread over eight SMs.
+// Pass 1 adds each lane's terms in walk order and the lanes in butterfly order (fixed); a CTA scans its warp totals
+// in warp order, the CTA totals cross the cluster once (every CTA adds them up in rank order, so all of them hold
+// the same prefixes bit for bit).  Pass 2 runs only in the one warp whose range holds the target: an inclusive
+// shuffle scan per 32 ids on top of the running prefix, the first id whose prefix exceeds u * total wins.
+constexpr int kSampleCluster = 8;
+__device__ __forceinline__ void dsmem_st_f64(uint32_t addr, double v) {
+    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
+}
+
+// grid (kSampleCluster, n_items), cluster (kSampleCluster, 1, 1).
 __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const float* __restrict__ logits, int V,
                                                                        const RowStat* __restrict__ stats,
                                                                        const RejectItem* __restrict__ items,
                                                                        const int32_t* __restrict__ row_tok,
                                                                        const float* __restrict__ u_all,
                                                                        RejectOut* __restrict__ out) {
-    const RejectItem it = items[blockIdx.x];
-    if (it.mode == 2) return;
+    pdl_wait();      // launched with programmatic serialisation: the row statistics must be complete
+    const int item = blockIdx.y, rank = (int)cluster_ctarank();
+    const RejectItem it = items[item];
+    if (it.mode == 2) return;                     // the whole cluster (one request) leaves together
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int kWarps = kSampleThreads / 32;
     __shared__ double s_m[kMaxItemRows], s_z[kMaxItemRows];
     __shared__ int s_arg[kMaxItemRows];
     __shared__ int s_ok[kMaxItemRows];
-    __shared__ int s_nacc, s_tok;
+    __shared__ int s_nacc;
     __shared__ double s_warp[kWarps];      // warp totals, then their exclusive prefixes
     __shared__ double s_incl[kWarps];      // inclusive prefixes of the warp totals
-    __shared__ double s_total;
+    __shared__ double s_total, s_base;
+    __shared__ double s_cta[2][kSampleCluster];   // the CTAs' totals, written by their owners; one set per attempt
 
     if (tid <= it.k) {   // rows 0..k: merge the column splits
         const RowStat* st = stats + (size_t)(it.row0 + tid) * kStatSplits;
@@ -137,20 +148,20 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
         int n = 0;
         while (n < it.k && s_ok[n]) ++n;
         s_nacc = n;
-        s_tok = -1;
     }
     __syncthreads();
     const int n_acc = s_nacc;
     if (it.mode == 1) {
-        if (tid == 0) { RejectOut r{n_acc, s_arg[n_acc], 0, 0}; out[blockIdx.x] = r; }
+        if (tid == 0 && rank == 0) { RejectOut r{n_acc, s_arg[n_acc], 0, 0}; out[item] = r; }
         return;
     }
     // Final draw from row n_acc: residual max(0, p - q) if a draft was rejected there, else p.
     const float* lr = logits + (size_t)(it.row0 + n_acc) * V;
     const double m = s_m[n_acc], inv_z = 1.0 / s_z[n_acc];
     const double uk = (double)u_all[it.u0 + it.k];
-    const int R = ((V + kWarps - 1) / kWarps + 31) / 32 * 32;     // ids per warp
-    const int j0 = min(V, warp * R), j1 = min(V, j0 + R);
+    constexpr int kAllWarps = kSampleCluster * kWarps;
+    const int R = ((V + kAllWarps - 1) / kAllWarps + 31) / 32 * 32;     // ids per warp
+    const int j0 = min(V, (rank * kWarps + warp) * R), j1 = min(V, j0 + R);
     bool use_q = n_acc < it.k;
     const float* qr = use_q ? it.q + (size_t)n_acc * V : nullptr;
     auto term = [&](int j) -> double {
@@ -176,7 +187,19 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
             if (lane == 0) excl = 0.0;
             s_warp[lane] = excl;         // exclusive prefix of the warp totals = the previous warp's inclusive one, exactly
             s_incl[lane] = winc;
-            if (lane == 31) s_total = winc;
+            const double cta_total = __shfl_sync(0xffffffffu, winc, 31);
+            if (lane < kSampleCluster)   // this CTA's total into every CTA's table
+                dsmem_st_f64(dsmem_addr(smem_u32(&s_cta[attempt][rank]), (uint32_t)lane), cta_total);
+        }
+        cluster_sync_all();
+        if (tid == 0) {
+            double run = 0.0, base = 0.0;
+            for (int r = 0; r < kSampleCluster; ++r) {
+                if (r == rank) base = run;
+                run += s_cta[attempt][r];
+            }
+            s_base = base;               // ranks before this one, added in rank order: equals the previous CTA's
+            s_total = run;               // base + total exactly, so the prefixes are monotone across CTAs as well
         }
         __syncthreads();
         const double total = s_total;
@@ -187,8 +210,8 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
         }
         const double target = uk * total;
         // the owner is the first warp whose inclusive prefix exceeds the target (warp-uniform test)
-        const double before = s_warp[warp];
-        const bool mine = s_incl[warp] > target && !(before > target);     // exactly one warp: prefixes are monotone
+        const double before = s_base + s_warp[warp];
+        const bool mine = s_base + s_incl[warp] > target && !(before > target);     // exactly one warp of the cluster
         if (mine) {
             double run = before;
             int tok = -1, last_mass = -1;
@@ -206,10 +229,10 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
                 run += __shfl_sync(0xffffffffu, inc, 31);
             }
             if (tok < 0) tok = last_mass;    // the walk's rounding fell short of the range's total: its last id with mass
-            if (lane == 0) s_tok = tok;
+            if (lane == 0) { RejectOut r{n_acc, tok, 0, 0}; out[item] = r; }
         }
-        __syncthreads();
-        if (s_tok < 0 && tid == 0) {
+        // u < 1, so target < total and some warp owns it; were rounding ever to say otherwise, rank 0 answers
+        if (!(total > target) && rank == 0 && tid == 0) {
             // target >= every prefix (rounding at the top of the CDF): last token with mass
             int tok = V - 1;
             for (int j = V - 1; j >= 0; --j) {
@@ -217,12 +240,11 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
                 if (use_q) r = fmax(0.0, r - (double)qr[j]);
                 if (r > 0.0) { tok = j; break; }
             }
-            s_tok = tok;
+            RejectOut r{n_acc, tok, 0, 0};
+            out[item] = r;
         }
-        __syncthreads();
         break;
     }
-    if (tid == 0) { RejectOut r{n_acc, s_tok, 0, 0}; out[blockIdx.x] = r; }
 }
 
 }  // namespace pipesd
