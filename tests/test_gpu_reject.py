@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 def ctxs():
     from paper_2605_13319_b200 import binding
     out = {}
-    for V in (1024, 32000, 128256):
+    for V in (1008, 1024, 32000, 50256, 128256):      # 1008 and 50256: multiples of 16 only (ragged last warp range)
         shape = synth.TINY.scaled(name=f"v{V}", vocab=V, n_layers=1, d_model=64, d_ffn=64, n_q_heads=1,
                                   n_kv_heads=1)
         w = synth.make_weights(shape, 0)
@@ -23,7 +23,7 @@ def ctxs():
         c.close()
 
 
-@pytest.mark.parametrize("V,k,trials", [(1024, 4, 60), (32000, 8, 24), (128256, 16, 8)])
+@pytest.mark.parametrize("V,k,trials", [(1008, 3, 40), (1024, 4, 60), (32000, 8, 24), (50256, 5, 12), (128256, 16, 8)])
 @pytest.mark.parametrize("sigma", [0.3, 1.0, 3.0])
 def test_reject_matches_oracle(ctxs, V, k, trials, sigma):
     ctx = ctxs[V]
