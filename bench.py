@@ -330,7 +330,7 @@ def main():
     req = fresh()
     replay(ctx, req, rounds[:args.warmup], False, torch, timed=False)
     ctx.profile_enable(True)
-    replay(ctx, req, rounds[args.warmup:], False, torch)
+    ms_prof, _, _ = replay(ctx, req, rounds[args.warmup:], False, torch)
     gprof = ctx.profile_read()
     ctx.profile_enable(False)
     ctx.req_close(req)
@@ -384,7 +384,8 @@ def main():
         "gpu_launches": int(prof["kernel_launches"]),
         "roofline": {"bound": "hbm", "kernel": "gemm_wstream_kernel" if args.engine == "tiled" else "mega_kernel", "achieved": gemm_gbs, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": gemm_gbs / peak,
-                     "launches": int(gprof["gemm_launches"]), "share_of_step": gprof["gemm_ms"] / ms,
+                     "launches": int(gprof["gemm_launches"]), "share_of_step": gprof["gemm_ms"] / ms_prof,
+                     "ms_per_step_with_events": ms_prof / steps,
                      "algorithmic_bytes_per_launch": gprof["gemm_bytes"] / max(1, gprof["gemm_launches"]),
                      "traffic": TRAFFIC_7B_K8.get(args.engine) if args.workload == "7b-k8" else None},
         "clocks": clocks,
