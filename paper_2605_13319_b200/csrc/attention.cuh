@@ -1,20 +1,23 @@
 // Multi-query decode attention over a paged bf16 KV cache: each request contributes a short chunk
 // of query rows (the pending token plus its k drafts) that attend to the cached prefix and, causally,
-// to each other.  The keys are cut into 8 splits ("split-K") handled by the 8 CTAs of a thread-block
+// to each other.  The keys are cut into 8 to 10 splits ("split-K") handled by the CTAs of a thread-block
 // cluster; every CTA produces an un-normalised partial output with its running max and sum in its own
 // shared memory, and after a cluster barrier the partials are merged over distributed shared memory and
 // written straight into the output projection's input format -- no partial results in global memory and
-// no separate merge kernel.  Tiles of keys that were cached before this pass do not depend on the
-// preceding QKV projection, so their copies are issued before the dependent-launch wait.
+// no separate merge kernel (requests of 4096 keys and more use several clusters and one more merge step).
+// Tiles of keys that were cached before this pass do not depend on the preceding QKV projection, so their
+// copies are issued before the dependent-launch wait.
 //
 // One CTA (4 warps) = one KV head of one request x one split x up to 64 query rows, where the rows are
 // all (query head of the group, chunk row) pairs that share the KV head (GQA).  K and V tiles of 64 keys
-// travel global -> shared with 16-byte cp.async in a two-stage ring (page table resolved per key row,
-// the pool stores every row with its 16-byte chunks XOR-permuted, so that ldmatrix is conflict-free).  QK^T and PV run on mma.sync m16n8k16 with fp32
-// accumulation; Q and the softmax probabilities are fp32 values split into bf16 hi + lo terms (two MMAs),
-// K and V are the cache's bf16.  How the 4 warps share a tile depends on the number of 16-row tiles:
-// 1 tile -> 4 key strips of 16, 2 tiles -> 2 x 2 strips of 32, 3-4 tiles -> one tile each over all 64 keys;
-// warps that split the keys keep independent online-softmax states that are merged in shared memory.
+// travel global -> shared by bulk copies in a two-stage ring: the rows of a page that belong to one KV head
+// are contiguous in the pool, so one thread issues one copy per page and K|V and every thread waits on the
+// stage's barrier (the pool stores every row with its 16-byte chunks XOR-permuted, so that ldmatrix is
+// conflict-free on the verbatim copy).  QK^T and PV run on mma.sync m16n8k16 with fp32 accumulation; Q and
+// the softmax probabilities are fp32 values split into bf16 hi + lo terms (two MMAs), K and V are the cache's
+// bf16.  How the 4 warps share a tile depends on the number of 16-row tiles: 1 tile -> 4 key strips of 16,
+// 2 tiles -> 2 x 2 strips of 32, 3-4 tiles -> one tile each over all 64 keys; warps that split the keys keep
+// independent online-softmax states that are merged in shared memory.
 #pragma once
 #include "common.cuh"
 #include "layers.cuh"
