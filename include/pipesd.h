@@ -219,6 +219,15 @@ int32_t pipesd_gemm_pack(const void *W, void *packed, int32_t N, int32_t K, void
 int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scratch, int32_t M, int32_t N,
                         int32_t K, void *cuda_stream);
 
+/* Host only, no CUDA call: how the attention kernel splits a request of `total_keys` keys (cached + this pass's
+ * rows) at the given page size.  resident_clusters[0..2] (host) = thread-block clusters of 8, 9 and 10 CTAs the
+ * device keeps resident at once for the request's footprint (0 = that width is unavailable), clusters_needed =
+ * clusters one layer launches for the request (KV heads x row groups).  out3 (host) receives {clusters sharing the
+ * keys, key splits per cluster, keys per split (a multiple of page_size)}.  The split is a function of the request
+ * alone, which is what keeps a request's result independent of its batch.  PIPESD_E_INVALID on bad arguments. */
+int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t *resident_clusters,
+                                int32_t clusters_needed, int32_t *out3);
+
 /* Tuning hook: force the number of K slices of every subsequent GEMM plan (0 = choose automatically). */
 int32_t pipesd_debug_gemm_force_split(int32_t S);
 

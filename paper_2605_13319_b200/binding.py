@@ -92,6 +92,7 @@ _SIGNATURES = {
     "pipesd_gemm_pack": (i32, [vp, vp, i32, i32, vp]),
     "pipesd_gemm_run": (i32, [vp, vp, vp, vp, i32, i32, i32, vp]),
     "pipesd_gemm_run_static": (i32, [vp, vp, vp, i32, i32, i32, vp]),
+    "pipesd_debug_attn_split": (i32, [i32, i32, ctypes.POINTER(ctypes.c_int32), i32, ctypes.POINTER(ctypes.c_int32)]),
     "pipesd_debug_gemm_force_split": (i32, [i32]),
 }
 
@@ -350,3 +351,13 @@ def gemm_run_static(packed, x, y, N, K, stream=None):
     rc = lib().pipesd_gemm_run_static(packed.data_ptr(), x.data_ptr(), y.data_ptr(), M, N, K, vp(st.cuda_stream))
     if rc != OK:
         raise PipesdError(rc, "pipesd_gemm_run_static")
+
+
+def debug_attn_split(total_keys: int, page_size: int, resident_clusters, clusters_needed: int):
+    """(clusters sharing the keys, key splits per cluster, keys per split) of one request: host arithmetic only."""
+    res = (ctypes.c_int32 * 3)(*[int(x) for x in resident_clusters])
+    out = (ctypes.c_int32 * 3)()
+    rc = lib().pipesd_debug_attn_split(total_keys, page_size, res, clusters_needed, out)
+    if rc != 0:
+        raise PipesdError(rc, "pipesd_debug_attn_split")
+    return tuple(out)

@@ -339,6 +339,28 @@ constexpr int kAttnSplits = 8;        // key splits per cluster of a request who
 constexpr int kAttnMaxCluster = 10;   // largest cluster along x (above 8: the non-portable sizes, opted into by the host;
                                       // a B200 keeps 41 clusters of 10 of this kernel resident but only 31 of 11 or 12)
 
+// Host: how one request's keys are split.  `resident[w - 8]` = clusters of width w (8, 9, 10) the device keeps
+// resident at once for this request's shared-memory footprint (0: width unavailable); `need` = clusters the request
+// launches per layer (KV heads x row groups).  One cluster of eight per 2048 keys up to four clusters; a single
+// cluster widens to the smallest width that leaves each CTA the fewest 64-key tiles, as long as all the request's
+// clusters still run in one wave.  Everything here depends on the request alone, never on its batch.
+struct AttnSplit { int clusters, width, keys_per_split; };
+static inline AttnSplit attn_split_plan(int total_keys, int page_size, const int* resident, int need) {
+    AttnSplit p;
+    p.clusters = total_keys / 2048 < 1 ? 1 : (total_keys / 2048 > kMaxSplits / kAttnSplits ? kMaxSplits / kAttnSplits : total_keys / 2048);
+    p.width = kAttnSplits;
+    auto chunk_of = [&](int splits) {
+        const int ch = (total_keys + splits - 1) / splits;
+        return (ch + page_size - 1) / page_size * page_size;
+    };
+    auto tiles_of = [&](int splits) { return (chunk_of(splits) + kAttnTile - 1) / kAttnTile; };
+    if (p.clusters == 1)
+        for (int w = kAttnSplits + 1; w <= kAttnMaxCluster; ++w)
+            if (resident[w - kAttnSplits] >= need && tiles_of(w) < tiles_of(p.width)) p.width = w;
+    p.keys_per_split = chunk_of(p.width * p.clusters);
+    return p;
+}
+
 #ifdef PIPESD_GEMM_TRACE
 // Development build only: per (layer, CTA) timestamps of the attention kernel's anatomy.
 __device__ unsigned long long g_attn_trace[64 * 512 * 8];

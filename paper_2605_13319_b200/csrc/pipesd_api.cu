@@ -363,27 +363,15 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         const ItemDesc& it = items[i];
         const Request& r = ctx->reqs[it.slot];
         const int total = r.len + it.rows;
-        // one cluster of eight key splits per (request, KV head, row group); a long context gets one more
-        // cluster per 2048 keys (up to four).  The count depends on the request alone, never on what else
-        // is in the batch, so that a request's summation order is the same in every batch.
-        const int ncl = std::max(1, std::min(kMaxSplits / kAttnSplits, total / 2048));
-        // A single cluster may be wider than eight: the width (8..10) that leaves each CTA the fewest 64-key tiles,
-        // the smallest such, provided the request's clusters still fit the device in one wave at that width.  (2057 keys: 8 splits of 272 keys are five tiles each, 9 splits of 240 are four.)
-        int cs_i = kAttnSplits;
-        auto chunk_of = [&](int splits) {
-            const int ch = (total + splits - 1) / splits;
-            return (ch + c.page_size - 1) / c.page_size * c.page_size;
-        };
-        if (ncl == 1) {
-            const int R_i = it.rows * (c.n_q_heads / c.n_kv_heads);                  // the request's own footprint: query
-            const int qt_i = std::min(kAttnMaxRowTiles, (R_i + 15) / 16);            // row tiles and row groups per KV head
-            const int rg_i = (R_i + kAttnMaxRowTiles * 16 - 1) / (kAttnMaxRowTiles * 16);
-            for (int s = kAttnSplits + 1; s <= kAttnMaxCluster; ++s)
-                if (ctx->attn_occ[s][qt_i] >= c.n_kv_heads * rg_i &&
-                    (chunk_of(s) + kAttnTile - 1) / kAttnTile < (chunk_of(cs_i) + kAttnTile - 1) / kAttnTile)
-                    cs_i = s;
-        }
-        const int chunk = chunk_of(cs_i * ncl);
+        // clusters that share the request's keys, key splits per cluster (8..10) and keys per split: from the request
+        // alone (its length, its rows), so that its summation order is the same in every batch
+        const int R_i = it.rows * (c.n_q_heads / c.n_kv_heads);                  // query rows per KV head
+        const int qt_i = std::min(kAttnMaxRowTiles, (R_i + 15) / 16);
+        const int rg_i = (R_i + kAttnMaxRowTiles * 16 - 1) / (kAttnMaxRowTiles * 16);
+        int resident[kAttnMaxCluster - kAttnSplits + 1];
+        for (int w = kAttnSplits; w <= kAttnMaxCluster; ++w) resident[w - kAttnSplits] = ctx->attn_occ[w][qt_i];
+        const AttnSplit sp = attn_split_plan(total, c.page_size, resident, c.n_kv_heads * rg_i);
+        const int ncl = sp.clusters, cs_i = sp.width, chunk = sp.keys_per_split;
         max_cs = std::max(max_cs, cs_i);
         int nsplit = ncl;   // stored per item: clusters sharing its keys
         I(ml.it_slot)[i] = it.slot;
@@ -1242,6 +1230,16 @@ int32_t pipesd_gemm_run(const void* packed, const float* x, float* y, void* scra
         attrs = true;
     }
     return gemm_run_with_scratch(packed, x, y, scratch, M, N, K, (cudaStream_t)cuda_stream);
+}
+
+int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t* resident_clusters,
+                                int32_t clusters_needed, int32_t* out3) {
+    if (!resident_clusters || !out3 || total_keys < 1 || page_size < 8 || page_size % 8) return PIPESD_E_INVALID;
+    int res[kAttnMaxCluster - kAttnSplits + 1];
+    for (int i = 0; i <= kAttnMaxCluster - kAttnSplits; ++i) res[i] = resident_clusters[i];
+    const AttnSplit p = attn_split_plan(total_keys, page_size, res, clusters_needed);
+    out3[0] = p.clusters; out3[1] = p.width; out3[2] = p.keys_per_split;
+    return PIPESD_OK;
 }
 
 int32_t pipesd_debug_gemm_force_split(int32_t S) {

@@ -41,3 +41,37 @@ def test_pure_host_entry_points():
     assert L.pipesd_query_sizes(ctypes.byref(bad), ctypes.byref(sz)) == binding.E_INVALID   # 32 % 5
     assert L.pipesd_gemm_packed_bytes(4096, 11008) == 4096 * 11008 * 2
     assert L.pipesd_gemm_scratch_bytes(9, 4096, 11008) >= 9 * 4096 * 4
+
+
+def test_attention_key_split_plan():
+    """The split of a request's keys over clusters and CTAs: a function of the request alone."""
+    wide = (48, 45, 41)            # clusters of 8, 9, 10 the device keeps resident (a B200, one query row tile)
+    # 2057 keys: 8 splits of 272 keys are five 64-key tiles per CTA, 9 splits of 240 are four, 10 no fewer
+    assert binding.debug_attn_split(2057, 16, wide, 32) == (1, 9, 240)
+    # the wider cluster must still hold the whole request in one wave
+    assert binding.debug_attn_split(2057, 16, (48, 31, 31), 32) == (1, 8, 272)
+    assert binding.debug_attn_split(2057, 16, (48, 0, 0), 32) == (1, 8, 272)          # widths unavailable
+    assert binding.debug_attn_split(2057, 16, (48, 31, 41), 32) == (1, 10, 208)       # 9 does not fit, 10 does: four tiles
+    # 521 keys: 9 splits of 64 keys are one tile each, 8 splits of 80 are two
+    assert binding.debug_attn_split(521, 16, wide, 8) == (1, 9, 64)
+    # short requests: nothing to gain, stay at eight; splits are whole pages
+    assert binding.debug_attn_split(9, 16, wide, 8) == (1, 8, 16)
+    assert binding.debug_attn_split(100, 8, wide, 8) == (1, 8, 16)
+    assert binding.debug_attn_split(100, 64, wide, 8) == (1, 8, 64)
+    # one more cluster per 2048 keys, up to four, eight splits each
+    assert binding.debug_attn_split(4096, 16, wide, 32) == (2, 8, 256)
+    assert binding.debug_attn_split(8209, 16, wide, 16) == (4, 8, 272)
+    assert binding.debug_attn_split(40000, 16, wide, 16) == (4, 8, 1264)
+    # every key is covered, splits are page multiples, whatever the length
+    for total in list(range(1, 300)) + [1023, 1024, 1025, 2047, 2048, 4095, 4097, 6143, 6144, 12345]:
+        for ps in (8, 16, 24, 64):
+            ncl, w, chunk = binding.debug_attn_split(total, ps, wide, 8)
+            assert 8 <= w <= 10 and 1 <= ncl <= 4 and chunk % ps == 0
+            assert ncl * w * chunk >= total
+            assert (w == 8) or ncl == 1
+            if w > 8:   # widened only for fewer tiles per CTA
+                c8 = -(-(-(-total // 8)) // ps) * ps
+                assert -(-chunk // 64) < -(-c8 // 64)
+    import pytest
+    with pytest.raises(binding.PipesdError):
+        binding.debug_attn_split(100, 12, wide, 8)
