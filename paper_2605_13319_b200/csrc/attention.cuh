@@ -11,7 +11,7 @@
 // One CTA (4 warps) = one KV head of one request x one split x up to 64 query rows, where the rows are
 // all (query head of the group, chunk row) pairs that share the KV head (GQA).  K and V tiles of 64 keys
 // travel global -> shared by bulk copies in a two-stage ring: the rows of a page that belong to one KV head
-// are contiguous in the pool, so one thread issues one copy per page and K|V and every thread waits on the
+// are contiguous in the pool, so the lanes of one warp issue one copy per page and K|V and every thread waits on the
 // stage's barrier (the pool stores every row with its 16-byte chunks XOR-permuted, so that ldmatrix is
 // conflict-free on the verbatim copy).  QK^T and PV run on mma.sync m16n8k16 with fp32 accumulation; Q and
 // the softmax probabilities are fp32 values split into bf16 hi + lo terms (two MMAs), K and V are the cache's
@@ -91,23 +91,23 @@ __device__ __forceinline__ void split2_bf16(float a, float b, uint32_t& hi, uint
     lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-// Issue (one thread) the copies of one 64-key tile into a ring stage: the rows of a page that belong to one KV head
+// Issue (one warp) the copies of one 64-key tile into a ring stage: the rows of a page that belong to one KV head
 // are contiguous in the pool (already chunk-permuted), so every page the tile touches is one bulk copy of K rows
-// and one of V rows, counted in bytes on the stage's barrier.  Rows at or beyond k1 are not copied.
+// and one of V rows, counted in bytes on the stage's barrier; lane l takes the l-th page of the tile (at most nine).
+// Rows at or beyond k1 are not copied.
 template <int HD>
 __device__ __forceinline__ void attn_issue_tile(const AttnCtx& c, uint32_t stage_addr, uint32_t bar, int j0) {
+    const int lane = threadIdx.x & 31;
     const int j1 = min(j0 + kAttnTile, c.k1);
-    mbar_expect_tx(bar, (uint32_t)(j1 - j0) * (HD * 2) * 2);
-    int pidx = j0 / c.page_size, slot = j0 - pidx * c.page_size;
-    for (int j = j0; j < j1;) {
-        const int n = min(c.page_size - slot, j1 - j);
-        const uint16_t* kp = c.kbase + (size_t)c.bt[pidx - c.bt_first] * c.page_stride + (size_t)slot * HD;
-        const uint32_t dst = stage_addr + (uint32_t)(j - j0) * (HD * 2);
-        bulk_g2s(dst, kp, (uint32_t)n * (HD * 2), bar);
-        bulk_g2s(dst + AttnSmem<HD>::kTileBytes, kp + c.v_off, (uint32_t)n * (HD * 2), bar);
-        j += n;
-        slot = 0;
-        ++pidx;
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)(j1 - j0) * (HD * 2) * 2);
+    __syncwarp();
+    const int pidx = j0 / c.page_size + lane;                          // this lane's page of the request
+    const int js = max(j0, pidx * c.page_size), je = min(j1, (pidx + 1) * c.page_size);
+    if (js < je) {
+        const uint16_t* kp = c.kbase + (size_t)c.bt[pidx - c.bt_first] * c.page_stride + (size_t)(js - pidx * c.page_size) * HD;
+        const uint32_t dst = stage_addr + (uint32_t)(js - j0) * (HD * 2);
+        bulk_g2s(dst, kp, (uint32_t)(je - js) * (HD * 2), bar);
+        bulk_g2s(dst + AttnSmem<HD>::kTileBytes, kp + c.v_off, (uint32_t)(je - js) * (HD * 2), bar);
     }
 }
 
@@ -149,7 +149,7 @@ __device__ __forceinline__ void attn_body(const AttnCtx& c, const AttnCtx* c_iss
         const int stg = it % kAttnStages;
         if (it > 0) {
             __syncthreads();      // everyone is done with tile it-1: its stage can take tile it+1
-            if (it + 1 < ntiles && threadIdx.x == 0) {
+            if (it + 1 < ntiles && warp == 0) {
                 fence_proxy_async_smem();      // the stage was read with ordinary loads; the copy engine writes it next
                 attn_issue_tile<HD>(*c_issue, ring + ((it + 1) % kAttnStages) * SM::kStageBytes,
                                     bars + 8 * ((it + 1) % kAttnStages), c.k0 + (it + 1) * kAttnTile);
@@ -435,22 +435,25 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
 
     // Tiles made only of keys cached before this pass do not depend on the QKV projection that precedes this
     // kernel: their copies are issued now, the others after the dependency has resolved.
-    __shared__ AttnCtx s_ctx;      // thread 0's copy: what issuing a tile needs stays out of everyone's registers
+    __shared__ AttnCtx s_ctx;      // warp 0's copy: what issuing a tile needs stays out of everyone's registers
     __shared__ __align__(8) unsigned long long s_bars[kAttnStages];
     const uint32_t bars = smem_u32(s_bars);
     const int ntiles = c.k1 > c.k0 ? (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile : 0;
     const bool early0 = ntiles > 0 && min(c.k0 + kAttnTile, c.k1) <= c.base;
     const bool early1 = ntiles > 1 && min(c.k0 + 2 * kAttnTile, c.k1) <= c.base;
-    if (threadIdx.x == 0) {
-        s_ctx = c;
-        for (int i = 0; i < kAttnStages; ++i) mbar_init(bars + 8 * i, 1);
-        fence_mbar_init();
+    if (threadIdx.x < 32) {          // warp 0 issues every tile
+        if (threadIdx.x == 0) {
+            s_ctx = c;
+            for (int i = 0; i < kAttnStages; ++i) mbar_init(bars + 8 * i, 1);
+            fence_mbar_init();
+        }
+        __syncwarp();
         if (early0) attn_issue_tile<HD>(s_ctx, ring, bars, c.k0);
         if (early1) attn_issue_tile<HD>(s_ctx, ring + SM::kStageBytes, bars + 8, c.k0 + kAttnTile);
     }
     pdl_wait();
     ATTN_TRACE(1);
-    if (threadIdx.x == 0) {
+    if (threadIdx.x < 32) {
         if (!early0 && ntiles > 0) attn_issue_tile<HD>(s_ctx, ring, bars, c.k0);
         if (!early1 && ntiles > 1) attn_issue_tile<HD>(s_ctx, ring + SM::kStageBytes, bars + 8, c.k0 + kAttnTile);
     }
