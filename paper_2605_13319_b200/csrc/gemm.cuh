@@ -94,10 +94,12 @@ static inline GemmPlan gemm_plan(int M, int N, int K) {
     // GEMM always leaves room for three CTAs per SM, even when it brings fewer: at two 113 KB CTAs per SM a B200
     // holds exactly the 32 clusters of eight that the O and down projections launch, so one foreign CTA in a GPC
     // pushed a cluster into a second wave, and the next kernel's CTAs found no room to start and prefetch their
-    // weights under this kernel's tail.  Three stages instead of five for those two: -0.14 ms per 7B pass.
+    // weights under this kernel's tail.  Three stages instead of five for those two: -0.14 ms per 7B pass at up to 16
+    // rows.  With three or four token tiles per block the MMA work per chunk is 1.5-2x and the deeper ring wins
+    // (7b, 17 rows: 3.81 ms with five stages, 4.00 ms with three), so those keep the depth by CTA count.
     long ctas = (long)p.RB * p.S * p.TB;
     int per_sm = (int)((ctas + 147) / 148);
-    if (p.S > 1) per_sm = kGemmCtasPerSm;
+    if (p.S > 1 && p.NT <= 2) per_sm = kGemmCtasPerSm;
     per_sm = per_sm < 1 ? 1 : (per_sm > kGemmCtasPerSm ? kGemmCtasPerSm : per_sm);
     int budget = (227 * 1024) / per_sm - 1024 - kGemmSmemTail;
     p.stages = budget / gemm_stage_bytes(p.NT);
