@@ -22,7 +22,9 @@
  * orc_rope, orc_softmax, orc_attend against closed forms and invariants; orc_forward against a
  * hand-worked two-token model, chunking invariance, causality and the GQA==replicated-MHA
  * identity; orc_reject against brute-force enumeration of the output distribution, the greedy
- * longest-matching-prefix property, p == q, one-hot q and the 1 - TV(p,q) acceptance rate.
+ * longest-matching-prefix property, p == q, one-hot q and the 1 - TV(p,q) acceptance rate;
+ * orc_set_kv / orc_set_len / orc_get_kv against a bit-exact round trip, a closed-form attention over
+ * hand-set rows and a cache transplanted row by row into a fresh instance.
  */
 #include <math.h>
 #include <stdint.h>

@@ -386,11 +386,15 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
                                                             int q_tiles_smem, int row_groups, float* __restrict__ o_part,
                                                             float* __restrict__ m_part, float* __restrict__ l_part,
                                                             int* __restrict__ tickets, uint16_t* __restrict__ xf_out,
-                                                            int xu_layout, int* __restrict__ err) {
+                                                            int xu_layout, int* __restrict__ err, const L2Prefetch pf) {
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = AttnSmem<HD>;
     pdl_launch_dependents();
     ATTN_TRACE(0);
+    // attention leaves most of the HBM bandwidth unused: the output projection's weights come into L2 meanwhile
+    if (threadIdx.x == 0)
+        l2_prefetch_issue(pf, (int)((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x),
+                          (int)(gridDim.x * gridDim.y * gridDim.z));
     const int item = blockIdx.z;
     const int cs = (int)cluster_nctaid_x();
     const int cl = blockIdx.x / cs, rank = blockIdx.x % cs;        // cluster of this (request, head), rank in it

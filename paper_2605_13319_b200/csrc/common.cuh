@@ -122,6 +122,29 @@ __device__ __forceinline__ void bulk_g2s_hint(uint32_t dst_smem, const void* src
                  "l"(src), "r"(bytes), "r"(bar), "l"(pol)
                  : "memory");
 }
+// Hint: pull a contiguous global range into L2 (no destination, no completion to wait for).  Address 16-byte
+// aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+// What a kernel pulls into L2 on behalf of its successor while its own demand on HBM ebbs (its tail: split-K
+// reduction, epilogue, grid hand-over leave HBM idle for several microseconds).  The successor's weights are cut
+// into `runs` contiguous ranges of `run_bytes` (one per successor CTA); the successor copies the first `skip`
+// bytes of its range into shared memory by itself before its dependency wait, so the hint covers the `len`
+// bytes after those.  Purely a hint: results never depend on it.
+struct L2Prefetch {
+    const unsigned char* ptr;   // null: nothing to prefetch
+    uint32_t run_bytes, skip, len;
+    int runs;
+};
+// CTA `cta` of `n_ctas` issues the hints of runs cta, cta + n_ctas, ... (one thread calls this).
+__device__ __forceinline__ void l2_prefetch_issue(const L2Prefetch& pf, int cta, int n_ctas) {
+    if (pf.ptr == nullptr) return;
+    for (int r = cta; r < pf.runs; r += n_ctas) {
+        const unsigned char* p = pf.ptr + (size_t)r * pf.run_bytes + pf.skip;
+        for (uint32_t o = 0; o < pf.len; o += 16384u) bulk_prefetch_l2(p + o, pf.len - o < 16384u ? pf.len - o : 16384u);
+    }
+}
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
 // while its predecessor drains; pdl_wait() blocks until the predecessor has completed and its writes
 // are visible, pdl_launch_dependents() lets the successor start early.

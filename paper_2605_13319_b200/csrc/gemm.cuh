@@ -198,7 +198,26 @@ struct GemmArgs {
     float* ssq_out;     // [RB][M] sums of squares of x_new over the row block's columns
     // kSwiglu
     uint16_t* xf_act;   // silu(gate)*up as split-bf16 fragments, feature-major K = N/2
+    // the successor's weights this kernel pulls into L2 once its own last chunk has been requested
+    L2Prefetch pf;
 };
+
+// Host: the L2 hint that covers `depth_bytes` of every CTA's weight range of the GEMM (M, N, K) over `W`, after the
+// chunks that GEMM's CTAs copy by themselves before their dependency wait (their whole ring).
+static inline L2Prefetch gemm_prefetch_of(const void* W, int M, int N, int K, uint32_t depth_bytes) {
+    L2Prefetch pf = {};
+    if (W == nullptr || depth_bytes == 0) return pf;
+    const GemmPlan p = gemm_plan(M, N, K);
+    const uint32_t run = (uint32_t)(p.KS / p.S) * 4096u;           // K slices differ by at most one k16 step: a hint may be off by that
+    const uint32_t skip = (uint32_t)p.stages * kGemmWStage;
+    if (run <= skip) return pf;
+    pf.ptr = reinterpret_cast<const unsigned char*>(W);
+    pf.run_bytes = run;
+    pf.skip = skip;
+    pf.len = run - skip < depth_bytes ? run - skip : depth_bytes;
+    pf.runs = p.RB * p.S;
+    return pf;
+}
 
 template <int NT, int MODE>
 __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_kernel(const GemmArgs a) {
@@ -272,6 +291,8 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                 issued = c + 1;
                 if (++st == stages) { st = 0; ph ^= 1u; }
             }
+            // this CTA has asked for its last weights: from here on HBM idles until the successor streams
+            if (ok) l2_prefetch_issue(a.pf, (int)(blockIdx.y * gridDim.x + blockIdx.x), (int)(gridDim.x * gridDim.y));
             if (!ok) {
                 if (a.err) atomicExch(a.err, 1);
                 // give up: let every copy already issued land before this CTA's shared memory is released

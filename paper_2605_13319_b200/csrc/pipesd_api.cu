@@ -3,6 +3,7 @@
 // page tables and request lengths, uploads the per-call metadata and launches.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -223,6 +224,7 @@ struct pipesd_ctx {
     int last_rows = 0;
     int attn_occ[kAttnMaxCluster + 1][kAttnMaxRowTiles + 1] = {};   // [cluster width 9..][query row tiles]: clusters of the
                                                                      // attention kernel the device keeps resident at once (0: width unavailable)
+    uint32_t pf_depth = 64u << 10;   // bytes per successor CTA that a GEMM pulls into L2 for the next GEMM
     int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
     int engine = 0;         // run-time switch (pipesd_debug_set_engine) inside a context of the persistent engine: 0: persistent
                             // kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only; 2: as 0, but attention
@@ -445,17 +447,20 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     base.eps = c.rms_eps;
     base.d_in = d;
     base.n_ssq = n_ssq;
+    // depth of the L2 hints a kernel issues for its successor's weights (bytes per successor CTA)
+    const uint32_t pf_depth = ctx->pf_depth;
     auto launch_attn = [&](int l) -> int {
+        const L2Prefetch pf = use_mega ? L2Prefetch{} : gemm_prefetch_of(ctx->layers[l].o.packed, M, d, dv.qd, 1u << 20);
         dim3 ag(max_cs * max_nsplit, Hkv * row_groups, n_items);   // cluster = the widest any request of the batch asks for
         int* tickets = ctx->W<int>(ctx->ws.tickets);
         if (hd == 128)
             CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, max_cs, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0, ctx->err_word()));
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0, ctx->err_word(), pf));
         else
             CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, max_cs, (const float*)qbuf,
                                   meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0, ctx->err_word()));
+                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0, ctx->err_word(), pf));
         ctx->n_launch += 1;
         return PIPESD_OK;
     };
@@ -546,6 +551,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             GemmArgs a = base;
             a.W = lw.o.packed; a.xf = (const uint4*)xf_attn; a.N = d; a.ssq_in = nullptr;
             a.x = x; a.xf_out = (uint16_t*)xf_h; a.gain_next = lw.n2; a.ssq_out = ssqB;
+            a.pf = gemm_prefetch_of(lw.gu.packed, M, 2 * F, d, pf_depth);
             int rc_ = launch_gemm(ctx, kResid, a, dv.qd);
             if (rc_) return rc_;
         }
@@ -553,6 +559,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             GemmArgs a = base;
             a.W = lw.gu.packed; a.xf = (const uint4*)xf_h; a.N = 2 * F; a.ssq_in = ssqB;
             a.xf_act = (uint16_t*)xf_act;
+            a.pf = gemm_prefetch_of(lw.dn.packed, M, d, F, pf_depth);
             int rc_ = launch_gemm(ctx, kSwiglu, a, d);
             if (rc_) return rc_;
         }
@@ -562,6 +569,8 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             a.x = x; a.xf_out = (uint16_t*)xf_h;
             a.gain_next = l + 1 < c.n_layers ? ctx->layers[l + 1].n1 : ctx->final_norm;
             a.ssq_out = ssqA;
+            if (l + 1 < c.n_layers) a.pf = gemm_prefetch_of(ctx->layers[l + 1].qkv.packed, M, dv.Nqkv, d, pf_depth);
+            else if (want_logits) a.pf = gemm_prefetch_of(ctx->lm.packed, M, c.vocab, d, pf_depth);
             int rc_ = launch_gemm(ctx, kResid, a, F);
             if (rc_) return rc_;
         }
@@ -675,6 +684,7 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         }
         (void)cudaGetLastError();
     }
+    if (const char* e_pf = getenv("PIPESD_PF_KB")) ctx->pf_depth = (uint32_t)atoi(e_pf) << 10;
     ctx->kv_pool = (uint16_t*)mem->kv;
     ctx->wsp = (char*)mem->workspace;
     for (int i = 0; i < pipesd_ctx::kStages; ++i) {

@@ -140,6 +140,77 @@ def test_verify_greedy_and_all_accept(tiny):
     assert o.len == 6 + 4
 
 
+def test_cache_load_and_read_back_round_trip_and_transplant(tiny):
+    """orc_set_kv / orc_set_len / orc_get_kv: what the full-size parity tests and the timed CPU baseline load
+    their prefix through.  (1) rows written at a non-zero layer and position come back bit for bit, widened from
+    bf16 exactly, and leave their neighbours alone; (2) a hand-sized cache (one key, V set by hand) gives the
+    closed-form attention result, so the loaded values are the ones the forward reads; (3) a cache built by a
+    prefill, copied row by row into a fresh instance, yields identical logits on the next forward."""
+    shape, w = tiny
+    wd = shape.n_kv_heads * shape.head_dim
+    o = oracle.Oracle(shape, w, 32)
+    # (1) bit-exact round trip, layer 1, positions 5..7; every bf16 exponent and sign pattern that is finite
+    bits_k = synth.tokens_i32(3 * wd, 11, 1, 0x7f00).astype(np.uint16).reshape(3, wd)
+    bits_v = (synth.tokens_i32(3 * wd, 11, 2, 0x7f00).astype(np.uint16) | np.uint16(0x8000)).reshape(3, wd)
+    o.set_synthetic_kv(1, bits_k, bits_v, pos0=5)
+    for p in range(3):
+        kk, vv = o.get_kv(1, 5 + p)
+        assert np.array_equal(kk.view(np.uint32), bits_k[p].astype(np.uint32) << 16)
+        assert np.array_equal(vv.view(np.uint32), bits_v[p].astype(np.uint32) << 16)
+    for layer, pos in ((0, 5), (1, 4), (1, 8)):          # neighbours in both directions stay zero
+        kk, vv = o.get_kv(layer, pos)
+        assert not kk.any() and not vv.any()
+    assert o.len == 0                                     # set_kv does not move the length
+    o.set_len(8)
+    assert o.len == 8
+    # (3) transplant: prefill -> get_kv -> set_kv + set_len into a fresh instance -> same logits, exactly
+    a = oracle.Oracle(shape, w, 32)
+    prefix = synth.tokens_i32(9, 12, 0, shape.vocab)
+    a.prefill(prefix)
+    b = oracle.Oracle(shape, w, 32)
+    for l in range(shape.n_layers):
+        rows = [a.get_kv(l, p) for p in range(9)]
+        kb = synth.f32_to_bf16(np.stack([r[0] for r in rows]))
+        vb = synth.f32_to_bf16(np.stack([r[1] for r in rows]))
+        b.set_synthetic_kv(l, kb, vb)
+    b.set_len(9)
+    nxt = synth.tokens_i32(4, 12, 1, shape.vocab)
+    assert np.array_equal(a.forward(nxt), b.forward(nxt))
+    # a row loaded one position off, or into the wrong layer, changes the result
+    c = oracle.Oracle(shape, w, 32)
+    for l in range(shape.n_layers):
+        rows = [a.get_kv(l, p) for p in range(9)]
+        kb = synth.f32_to_bf16(np.stack([r[0] for r in rows]))
+        vb = synth.f32_to_bf16(np.stack([r[1] for r in rows]))
+        c.set_synthetic_kv(shape.n_layers - 1 - l, kb, vb)
+    c.set_len(9)
+    a.truncate(9)
+    assert not np.array_equal(a.forward(nxt), c.forward(nxt))
+
+
+def test_loaded_cache_is_what_attention_reads():
+    """Closed form on the hand-sized model: with the prefix K rows all zero every cached score is 0, so a query row
+    attends uniformly over the loaded V rows and itself; the loaded V values (exact small integers) appear in the
+    logits through the known tail of that model."""
+    shape = synth.ModelShape("hand", 1, 2, 1, 1, 2, 1, 3, rms_eps=0.0, rope_base=10000.0)
+    I2 = [[1.0, 0.0], [0.0, 1.0]]
+    Z2 = [[0.0, 0.0], [0.0, 0.0]]
+    w = {"tok_emb": _bf16([[1, 1], [1, -1], [2, 0]]), "lm_head": _bf16([[1, 0], [0, 1], [1, 1]]),
+         "final_norm": np.ones(2, np.float32),
+         "layers": [{"wq": _bf16(I2), "wk": _bf16(Z2), "wv": _bf16(Z2), "wo": _bf16(I2),
+                     "wg": _bf16([[0, 0]]), "wu": _bf16([[0, 0]]), "wd": _bf16([[0], [0]]),
+                     "attn_norm": np.ones(2, np.float32), "ffn_norm": np.ones(2, np.float32)}]}
+    o = oracle.Oracle(shape, w, 8)
+    # three loaded positions: K = 0, V = (3, -6), (6, 0), (-3, 9); the new row's own K and V are 0 (zero matrices)
+    o.set_synthetic_kv(0, _bf16([[0, 0]] * 3), _bf16([[3, -6], [6, 0], [-3, 9]]))
+    o.set_len(3)
+    logits = o.forward([0])[0]                 # x = (1, 1); attention = mean of the 4 V rows = (1.5, 0.75)
+    x0, x1 = 1 + 6 / 4, 1 + 3 / 4
+    r = math.sqrt((x0 ** 2 + x1 ** 2) / 2)
+    assert np.allclose(logits, [x0 / r, x1 / r, (x0 + x1) / r], atol=1e-14)
+    assert o.len == 4
+
+
 def test_numpy_restatement_cross_check(tiny):
     """Not a pin (it re-states the formulas): a compact fp64 numpy forward as a second opinion."""
     shape, w = tiny
