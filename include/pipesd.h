@@ -47,7 +47,25 @@ typedef enum pipesd_status {
 #define PIPESD_MODE_STOCHASTIC 0 /* u_i < min(1, p/q), residual resample, extra token ~ p */
 #define PIPESD_MODE_GREEDY 1     /* accept while draft == argmax (Sec. 2.2 prose); emit the argmax */
 
-#define PIPESD_Q_HOST 1u /* verify flag: item.q pointers are host memory; the library copies them */
+/* pipesd_verify flags */
+#define PIPESD_Q_HOST 1u     /* item.q pointers are host memory; the library copies them on its stream.  The q arrays
+                              * (like tokens, u and the results array) must then stay valid and unchanged until the
+                              * next pipesd_ctx_sync returns: from pinned memory the copy is truly asynchronous */
+#define PIPESD_AUTOCOMMIT 2u /* commit on the device: the kernel that takes the accept decision also writes the request's
+                              * new length (base + 1 + n_accepted) and pending token to device-resident state; the host
+                              * applies the same commit to its bookkeeping at the next pipesd_ctx_sync.  No
+                              * pipesd_kv_rollback call follows such a verify */
+#define PIPESD_CHAIN 4u      /* the cloud side of proactive transmission (App. B): this call verifies early drafts that the
+                              * edge sent before it knew the outcome of the call in flight for the same requests.  They
+                              * are valid iff that call accepts every draft and emits, as its extra token, this call's
+                              * tokens[0]; the library plans this pass for exactly that outcome, enqueues it behind the
+                              * call in flight without a host round trip, and the device decides: a pass whose condition
+                              * fails returns status PIPESD_DISCARDED and commits nothing.  Implies PIPESD_AUTOCOMMIT;
+                              * the call in flight must have been made with PIPESD_AUTOCOMMIT (or PIPESD_CHAIN) */
+
+#define PIPESD_TOKEN_PENDING (-1) /* as tokens[0] of a verify item: use the pending token the library recorded for the
+                                   * request (pipesd_kv_rollback's next_token, or a commit on the device) */
+#define PIPESD_DISCARDED 1        /* pipesd_verify_result.status of a chained pass whose condition failed (not an error) */
 
 /* Which kernels run the layer stack (both compute the same forward; their summation orders differ, so results
  * agree to rounding, not bit for bit).
@@ -122,7 +140,7 @@ typedef struct pipesd_verify_item {
 typedef struct pipesd_verify_result {
     int32_t n_accepted; /* 0..k                                                            */
     int32_t next_token; /* correction token if n_accepted < k, else the extra token        */
-    int32_t status;     /* PIPESD_OK, or the device-side error of this request             */
+    int32_t status;     /* PIPESD_OK, PIPESD_DISCARDED, or the device-side error of the call */
     int32_t reserved;
 } pipesd_verify_result;
 
@@ -132,27 +150,34 @@ const char *pipesd_strerror(int32_t status);
 /* Text of the most recent error on this context (host string owned by the context). */
 const char *pipesd_last_error(const pipesd_ctx *ctx);
 
-/* Bytes the caller must provide for a configuration.  Pure function of cfg. */
+/* Bytes the caller must provide for a configuration.  Pure function of cfg.  (Set-up around the method: the paper's
+ * cloud "only starts a server and executes NAV using the target model", Sec. 4.2, and says nothing about memory.) */
 int32_t pipesd_query_sizes(const pipesd_model_cfg *cfg, pipesd_sizes *out);
 
-/* Create a context: validates cfg, repacks the caller's weights into mem->weights (the caller may
- * free its own weight tensors once pipesd_ctx_sync has returned), zero-initialises metadata.
+/* Create a context = load the target model that performs NAV (Sec. 4.2, cloud component "Target Model"; Sec. 5.1 for
+ * the model family): validates cfg, repacks the caller's weights into mem->weights (the caller may free its own
+ * weight tensors once pipesd_ctx_sync has returned), zero-initialises metadata.
  * `cuda_stream` is a cudaStream_t (null = the legacy default stream). */
 int32_t pipesd_ctx_create(const pipesd_model_cfg *cfg, const pipesd_weights *w, const pipesd_mem *mem,
                           void *cuda_stream, pipesd_ctx **out);
 /* Releases host state and pinned staging; the caller's device buffers are untouched. */
 int32_t pipesd_ctx_destroy(pipesd_ctx *ctx);
-/* Waits for the stream; delivers pending verify results to the caller's array. */
+/* Waits for the stream; delivers the results of every verify call in flight to the callers' arrays (the NAV result
+ * that the cloud returns to the edge, Sec. 3.1 step 4) and applies commits made on the device to the host's
+ * bookkeeping.  PIPESD_E_CUDA if a bounded device-side wait gave up since the last call: the results of the calls in
+ * flight are then void (status PIPESD_E_CUDA each), nothing of them is committed, and the context stays usable. */
 int32_t pipesd_ctx_sync(pipesd_ctx *ctx);
 
-/* Request slots: an empty block table / return of all its pages to the pool. */
+/* Request slots, one per edge device served by this cloud model (App. I: every edge is independent, one target model
+ * handles the requests of all): an empty block table / return of all its pages to the pool. */
 int32_t pipesd_req_open(pipesd_ctx *ctx, int32_t *req);
 int32_t pipesd_req_close(pipesd_ctx *ctx, int32_t req);
 /* Committed length (cached positions) of a request. */
 int32_t pipesd_req_len(pipesd_ctx *ctx, int32_t req, int32_t *len);
 
-/* Append n prompt tokens (host ids) to the request's cache: the same layer stack as verify run in
- * chunks of max_rows rows, no acceptance step.  If last_logits (host, vocab floats) is non-null it
+/* Append n prompt tokens (host ids) to the request's cache -- the accepted prefix that every NAV pass runs against
+ * (Sec. 2.2: drafts are validated "against the accepted prefix"): the same layer stack as verify, run in chunks of
+ * at most min(max_rows, 32) rows, no acceptance step.  If last_logits (host, vocab floats) is non-null it
  * receives the logits of the final position; the call then synchronises. */
 int32_t pipesd_prefill(pipesd_ctx *ctx, int32_t req, const int32_t *tokens, int32_t n, float *last_logits);
 
@@ -167,8 +192,13 @@ int32_t pipesd_verify(pipesd_ctx *ctx, int32_t n_req, const pipesd_verify_item *
 /* Commit / rollback (App. B: rejected drafts are discarded, generation restarts after the last
  * accepted token): length <- base + 1 + n_accepted[i] with 0 <= n_accepted[i] <= k of the
  * request's last verify; pages wholly beyond the new length return to the pool.  No KV bytes move;
- * rows of the rejected tail are never read again. */
-int32_t pipesd_kv_rollback(pipesd_ctx *ctx, int32_t n_req, const int32_t *reqs, const int32_t *n_accepted);
+ * rows of the rejected tail are never read again.  next_token (host, n_req ids; may be null) records each
+ * request's pending token -- the correction or extra token, which opens the next round's chunk (Sec. 2.2: accepted and
+ * corrected tokens become the next prefix) -- so that the next verify may pass PIPESD_TOKEN_PENDING as tokens[0].
+ * A request may appear once per call (PIPESD_E_INVALID otherwise; nothing is changed then).  The arguments are
+ * explicit so that a harness can impose a reference decision. */
+int32_t pipesd_kv_rollback(pipesd_ctx *ctx, int32_t n_req, const int32_t *reqs, const int32_t *n_accepted,
+                           const int32_t *next_token);
 
 /* ---- component entry points (used for per-kernel parity and bandwidth measurements) ---- */
 
@@ -185,6 +215,16 @@ int32_t pipesd_debug_write_kv(pipesd_ctx *ctx, int32_t req, int32_t layer, int32
 int32_t pipesd_reject_from_logits(pipesd_ctx *ctx, int32_t k, int32_t mode, const float *logits,
                                   const float *q, const int32_t *drafts, const float *u,
                                   pipesd_verify_result *result);
+
+/* Device-resident state of a request as the commit-on-device path left it: out3 (host) = {committed length, pending
+ * token, 1 if the last such pass accepted every draft}.  Synchronises.  Only passes made with PIPESD_AUTOCOMMIT or
+ * PIPESD_CHAIN write this state. */
+int32_t pipesd_debug_req_state(pipesd_ctx *ctx, int32_t req, int32_t *out3);
+/* Self-test of the error path that every bounded device-side wait of the library takes: enqueues a one-warp kernel
+ * that polls a flag nothing ever sets, gives up after limit_us (1..100000) microseconds, records that in the device
+ * error word and returns.  The next pipesd_ctx_sync then reports PIPESD_E_CUDA and clears the word; the context and
+ * the GPU stay usable. */
+int32_t pipesd_debug_wait_timeout(pipesd_ctx *ctx, int32_t limit_us);
 
 /* Truncate a request's committed length to new_len <= its current length (pages beyond return to the
  * pool).  Lets a harness replay rounds from a recorded point; the serving path uses pipesd_kv_rollback. */
@@ -228,9 +268,6 @@ int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scra
 int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t *resident_clusters,
                                 int32_t clusters_needed, int32_t *out3);
 
-/* Tuning hook: force the number of K slices of every subsequent GEMM plan (0 = choose automatically). */
-int32_t pipesd_debug_gemm_force_split(int32_t S);
-
 /* The same GEMM for callers that cannot allocate device memory.  (The paper has no counterpart: this
  * is a convenience of the library, not a step of the method.)
  *
@@ -246,7 +283,9 @@ int32_t pipesd_debug_gemm_force_split(int32_t S);
  *
  * Limits and rules:
  *   - If pipesd_gemm_scratch_bytes(M, N, K) is larger than PIPESD_STATIC_SCRATCH_BYTES the call returns
- *     PIPESD_E_TOO_LARGE and launches nothing (8 MiB covers M*K up to 2M elements, e.g. 190 rows at K=11008).
+ *     PIPESD_E_TOO_LARGE and launches nothing.  The scratch holds 4 bytes per (token, k) with the tokens padded to
+ *     whole blocks of 32 once M > 24: ceil(M/32)*32 * K * 4 bytes must fit 8 MiB, e.g. 160 rows at K=11008 (161 do
+ *     not), 512 rows at K=4096.  Ask pipesd_gemm_scratch_bytes when in doubt.
  *   - The first call on each device looks up the array's device address (with that device current)
  *     and sets kernel attributes; make that first call during set-up, before any stream capture.
  *   - All calls share the one array and it keeps whatever the last call left there.  Nothing needs

@@ -236,6 +236,26 @@ class Oracle:
         """Keep the pending token's row and the accepted drafts' rows; drop the rejected tail."""
         self.truncate(base_len + 1 + n_accepted)
 
+    def verify_chain(self, tokens, q, u, buffered, q_buf, u_buf, greedy=False):
+        """One round followed by the cloud's handling of proactively sent drafts (paper App. B).  While this round
+        was being verified the edge kept drafting: `buffered` = [b_1..b_m] are those early tokens, where b_1 is the
+        edge's own guess at this round's extra token and b_2..b_m continue from it (q_buf [m-1, V], u_buf [m] belong
+        to them).  After the round the cloud checks (i) every draft accepted and (ii) extra token == b_1.  If both
+        hold the buffered tokens stay valid: the round is committed in full and b_1 (now the pending token) with
+        b_2..b_m as drafts is the next round, verified at once.  Otherwise they are discarded and only the first
+        round is committed.  Either way the cache is left committed.
+        Returns (first round's dict, second round's dict or None when the buffered tokens were discarded)."""
+        tokens = np.ascontiguousarray(tokens, np.int32)
+        buffered = np.ascontiguousarray(buffered, np.int32)
+        k = tokens.size - 1
+        r1 = self.verify(tokens, q, u, greedy)
+        self.rollback(r1["base_len"], r1["n_accepted"])
+        if not (r1["n_accepted"] == k and r1["next_token"] == int(buffered[0])):
+            return r1, None
+        r2 = self.verify(buffered, q_buf, u_buf, greedy)
+        self.rollback(r2["base_len"], r2["n_accepted"])
+        return r1, r2
+
     def draft_round(self, pending: int, k: int, sigma: float, noise, draft_u):
         """Make one round's inputs by running the target one token at a time:
         q_i = softmax(l_{i-1} + sigma * eps_i), d_i drawn from q_i by inverse CDF with draft_u[i-1].

@@ -22,7 +22,9 @@ MODE_STOCHASTIC, MODE_GREEDY = 0, 1
 ENGINE_TILED, ENGINE_PERSISTENT = 0, 1
 ENGINES = {"tiled": ENGINE_TILED, "persistent": ENGINE_PERSISTENT}
 DEFAULT_ENGINE = "tiled"
-Q_HOST = 1
+Q_HOST, AUTOCOMMIT, CHAIN = 1, 2, 4
+TOKEN_PENDING = -1
+DISCARDED = 1
 
 i32, u32, u64, f32, vp = ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float, ctypes.c_void_p
 
@@ -78,7 +80,7 @@ _SIGNATURES = {
     "pipesd_req_len": (i32, [vp, i32, ctypes.POINTER(i32)]),
     "pipesd_prefill": (i32, [vp, i32, vp, i32, vp]),
     "pipesd_verify": (i32, [vp, i32, ctypes.POINTER(VerifyItem), ctypes.POINTER(VerifyResult), u32]),
-    "pipesd_kv_rollback": (i32, [vp, i32, vp, vp]),
+    "pipesd_kv_rollback": (i32, [vp, i32, vp, vp, vp]),
     "pipesd_debug_get_logits": (i32, [vp, vp, i32]),
     "pipesd_debug_read_kv": (i32, [vp, i32, i32, i32, i32, vp, vp]),
     "pipesd_debug_write_kv": (i32, [vp, i32, i32, i32, i32, vp, vp]),
@@ -93,7 +95,8 @@ _SIGNATURES = {
     "pipesd_gemm_run": (i32, [vp, vp, vp, vp, i32, i32, i32, vp]),
     "pipesd_gemm_run_static": (i32, [vp, vp, vp, i32, i32, i32, vp]),
     "pipesd_debug_attn_split": (i32, [i32, i32, ctypes.POINTER(ctypes.c_int32), i32, ctypes.POINTER(ctypes.c_int32)]),
-    "pipesd_debug_gemm_force_split": (i32, [i32]),
+    "pipesd_debug_req_state": (i32, [vp, i32, ctypes.POINTER(ctypes.c_int32)]),
+    "pipesd_debug_wait_timeout": (i32, [vp, i32]),
 }
 
 
@@ -130,7 +133,7 @@ class Context:
 
     def __init__(self, shape, weights: dict, *, n_pages: int, max_requests: int = 1, max_draft: int = 16,
                  max_rows: int | None = None, max_seq: int = 4096, page_size: int = 16, device: int = 0,
-                 stream=None, engine: str | None = None):
+                 stream=None, engine: str | None = None, poison: bool = False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: the verify pass has no CPU path")
@@ -155,6 +158,12 @@ class Context:
             self._wbuf = torch.empty(sz.weights_bytes, dtype=torch.uint8, device=self.device)
             self._kvbuf = torch.empty(sz.kv_bytes, dtype=torch.uint8, device=self.device)
             self._wsbuf = torch.zeros(sz.workspace_bytes, dtype=torch.uint8, device=self.device)
+            if poison:
+                # Every byte 0xFF: NaN as bf16 and as fp32, -1 as an index.  A read of a K/V row or of a workspace
+                # element that this library did not write first then shows up in the results instead of passing
+                # silently (pipesd_ctx_create initialises what it relies on itself).
+                self._kvbuf.fill_(0xFF)
+                self._wsbuf.fill_(0xFF)
             # upload the caller's row-major bf16 tensors; they are released after the repack
             up = lambda a: torch.from_numpy(a).to(self.device, non_blocking=False)
             lw = (LayerWeights * shape.n_layers)()
@@ -250,17 +259,26 @@ class Context:
             alive += [tok, u, q]
             arr[i] = VerifyItem(it["req"], k, it.get("mode", MODE_STOCHASTIC), 0, tok.ctypes.data, qp,
                                 u.ctypes.data if u is not None else None)
-        self._alive = alive
+        self._alive = self._alive + alive if (flags & CHAIN) else alive
         self._check(lib().pipesd_verify(self._h, n, arr, res, flags), "pipesd_verify")
         if not sync:
             return res
         self.ctx_sync()
         return [(r.n_accepted, r.next_token) for r in res]
 
-    def kv_rollback(self, reqs, n_accepted):
+    def kv_rollback(self, reqs, n_accepted, next_token=None):
         r = np.ascontiguousarray(reqs, np.int32)
         a = np.ascontiguousarray(n_accepted, np.int32)
-        self._check(lib().pipesd_kv_rollback(self._h, r.size, _np_ptr(r), _np_ptr(a)), "pipesd_kv_rollback")
+        t = np.ascontiguousarray(next_token, np.int32) if next_token is not None else None
+        self._check(lib().pipesd_kv_rollback(self._h, r.size, _np_ptr(r), _np_ptr(a), _np_ptr(t)), "pipesd_kv_rollback")
+
+    def debug_req_state(self, req: int):
+        out = (ctypes.c_int32 * 3)()
+        self._check(lib().pipesd_debug_req_state(self._h, req, out), "pipesd_debug_req_state")
+        return tuple(out)
+
+    def debug_wait_timeout(self, limit_us: int):
+        self._check(lib().pipesd_debug_wait_timeout(self._h, limit_us), "pipesd_debug_wait_timeout")
 
     def debug_get_logits(self, rows: int) -> np.ndarray:
         out = np.empty((rows, self.shape.vocab), np.float32)

@@ -361,17 +361,6 @@ static inline AttnSplit attn_split_plan(int total_keys, int page_size, const int
     return p;
 }
 
-#ifdef PIPESD_GEMM_TRACE
-// Development build only: per (layer, CTA) timestamps of the attention kernel's anatomy.
-__device__ unsigned long long g_attn_trace[64 * 512 * 8];
-#define ATTN_TRACE(k)                                                                                               \
-    do {                                                                                                             \
-        if (threadIdx.x == 0 && layer < 64 && blockIdx.z == 0)                                                       \
-            g_attn_trace[((size_t)layer * 512 + blockIdx.y * gridDim.x + blockIdx.x) * 8 + (k)] = global_ns();       \
-    } while (0)
-#else
-#define ATTN_TRACE(k) do { } while (0)
-#endif
 
 // grid (cs * max clusters per request, n_kv_heads * row_groups, n_items), cluster (cs,1,1), 8 <= cs <= 10, block 128.
 // A request uses the first it_cs <= cs CTAs of its cluster; the others hold an empty split (exact zeros in the
@@ -390,7 +379,6 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = AttnSmem<HD>;
     pdl_launch_dependents();
-    ATTN_TRACE(0);
     // attention leaves most of the HBM bandwidth unused: the output projection's weights come into L2 meanwhile
     if (threadIdx.x == 0)
         l2_prefetch_issue(pf, (int)((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x),
@@ -456,7 +444,6 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
         if (early1) attn_issue_tile<HD>(s_ctx, ring + SM::kStageBytes, bars + 8, c.k0 + kAttnTile);
     }
     pdl_wait();
-    ATTN_TRACE(1);
     if (threadIdx.x < 32) {
         if (!early0 && ntiles > 0) attn_issue_tile<HD>(s_ctx, ring, bars, c.k0);
         if (!early1 && ntiles > 1) attn_issue_tile<HD>(s_ctx, ring + SM::kStageBytes, bars + 8, c.k0 + kAttnTile);
@@ -493,7 +480,6 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
             make_uint4(pack2(l[0], l[1]), pack2(l[2], l[3]), pack2(l[4], l[5]), pack2(l[6], l[7]));
     }
     __syncthreads();
-    ATTN_TRACE(2);
 
     // partial result of this CTA: takes over the Q-fragment region once the tile loop is done
     float* Fo = reinterpret_cast<float*>(smem + SM::kRing);     // [row_tiles*16][HD]
@@ -506,10 +492,8 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
     else if (row_tiles == 2) attn_body<HD, 2>(c, &s_ctx, smem, bars, err, Fo, Fm, Fl);
     else attn_body<HD, 4>(c, &s_ctx, smem, bars, err, Fo, Fm, Fl);
 
-    ATTN_TRACE(3);
     // ---- merge the cluster's splits over distributed shared memory; rank r owns rows r, r+cs, ... of the group
     cluster_sync_all();
-    ATTN_TRACE(4);
     constexpr int EPT = HD / kAttnThreads > 0 ? HD / kAttnThreads : 1;   // output columns per thread
     const uint32_t fo_a = smem_u32(Fo), fm_a = smem_u32(Fm), fl_a = smem_u32(Fl);
     const int n_rows = min(row_tiles * 16, c.R - c.rho0);
@@ -565,10 +549,8 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const float* __re
         }
     }
     __shared__ int s_last;
-    ATTN_TRACE(5);
     if (ncl > 1) __threadfence();
     cluster_sync_all();   // nobody leaves while its shared memory may still be read; partials are published
-    ATTN_TRACE(6);
     if (ncl == 1) return;
     // ---- several clusters share the keys: the last one to arrive merges their partials
     if (rank == 0 && threadIdx.x == 0) {

@@ -8,7 +8,6 @@ namespace pipesd {
 
 constexpr int kMaxItemRows = 32;   // rows (k+1, or a prefill chunk) one request contributes to a pass
 constexpr int kMaxSplits = 32;     // split-K partitions of one request's KV range
-constexpr int kWaveCtas = 296;     // 148 SMs x 2 resident CTAs: the grid-sizing unit of the GEMMs
 
 __device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
 
@@ -32,15 +31,6 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint4& a, ui
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
-}
-
-// Streaming 16-byte load of read-once data: bypass L1 allocation.
-__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
 }
 
 __device__ __forceinline__ float warp_sum(float v) {

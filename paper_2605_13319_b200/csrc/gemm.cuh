@@ -39,17 +39,6 @@ constexpr int kGemmSmemTail = 128 + 128 + 1024;             // barriers | rstd[3
 
 enum GemmMode { kPlain = 0, kQkvRope = 1, kResid = 2, kSwiglu = 3 };
 
-#ifdef PIPESD_GEMM_TRACE
-// Development build only: per (launch, CTA) timestamps of the kernel's anatomy.
-__device__ unsigned long long g_gemm_trace[512 * 512 * 8];
-#define GEMM_TRACE(k)                                                                                              \
-    do {                                                                                                            \
-        if (a.trace_idx >= 0 && a.trace_idx < 512 && blockIdx.x < 512 && blockIdx.y == 0)                           \
-            g_gemm_trace[((size_t)a.trace_idx * 512 + blockIdx.x) * 8 + (k)] = global_ns();                         \
-    } while (0)
-#else
-#define GEMM_TRACE(k) do { } while (0)
-#endif
 
 __host__ __device__ constexpr int gemm_stage_bytes(int NT) { return kGemmWStage + kGemmKC * NT * 512; }
 __host__ __device__ constexpr int gemm_smem_bytes(int NT, int stages) { return stages * gemm_stage_bytes(NT) + kGemmSmemTail; }
@@ -69,8 +58,6 @@ __host__ __device__ inline int xf_tb(int M) { int nt = xf_nt(M); return (M + nt 
 // uint4 elements of the xf array of an [M, K] activation.
 __host__ __device__ inline size_t xf_elems(int M, int K) { return (size_t)xf_tb(M) * (K / 16) * xf_nt(M) * 32; }
 
-static int g_gemm_force_split = 0;   // 0: choose automatically (tuning hook)
-
 // Host: choose the K split (cluster size).  What matters is enough CTAs to keep ~100 KB of copies in
 // flight per SM and a last wave that is nearly full.
 static inline GemmPlan gemm_plan(int M, int N, int K) {
@@ -88,8 +75,7 @@ static inline GemmPlan gemm_plan(int M, int N, int K) {
         if (s > 1 && p.KS / s < 2 * kGemmKC) break;
         if ((long)p.RB * s <= kGemmWave) best = s;
     }
-    p.S = g_gemm_force_split > 0 && g_gemm_force_split <= kGemmMaxSplit && g_gemm_force_split <= p.KS
-              ? g_gemm_force_split : best;
+    p.S = best;
     // ring depth: as deep as the shared memory of an SM allows for the number of CTAs it will hold.  A clustered
     // GEMM always leaves room for three CTAs per SM, even when it brings fewer: at two 113 KB CTAs per SM a B200
     // holds exactly the 32 clusters of eight that the O and down projections launch, so one foreign CTA in a GPC
@@ -175,7 +161,6 @@ struct GemmArgs {
     const uint4* W;     // packed weights
     const uint4* xf;    // activations, split-bf16 B fragments [tb][ks][nt][32]
     int* err;           // device error word (nullable): set when a bounded wait gives up
-    int trace_idx;      // development build: slot of this launch in the trace array
     int M, N, S, KS, stages;
     // input normalisation (nullable): ssq_in[b*M + tok], b < n_ssq, are sums of squares of the un-normalised
     // input row; the result rows are scaled by rsqrt(sum / d_in + eps)
@@ -239,7 +224,6 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
     const int tok0 = tb * MT;
 
     if (threadIdx.x == 0) {
-        GEMM_TRACE(0);
         for (int i = 0; i < stages; ++i) {
             mbar_init(full0 + 8 * i, 1);
             mbar_init(empty0 + 8 * i, kGemmConsumerWarps);
@@ -272,7 +256,6 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                 bulk_g2s_hint(smem_base + c * kStageBytes, wsrc + (size_t)c * kGemmWStage, (uint32_t)kc * 4096, full0 + 8 * c, pol);
             }
             pdl_wait();
-            GEMM_TRACE(1);
             for (int c = 0; c < pre; ++c) {
                 const int kc = chunk_ks(c);
                 bulk_g2s(smem_base + c * kStageBytes + kGemmWStage, bsrc + (size_t)c * kBStage, (uint32_t)kc * NT * 512,
@@ -365,7 +348,6 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
         for (int c = 0; c < nchunks; ++c) {
             ok = mbar_wait(full0 + 8 * st, ph);
             if (!ok) break;
-            if (c == 0 && threadIdx.x == 0) GEMM_TRACE(2);
             const unsigned char* wst = smem + st * kStageBytes;
             const unsigned char* bst = wst + kGemmWStage;
             int kc = nks - c * kGemmKC;
@@ -390,7 +372,6 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             if (++st == stages) { st = 0; ph ^= 1u; }
         }
         if (!ok && a.err && lane == 0) atomicExch(a.err, 2);
-        if (threadIdx.x == 0) GEMM_TRACE(3);
         // All consumers are past their last ring read before the ring is reused for the partial tile.
         asm volatile("bar.sync 1, %0;" ::"n"(kGemmConsumers) : "memory");
         // partial tile P[tile 8][token MT][row 16] (fp32) at the start of the ring
@@ -410,7 +391,6 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
 
     // ---------------- cluster reduction + epilogue (all 160 threads reach both barriers, also on errors)
     if (a.S > 1) cluster_sync_all(); else __syncthreads();
-    if (threadIdx.x == 0) GEMM_TRACE(4);
     pdl_wait();   // (long satisfied) every thread that touches the predecessors' global data has waited itself
     if (warp < kGemmConsumerWarps) {
         const int row = threadIdx.x & 15, tg = threadIdx.x >> 4;   // 16 lanes = the 16 rows of a tile
@@ -500,9 +480,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             for (int tile = s; tile < 8; tile += a.S) epi_tile(tile, nullptr, nullptr, nullptr, nullptr);
         }
     }
-    if (threadIdx.x == 0) GEMM_TRACE(5);
     if (a.S > 1) cluster_sync_all(); else __syncthreads();
-    if (threadIdx.x == 0) GEMM_TRACE(6);
     if (MODE == kResid && s == 0 && threadIdx.x < MT) {
         const int tok = tok0 + threadIdx.x;
         if (tok < a.M) {
@@ -511,16 +489,6 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             for (int tile = 0; tile < 8; ++tile) q += tss_s[tile * 32 + threadIdx.x];
             a.ssq_out[(size_t)rb * a.M + tok] = q;
         }
-    }
-}
-
-// y[i] = sum_s part[s][i], fixed order.
-__global__ void reduce_partials_kernel(const float* __restrict__ part, float* __restrict__ y, size_t n, int S) {
-    pdl_wait();
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        float v = 0.f;
-        for (int s = 0; s < S; ++s) v += part[(size_t)s * n + i];
-        y[i] = v;
     }
 }
 

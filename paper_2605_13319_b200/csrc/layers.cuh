@@ -87,4 +87,19 @@ __global__ void rope_table_kernel(PassMeta meta, int M, int hd, double log_base,
     sn[i] = (float)s;
 }
 
+// Self-test of the bounded-wait convention every kernel of the library follows: poll a flag that nothing ever sets,
+// give up when the time limit is reached, record that in the device error word and return normally.  The host then
+// reports the error at its next synchronisation and the context stays usable.
+__global__ void wait_never_kernel(const int* __restrict__ flag, int* __restrict__ err, unsigned long long limit_ns) {
+    if (threadIdx.x != 0) return;
+    const unsigned long long t0 = global_ns();
+    bool seen = false;
+    for (unsigned it = 0; !seen; ++it) {
+        seen = *reinterpret_cast<const volatile int*>(flag) != 0;
+        if (!seen && global_ns() - t0 > limit_ns) break;
+        if (it > (1u << 28)) break;       // an iteration cap on top of the clock
+    }
+    if (!seen) atomicExch(err, 77);
+}
+
 }  // namespace pipesd

@@ -192,17 +192,6 @@ __device__ __forceinline__ int ld_acquire_cta(const int* smem_p) {
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-#ifdef PIPESD_MEGA_TRACE
-// Development build only: per (launch, phase, CTA) timestamps of the phase-boundary anatomy.
-__device__ unsigned long long g_mega_trace[64 * 4 * kMegaMaxCtas * 8];
-#define MEGA_TRACE(k)                                                                                          \
-    do {                                                                                                        \
-        if (a.launch_idx < 64)                                                                                  \
-            g_mega_trace[(((size_t)a.launch_idx * 4 + (p - a.p0)) * kMegaMaxCtas + cta) * 8 + (k)] = global_ns(); \
-    } while (0)
-#else
-#define MEGA_TRACE(k) do { } while (0)
-#endif
 
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -587,7 +576,6 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     }
     int last_st = st;
     for (int tile = tile0; tile < tile1; ++tile, ++n) {
-        if (threadIdx.x == 0 && tile == tile0) MEGA_TRACE(1);
         if (ok) {
             const uint32_t par = (uint32_t)(n / kStages) & 1u;
             ok = mbar_wait_err(fullW0 + 8 * st, par, a.err) && mbar_wait_err(fullX0 + 8 * st, par, a.err);
@@ -676,7 +664,6 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
         }
         if (++st == kStages) st = 0;
     }
-    if (threadIdx.x == 0) MEGA_TRACE(6);
     // ---- merge the eight warps: common maximum, rescaled sums, outputs added in the order
     // ((w0 + w4) + (w1 + w5)) + (w2 + w6) + (w3 + w7)
 #pragma unroll
@@ -736,7 +723,6 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
     asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
     if (warp == 0) { add(1); add(2); add(3); }
     // warp 0 now holds the CTA's un-normalised output for the head, relative to m_tot, with the sum l_tot
-    if (threadIdx.x == 0) MEGA_TRACE(2);
     const int i0 = mega_owner(ub, T, G), i1 = mega_owner(ub + CPR - 1, T, G);
     constexpr int kSlotFloats = 8 * kMegaEpiThreads * 4;       // one CTA's slot of the exchange array
     if (i0 != i1 && cta != i0) {
@@ -756,7 +742,6 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
             fence_proxy_async_all();      // the stage served as scratch: ordinary stores before the next bulk copy into it
             if (ok) mbar_arrive(empty0 + 8 * last_st);
             st_release_cta(pub_seq, pseg);
-            MEGA_TRACE(3);
         }
         return;
     }
@@ -825,7 +810,6 @@ __device__ __forceinline__ void att_segment(const MegaArgs& a, const MegaPhase& 
         fence_proxy_async_all();
         if (ok) mbar_arrive(empty0 + 8 * last_st);
         st_release_cta(pub_seq, pseg);
-        MEGA_TRACE(5);
     }
 }
 
@@ -986,7 +970,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 ok = __shfl_sync(0xffffffffu, ok, 0);
             }
             if (!ok) break;
-            if (lane == 0) { st_release_cta(dep_seq, p + 1); MEGA_TRACE(0); }
+            if (lane == 0) st_release_cta(dep_seq, p + 1);
             if (p == a.p1 - 1) {
                 // Successor kernels may be scheduled from here on -- but only once every CTA of this grid
                 // is resident: a successor that took the place of a CTA still to come would wait for this
@@ -1113,8 +1097,6 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                                 accumulate = 1;
                             }
                             umma_commit(empty0 + 8 * st);      // the stage is free when these MMAs have read it
-                            if (c == cb) MEGA_TRACE(1);
-                            if (c == ce - 1) MEGA_TRACE(6);
                         }
                         if (++st == kStages) st = 0;
                     }
@@ -1222,7 +1204,6 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 }
                 ++seg;
                 ++pseg;
-                if (threadIdx.x == 0) MEGA_TRACE(2);
                 // ---- the CTA's part of unit u is summed.  Alone on the unit: epilogue.  Otherwise the CTA that
                 // owns the unit's first chunk collects (the unit is the last thing that CTA does in the phase,
                 // so it waits for little): the others leave their rows in global memory and count themselves
@@ -1238,7 +1219,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                         // all stores of the CTA happen before thread 0's signal to the publisher thread (ordered by
                         // the named barrier), which counts the CTA in with a release
                         asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
-                        if (threadIdx.x == 0) { st_release_cta(pub_seq, pseg); MEGA_TRACE(3); }
+                        if (threadIdx.x == 0) st_release_cta(pub_seq, pseg);
                         continue;
                     }
                     if (threadIdx.x == 0) {
@@ -1248,7 +1229,6 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                         if (!poll_counter(a.tickets + ph.ticket0 + u, n_contrib - 1, a.err)) atomicCAS(a.err, 0, 14000 + p);
                     }
                     asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
-                    if (threadIdx.x == 0) MEGA_TRACE(3);
                     // contributions are fetched eight CTAs at a time, two 16-byte words each (16 loads in flight),
                     // and added in CTA order
                     for (int q0 = 0; q0 < 2 * NT; q0 += 2) {
@@ -1275,7 +1255,6 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                         }
                     }
                 }
-                if (threadIdx.x == 0) MEGA_TRACE(4);
                 if (mode == kPlain) mega_epilogue<NT, kPlain>(a, ph, p, cta, u, warp, lane, v, pa, pb, rstd_s, ssq_w, kvoff_s);
                 else if (mode == kQkvRope) mega_epilogue<NT, kQkvRope>(a, ph, p, cta, u, warp, lane, v, pa, pb, rstd_s, ssq_w, kvoff_s);
                 else if (mode == kResid) mega_epilogue<NT, kResid>(a, ph, p, cta, u, warp, lane, v, pa, pb, rstd_s, ssq_w, kvoff_s);
@@ -1284,7 +1263,7 @@ __global__ void __launch_bounds__(kMegaThreads, 1) mega_kernel(const MegaArgs a)
                 // thread counts the unit as done with a release, so that no epilogue warp waits for the fence;
                 // readers acquire the counter (and fence the asynchronous proxy before their bulk copies)
                 asm volatile("bar.sync 1, %0;" ::"n"(kMegaEpiThreads) : "memory");
-                if (threadIdx.x == 0) { st_release_cta(pub_seq, pseg); MEGA_TRACE(5); }
+                if (threadIdx.x == 0) st_release_cta(pub_seq, pseg);
             }
         }
     }

@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <deque>
 #include <mutex>
 #include <new>
 #include <string>
@@ -30,6 +31,9 @@ struct Request {
     bool open = false;
     int len = 0;        // committed positions
     int tentative = 0;  // rows written by a verify that has not been committed yet (k+1), else 0
+    int spec = 0;       // rows written by commit-on-device verifies still in flight (each planned as if its predecessors
+                        // had accepted every draft); the host learns the committed length at the next pipesd_ctx_sync
+    int pending = -1;   // recorded pending token (pipesd_kv_rollback with next_token, or a commit on device), -1: none
     std::vector<int> pages;
 };
 
@@ -92,7 +96,7 @@ Derived derive(const pipesd_model_cfg& c) {
 
 struct WsLayout {
     size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, tickets, cs, sn, kvoff, stats, results, meta,
-        block_tab, qstage, mega_phases, mega_phases_att, mega_ctr, mega_scratch, total;
+        block_tab, qstage, req_state, never_flag, mega_phases, mega_phases_att, mega_ctr, mega_scratch, total;
     size_t mega_ctr_ints;
 };
 
@@ -126,6 +130,8 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     w.meta = take(meta_layout(c.max_rows, d.max_items).total);
     w.block_tab = take(4 * (size_t)c.max_requests * d.max_pages);
     w.qstage = take(4 * M * c.vocab);
+    w.req_state = take(sizeof(ReqState) * (size_t)c.max_requests);
+    w.never_flag = take(16);
     // persistent layer-stack kernel: phase table, counters (finished units per phase | started CTAs per launch |
     // one ticket per 256-row unit), accumulator fragments of units shared by several CTAs
     const size_t n_phases = 5 * (size_t)c.n_layers + 1;      // with the attention phases
@@ -160,6 +166,33 @@ size_t weights_bytes(const pipesd_model_cfg& c, const Derived& d) {
 
 size_t kv_bytes(const pipesd_model_cfg& c) {
     return (size_t)c.n_layers * c.n_pages * 2 * c.n_kv_heads * c.page_size * c.head_dim * 2;
+}
+
+// Kernel attributes (shared-memory limits, cluster sizes) belong to a device: set once per device ordinal, with that
+// device current, whichever entry point gets there first.
+constexpr int kMaxDevices = 64;
+std::mutex g_dev_mu;
+bool g_dev_ready[kMaxDevices] = {false};
+
+cudaError_t init_attrs_current_device() {
+    cudaError_t e;
+    if ((e = gemm_init_attrs()) != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes(128, kAttnMaxRowTiles));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)attn_smem_bytes(64, kAttnMaxRowTiles));
+}
+
+int ensure_device_ready() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PIPESD_E_CUDA;
+    std::lock_guard<std::mutex> lock(g_dev_mu);
+    if (!g_dev_ready[dev]) {
+        if (init_attrs_current_device() != cudaSuccess) return PIPESD_E_CUDA;
+        g_dev_ready[dev] = true;
+    }
+    return PIPESD_OK;
 }
 
 int check_cfg(const pipesd_model_cfg* c) {
@@ -217,10 +250,17 @@ struct pipesd_ctx {
     char* h_meta[kStages] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ev_meta[kStages] = {nullptr, nullptr, nullptr, nullptr};
     int stage = 0;
-    RejectOut* h_results = nullptr;
-    pipesd_verify_result* pend_dst = nullptr;
-    int pend_n = 0;
-    bool pend_check = false;   // a prefill is in flight whose device error word has not been looked at yet
+    // Calls whose results (and device error word) have been copied towards the host but not looked at yet, oldest
+    // first; at most kStages of them (one pinned staging buffer each).
+    struct InflightItem { int slot, k, commit; };
+    struct Inflight {
+        pipesd_verify_result* dst = nullptr;   // caller's array (null: a prefill or a self-test, only the error word matters)
+        std::vector<InflightItem> items;
+        int buf = 0;                           // staging buffer
+    };
+    RejectOut* h_results[kStages] = {nullptr, nullptr, nullptr, nullptr};
+    std::deque<Inflight> inflight;
+    int res_buf = 0;
     int last_rows = 0;
     int attn_occ[kAttnMaxCluster + 1][kAttnMaxRowTiles + 1] = {};   // [cluster width 9..][query row tiles]: clusters of the
                                                                      // attention kernel the device keeps resident at once (0: width unavailable)
@@ -234,7 +274,6 @@ struct pipesd_ctx {
     std::string err;
     // launch accounting
     int64_t n_launch = 0, n_gemm = 0;
-    int n_gemm_in_pass = 0;   // position of the next GEMM launch in the current pass (development traces)
     double gemm_bytes = 0.0;
     bool time_gemms = false;
     std::vector<cudaEvent_t> prof_ev;   // start/stop pairs
@@ -285,7 +324,6 @@ int cuda_fail(pipesd_ctx* c, cudaError_t e, const char* where) {
 int launch_gemm(pipesd_ctx* ctx, int mode, GemmArgs a, int K) {
     const GemmPlan p = gemm_plan(a.M, a.N, K);
     a.err = ctx->err_word();
-    a.trace_idx = (int)(ctx->n_gemm_in_pass++);
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (ctx->time_gemms) {
         if (ctx->prof_used + 2 > ctx->prof_ev.size()) {
@@ -313,7 +351,23 @@ struct ItemDesc {
     const int32_t* tokens;  // host, rows ids
     const float* q;         // device
     const float* u;         // host, k+1 (null when mode == 2)
+    int base;               // cached positions the pass runs against
+    int commit;             // kCommit*
+    int tok0;               // id of the first row when tokens[0] asks for the recorded pending token
 };
+
+// Enqueue the copy of the result slots and the device error word into the next staging buffer and remember the call.
+int push_inflight(pipesd_ctx* ctx, pipesd_verify_result* dst, std::vector<pipesd_ctx::InflightItem> items) {
+    pipesd_ctx::Inflight f;
+    f.dst = dst;
+    f.items = std::move(items);
+    f.buf = ctx->res_buf;
+    ctx->res_buf = (ctx->res_buf + 1) % pipesd_ctx::kStages;
+    CU(cudaMemcpyAsync(ctx->h_results[f.buf], ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut) * ctx->dv.max_items + 4,
+                       cudaMemcpyDeviceToHost, ctx->st));
+    ctx->inflight.push_back(std::move(f));
+    return PIPESD_OK;
+}
 
 // Make sure the request owns pages for `need_len` positions. All-or-nothing is checked by the caller.
 int pages_needed(const pipesd_ctx* c, const Request& r, int need_len) {
@@ -363,8 +417,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     int row = 0, part0 = 0, max_nsplit = 1, u0 = 0, max_cs = kAttnSplits;
     for (int i = 0; i < n_items; ++i) {
         const ItemDesc& it = items[i];
-        const Request& r = ctx->reqs[it.slot];
-        const int total = r.len + it.rows;
+        const int total = it.base + it.rows;
         // clusters that share the request's keys, key splits per cluster (8..10) and keys per split: from the request
         // alone (its length, its rows), so that its summation order is the same in every batch
         const int R_i = it.rows * (c.n_q_heads / c.n_kv_heads);                  // query rows per KV head
@@ -379,7 +432,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         I(ml.it_slot)[i] = it.slot;
         I(ml.it_row0)[i] = row;
         I(ml.it_rows)[i] = it.rows;
-        I(ml.it_base)[i] = r.len;
+        I(ml.it_base)[i] = it.base;
         I(ml.it_nsplit)[i] = nsplit;
         I(ml.it_chunk)[i] = chunk;
         I(ml.it_cs)[i] = cs_i;
@@ -391,10 +444,14 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         hr[i].mode = it.mode;
         hr[i].u0 = u0;
         hr[i].q = it.q;
+        hr[i].slot = it.slot;
+        hr[i].base = it.base;
+        hr[i].commit = it.commit;
+        hr[i].reserved = 0;
         for (int j = 0; j < it.rows; ++j) {
             I(ml.row_item)[row + j] = i;
-            I(ml.row_pos)[row + j] = r.len + j;
-            I(ml.row_tok)[row + j] = it.tokens[j];
+            I(ml.row_pos)[row + j] = it.base + j;
+            I(ml.row_tok)[row + j] = j == 0 && it.tokens[0] < 0 ? it.tok0 : it.tokens[j];
         }
         for (int j = 0; j <= it.k; ++j) hu[u0 + j] = it.u ? it.u[j] : 0.f;
         u0 += it.k + 1;
@@ -404,7 +461,6 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     CU(cudaEventRecord(ctx->ev_meta[sidx], ctx->st));
 
     // ---- layer stack
-    ctx->n_gemm_in_pass = 0;
     const PassMeta meta = ctx->pass_meta();
     cudaStream_t st = ctx->st;
     float* x = ctx->W<float>(ctx->ws.x);
@@ -476,10 +532,9 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         int* ctr = ctx->W<int>(ctx->ws.mega_ctr);
         const int n_phases = 5 * c.n_layers + 1;      // counters are laid out for the longer table
         if (one_launch) {
-            const Request& r = ctx->reqs[items[0].slot];
-            ma.att_base = r.len;
+            ma.att_base = items[0].base;
             ma.att_rows = items[0].rows;
-            ma.att_cpr = (r.len + items[0].rows + kAttTile - 1) / kAttTile;
+            ma.att_cpr = (items[0].base + items[0].rows + kAttTile - 1) / kAttTile;
             ma.att_bt = ctx->W<int32_t>(ctx->ws.block_tab) + (size_t)items[0].slot * dv.max_pages;
         }
         ma.done = ctr;
@@ -586,14 +641,14 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             if (rc_) return rc_;
         }
         // plain launches from here on: they start after the GEMM has fully completed
-        row_stats_kernel<<<dim3(M, kStatSplits), 256, 0, st>>>(nullptr, 1, M, c.vocab, logits, stats);
+        row_stats_kernel<<<dim3(M, kStatSplits), 256, 0, st>>>(c.vocab, logits, stats);
         ctx->last_rows = M;
         if (want_reject) {
             CU(launch_pdl_cluster(accept_sample_kernel, dim3(kSampleCluster, n_items), dim3(kSampleThreads), 0, st,
                                   kSampleCluster, (const float*)logits, c.vocab, (const RowStat*)stats,
                                   reinterpret_cast<const RejectItem*>(ctx->wsp + ctx->ws.meta + ml.rej), meta.row_tok,
                                   reinterpret_cast<const float*>(ctx->wsp + ctx->ws.meta + ml.u),
-                                  ctx->W<RejectOut>(ctx->ws.results)));
+                                  ctx->W<RejectOut>(ctx->ws.results), ctx->W<ReqState>(ctx->ws.req_state)));
         }
     }
     CU(cudaGetLastError());
@@ -654,13 +709,7 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     if (((uintptr_t)mem->weights | (uintptr_t)mem->kv | (uintptr_t)mem->workspace) & 255) return bail(PIPESD_E_INVALID);
     cudaError_t e = cudaSetDevice(c.device);
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
-    if ((e = gemm_init_attrs()) != cudaSuccess) return bail(PIPESD_E_CUDA);
-    e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_smem_bytes(128, kAttnMaxRowTiles));
-    if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
-    e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_smem_bytes(64, kAttnMaxRowTiles));
-    if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
+    if (ensure_device_ready() != PIPESD_OK) return bail(PIPESD_E_CUDA);
 
     {   // clusters of 9 or 10 CTAs are non-portable sizes: opt in and ask how many such clusters the device keeps
         // resident for each shared-memory footprint (query row tiles); run_pass widens a request's cluster only if
@@ -693,8 +742,9 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         if (cudaEventCreateWithFlags(&ctx->ev_meta[i], cudaEventDisableTiming) != cudaSuccess)
             return bail(PIPESD_E_CUDA);
     }
-    if (cudaHostAlloc((void**)&ctx->h_results, sizeof(RejectOut) * dv.max_items + 16, cudaHostAllocDefault) != cudaSuccess)
-        return bail(PIPESD_E_CUDA);
+    for (int i = 0; i < pipesd_ctx::kStages; ++i)
+        if (cudaHostAlloc((void**)&ctx->h_results[i], sizeof(RejectOut) * dv.max_items + 16, cudaHostAllocDefault) != cudaSuccess)
+            return bail(PIPESD_E_CUDA);
 
     cudaStream_t st = ctx->st;
     // the device error word and the attention tickets start at zero (the tickets reset themselves after use)
@@ -836,7 +886,8 @@ int32_t pipesd_ctx_destroy(pipesd_ctx* ctx) {
         if (ctx->h_meta[i]) cudaFreeHost(ctx->h_meta[i]);
         if (ctx->ev_meta[i]) cudaEventDestroy(ctx->ev_meta[i]);
     }
-    if (ctx->h_results) cudaFreeHost(ctx->h_results);
+    for (int i = 0; i < pipesd_ctx::kStages; ++i)
+        if (ctx->h_results[i]) cudaFreeHost(ctx->h_results[i]);
     for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
     delete ctx;
     return PIPESD_OK;
@@ -845,28 +896,46 @@ int32_t pipesd_ctx_destroy(pipesd_ctx* ctx) {
 int32_t pipesd_ctx_sync(pipesd_ctx* ctx) {
     if (!ctx) return PIPESD_E_INVALID;
     CU(cudaStreamSynchronize(ctx->st));
-    if (ctx->pend_dst || ctx->pend_check) {
-        ctx->pend_check = false;
-        const int dev_err = *reinterpret_cast<const int*>(ctx->h_results + ctx->dv.max_items);
-        if (dev_err) {   // a bounded device-side wait gave up: the results of this call are void
-            for (int i = 0; i < ctx->pend_n; ++i) ctx->pend_dst[i].status = PIPESD_E_CUDA;
-            ctx->pend_dst = nullptr;
-            ctx->pend_n = 0;
-            cudaMemsetAsync(ctx->err_word(), 0, 4, ctx->st);
-            cudaMemsetAsync(ctx->wsp + ctx->ws.tickets, 0, 4 * (size_t)ctx->cfg.max_rows * ctx->cfg.n_q_heads, ctx->st);
-            char msg[96];
-            snprintf(msg, sizeof msg, "a device-side wait timed out (kernel error word %d)", dev_err);
-            return fail(ctx, PIPESD_E_CUDA, msg);
+    if (ctx->inflight.empty()) return PIPESD_OK;
+    // The device error word travels with every call's results; the kernels only ever set it, so the newest copy
+    // tells whether any bounded device-side wait of the calls in flight gave up.
+    const int dev_err = *reinterpret_cast<const int*>(ctx->h_results[ctx->inflight.back().buf] + ctx->dv.max_items);
+    if (dev_err) {   // the results of every call in flight are void; nothing is committed
+        for (const pipesd_ctx::Inflight& f : ctx->inflight) {
+            for (size_t i = 0; i < f.items.size(); ++i) {
+                if (f.dst) f.dst[i].status = PIPESD_E_CUDA;
+                if (f.items[i].commit != kCommitNone) ctx->reqs[f.items[i].slot].spec = 0;
+            }
         }
-        for (int i = 0; i < ctx->pend_n; ++i) {
-            ctx->pend_dst[i].n_accepted = ctx->h_results[i].n_accepted;
-            ctx->pend_dst[i].next_token = ctx->h_results[i].next_token;
-            ctx->pend_dst[i].status = ctx->h_results[i].status;
-            ctx->pend_dst[i].reserved = 0;
-        }
-        ctx->pend_dst = nullptr;
-        ctx->pend_n = 0;
+        ctx->inflight.clear();
+        cudaMemsetAsync(ctx->err_word(), 0, 4, ctx->st);
+        cudaMemsetAsync(ctx->wsp + ctx->ws.tickets, 0, 4 * (size_t)ctx->cfg.max_rows * ctx->cfg.n_q_heads, ctx->st);
+        char msg[96];
+        snprintf(msg, sizeof msg, "a device-side wait timed out (kernel error word %d)", dev_err);
+        return fail(ctx, PIPESD_E_CUDA, msg);
     }
+    for (const pipesd_ctx::Inflight& f : ctx->inflight) {
+        const RejectOut* res = ctx->h_results[f.buf];
+        for (size_t i = 0; i < f.items.size(); ++i) {
+            if (f.dst) {
+                f.dst[i].n_accepted = res[i].n_accepted;
+                f.dst[i].next_token = res[i].next_token;
+                f.dst[i].status = res[i].status;
+                f.dst[i].reserved = 0;
+            }
+            const pipesd_ctx::InflightItem& it = f.items[i];
+            if (it.commit == kCommitNone) continue;
+            // what the kernel committed on the device, applied to the host's bookkeeping (calls in order)
+            Request& r = ctx->reqs[it.slot];
+            r.spec -= it.k + 1;
+            if (res[i].status == 0) {
+                r.len += 1 + res[i].n_accepted;
+                r.pending = res[i].next_token;
+            }
+            if (r.spec == 0) shrink_pages(ctx, r, r.len);
+        }
+    }
+    ctx->inflight.clear();
     return PIPESD_OK;
 }
 
@@ -903,7 +972,11 @@ int32_t pipesd_req_len(pipesd_ctx* ctx, int32_t req, int32_t* len) {
 int32_t pipesd_prefill(pipesd_ctx* ctx, int32_t req, const int32_t* tokens, int32_t n, float* last_logits) {
     if (!ctx || !tokens || n < 1 || bad_req(ctx, req)) return fail(ctx, PIPESD_E_INVALID, "pipesd_prefill");
     Request& r = ctx->reqs[req];
-    if (r.tentative) return fail(ctx, PIPESD_E_STATE, "prefill on a request with an uncommitted verify");
+    if (r.tentative || r.spec) return fail(ctx, PIPESD_E_STATE, "prefill on a request with an uncommitted verify");
+    if ((int)ctx->inflight.size() >= pipesd_ctx::kStages) {
+        int rc0 = pipesd_ctx_sync(ctx);
+        if (rc0 != PIPESD_OK) return rc0;
+    }
     if (r.len + n > ctx->cfg.max_seq) return fail(ctx, PIPESD_E_RANGE, "prefill beyond max_seq");
     for (int i = 0; i < n; ++i)
         if (tokens[i] < 0 || tokens[i] >= ctx->cfg.vocab) return fail(ctx, PIPESD_E_INVALID, "token id out of range");
@@ -916,14 +989,14 @@ int32_t pipesd_prefill(pipesd_ctx* ctx, int32_t req, const int32_t* tokens, int3
         int rows = std::min(chunk, n - done);
         bool last = done + rows == n;
         std::vector<ItemDesc> items(1);
-        items[0] = ItemDesc{req, rows, 2, 0, tokens + done, nullptr, nullptr};
+        items[0] = ItemDesc{req, rows, 2, 0, tokens + done, nullptr, nullptr, r.len, kCommitNone, 0};
         rc = run_pass(ctx, items, last && last_logits, false);
         if (rc != PIPESD_OK) return rc;
         r.len += rows;
+        r.pending = -1;
         if (last) {   // the device error word travels back with the (unused) result slots; pipesd_ctx_sync reads it
-            CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results),
-                               sizeof(RejectOut) * ctx->dv.max_items + 4, cudaMemcpyDeviceToHost, ctx->st));
-            ctx->pend_check = true;
+            rc = push_inflight(ctx, nullptr, {});
+            if (rc != PIPESD_OK) return rc;
         }
         if (last && last_logits) {
             CU(cudaMemcpyAsync(last_logits, ctx->W<float>(ctx->ws.logits) + (size_t)(rows - 1) * ctx->cfg.vocab,
@@ -939,8 +1012,14 @@ int32_t pipesd_verify(pipesd_ctx* ctx, int32_t n_req, const pipesd_verify_item* 
                       pipesd_verify_result* results, uint32_t flags) {
     if (!ctx || !items_in || !results || n_req < 1 || n_req > ctx->dv.max_items)
         return fail(ctx, PIPESD_E_INVALID, "pipesd_verify: arguments");
+    if (flags & ~(uint32_t)(PIPESD_Q_HOST | PIPESD_AUTOCOMMIT | PIPESD_CHAIN))
+        return fail(ctx, PIPESD_E_INVALID, "pipesd_verify: unknown flag");
     const pipesd_model_cfg& c = ctx->cfg;
-    if (ctx->pend_dst || ctx->pend_check) {  // deliver the previous call's results before their staging is reused
+    const bool chain = (flags & PIPESD_CHAIN) != 0;
+    const int commit = chain ? kCommitChain : ((flags & PIPESD_AUTOCOMMIT) ? kCommitAuto : kCommitNone);
+    // A chained call rides behind the calls in flight; any other call first takes delivery of their results (the host
+    // needs the committed lengths), and so does a chained one once every staging buffer is taken.
+    if (!ctx->inflight.empty() && (!chain || (int)ctx->inflight.size() >= pipesd_ctx::kStages)) {
         int rc = pipesd_ctx_sync(ctx);
         if (rc != PIPESD_OK) return rc;
     }
@@ -955,25 +1034,32 @@ int32_t pipesd_verify(pipesd_ctx* ctx, int32_t n_req, const pipesd_verify_item* 
         if (it.mode != PIPESD_MODE_STOCHASTIC && it.mode != PIPESD_MODE_GREEDY)
             return fail(ctx, PIPESD_E_INVALID, "verify: mode");
         if (it.mode == PIPESD_MODE_STOCHASTIC && !it.q) return fail(ctx, PIPESD_E_INVALID, "verify: q missing");
+        const Request& r = ctx->reqs[it.req];
         for (int j = 0; j <= it.k; ++j) {
-            if (it.tokens[j] < 0 || it.tokens[j] >= c.vocab) return fail(ctx, PIPESD_E_INVALID, "verify: token id");
+            const bool use_pending = j == 0 && it.tokens[0] == PIPESD_TOKEN_PENDING && !chain;
+            if (use_pending && r.pending < 0) return fail(ctx, PIPESD_E_STATE, "verify: no pending token recorded for the request");
+            if (!use_pending && (it.tokens[j] < 0 || it.tokens[j] >= c.vocab)) return fail(ctx, PIPESD_E_INVALID, "verify: token id");
             if (it.u && !(it.u[j] >= 0.f && it.u[j] < 1.f)) return fail(ctx, PIPESD_E_INVALID, "verify: uniform outside [0,1)");
         }
-        const Request& r = ctx->reqs[it.req];
         if (r.tentative) return fail(ctx, PIPESD_E_STATE, "verify on a request with an uncommitted tail");
-        if (r.len + it.k + 1 > c.max_seq) return fail(ctx, PIPESD_E_RANGE, "verify beyond max_seq");
+        if (chain && !r.spec) return fail(ctx, PIPESD_E_STATE, "chained verify without a commit-on-device verify in flight");
+        if (!chain && r.spec) return fail(ctx, PIPESD_E_STATE, "verify on a request with an uncommitted tail");
+        if (r.len + r.spec + it.k + 1 > c.max_seq) return fail(ctx, PIPESD_E_RANGE, "verify beyond max_seq");
         M += it.k + 1;
-        pages += pages_needed(ctx, r, r.len + it.k + 1);
+        pages += pages_needed(ctx, r, r.len + r.spec + it.k + 1);
     }
     if (M > c.max_rows) return fail(ctx, PIPESD_E_RANGE, "verify: more rows than max_rows");
     if (pages > (int)ctx->free_pages.size()) return fail(ctx, PIPESD_E_OOM_PAGES, "pipesd_verify");
 
     std::vector<ItemDesc> items(n_req);
+    std::vector<pipesd_ctx::InflightItem> fl(n_req);
     float* qstage = ctx->W<float>(ctx->ws.qstage);
     size_t qrow = 0;
     for (int i = 0; i < n_req; ++i) {
         const pipesd_verify_item& it = items_in[i];
-        int rc = grow_pages(ctx, it.req, ctx->reqs[it.req].len + it.k + 1);
+        const Request& r = ctx->reqs[it.req];
+        const int base = r.len + r.spec;      // a chained pass is planned as if its predecessors had accepted every draft
+        int rc = grow_pages(ctx, it.req, base + it.k + 1);
         if (rc != PIPESD_OK) return rc;
         const float* q = it.q;
         if (it.mode == PIPESD_MODE_STOCHASTIC && (flags & PIPESD_Q_HOST)) {
@@ -982,31 +1068,41 @@ int32_t pipesd_verify(pipesd_ctx* ctx, int32_t n_req, const pipesd_verify_item* 
             q = dst;
             qrow += it.k;
         }
-        items[i] = ItemDesc{it.req, it.k + 1, it.mode, it.k, it.tokens, q, it.u};
+        items[i] = ItemDesc{it.req, it.k + 1, it.mode, it.k, it.tokens, q, it.u, base, commit, r.pending};
+        fl[i] = pipesd_ctx::InflightItem{it.req, it.k, commit};
     }
     int rc = run_pass(ctx, items, true, true);
     if (rc != PIPESD_OK) return rc;
-    CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut) * ctx->dv.max_items + 4,
-                       cudaMemcpyDeviceToHost, ctx->st));
-    ctx->pend_dst = results;
-    ctx->pend_n = n_req;
-    for (int i = 0; i < n_req; ++i) ctx->reqs[items_in[i].req].tentative = items_in[i].k + 1;
+    rc = push_inflight(ctx, results, std::move(fl));
+    if (rc != PIPESD_OK) return rc;
+    for (int i = 0; i < n_req; ++i) {
+        Request& r = ctx->reqs[items_in[i].req];
+        if (commit == kCommitNone) r.tentative = items_in[i].k + 1;
+        else r.spec += items_in[i].k + 1;
+    }
     return PIPESD_OK;
 }
 
-int32_t pipesd_kv_rollback(pipesd_ctx* ctx, int32_t n_req, const int32_t* reqs, const int32_t* n_accepted) {
+int32_t pipesd_kv_rollback(pipesd_ctx* ctx, int32_t n_req, const int32_t* reqs, const int32_t* n_accepted,
+                           const int32_t* next_token) {
     if (!ctx || !reqs || !n_accepted || n_req < 1) return fail(ctx, PIPESD_E_INVALID, "pipesd_kv_rollback");
+    std::vector<char> seen(ctx->cfg.max_requests, 0);
     for (int i = 0; i < n_req; ++i) {
         if (bad_req(ctx, reqs[i])) return fail(ctx, PIPESD_E_INVALID, "rollback: bad request");
+        if (seen[reqs[i]]) return fail(ctx, PIPESD_E_INVALID, "rollback: repeated request");
+        seen[reqs[i]] = 1;
         const Request& r = ctx->reqs[reqs[i]];
         if (!r.tentative) return fail(ctx, PIPESD_E_STATE, "rollback without a preceding verify");
         if (n_accepted[i] < 0 || n_accepted[i] > r.tentative - 1)
             return fail(ctx, PIPESD_E_RANGE, "rollback: n_accepted outside 0..k");
+        if (next_token && (next_token[i] < 0 || next_token[i] >= ctx->cfg.vocab))
+            return fail(ctx, PIPESD_E_INVALID, "rollback: next_token is not a token id");
     }
     for (int i = 0; i < n_req; ++i) {
         Request& r = ctx->reqs[reqs[i]];
         r.len += 1 + n_accepted[i];
         r.tentative = 0;
+        r.pending = next_token ? next_token[i] : -1;
         shrink_pages(ctx, r, r.len);
     }
     return PIPESD_OK;
@@ -1026,7 +1122,7 @@ static int32_t kv_rw(pipesd_ctx* ctx, int32_t req, int32_t layer, int32_t pos0, 
         return fail(ctx, PIPESD_E_INVALID, "kv read/write");
     const pipesd_model_cfg& c = ctx->cfg;
     Request& r = ctx->reqs[req];
-    if (r.tentative) return fail(ctx, PIPESD_E_STATE, "kv read/write with an uncommitted verify");
+    if (r.tentative || r.spec) return fail(ctx, PIPESD_E_STATE, "kv read/write with an uncommitted verify");
     const int end = pos0 + n_pos;
     if (write) {
         if (end > c.max_seq) return fail(ctx, PIPESD_E_RANGE, "kv write beyond max_seq");
@@ -1080,7 +1176,7 @@ int32_t pipesd_reject_from_logits(pipesd_ctx* ctx, int32_t k, int32_t mode, cons
         return fail(ctx, PIPESD_E_INVALID, "pipesd_reject_from_logits");
     if (mode != PIPESD_MODE_GREEDY && (mode != PIPESD_MODE_STOCHASTIC || !q))
         return fail(ctx, PIPESD_E_INVALID, "pipesd_reject_from_logits: mode / q");
-    if (ctx->pend_dst) {
+    if (!ctx->inflight.empty()) {
         int rc = pipesd_ctx_sync(ctx);
         if (rc != PIPESD_OK) return rc;
     }
@@ -1100,26 +1196,27 @@ int32_t pipesd_reject_from_logits(pipesd_ctx* ctx, int32_t k, int32_t mode, cons
     float* dl = ctx->W<float>(ctx->ws.logits);
     float* dq = ctx->W<float>(ctx->ws.qstage);
     RejectItem* hr = reinterpret_cast<RejectItem*>(hm + ml.rej);
-    hr[0] = RejectItem{0, k, mode, 0, dq};
+    hr[0] = RejectItem{0, k, mode, 0, dq, 0, 0, kCommitNone, 0};
     cudaStream_t st = ctx->st;
     CU(cudaMemcpyAsync(ctx->wsp + ctx->ws.meta, hm, ml.total, cudaMemcpyHostToDevice, st));
     CU(cudaEventRecord(ctx->ev_meta[sidx], st));
     CU(cudaMemcpyAsync(dl, logits, 4 * (size_t)(k + 1) * V, cudaMemcpyHostToDevice, st));
     if (mode == PIPESD_MODE_STOCHASTIC) CU(cudaMemcpyAsync(dq, q, 4 * (size_t)k * V, cudaMemcpyHostToDevice, st));
     RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
-    row_stats_kernel<<<dim3(k + 1, kStatSplits), 256, 0, st>>>(nullptr, 1, k + 1, V, dl, stats);
+    row_stats_kernel<<<dim3(k + 1, kStatSplits), 256, 0, st>>>(V, dl, stats);
     CU(cudaGetLastError());
     CU(launch_pdl_cluster(accept_sample_kernel, dim3(kSampleCluster, 1), dim3(kSampleThreads), 0, st, kSampleCluster,
                           (const float*)dl, V, (const RowStat*)stats,
                           reinterpret_cast<const RejectItem*>(ctx->wsp + ctx->ws.meta + ml.rej),
                           reinterpret_cast<const int32_t*>(ctx->wsp + ctx->ws.meta + ml.row_tok),
                           reinterpret_cast<const float*>(ctx->wsp + ctx->ws.meta + ml.u),
-                          ctx->W<RejectOut>(ctx->ws.results)));
-    CU(cudaMemcpyAsync(ctx->h_results, ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut), cudaMemcpyDeviceToHost, st));
+                          ctx->W<RejectOut>(ctx->ws.results), ctx->W<ReqState>(ctx->ws.req_state)));
+    RejectOut* hres = ctx->h_results[0];   // nothing is in flight here (synchronised above)
+    CU(cudaMemcpyAsync(hres, ctx->W<RejectOut>(ctx->ws.results), sizeof(RejectOut), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
-    result->n_accepted = ctx->h_results[0].n_accepted;
-    result->next_token = ctx->h_results[0].next_token;
-    result->status = ctx->h_results[0].status;
+    result->n_accepted = hres[0].n_accepted;
+    result->next_token = hres[0].next_token;
+    result->status = hres[0].status;
     result->reserved = 0;
     ctx->last_rows = k + 1;
     return PIPESD_OK;
@@ -1128,26 +1225,34 @@ int32_t pipesd_reject_from_logits(pipesd_ctx* ctx, int32_t k, int32_t mode, cons
 int32_t pipesd_debug_set_len(pipesd_ctx* ctx, int32_t req, int32_t new_len) {
     if (!ctx || bad_req(ctx, req)) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_len");
     Request& r = ctx->reqs[req];
-    if (r.tentative) return fail(ctx, PIPESD_E_STATE, "set_len with an uncommitted verify");
+    if (r.tentative || r.spec) return fail(ctx, PIPESD_E_STATE, "set_len with an uncommitted verify");
     if (new_len < 0 || new_len > r.len) return fail(ctx, PIPESD_E_RANGE, "set_len can only truncate");
     r.len = new_len;
+    r.pending = -1;
     shrink_pages(ctx, r, r.len);
     return PIPESD_OK;
 }
 
-#ifdef PIPESD_GEMM_TRACE
-int32_t pipesd_debug_attn_trace(unsigned long long* dst, int32_t n) {
-    return cudaMemcpyFromSymbol(dst, g_attn_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
+int32_t pipesd_debug_req_state(pipesd_ctx* ctx, int32_t req, int32_t* out3) {
+    if (!ctx || !out3 || bad_req(ctx, req)) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_req_state");
+    ReqState s;
+    CU(cudaMemcpyAsync(&s, ctx->W<ReqState>(ctx->ws.req_state) + req, sizeof s, cudaMemcpyDeviceToHost, ctx->st));
+    CU(cudaStreamSynchronize(ctx->st));
+    out3[0] = s.len; out3[1] = s.pending; out3[2] = s.all_accepted;
+    return PIPESD_OK;
 }
-int32_t pipesd_debug_gemm_trace(unsigned long long* dst, int32_t n) {
-    return cudaMemcpyFromSymbol(dst, g_gemm_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
+
+int32_t pipesd_debug_wait_timeout(pipesd_ctx* ctx, int32_t limit_us) {
+    if (!ctx || limit_us < 1 || limit_us > 100000) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_wait_timeout");
+    if ((int)ctx->inflight.size() >= pipesd_ctx::kStages) {
+        int rc = pipesd_ctx_sync(ctx);
+        if (rc != PIPESD_OK) return rc;
+    }
+    CU(cudaMemsetAsync(ctx->wsp + ctx->ws.never_flag, 0, 16, ctx->st));
+    wait_never_kernel<<<1, 32, 0, ctx->st>>>(ctx->W<int>(ctx->ws.never_flag), ctx->err_word(), (unsigned long long)limit_us * 1000ull);
+    CU(cudaGetLastError());
+    return push_inflight(ctx, nullptr, {});
 }
-#endif
-#ifdef PIPESD_MEGA_TRACE
-int32_t pipesd_debug_mega_trace(unsigned long long* dst, int32_t n) {
-    return cudaMemcpyFromSymbol(dst, g_mega_trace, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -6;
-}
-#endif
 
 int32_t pipesd_debug_set_engine(pipesd_ctx* ctx, int32_t engine) {
     if (!ctx || engine < 0 || engine > 2) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine");
@@ -1234,11 +1339,7 @@ static int32_t gemm_run_with_scratch(const void* packed, const float* x, float* 
 int32_t pipesd_gemm_run(const void* packed, const float* x, float* y, void* scratch, int32_t M, int32_t N,
                         int32_t K, void* cuda_stream) {
     if (!packed || !x || !y || !scratch || M < 1 || N < 16 || K < 16 || N % 16 || K % 16) return PIPESD_E_INVALID;
-    static bool attrs = false;
-    if (!attrs) {
-        if (gemm_init_attrs() != cudaSuccess) return PIPESD_E_CUDA;
-        attrs = true;
-    }
+    if (ensure_device_ready() != PIPESD_OK) return PIPESD_E_CUDA;
     return gemm_run_with_scratch(packed, x, y, scratch, M, N, K, (cudaStream_t)cuda_stream);
 }
 
@@ -1249,11 +1350,6 @@ int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int
     for (int i = 0; i <= kAttnMaxCluster - kAttnSplits; ++i) res[i] = resident_clusters[i];
     const AttnSplit p = attn_split_plan(total_keys, page_size, res, clusters_needed);
     out3[0] = p.clusters; out3[1] = p.width; out3[2] = p.keys_per_split;
-    return PIPESD_OK;
-}
-
-int32_t pipesd_debug_gemm_force_split(int32_t S) {
-    g_gemm_force_split = S > 0 ? S : 0;
     return PIPESD_OK;
 }
 
@@ -1268,7 +1364,6 @@ extern "C" {
 static __device__ __align__(256) unsigned char g_static_gemm_scratch[PIPESD_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mu;
 void* g_static_ptr[kMaxDevices] = {nullptr};   // device address of the array, per device ordinal
 
@@ -1277,11 +1372,11 @@ void* g_static_ptr[kMaxDevices] = {nullptr};   // device address of the array, p
 int static_scratch_for_current_device(void** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PIPESD_E_CUDA;
+    if (ensure_device_ready() != PIPESD_OK) return PIPESD_E_CUDA;
     std::lock_guard<std::mutex> lock(g_static_mu);
     if (!g_static_ptr[dev]) {
         void* p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_gemm_scratch) != cudaSuccess || !p) return PIPESD_E_CUDA;
-        if (gemm_init_attrs() != cudaSuccess) return PIPESD_E_CUDA;
         g_static_ptr[dev] = p;
     }
     *out = g_static_ptr[dev];

@@ -19,25 +19,17 @@ struct RowStat {
     double z;      // sum exp(l - m) over the split
 };
 
-// logits[row][j] = sum_s part[s][row][j] (written out), and per (row, split): max, argmax, sum-exp.
-// grid (M, kStatSplits), block 256.
-__global__ void __launch_bounds__(256) row_stats_kernel(const float* __restrict__ part, int S, int M, int V,
-                                                        float* __restrict__ logits, RowStat* __restrict__ stats) {
+// Per (row, split) of the logits: max, argmax, sum-exp.  grid (M, kStatSplits), block 256.
+__global__ void __launch_bounds__(256) row_stats_kernel(int V, const float* __restrict__ logits,
+                                                        RowStat* __restrict__ stats) {
     const int row = blockIdx.x, sp = blockIdx.y;
     const int per = (V + kStatSplits - 1) / kStatSplits;
     const int j0 = sp * per, j1 = min(V, j0 + per);
-    float* lr = logits + (size_t)row * V;
+    const float* lr = logits + (size_t)row * V;
     float m = -INFINITY;
     int arg = 0x7fffffff;
     for (int j = j0 + threadIdx.x; j < j1; j += 256) {
-        float v;
-        if (part) {
-            v = 0.f;
-            for (int s = 0; s < S; ++s) v += part[((size_t)s * M + row) * V + j];
-            lr[j] = v;
-        } else {
-            v = lr[j];
-        }
+        const float v = lr[j];
         if (v > m) { m = v; arg = j; }
     }
     __shared__ float sm_m[8];
@@ -76,9 +68,24 @@ struct RejectItem {
     int mode;          // 0 stochastic, 1 greedy, 2 none (prefill)
     int u0;            // offset of the request's k+1 uniforms
     const float* q;    // device [k][V]
+    int slot;          // request slot (row of the request-state array)
+    int base;          // cached positions before this pass, as the host planned it
+    int commit;        // kCommit*: what the kernel does with the request's device-resident state
+    int reserved;
 };
 
 struct RejectOut { int n_accepted, next_token, status, reserved; };
+
+// Device-resident request state, kept by the commit-on-device path: the committed length and the pending token
+// (the last correction or extra token, whose K/V is not cached yet), and whether the last pass accepted every draft.
+struct ReqState { int len, pending, all_accepted, reserved; };
+constexpr int kCommitNone = 0;      // the host commits later (pipesd_kv_rollback)
+constexpr int kCommitAuto = 1;      // write {base + 1 + n_accepted, emitted token} to the state
+constexpr int kCommitChain = 2;     // as kCommitAuto, but only if the state says that the pass before this one accepted every
+                                    // draft, left exactly `base` positions and emitted this pass's first token
+                                    // (early drafts kept by the cloud are valid under exactly that condition); otherwise the pass
+                                    // is void: status kStatusDiscarded, state untouched apart from all_accepted = 0
+constexpr int kStatusDiscarded = 1;
 
 // One CTA per request: combine the row statistics, run the accept chain, make the final draw.
 //
@@ -102,12 +109,34 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
                                                                        const RejectItem* __restrict__ items,
                                                                        const int32_t* __restrict__ row_tok,
                                                                        const float* __restrict__ u_all,
-                                                                       RejectOut* __restrict__ out) {
+                                                                       RejectOut* __restrict__ out,
+                                                                       ReqState* __restrict__ req_state) {
     pdl_wait();      // launched with programmatic serialisation: the row statistics must be complete
     const int item = blockIdx.y, rank = (int)cluster_ctarank();
     const RejectItem it = items[item];
     if (it.mode == 2) return;                     // the whole cluster (one request) leaves together
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (it.commit == kCommitChain) {
+        // the state was written by the pass before this one (an earlier launch): every thread reads the same values
+        const ReqState s = req_state[it.slot];
+        if (!(s.all_accepted && s.len == it.base && s.pending == row_tok[it.row0])) {
+            if (rank == 0 && tid == 0) {
+                RejectOut r{0, -1, kStatusDiscarded, 0};
+                out[item] = r;
+                req_state[it.slot].all_accepted = 0;
+            }
+            return;
+        }
+    }
+    // exactly one thread of the cluster publishes the result and, on the commit-on-device path, the new state
+    auto emit = [&](int n_acc_, int tok_) {
+        RejectOut r{n_acc_, tok_, 0, 0};
+        out[item] = r;
+        if (it.commit != kCommitNone) {
+            ReqState s{it.base + 1 + n_acc_, tok_, n_acc_ == it.k ? 1 : 0, 0};
+            req_state[it.slot] = s;
+        }
+    };
     constexpr int kWarps = kSampleThreads / 32;
     __shared__ double s_m[kMaxItemRows], s_z[kMaxItemRows];
     __shared__ int s_arg[kMaxItemRows];
@@ -152,7 +181,7 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
     __syncthreads();
     const int n_acc = s_nacc;
     if (it.mode == 1) {
-        if (tid == 0 && rank == 0) { RejectOut r{n_acc, s_arg[n_acc], 0, 0}; out[item] = r; }
+        if (tid == 0 && rank == 0) emit(n_acc, s_arg[n_acc]);
         return;
     }
     // Final draw from row n_acc: residual max(0, p - q) if a draft was rejected there, else p.
@@ -229,7 +258,7 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
                 run += __shfl_sync(0xffffffffu, inc, 31);
             }
             if (tok < 0) tok = last_mass;    // the walk's rounding fell short of the range's total: its last id with mass
-            if (lane == 0) { RejectOut r{n_acc, tok, 0, 0}; out[item] = r; }
+            if (lane == 0) emit(n_acc, tok);
         }
         // u < 1, so target < total and some warp owns it; were rounding ever to say otherwise, rank 0 answers
         if (!(total > target) && rank == 0 && tid == 0) {
@@ -240,8 +269,7 @@ __global__ void __launch_bounds__(kSampleThreads) accept_sample_kernel(const flo
                 if (use_q) r = fmax(0.0, r - (double)qr[j]);
                 if (r > 0.0) { tok = j; break; }
             }
-            RejectOut r{n_acc, tok, 0, 0};
-            out[item] = r;
+            emit(n_acc, tok);
         }
         break;
     }

@@ -35,7 +35,7 @@ def test_1b_shape_real_prefill_sigma_sweep(engine):
     from paper_2605_13319_b200 import binding
     shape, P, k = synth.B1, 512, 8
     w = synth.make_weights(shape, 0)
-    ctx = binding.Context(shape, w, n_pages=P // 16 + 8, max_seq=P + 64, engine=engine)
+    ctx = binding.Context(shape, w, n_pages=P // 16 + 8, max_seq=P + 64, engine=engine, poison=True)
     orc = oracle.Oracle(shape, w, P + 64)
     prefix = synth.make_prefix(shape, P, 0)
     t0 = time.time()
@@ -64,6 +64,43 @@ def test_1b_shape_real_prefill_sigma_sweep(engine):
     ctx.close()
 
 
+def test_1b_shape_64_lockstep_rounds_real_prefill():
+    """The method's multi-round configuration for real: 64 rounds of verify + rollback against a REAL prefill on both
+    sides (1b shape, 512-token prefix), the checker in lock-step and leading, k cycling through 4, 8 and 16, the two
+    sets of kernels taking turns on the same growing cache."""
+    from paper_2605_13319_b200 import binding
+    shape, P, rounds = synth.B1, 512, 64
+    w = synth.make_weights(shape, 0)
+    max_seq = P + rounds * 17 + 32
+    ctx = binding.Context(shape, w, n_pages=max_seq // 16 + 8, max_seq=max_seq, max_rows=40, engine="persistent", poison=True)
+    orc = oracle.Oracle(shape, w, max_seq)
+    prefix = synth.make_prefix(shape, P, 5)
+    orc.prefill(prefix)
+    req = ctx.req_open()
+    ctx.prefill(req, prefix)
+    tally = Tally()
+    pending = synth.make_pending(shape, 5)
+    t0 = time.time()
+    for r in range(rounds):
+        k = (4, 8, 16)[r % 3]
+        sigma = (0.3, 1.0)[(r // 3) % 2]
+        ctx.debug_set_engine(r % 2)                        # 0: persistent kernel, 1: tiled kernels
+        toks, q, u, _ = draft_inputs(orc, shape, k, sigma, 5, round_=r, pending=pending)
+        ref = orc.verify(toks, q, u)
+        (got,) = ctx.verify([dict(req=req, tokens=toks, q=q, u=u)], flags=binding.Q_HOST)
+        err = logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max()
+        assert err < LOGIT_TOL
+        tally.max_logit_err = max(tally.max_logit_err, err)
+        tally.check(got, ref, ref["logits"], q, u, where=f"round {r}")
+        orc.rollback(ref["base_len"], ref["n_accepted"])
+        ctx.kv_rollback([req], [ref["n_accepted"]], [ref["next_token"]])
+        assert ctx.req_len(req) == orc.len
+        pending = ref["next_token"]
+    print(f"\n{rounds} rounds in {time.time() - t0:.0f} s, final length {orc.len}; " + tally.report())
+    assert tally.max_logit_err < 2e-3
+    ctx.close()
+
+
 @pytest.fixture(scope="module")
 def seven_b():
     from paper_2605_13319_b200 import binding
@@ -75,7 +112,7 @@ def seven_b():
     # persistent engine with room for the 300-row batch: the context keeps the weights in both orders, single
     # requests run on the persistent kernel, the batch (and whatever debug_set_engine(1) asks for) on the tiled ones
     ctx = binding.Context(shape, w, n_pages=pages, max_seq=4096 + 32, max_requests=34,
-                          max_rows=int(ks.sum()) + 32, max_draft=16, engine="persistent")
+                          max_rows=int(ks.sum()) + 32, max_draft=16, engine="persistent", poison=True)
     print(f"\n7b weights + context: {time.time() - t0:.1f} s")
     yield shape, w, ctx, (lens, ks, sig)
     ctx.close()
@@ -109,7 +146,7 @@ def test_7b_shape_k_4_8_16_and_lockstep_rounds(seven_b):
             ctx.debug_set_len(req, P)
         ctx.debug_set_engine(0)
     pending = synth.make_pending(shape, 7)
-    for r in range(64 if FULL else 3):
+    for r in range(64 if FULL else 8):
         k = 8
         toks, q, u, _ = draft_inputs(orc, shape, k, 1.0, 7, round_=r, pending=pending)
         ref = orc.verify(toks, q, u)
@@ -122,6 +159,49 @@ def test_7b_shape_k_4_8_16_and_lockstep_rounds(seven_b):
         ctx.kv_rollback([req], [ref["n_accepted"]])
         assert ctx.req_len(req) == orc.len
         pending = ref["next_token"]
+    print(tally.report())
+    assert tally.max_logit_err < 5e-3
+    ctx.req_close(req)
+
+
+def test_7b_shape_real_prefill_short_prefix(seven_b):
+    """The GPU prefill checked against the checker's at the 7b shape: a 160-token prefix prefilled on BOTH sides (no
+    seeded K/V rows), K/V rows of the first and last layer read back, then a k=8 verify on each set of kernels."""
+    from paper_2605_13319_b200 import binding
+    shape, w, ctx, _ = seven_b
+    P, k = 160, 8
+    orc = oracle.Oracle(shape, w, P + 32)
+    prefix = synth.make_prefix(shape, P, 9)
+    t0 = time.time()
+    orc.prefill(prefix)
+    print(f"\noracle prefill of {P} tokens at the 7b shape: {time.time() - t0:.0f} s")
+    req = ctx.req_open()
+    ctx.prefill(req, prefix)
+    for layer in (0, shape.n_layers - 1):
+        kg, vg = ctx.debug_read_kv(req, layer, 0, P)
+        ko = np.stack([orc.get_kv(layer, p)[0] for p in range(P)])
+        vo = np.stack([orc.get_kv(layer, p)[1] for p in range(P)])
+        for got_bits, want in ((kg, ko), (vg, vo)):
+            diff = np.abs(synth.bf16_to_f32(got_bits) - want)
+            # one bf16 ulp where the fp32-vs-fp64 difference crosses a rounding boundary, plus the accumulated
+            # difference of the layers below (the same bound as on the tiny shape)
+            slack, l1 = (2e-5, 1e-4) if layer == 0 else (2e-3, 1e-3)
+            assert np.all(diff <= 2.0 ** -7 * np.abs(want) + slack * max(1.0, float(np.abs(want).max())))
+            assert diff.sum() / np.abs(want).sum() < l1
+    toks, q, u, _ = draft_inputs(orc, shape, k, 1.0, 9)
+    ref = orc.verify(toks, q, u)
+    tally = Tally()
+    for eng, name in ((0, "persistent"), (1, "tiled")):
+        ctx.debug_set_engine(eng)
+        (got,) = ctx.verify([dict(req=req, tokens=toks, q=q, u=u)], flags=binding.Q_HOST)
+        err = logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max()
+        print(f"{name}: n_accepted {ref['n_accepted']}, gpu {got}, rel logit err {err:.2e}")
+        assert err < LOGIT_TOL
+        tally.max_logit_err = max(tally.max_logit_err, err)
+        tally.check(got, ref, ref["logits"], q, u, where=name)
+        ctx.kv_rollback([req], [0])
+        ctx.debug_set_len(req, P)
+    ctx.debug_set_engine(0)
     print(tally.report())
     assert tally.max_logit_err < 5e-3
     ctx.req_close(req)
@@ -192,7 +272,7 @@ def test_8b_shape_long_context_large_vocab(engine):
     from paper_2605_13319_b200 import binding
     shape, P, k = synth.B8, 8192, 16
     w = synth.make_weights(shape, 0)
-    ctx = binding.Context(shape, w, n_pages=P // 16 + 8, max_seq=P + 64, engine=engine)
+    ctx = binding.Context(shape, w, n_pages=P // 16 + 8, max_seq=P + 64, engine=engine, poison=True)
     orc = oracle.Oracle(shape, w, P + 64)
     req = ctx.req_open()
     _load_synthetic_prefix(ctx, orc, shape, req, P, seed=3)

@@ -15,7 +15,7 @@ def _mk(shape, seed, P, n_pages=None, **kw):
     w = synth.make_weights(shape, seed)
     max_seq = kw.pop("max_seq", P + 256)
     n_pages = n_pages or (max_seq // 16 + 2) * kw.get("max_requests", 1)
-    ctx = binding.Context(shape, w, n_pages=n_pages, max_seq=max_seq, **kw)
+    ctx = binding.Context(shape, w, n_pages=n_pages, max_seq=max_seq, poison=True, **kw)
     orc = oracle.Oracle(shape, w, max_seq)
     return w, ctx, orc
 
@@ -119,7 +119,7 @@ def test_batched_ragged_verify_and_batch_invariance(engine):
     lens, ks, sig = synth.ragged_requests(3, n_req, 5, 150, 1, 16)
     w = synth.make_weights(shape, 2)
     ctx = binding.Context(shape, w, n_pages=(200 // 16 + 2) * n_req * 2, max_seq=200, max_requests=2 * n_req,
-                          max_rows=max(33, int(ks.sum() + n_req)), max_draft=16, engine=engine)
+                          max_rows=max(33, int(ks.sum() + n_req)), max_draft=16, engine=engine, poison=True)
     assert int(ks.sum() + n_req) > 32
     tally = Tally()
     items, refs, solo = [], [], []
@@ -162,7 +162,7 @@ def test_draft_lengths_across_token_tile_counts(engine):
     w = synth.make_weights(shape, 5)
     tally = Tally()
     for n, (k, P) in enumerate(((1, 1), (7, 63), (8, 64), (15, 65), (16, 127), (31, 130))):
-        ctx = binding.Context(shape, w, n_pages=16, max_seq=200, max_draft=31, engine=engine)
+        ctx = binding.Context(shape, w, n_pages=16, max_seq=200, max_draft=31, engine=engine, poison=True)
         orc = oracle.Oracle(shape, w, 200)
         prefix = synth.make_prefix(shape, P, 5, request=n)
         orc.prefill(prefix)
@@ -197,7 +197,7 @@ def test_page_sizes_other_than_16(engine):
     tally = Tally()
     for n, (ps, P, k) in enumerate(((8, 150, 5), (24, 101, 8), (32, 193, 3), (64, 130, 8), (128, 200, 12))):
         ctx = binding.Context(shape, w, n_pages=(P + 48) // ps + 3, max_seq=P + 40, max_draft=16, page_size=ps,
-                              engine=engine)
+                              engine=engine, poison=True)
         orc = oracle.Oracle(shape, w, P + 40)
         prefix = synth.make_prefix(shape, P, 6, request=n)
         orc.prefill(prefix)
@@ -247,8 +247,17 @@ def test_host_side_errors_and_page_accounting():
     with pytest.raises(binding.PipesdError) as e:
         ctx.kv_rollback([r0], [5])
     assert e.value.code == binding.E_RANGE
+    with pytest.raises(binding.PipesdError) as e:     # a request listed twice would be committed twice
+        ctx.kv_rollback([r0, r0], [1, 1])
+    assert e.value.code == binding.E_INVALID and ctx.req_len(r0) == 60
+    with pytest.raises(binding.PipesdError) as e:
+        ctx.kv_rollback([r0], [1], [shape.vocab])
+    assert e.value.code == binding.E_INVALID and ctx.req_len(r0) == 60
     ctx.kv_rollback([r0], [4])
     assert ctx.req_len(r0) == 65
+    with pytest.raises(binding.PipesdError) as e:     # no pending token was recorded at that rollback
+        ctx.verify([dict(req=r0, tokens=np.array([binding.TOKEN_PENDING, 2], np.int32), u=u[:2], mode=binding.MODE_GREEDY)])
+    assert e.value.code == binding.E_STATE
     with pytest.raises(binding.PipesdError) as e:
         ctx.verify([dict(req=r0, tokens=np.array([1, 99999], np.int32), u=u[:2], mode=binding.MODE_GREEDY)])
     assert e.value.code == binding.E_INVALID

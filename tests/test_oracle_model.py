@@ -211,6 +211,63 @@ def test_loaded_cache_is_what_attention_reads():
     assert o.len == 4
 
 
+def test_chained_rounds_equal_two_separate_rounds_by_enumeration():
+    """App. B, cloud side of proactive transmission, enumerated on a small vocabulary: for EVERY candidate first
+    buffered token b_1 and a grid of uniforms, the buffered tokens are kept exactly when all drafts were accepted
+    and the extra token equals b_1; when kept, the second round's outcome and logits equal those of an instance
+    that never chained (prefilled directly with the committed sequence, then verified); when discarded, the cache
+    holds the first round's commit only and behaves like an instance that was never offered the buffered tokens."""
+    shape = synth.TINY.scaled(name="chain", vocab=16, n_layers=1, d_model=32, n_q_heads=2, n_kv_heads=1, head_dim=16,
+                              d_ffn=48)
+    w = synth.make_weights(shape, 9)
+    V, P, k, m = shape.vocab, 5, 2, 3
+    prefix = synth.tokens_i32(P, 9, 0, V)
+    kept = dropped = 0
+    for trial in range(6):
+        a = oracle.Oracle(shape, w, 32)
+        a.prefill(prefix)
+        pending = int(synth.tokens_i32(1, 9, 100 + trial, V)[0])
+        # drafts from q = p (sigma 0) half of the time so that full acceptance is common, else noisy
+        sigma = 0.0 if trial % 2 == 0 else 1.5
+        toks, q, _ = a.draft_round(pending, k, sigma, synth.normal_f32((k, V), 9, 200 + trial),
+                                   synth.uniform_f32(k, 9, 300 + trial))
+        u = synth.uniform_f32(k + 1, 9, 400 + trial)
+        rest = synth.tokens_i32(m - 1, 9, 500 + trial, V)
+        q_buf = np.stack([oracle.softmax(synth.normal_f32(V, 9, 600 + trial + 50 * j).astype(np.float64))
+                          for j in range(m - 1)]).astype(np.float32)
+        u_buf = synth.uniform_f32(m, 9, 700 + trial)
+        for b1 in range(V):
+            buffered = np.concatenate([[b1], rest]).astype(np.int32)
+            c = oracle.Oracle(shape, w, 32)
+            c.prefill(prefix)
+            r1, r2 = c.verify_chain(toks, q, u, buffered, q_buf, u_buf)
+            # the first round is an ordinary round
+            s = oracle.Oracle(shape, w, 32)
+            s.prefill(prefix)
+            ref1 = s.verify(toks, q, u)
+            assert (r1["n_accepted"], r1["next_token"]) == (ref1["n_accepted"], ref1["next_token"])
+            assert np.array_equal(r1["logits"], ref1["logits"])
+            keep = ref1["n_accepted"] == k and ref1["next_token"] == b1
+            assert (r2 is not None) == keep
+            committed = list(prefix) + list(toks[:1 + ref1["n_accepted"]])
+            if keep:
+                kept += 1
+                f = oracle.Oracle(shape, w, 32)
+                f.prefill(np.array(committed, np.int32))
+                ref2 = f.verify(buffered, q_buf, u_buf)
+                assert (r2["n_accepted"], r2["next_token"]) == (ref2["n_accepted"], ref2["next_token"])
+                assert np.allclose(r2["logits"], ref2["logits"], atol=1e-12)    # same values; prefill chunks differ
+                assert c.len == len(committed) + 1 + ref2["n_accepted"]
+            else:
+                dropped += 1
+                assert c.len == len(committed)
+                nxt = np.array([ref1["next_token"], 3, 7], np.int32)
+                f = oracle.Oracle(shape, w, 32)
+                f.prefill(np.array(committed, np.int32))
+                assert np.allclose(c.forward(nxt), f.forward(nxt), atol=1e-12)
+    assert kept >= 2 and dropped >= 2 * 15, (kept, dropped)
+
+
 def test_numpy_restatement_cross_check(tiny):
     """Not a pin (it re-states the formulas): a compact fp64 numpy forward as a second opinion."""
     shape, w = tiny
