@@ -67,18 +67,6 @@ typedef enum pipesd_status {
                                    * request (pipesd_kv_rollback's next_token, or a commit on the device) */
 #define PIPESD_DISCARDED 1        /* pipesd_verify_result.status of a chained pass whose condition failed (not an error) */
 
-/* Which kernels run the layer stack (both compute the same forward; their summation orders differ, so results
- * agree to rounding, not bit for bit).
- *   TILED       one kernel per projection (weight-streaming GEMMs with fused epilogues, split-K summed over a
- *               thread-block cluster) and one attention kernel per layer; any number of rows per pass.
- *   PERSISTENT  passes of at most 32 rows run in a persistent kernel: one CTA per SM streams the weights of
- *               consecutive projections through the tcgen05 tensor cores without a kernel boundary; when the pass
- *               is a single request whose query rows per KV head fit one 16-row tile, attention is a phase of the
- *               same kernel and the whole pass is one launch.  Larger passes fall back to the tiled kernels (the
- *               context then keeps the weights in both orders, i.e. twice the weight memory, if max_rows > 32). */
-#define PIPESD_ENGINE_TILED 0
-#define PIPESD_ENGINE_PERSISTENT 1
-
 typedef struct pipesd_model_cfg {
     int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
     float rms_eps;
@@ -90,7 +78,7 @@ typedef struct pipesd_model_cfg {
     int32_t max_rows;     /* largest sum of (k+1) over the items of one verify call            */
     int32_t max_seq;      /* largest number of cached positions per request                    */
     int32_t device;       /* CUDA device ordinal                                               */
-    int32_t engine;       /* PIPESD_ENGINE_*: which kernels run the layer stack (0 = tiled)    */
+    int32_t reserved;     /* must be 0                                                         */
 } pipesd_model_cfg;
 
 /* Device pointers to row-major [out, in] bf16 matrices; norm gains are fp32 [d_model]. */
@@ -230,12 +218,6 @@ int32_t pipesd_debug_wait_timeout(pipesd_ctx *ctx, int32_t limit_us);
  * pool).  Lets a harness replay rounds from a recorded point; the serving path uses pipesd_kv_rollback. */
 int32_t pipesd_debug_set_len(pipesd_ctx *ctx, int32_t req, int32_t new_len);
 
-/* Run-time switch inside a context created with PIPESD_ENGINE_PERSISTENT (a harness compares the kernels with it).
- * 0 (initial): as the engine is described above.  1: the tiled kernels for every pass; needs the weights in their
- * order (max_rows > 32), PIPESD_E_INVALID otherwise.  2: as 0, but attention always runs as its own kernel between
- * persistent launches.  A context of the tiled engine accepts the values and ignores them. */
-int32_t pipesd_debug_set_engine(pipesd_ctx *ctx, int32_t engine);
-
 /* Launch accounting.  While enabled, every kernel launch of the context is counted and every
  * weight-streaming GEMM launch is bracketed by CUDA events on the context's stream.
  * pipesd_profile_read synchronises, reports the totals since the last read and resets them. */
@@ -260,7 +242,7 @@ int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scra
                         int32_t K, void *cuda_stream);
 
 /* Host only, no CUDA call: how the attention kernel splits a request of `total_keys` keys (cached + this pass's
- * rows) at the given page size.  resident_clusters[0..2] (host) = thread-block clusters of 8, 9 and 10 CTAs the
+ * rows) at the given page size (tiles of 128 keys).  resident_clusters[0..2] (host) = thread-block clusters of 8, 9 and 10 CTAs the
  * device keeps resident at once for the request's footprint (0 = that width is unavailable), clusters_needed =
  * clusters one layer launches for the request (KV heads x row groups).  out3 (host) receives {clusters sharing the
  * keys, key splits per cluster, keys per split (a multiple of page_size)}.  The split is a function of the request

@@ -19,9 +19,6 @@ OK, E_INVALID, E_FULL, E_OOM_PAGES, E_STATE, E_RANGE, E_CUDA, E_NOMEM = 0, -1, -
 E_TOO_LARGE = -8
 STATIC_SCRATCH_BYTES = 8 << 20
 MODE_STOCHASTIC, MODE_GREEDY = 0, 1
-ENGINE_TILED, ENGINE_PERSISTENT = 0, 1
-ENGINES = {"tiled": ENGINE_TILED, "persistent": ENGINE_PERSISTENT}
-DEFAULT_ENGINE = "tiled"
 Q_HOST, AUTOCOMMIT, CHAIN = 1, 2, 4
 TOKEN_PENDING = -1
 DISCARDED = 1
@@ -32,7 +29,7 @@ i32, u32, u64, f32, vp = ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64, ctype
 class ModelCfg(ctypes.Structure):
     _fields_ = [(n, i32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab")] \
         + [("rms_eps", f32), ("rope_base", f32)] \
-        + [(n, i32) for n in ("page_size", "n_pages", "max_requests", "max_draft", "max_rows", "max_seq", "device", "engine")]
+        + [(n, i32) for n in ("page_size", "n_pages", "max_requests", "max_draft", "max_rows", "max_seq", "device", "reserved")]
 
 
 class LayerWeights(ctypes.Structure):
@@ -86,7 +83,6 @@ _SIGNATURES = {
     "pipesd_debug_write_kv": (i32, [vp, i32, i32, i32, i32, vp, vp]),
     "pipesd_reject_from_logits": (i32, [vp, i32, i32, vp, vp, vp, vp, ctypes.POINTER(VerifyResult)]),
     "pipesd_debug_set_len": (i32, [vp, i32, i32]),
-    "pipesd_debug_set_engine": (i32, [vp, i32]),
     "pipesd_profile_enable": (i32, [vp, i32]),
     "pipesd_profile_read": (i32, [vp, ctypes.POINTER(ProfileInfo)]),
     "pipesd_gemm_packed_bytes": (u64, [i32, i32]),
@@ -133,7 +129,7 @@ class Context:
 
     def __init__(self, shape, weights: dict, *, n_pages: int, max_requests: int = 1, max_draft: int = 16,
                  max_rows: int | None = None, max_seq: int = 4096, page_size: int = 16, device: int = 0,
-                 stream=None, engine: str | None = None, poison: bool = False):
+                 stream=None, poison: bool = False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required: the verify pass has no CPU path")
@@ -146,8 +142,7 @@ class Context:
             max_rows = max(max_draft + 1, 32)
         self.cfg = ModelCfg(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                             shape.d_ffn, shape.vocab, shape.rms_eps, shape.rope_base, page_size, n_pages,
-                            max_requests, max_draft, max_rows, max_seq, device, ENGINES[engine or DEFAULT_ENGINE])
-        self.engine = engine or DEFAULT_ENGINE
+                            max_requests, max_draft, max_rows, max_seq, device, 0)
         L = lib()
         sz = Sizes()
         rc = L.pipesd_query_sizes(ctypes.byref(self.cfg), ctypes.byref(sz))
@@ -298,10 +293,6 @@ class Context:
         v = np.ascontiguousarray(v_bf16, np.uint16)
         self._check(lib().pipesd_debug_write_kv(self._h, req, layer, pos0, k.shape[0], _np_ptr(k), _np_ptr(v)),
                     "pipesd_debug_write_kv")
-
-    def debug_set_engine(self, engine: int):
-        """0: persistent kernel for passes of <= 32 rows (default); 1: tiled kernels for every pass."""
-        self._check(lib().pipesd_debug_set_engine(self._h, engine), "pipesd_debug_set_engine")
 
     def debug_set_len(self, req: int, new_len: int):
         self._check(lib().pipesd_debug_set_len(self._h, req, new_len), "pipesd_debug_set_len")

@@ -127,12 +127,15 @@ struct L2Prefetch {
     uint32_t run_bytes, skip, len;
     int runs;
 };
-// CTA `cta` of `n_ctas` issues the hints of runs cta, cta + n_ctas, ... (one thread calls this).
-__device__ __forceinline__ void l2_prefetch_issue(const L2Prefetch& pf, int cta, int n_ctas) {
+// CTA `cta` of `n_ctas` issues the hints of runs cta, cta + n_ctas, ...: `n_thr` threads call this with their index
+// `tid`, one 128-byte line per thread and step, through the load/store path (the copy engine's queue stays free for
+// the successor's own copies).
+__device__ __forceinline__ void l2_prefetch_issue(const L2Prefetch& pf, int cta, int n_ctas, int tid, int n_thr) {
     if (pf.ptr == nullptr) return;
     for (int r = cta; r < pf.runs; r += n_ctas) {
         const unsigned char* p = pf.ptr + (size_t)r * pf.run_bytes + pf.skip;
-        for (uint32_t o = 0; o < pf.len; o += 16384u) bulk_prefetch_l2(p + o, pf.len - o < 16384u ? pf.len - o : 16384u);
+        for (uint32_t o = (uint32_t)tid * 128u; o < pf.len; o += (uint32_t)n_thr * 128u)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p + o) : "memory");
     }
 }
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
@@ -208,23 +211,6 @@ __device__ __forceinline__ void xf_store_one(uint16_t* xf, int tok, int k, float
     xf[slot * 8 + 4 + half * 2 + (kk & 1)] = l;
 }
 
-// ---- "xu" activation arrays: the token-major B operand of tcgen05.mma, in global memory ------------------
-// One token block of at most 32 tokens (NT = tiles of 8 tokens).  Per k16 step NT*512 bytes, cut into 16-byte
-// pieces = 8 consecutive tokens of one k: piece (k half kg, token group ng, k row) at ((kg*2NT + ng)*8 + row)*16,
-// token groups 0..NT-1 hold the bf16 hi terms, NT..2NT-1 the lo terms.  A chunk of consecutive k16 steps is one
-// contiguous run, copied into shared memory as it is.
-__host__ __device__ __forceinline__ size_t xu_piece_offset(int k, int ng, int NT) {
-    return (size_t)(k >> 4) * NT * 512 + (size_t)(((((k >> 3) & 1) * 2 * NT + ng) * 8 + (k & 7)) * 16);
-}
-// Stores one element (its hi and lo terms) of an xu array.
-__device__ __forceinline__ void xu_store_one(uint16_t* xu, int tok, int k, float v, int NT) {
-    uint16_t h, l;
-    split_bf16(v, h, l);
-    unsigned char* b = reinterpret_cast<unsigned char*>(xu);
-    *reinterpret_cast<uint16_t*>(b + xu_piece_offset(k, tok >> 3, NT) + (tok & 7) * 2) = h;
-    *reinterpret_cast<uint16_t*>(b + xu_piece_offset(k, NT + (tok >> 3), NT) + (tok & 7) * 2) = l;
-}
-
 // ---- thread-block clusters: barrier and distributed shared memory --------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -273,15 +259,19 @@ struct PassMeta {
 };
 
 // Offset (in elements) of K (kv=0) or V (kv=1) element (slot, e) of a head inside the paged pool:
-// layout [layer][page][kv][head][slot][e'], where the 16-byte chunks of a row are XOR-permuted by the slot's low
-// three bits (e' = kv_swizzle(e, slot)): a tile of rows copied to shared memory as it is can then be read with
-// ldmatrix without bank conflicts.  The page size is a multiple of 8, so a row's permutation is also that of
-// its index in any 8-aligned tile.
-__device__ __host__ __forceinline__ int kv_swizzle(int e, int slot) { return ((((e >> 3) ^ (slot & 7)) << 3) | (e & 7)); }
+// layout [layer][page][kv][head][slot/8][e/8][slot%8][e%8].  Inside a (page, head) block the rows sit in groups of
+// eight, cut into 8-element (16-byte) pieces, the eight rows' pieces of the same columns next to each other: 128
+// contiguous bytes are an 8 x 8 "core matrix" of the tensor cores' shared-memory operands, so a page copied to
+// shared memory as it is serves as the K-major operand of Q K^T (rows = keys) and as the MN-major operand of P V
+// (rows = head dimensions) alike.  The page size is a multiple of 8.
+__device__ __host__ __forceinline__ size_t kv_row_offset(int slot, int hd) {          // of element 0 of a row inside its block
+    return (size_t)(slot >> 3) * hd * 8 + (size_t)(slot & 7) * 8;
+}
+__device__ __host__ __forceinline__ size_t kv_col_offset(int e) { return (size_t)(e >> 3) * 64 + (size_t)(e & 7); }
 __device__ __host__ __forceinline__ size_t kv_index(int layer, int n_pages, int page, int kv, int n_kv_heads,
                                                     int head, int page_size, int slot, int hd, int e) {
-    return (((((size_t)layer * n_pages + page) * 2 + kv) * n_kv_heads + head) * page_size + slot) * (size_t)hd +
-           kv_swizzle(e, slot);
+    return ((((size_t)layer * n_pages + page) * 2 + kv) * n_kv_heads + head) * page_size * (size_t)hd +
+           kv_row_offset(slot, hd) + kv_col_offset(e);
 }
 
 }  // namespace pipesd

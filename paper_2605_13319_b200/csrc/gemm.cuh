@@ -174,7 +174,7 @@ struct GemmArgs {
     uint16_t* kv_pool;
     const float* cs;    // [M][hd/2] cos / sin of the row's position
     const float* sn;
-    const long long* row_kvoff;   // [M] element offset of the row's K slot inside a layer (head 0)
+    const long long* row_kvoff;   // [M] element offset of the row's K row inside a layer (head 0, column 0)
     int Hq, Hkv, hd, layer, n_pages, page_size;
     // kResid
     float* x;           // residual stream [M][N], updated in place
@@ -274,8 +274,6 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                 issued = c + 1;
                 if (++st == stages) { st = 0; ph ^= 1u; }
             }
-            // this CTA has asked for its last weights: from here on HBM idles until the successor streams
-            if (ok) l2_prefetch_issue(a.pf, (int)(blockIdx.y * gridDim.x + blockIdx.x), (int)(gridDim.x * gridDim.y));
             if (!ok) {
                 if (a.err) atomicExch(a.err, 1);
                 // give up: let every copy already issued land before this CTA's shared memory is released
@@ -372,6 +370,8 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             if (++st == stages) { st = 0; ph ^= 1u; }
         }
         if (!ok && a.err && lane == 0) atomicExch(a.err, 2);
+        // this CTA has consumed its last weights: from here on HBM idles until the successor streams
+        if (ok) l2_prefetch_issue(a.pf, (int)(blockIdx.y * gridDim.x + blockIdx.x), (int)(gridDim.x * gridDim.y), threadIdx.x, kGemmConsumers);
         // All consumers are past their last ring read before the ring is reused for the partial tile.
         asm volatile("bar.sync 1, %0;" ::"n"(kGemmConsumers) : "memory");
         // partial tile P[tile 8][token MT][row 16] (fp32) at the start of the ring
@@ -461,9 +461,9 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                             const int kv = head < a.Hq + a.Hkv ? 0 : 1;
                             const int kvh = kv ? head - a.Hq - a.Hkv : head - a.Hq;
                             const size_t per_head = (size_t)a.page_size * a.hd;
-                            const long long rk = cin ? pf_kv[i] : a.row_kvoff[tok];   // row offset | slot & 7
-                            const size_t off = (size_t)a.layer * a.n_pages * 2 * a.Hkv * per_head + (size_t)(rk & ~7ll) +
-                                               ((size_t)kv * a.Hkv + kvh) * per_head + kv_swizzle(dim, (int)(rk & 7));
+                            const long long rk = cin ? pf_kv[i] : a.row_kvoff[tok];   // the row's offset inside a layer (head 0, K)
+                            const size_t off = (size_t)a.layer * a.n_pages * 2 * a.Hkv * per_head + (size_t)rk +
+                                               ((size_t)kv * a.Hkv + kvh) * per_head + kv_col_offset(dim);
                             a.kv_pool[off] = f32_to_bf16_bits(val);
                         }
                     }

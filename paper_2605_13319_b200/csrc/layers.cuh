@@ -7,7 +7,7 @@
 namespace pipesd {
 
 // x = bf16 embedding row (residual stream, fp32); xf = x * gain of the first RMSNorm as split-bf16
-// fragments (or, with xu_layout, in the persistent kernel's xu layout); ssq[0][row] = sum x^2, ssq[b > 0][row] = 0 (the consumer adds n_ssq block sums up).
+// fragments; ssq[0][row] = sum x^2, ssq[b > 0][row] = 0 (the consumer adds n_ssq block sums up).
 // One CTA of 1024 threads per row, four columns per thread.
 constexpr int kEmbedThreads = 1024;
 constexpr int kEmbedMaxVec = 2;   // float4 per thread: d <= 8192
@@ -15,7 +15,7 @@ __global__ void __launch_bounds__(kEmbedThreads) embed_kernel(float* __restrict_
                                                               const int32_t* __restrict__ row_tok, int M,
                                                               const float* __restrict__ gain, int d,
                                                               uint32_t* __restrict__ xf_out, float* __restrict__ ssq,
-                                                              int n_ssq, int xu_layout) {
+                                                              int n_ssq) {
     pdl_wait();
     pdl_launch_dependents();
     const int row = blockIdx.x;
@@ -33,16 +33,8 @@ __global__ void __launch_bounds__(kEmbedThreads) embed_kernel(float* __restrict_
             *reinterpret_cast<float4*>(xr + e) = a;
             ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
             const float4 g = *reinterpret_cast<const float4*>(gain + e);
-            if (xu_layout) {
-                uint16_t* xu = reinterpret_cast<uint16_t*>(xf_out);
-                xu_store_one(xu, row, e, a.x * g.x, NT);
-                xu_store_one(xu, row, e + 1, a.y * g.y, NT);
-                xu_store_one(xu, row, e + 2, a.z * g.z, NT);
-                xu_store_one(xu, row, e + 3, a.w * g.w, NT);
-            } else {
-                xf_store_pair(xf_out, row, e, a.x * g.x, a.y * g.y, KS, NT);
-                xf_store_pair(xf_out, row, e + 2, a.z * g.z, a.w * g.w, KS, NT);
-            }
+            xf_store_pair(xf_out, row, e, a.x * g.x, a.y * g.y, KS, NT);
+            xf_store_pair(xf_out, row, e + 2, a.z * g.z, a.w * g.w, KS, NT);
         }
     }
     ss = warp_sum(ss);
@@ -59,8 +51,8 @@ __global__ void __launch_bounds__(kEmbedThreads) embed_kernel(float* __restrict_
 }
 
 // cos/sin of pos * base^(-2j/hd), evaluated in fp64 (positions reach 10^4, fp32 angles would lose
-// three digits), stored fp32 [M][hd/2]; and, per row, the element offset of its K slot (head 0) inside a
-// layer of the paged pool (with the slot's chunk permutation in the low bits), so that the QKV epilogue appends K/V without walking the page table.
+// three digits), stored fp32 [M][hd/2]; and, per row, the element offset of its K row (head 0) inside a
+// layer of the paged pool, so that the QKV epilogue appends K/V without walking the page table.
 __global__ void rope_table_kernel(PassMeta meta, int M, int hd, double log_base, float* __restrict__ cs,
                                   float* __restrict__ sn, long long* __restrict__ row_kvoff, int n_pages, int Hkv,
                                   int page_size) {
@@ -74,10 +66,7 @@ __global__ void rope_table_kernel(PassMeta meta, int M, int hd, double log_base,
     if (j == 0) {
         const int item = meta.row_item[row];
         const int page = meta.block_tab[(size_t)meta.it_slot[item] * meta.max_pages + pos / page_size];
-        // element offset of the row inside a layer (head 0, K); its low three bits carry slot & 7, the row's
-        // chunk permutation (the offset itself is a multiple of the head width)
-        const int slot = pos % page_size;
-        row_kvoff[row] = (long long)(kv_index(0, n_pages, page, 0, Hkv, 0, page_size, 0, hd, 0) + (size_t)slot * hd) | (slot & 7);
+        row_kvoff[row] = (long long)kv_index(0, n_pages, page, 0, Hkv, 0, page_size, pos % page_size, hd, 0);
     }
     double theta = exp(-2.0 * (double)j / (double)hd * log_base);
     double ang = (double)pos * theta;

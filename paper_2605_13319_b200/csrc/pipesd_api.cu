@@ -18,7 +18,6 @@
 #include "common.cuh"
 #include "gemm.cuh"
 #include "layers.cuh"
-#include "mega_tc.cuh"
 #include "reject.cuh"
 
 using namespace pipesd;
@@ -38,8 +37,7 @@ struct Request {
 };
 
 struct GemmW {
-    uint4* packed = nullptr;     // MMA-fragment order (tiled kernels; only packed when max_rows > 32)
-    uint4* packed_u = nullptr;   // tensor-core operand order (persistent kernel)
+    uint4* packed = nullptr;     // MMA-fragment order
     int N = 0, K = 0;
 };
 
@@ -96,8 +94,7 @@ Derived derive(const pipesd_model_cfg& c) {
 
 struct WsLayout {
     size_t x, xf_h, qbuf, xf_attn, xf_act, logits, partA, partB, ssqA, ssqB, o_part, m_part, l_part, tickets, cs, sn, kvoff, stats, results, meta,
-        block_tab, qstage, req_state, never_flag, mega_phases, mega_phases_att, mega_ctr, mega_scratch, total;
-    size_t mega_ctr_ints;
+        block_tab, qstage, req_state, never_flag, total;
 };
 
 WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
@@ -132,31 +129,14 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     w.qstage = take(4 * M * c.vocab);
     w.req_state = take(sizeof(ReqState) * (size_t)c.max_requests);
     w.never_flag = take(16);
-    // persistent layer-stack kernel: phase table, counters (finished units per phase | started CTAs per launch |
-    // one ticket per 256-row unit), accumulator fragments of units shared by several CTAs
-    const size_t n_phases = 5 * (size_t)c.n_layers + 1;      // with the attention phases
-    auto units = [](size_t N) { return ((N + 127) / 128 + 1) / 2; };
-    const size_t n_tickets = (size_t)c.n_layers * (units(d.Nqkv) + 2 * units(c.d_model) + units(2 * (size_t)c.d_ffn) + c.n_kv_heads) +
-                             units(c.vocab);
-    w.mega_phases = take(sizeof(MegaPhase) * n_phases);
-    w.mega_phases_att = take(sizeof(MegaPhase) * n_phases);
-    w.mega_ctr_ints = n_phases + (size_t)c.n_layers + 2 + n_tickets;
-    w.mega_ctr = take(4 * w.mega_ctr_ints);
-    w.mega_scratch = take((size_t)kMegaMaxCtas * 8 * kMegaEpiThreads * sizeof(float4));
     w.total = o;
     return w;
 }
 
 size_t packed_bytes(int N, int K) { return align_up(gemm_packed_bytes(N, K)); }
 
-// Two sets of kernels run the layer stack and each reads the weights in its own order.  The tiled per-projection
-// kernels (cfg.engine == PIPESD_ENGINE_TILED) take any pass.  The persistent kernel (PIPESD_ENGINE_PERSISTENT) takes
-// passes of at most 32 rows; a context that selects it and admits larger passes keeps both copies of the matrices.
-bool has_mega(const pipesd_model_cfg& c) { return c.engine == PIPESD_ENGINE_PERSISTENT; }
-bool needs_tiled(const pipesd_model_cfg& c) { return !has_mega(c) || c.max_rows > 32; }
-
 size_t weights_bytes(const pipesd_model_cfg& c, const Derived& d) {
-    const size_t copies = (needs_tiled(c) ? 1 : 0) + (has_mega(c) ? 1 : 0);
+    const size_t copies = 1;
     size_t per_layer = copies * (packed_bytes(d.Nqkv, c.d_model) + packed_bytes(c.d_model, d.qd) +
                                  packed_bytes(2 * c.d_ffn, c.d_model) + packed_bytes(c.d_model, c.d_ffn)) +
                        2 * align_up(4 * (size_t)c.d_model);
@@ -178,10 +158,10 @@ cudaError_t init_attrs_current_device() {
     cudaError_t e;
     if ((e = gemm_init_attrs()) != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_smem_bytes(128, kAttnMaxRowTiles));
+                             (int)attn_smem_bytes(128, kAttnMaxRows));
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)attn_smem_bytes(64, kAttnMaxRowTiles));
+                                (int)attn_smem_bytes(64, kAttnMaxRows));
 }
 
 int ensure_device_ready() {
@@ -208,7 +188,7 @@ int check_cfg(const pipesd_model_cfg* c) {
     if (c->max_draft < 1 || c->max_draft > kMaxItemRows - 1) return PIPESD_E_INVALID;
     if (c->max_rows < c->max_draft + 1 || c->max_rows > 4096 || c->max_seq < 1) return PIPESD_E_INVALID;
     if (!(c->rms_eps >= 0.f) || !(c->rope_base > 1.f)) return PIPESD_E_INVALID;
-    if (c->engine != PIPESD_ENGINE_TILED && c->engine != PIPESD_ENGINE_PERSISTENT) return PIPESD_E_INVALID;
+    if (c->reserved != 0) return PIPESD_E_INVALID;
     return PIPESD_OK;
 }
 
@@ -262,15 +242,9 @@ struct pipesd_ctx {
     std::deque<Inflight> inflight;
     int res_buf = 0;
     int last_rows = 0;
-    int attn_occ[kAttnMaxCluster + 1][kAttnMaxRowTiles + 1] = {};   // [cluster width 9..][query row tiles]: clusters of the
+    int attn_occ[kAttnMaxCluster + 1][kAttnMaxRows / 16 + 1] = {};  // [cluster width 9..][query rows / 16]: clusters of the
                                                                      // attention kernel the device keeps resident at once (0: width unavailable)
-    uint32_t pf_depth = 64u << 10;   // bytes per successor CTA that a GEMM pulls into L2 for the next GEMM
-    int mega_grid = 0;      // CTAs of the persistent kernel (one per SM)
-    int engine = 0;         // run-time switch (pipesd_debug_set_engine) inside a context of the persistent engine: 0: persistent
-                            // kernel for passes of <= 32 rows, tiled kernels otherwise; 1: tiled only; 2: as 0, but attention
-                            // always as its own kernel between the persistent launches
-    std::vector<MegaPhase> phases;       // GEMM phases only: attention runs as its own kernel between launches
-    std::vector<MegaPhase> phases_att;   // with one attention phase per layer: the whole pass is one launch
+    uint32_t pf_depth = 32u << 10;   // bytes per successor CTA that a GEMM pulls into L2 for the next GEMM
     std::string err;
     // launch accounting
     int64_t n_launch = 0, n_gemm = 0;
@@ -421,8 +395,8 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         // clusters that share the request's keys, key splits per cluster (8..10) and keys per split: from the request
         // alone (its length, its rows), so that its summation order is the same in every batch
         const int R_i = it.rows * (c.n_q_heads / c.n_kv_heads);                  // query rows per KV head
-        const int qt_i = std::min(kAttnMaxRowTiles, (R_i + 15) / 16);
-        const int rg_i = (R_i + kAttnMaxRowTiles * 16 - 1) / (kAttnMaxRowTiles * 16);
+        const int qt_i = attn_rows_n(R_i) / 16;
+        const int rg_i = (R_i + kAttnMaxRows - 1) / kAttnMaxRows;
         int resident[kAttnMaxCluster - kAttnSplits + 1];
         for (int w = kAttnSplits; w <= kAttnMaxCluster; ++w) resident[w - kAttnSplits] = ctx->attn_occ[w][qt_i];
         const AttnSplit sp = attn_split_plan(total, c.page_size, resident, c.n_kv_heads * rg_i);
@@ -478,10 +452,6 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     const int hd = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads, d = c.d_model, F = c.d_ffn;
     const int n_ssq = (d + 127) / 128;
 
-    // Passes of at most 32 rows (one token block) run their GEMMs in the persistent kernel, whose counters
-    // start every pass at zero.
-    const bool use_mega = has_mega(c) && ((ctx->engine != 1 && M <= 32) || !needs_tiled(c));
-    if (use_mega) CU(cudaMemsetAsync(ctx->wsp + ctx->ws.mega_ctr, 0, 4 * ctx->ws.mega_ctr_ints, st));
     // Every kernel of the chain is launched with programmatic stream serialisation: it may start while its
     // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
     {
@@ -489,15 +459,15 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         CU(launch_pdl(rope_table_kernel, dim3((n + 127) / 128), dim3(128), 0, st, meta, M, hd, log((double)c.rope_base),
                       cs, sn, ctx->W<long long>(ctx->ws.kvoff), c.n_pages, Hkv, c.page_size));
         CU(launch_pdl(embed_kernel, dim3(M), dim3(kEmbedThreads), 0, st, x, (const uint16_t*)ctx->emb, meta.row_tok, M,
-                      (const float*)ctx->layers[0].n1, d, xf_h, ssqA, n_ssq, use_mega ? 1 : 0));
+                      (const float*)ctx->layers[0].n1, d, xf_h, ssqA, n_ssq));
         ctx->n_launch += 2;
     }
     int max_item_rows = 1;
     for (auto& it : items) max_item_rows = std::max(max_item_rows, it.rows);
     const int maxR = max_item_rows * (Hq / Hkv);                      // query rows that share one KV head
-    const int q_tiles = std::min(kAttnMaxRowTiles, (maxR + 15) / 16);
-    const int row_groups = (maxR + kAttnMaxRowTiles * 16 - 1) / (kAttnMaxRowTiles * 16);
-    const size_t asmem = attn_smem_bytes(hd, q_tiles);
+    const int n_max = attn_rows_n(maxR);
+    const int row_groups = (maxR + kAttnMaxRows - 1) / kAttnMaxRows;
+    const size_t asmem = attn_smem_bytes(hd, n_max);
     GemmArgs base = {};
     base.M = M;
     base.eps = c.rms_eps;
@@ -506,90 +476,18 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     // depth of the L2 hints a kernel issues for its successor's weights (bytes per successor CTA)
     const uint32_t pf_depth = ctx->pf_depth;
     auto launch_attn = [&](int l) -> int {
-        const L2Prefetch pf = use_mega ? L2Prefetch{} : gemm_prefetch_of(ctx->layers[l].o.packed, M, d, dv.qd, 1u << 20);
         dim3 ag(max_cs * max_nsplit, Hkv * row_groups, n_items);   // cluster = the widest any request of the batch asks for
-        int* tickets = ctx->W<int>(ctx->ws.tickets);
-        if (hd == 128)
-            CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, max_cs, (const float*)qbuf,
-                                  meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0, ctx->err_word(), pf));
-        else
-            CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, max_cs, (const float*)qbuf,
-                                  meta, (const uint16_t*)ctx->kv_pool, l, c.n_pages, c.page_size, M, Hq, Hkv, q_tiles,
-                                  row_groups, o_part, m_part, l_part, tickets, (uint16_t*)xf_attn, use_mega ? 1 : 0, ctx->err_word(), pf));
+        AttnArgs aa = {};
+        aa.q = qbuf; aa.meta = meta; aa.kv_pool = ctx->kv_pool;
+        aa.layer = l; aa.n_pages = c.n_pages; aa.page_size = c.page_size; aa.M = M; aa.Hq = Hq; aa.Hkv = Hkv;
+        aa.n_max = n_max; aa.row_groups = row_groups;
+        aa.o_part = o_part; aa.m_part = m_part; aa.l_part = l_part; aa.tickets = ctx->W<int>(ctx->ws.tickets);
+        aa.xf_out = (uint16_t*)xf_attn; aa.err = ctx->err_word();
+        if (hd == 128) CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, max_cs, aa));
+        else CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, max_cs, aa));
         ctx->n_launch += 1;
         return PIPESD_OK;
     };
-    if (use_mega) {
-        // Persistent kernel: [QKV 0] attn [O, gate/up, down, QKV 1] attn ... [O, gate/up, down, LM head]
-        // One request whose query rows per KV head fit one 16-row MMA tile (and 16-position pages): attention
-        // runs as a phase of the same launch, and the whole pass is ONE persistent kernel.
-        const bool one_launch = ctx->engine == 0 && n_items == 1 && (Hq / Hkv) * items[0].rows <= 16 && c.page_size == 16;
-        const std::vector<MegaPhase>& table = one_launch ? ctx->phases_att : ctx->phases;
-        MegaArgs ma = {};
-        ma.phases = ctx->W<MegaPhase>(one_launch ? ctx->ws.mega_phases_att : ctx->ws.mega_phases);
-        ma.M = M;
-        int* ctr = ctx->W<int>(ctx->ws.mega_ctr);
-        const int n_phases = 5 * c.n_layers + 1;      // counters are laid out for the longer table
-        if (one_launch) {
-            ma.att_base = items[0].base;
-            ma.att_rows = items[0].rows;
-            ma.att_cpr = (items[0].base + items[0].rows + kAttTile - 1) / kAttTile;
-            ma.att_bt = ctx->W<int32_t>(ctx->ws.block_tab) + (size_t)items[0].slot * dv.max_pages;
-        }
-        ma.done = ctr;
-        ma.tickets = ctr + n_phases + c.n_layers + 2;
-        ma.scratch = ctx->W<float4>(ctx->ws.mega_scratch);
-        ma.err = ctx->err_word();
-        ma.eps = c.rms_eps;
-        ma.d_in = d;
-        ma.q_out = qbuf; ma.kv_pool = ctx->kv_pool; ma.cs = cs; ma.sn = sn;
-        ma.row_kvoff = ctx->W<long long>(ctx->ws.kvoff);
-        ma.Hq = Hq; ma.Hkv = Hkv; ma.hd = hd; ma.n_pages = c.n_pages; ma.page_size = c.page_size;
-        const int NT = xf_nt(M);
-        auto launch_mega = [&](int launch_idx, int p0, int p1) -> int {
-            MegaArgs a = ma;
-            a.p0 = p0; a.p1 = p1;
-            a.launch_idx = launch_idx;
-            a.arrived = ctr + n_phases + launch_idx;
-            cudaEvent_t e1 = nullptr;
-            if (ctx->time_gemms) {
-                if (ctx->prof_used + 2 > ctx->prof_ev.size())
-                    for (int i = 0; i < 2; ++i) {
-                        cudaEvent_t e;
-                        CU(cudaEventCreate(&e));
-                        ctx->prof_ev.push_back(e);
-                    }
-                CU(cudaEventRecord(ctx->prof_ev[ctx->prof_used], st));
-                e1 = ctx->prof_ev[ctx->prof_used + 1];
-                ctx->prof_used += 2;
-            }
-            CU(mega_launch(NT, a, ctx->mega_grid, st));
-            if (e1) CU(cudaEventRecord(e1, st));
-            ctx->n_launch += 1;
-            ctx->n_gemm += 1;
-            for (int p = p0; p < p1; ++p) {
-                const MegaPhase& ph = table[p];
-                if (ph.mode == kPhaseAttn)   // K and V of every key once
-                    ctx->gemm_bytes += 2.0 * (ma.att_base + ma.att_rows) * Hkv * hd * 2.0;
-                else
-                    ctx->gemm_bytes += 2.0 * ph.N * ph.KS * 16 + 4.0 * M * ph.KS * 16 + 4.0 * M * ph.N;
-            }
-            return PIPESD_OK;
-        };
-        int rc_;
-        if (one_launch) {
-            if ((rc_ = launch_mega(0, 0, want_logits ? 5 * c.n_layers + 1 : 5 * c.n_layers))) return rc_;
-        } else {
-        if ((rc_ = launch_mega(0, 0, 1))) return rc_;
-        for (int l = 0; l < c.n_layers; ++l) {
-            if ((rc_ = launch_attn(l))) return rc_;
-            const bool last = l + 1 == c.n_layers;
-            const int p1 = last ? (want_logits ? 4 * l + 5 : 4 * l + 4) : 4 * l + 5;
-            if ((rc_ = launch_mega(l + 1, 4 * l + 1, p1))) return rc_;
-        }
-        }
-    } else
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& lw = ctx->layers[l];
         {   // q, k, v = W_qkv . norm(x); RoPE; K/V appended to the pages
@@ -634,7 +532,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         ctx->n_launch += 1 + (want_reject ? 1 : 0);   // row_stats, accept_sample
         float* logits = ctx->W<float>(ctx->ws.logits);
         RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
-        if (!use_mega) {
+        {
             GemmArgs a = base;
             a.W = ctx->lm.packed; a.xf = (const uint4*)xf_h; a.N = c.vocab; a.ssq_in = ssqA; a.out = logits;
             int rc_ = launch_gemm(ctx, kPlain, a, d);
@@ -718,11 +616,11 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         const void* fn = hd128 ? (const void*)attn_kernel<128> : (const void*)attn_kernel<64>;
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
             for (int w = kAttnSplits + 1; w <= kAttnMaxCluster; ++w)
-                for (int qt = 1; qt <= kAttnMaxRowTiles; ++qt) {
+                for (int qt = 1; qt <= kAttnMaxRows / 16; ++qt) {
                     cudaLaunchConfig_t lc = {};
                     lc.gridDim = dim3(w, 1, 1);
                     lc.blockDim = dim3(kAttnThreads);
-                    lc.dynamicSmemBytes = attn_smem_bytes(c.head_dim, qt);
+                    lc.dynamicSmemBytes = attn_smem_bytes(c.head_dim, 16 * qt);
                     cudaLaunchAttribute at[1];
                     at[0].id = cudaLaunchAttributeClusterDimension;
                     at[0].val.clusterDim.x = w; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -756,7 +654,6 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     char* wp = (char*)mem->weights;
     size_t off = 0;
     auto take = [&](size_t bytes) { char* p = wp + off; off += align_up(bytes); return p; };
-    const bool tiled = needs_tiled(c);
     auto pack = [&](GemmW& g, int N, int K, int mode, std::initializer_list<std::pair<const void*, int>> srcs) {
         g.N = N;
         g.K = K;
@@ -767,14 +664,8 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         for (auto& s : srcs) { ps.w[i] = (const uint16_t*)s.first; ps.rows[i] = s.second; ++i; }
         size_t total = (size_t)((N + 127) / 128 * 8) * (K / 16) * 32;
         int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
-        if (has_mega(c)) {
-            g.packed_u = (uint4*)take(gemm_packed_bytes(N, K));
-            gemm_pack_umma_kernel<<<blocks, 256, 0, st>>>(ps, g.packed_u, N, K);
-        }
-        if (tiled) {
-            g.packed = (uint4*)take(gemm_packed_bytes(N, K));
-            gemm_pack_kernel<<<blocks, 256, 0, st>>>(ps, g.packed, N, K);
-        }
+        g.packed = (uint4*)take(gemm_packed_bytes(N, K));
+        gemm_pack_kernel<<<blocks, 256, 0, st>>>(ps, g.packed, N, K);
     };
     ctx->emb = (uint16_t*)take((size_t)c.vocab * c.d_model * 2);
     if (cudaMemcpyAsync(ctx->emb, w->tok_emb, (size_t)c.vocab * c.d_model * 2, cudaMemcpyDeviceToDevice, st) !=
@@ -799,78 +690,6 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     ctx->final_norm = (float*)take(4 * (size_t)c.d_model);
     cudaMemcpyAsync(ctx->final_norm, w->final_norm, 4 * (size_t)c.d_model, cudaMemcpyDeviceToDevice, st);
     if (cudaGetLastError() != cudaSuccess) return bail(PIPESD_E_CUDA);
-
-    // ---- phase table of the persistent kernel: QKV(0) | O, gate/up, down, QKV(l+1) per layer | ... | LM head
-    if (has_mega(c)) {
-        int n_sm = 0;
-        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, c.device) != cudaSuccess || n_sm < 1)
-            return bail(PIPESD_E_CUDA);
-        ctx->mega_grid = std::min(n_sm, kMegaMaxCtas);
-        if (mega_init_attrs() != cudaSuccess) return bail(PIPESD_E_CUDA);
-        const int d = c.d_model;
-        const int n_ssq = ((d + 127) / 128 + 1) / 2;      // 256-row units of the residual stream
-        uint32_t* xf_h = ctx->W<uint32_t>(ctx->ws.xf_h);
-        uint32_t* xf_attn = ctx->W<uint32_t>(ctx->ws.xf_attn);
-        uint32_t* xf_act = ctx->W<uint32_t>(ctx->ws.xf_act);
-        float* ssqA = ctx->W<float>(ctx->ws.ssqA);
-        float* ssqB = ctx->W<float>(ctx->ws.ssqB);
-        float* x = ctx->W<float>(ctx->ws.x);
-        for (int with_att = 0; with_att < 2; ++with_att) {
-        std::vector<MegaPhase>& table = with_att ? ctx->phases_att : ctx->phases;
-        int ticket0 = 0;
-        auto add = [&](const GemmW& g, int mode, const uint32_t* xf) -> MegaPhase& {
-            MegaPhase ph = {};
-            ph.W = g.packed_u;
-            ph.xf = (const uint4*)xf;
-            ph.mode = mode;
-            mega_phase_geometry(ph, g.N, g.K);
-            ph.ticket0 = ticket0;
-            ticket0 += ph.UB;
-            table.push_back(ph);
-            return table.back();
-        };
-        for (int l = 0; l < c.n_layers; ++l) {
-            const LayerW& lw = ctx->layers[l];
-            {
-                MegaPhase& ph = add(lw.qkv, kQkvRope, xf_h);
-                ph.ssq_in = ssqA; ph.n_ssq = n_ssq; ph.layer = l;
-            }
-            if (with_att) {
-                MegaPhase ph = {};
-                ph.mode = kPhaseAttn;
-                ph.UB = c.n_kv_heads;          // one unit per KV head; tiles per head come with each launch
-                ph.layer = l;
-                ph.xf_out = (uint16_t*)xf_attn;
-                ph.ticket0 = ticket0;
-                ticket0 += ph.UB;
-                table.push_back(ph);
-            }
-            {
-                MegaPhase& ph = add(lw.o, kResid, xf_attn);
-                ph.x = x; ph.xf_out = (uint16_t*)xf_h; ph.gain_next = lw.n2; ph.ssq_out = ssqB;
-            }
-            {
-                MegaPhase& ph = add(lw.gu, kSwiglu, xf_h);
-                ph.ssq_in = ssqB; ph.n_ssq = n_ssq; ph.xf_out = (uint16_t*)xf_act;
-            }
-            {
-                MegaPhase& ph = add(lw.dn, kResid, xf_act);
-                ph.x = x; ph.xf_out = (uint16_t*)xf_h;
-                ph.gain_next = l + 1 < c.n_layers ? ctx->layers[l + 1].n1 : ctx->final_norm;
-                ph.ssq_out = ssqA;
-            }
-        }
-        {
-            MegaPhase& ph = add(ctx->lm, kPlain, xf_h);
-            ph.ssq_in = ssqA; ph.n_ssq = n_ssq; ph.out = ctx->W<float>(ctx->ws.logits);
-        }
-        if ((size_t)ticket0 + table.size() + c.n_layers + 2 > ctx->ws.mega_ctr_ints) return bail(PIPESD_E_INVALID);
-        if (cudaMemcpyAsync(ctx->wsp + (with_att ? ctx->ws.mega_phases_att : ctx->ws.mega_phases), table.data(),
-                            sizeof(MegaPhase) * table.size(), cudaMemcpyHostToDevice, st) != cudaSuccess)
-            return bail(PIPESD_E_CUDA);
-        }
-        if (cudaStreamSynchronize(st) != cudaSuccess) return bail(PIPESD_E_CUDA);   // the table is read from pageable memory
-    }
 
     ctx->reqs.resize(c.max_requests);
     ctx->free_pages.resize(c.n_pages);
@@ -1252,15 +1071,6 @@ int32_t pipesd_debug_wait_timeout(pipesd_ctx* ctx, int32_t limit_us) {
     wait_never_kernel<<<1, 32, 0, ctx->st>>>(ctx->W<int>(ctx->ws.never_flag), ctx->err_word(), (unsigned long long)limit_us * 1000ull);
     CU(cudaGetLastError());
     return push_inflight(ctx, nullptr, {});
-}
-
-int32_t pipesd_debug_set_engine(pipesd_ctx* ctx, int32_t engine) {
-    if (!ctx || engine < 0 || engine > 2) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_set_engine");
-    if (engine == 1 && !needs_tiled(ctx->cfg))
-        return fail(ctx, PIPESD_E_INVALID,
-                    "pipesd_debug_set_engine: this context keeps no weights in the tiled kernels' order (persistent engine, max_rows <= 32)");
-    ctx->engine = engine;
-    return PIPESD_OK;
 }
 
 int32_t pipesd_profile_enable(pipesd_ctx* ctx, int32_t time_gemms) {

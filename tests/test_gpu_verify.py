@@ -7,7 +7,6 @@ from paper_2605_13319_b200 import synth
 from harness import LOGIT_TOL, Tally, draft_inputs, logit_rel_err
 
 pytestmark = pytest.mark.gpu
-ENGINES = pytest.mark.parametrize("engine", ["tiled", "persistent"])
 
 
 def _mk(shape, seed, P, n_pages=None, **kw):
@@ -20,13 +19,11 @@ def _mk(shape, seed, P, n_pages=None, **kw):
     return w, ctx, orc
 
 
-@ENGINES
-def test_tiny_config_many_seeds(engine):
-    """2 layers, d 256, 4 heads x 64, FFN 688, vocab 1024; P=64, k=4, sigma=1; stochastic and greedy.
-    With the persistent engine every verify here is ONE launch (attention inside the kernel)."""
+def test_tiny_config_many_seeds():
+    """2 layers, d 256, 4 heads x 64, FFN 688, vocab 1024; P=64, k=4, sigma=1; stochastic and greedy."""
     from paper_2605_13319_b200 import binding
     shape, P, k = synth.TINY, 64, 4
-    w, ctx, orc = _mk(shape, 0, P, engine=engine)
+    w, ctx, orc = _mk(shape, 0, P)
     tally, gt = Tally(), Tally()
     prefix = synth.make_prefix(shape, P, 0)
     orc.prefill(prefix)
@@ -73,16 +70,14 @@ def test_tiny_config_many_seeds(engine):
     ctx.close()
 
 
-@ENGINES
-def test_multi_round_verify_rollback_lockstep(engine):
+def test_multi_round_verify_rollback_lockstep():
     """Rounds of verify + rollback: the cache grows by n_accepted+1 and is truncated each round; the checker
     leads (its decision is committed on both sides) so a counted near-tie cannot desynchronise later rounds.
-    Two query heads per KV head and k up to 8: with the persistent engine the rounds alternate between attention
-    inside the kernel (at most 16 query rows per KV head) and attention as its own kernel."""
+    Two query heads per KV head and k up to 8: 4 to 18 query rows per KV head (one or two 16-row column blocks)."""
     from paper_2605_13319_b200 import binding
     shape = synth.TINY.scaled(name="tiny-gqa", n_kv_heads=2)
     P, rounds = 37, 24                       # prefix not a multiple of the page size
-    w, ctx, orc = _mk(shape, 1, P, max_seq=P + rounds * 9 + 16, engine=engine)
+    w, ctx, orc = _mk(shape, 1, P, max_seq=P + rounds * 9 + 16)
     prefix = synth.make_prefix(shape, P, 1)
     orc.prefill(prefix)
     req = ctx.req_open()
@@ -108,18 +103,15 @@ def test_multi_round_verify_rollback_lockstep(engine):
     ctx.close()
 
 
-@ENGINES
-def test_batched_ragged_verify_and_batch_invariance(engine):
-    """Several requests with different prefix lengths and draft counts in ONE call == each alone == checker.
-    The bit-for-bit comparison holds on one set of kernels: the batch (more than 32 rows) runs on the tiled ones,
-    so under the persistent engine the single requests are switched to them as well."""
+def test_batched_ragged_verify_and_batch_invariance():
+    """Several requests with different prefix lengths and draft counts in ONE call == each alone == checker."""
     from paper_2605_13319_b200 import binding
     shape = synth.TINY.scaled(name="tiny-gqa", n_kv_heads=2)
     n_req = 6
     lens, ks, sig = synth.ragged_requests(3, n_req, 5, 150, 1, 16)
     w = synth.make_weights(shape, 2)
     ctx = binding.Context(shape, w, n_pages=(200 // 16 + 2) * n_req * 2, max_seq=200, max_requests=2 * n_req,
-                          max_rows=max(33, int(ks.sum() + n_req)), max_draft=16, engine=engine, poison=True)
+                          max_rows=max(33, int(ks.sum() + n_req)), max_draft=16, poison=True)
     assert int(ks.sum() + n_req) > 32
     tally = Tally()
     items, refs, solo = [], [], []
@@ -135,7 +127,6 @@ def test_batched_ragged_verify_and_batch_invariance(engine):
             bank.append(dict(req=req, tokens=toks, q=q, u=u))
     got = ctx.verify(items, flags=binding.Q_HOST)
     logits = ctx.debug_get_logits(int(ks.sum() + n_req))
-    ctx.debug_set_engine(1)
     row = 0
     for i in range(n_req):
         ref, q, u = refs[i]
@@ -152,17 +143,16 @@ def test_batched_ragged_verify_and_batch_invariance(engine):
     ctx.close()
 
 
-@ENGINES
-def test_draft_lengths_across_token_tile_counts(engine):
+def test_draft_lengths_across_token_tile_counts():
     """k = 1, 7, 8, 15, 16, 31 (the maximum): 2, 8, 9, 16, 17 and 32 rows per pass, i.e. one to four 8-token
-    tiles in the GEMMs and, with the persistent engine, both sides of the 16-query-row limit up to which
-    attention runs inside the kernel.  Prefix lengths straddle page and 64-key tile boundaries."""
+    tiles in the GEMMs and one or two 16-row column blocks in attention.  Prefix lengths straddle page and 128-key
+    tile boundaries."""
     from paper_2605_13319_b200 import binding
     shape = synth.TINY
     w = synth.make_weights(shape, 5)
     tally = Tally()
-    for n, (k, P) in enumerate(((1, 1), (7, 63), (8, 64), (15, 65), (16, 127), (31, 130))):
-        ctx = binding.Context(shape, w, n_pages=16, max_seq=200, max_draft=31, engine=engine, poison=True)
+    for n, (k, P) in enumerate(((1, 1), (7, 63), (8, 127), (15, 128), (16, 129), (31, 130))):
+        ctx = binding.Context(shape, w, n_pages=16, max_seq=200, max_draft=31, poison=True)
         orc = oracle.Oracle(shape, w, 200)
         prefix = synth.make_prefix(shape, P, 5, request=n)
         orc.prefill(prefix)
@@ -186,18 +176,16 @@ def test_draft_lengths_across_token_tile_counts(engine):
     assert tally.max_logit_err < 1e-3
 
 
-@ENGINES
-def test_page_sizes_other_than_16(engine):
-    """Pages of 8, 24, 32, 64 and 128 positions: a 64-key attention tile then covers eight pages, straddles pages
-    unevenly, covers two, one, or half of one; the appended rows land across page boundaries.  (The persistent
-    engine runs attention inside its kernel only for 16-position pages: here it uses the separate kernel.)"""
+def test_page_sizes_other_than_16():
+    """Pages of 8, 24, 32, 64, 128 and 256 positions: a 128-key attention tile then covers sixteen pages, straddles
+    pages unevenly, covers four, two, one, or half of one; the appended rows land across page boundaries."""
     from paper_2605_13319_b200 import binding
     shape = synth.TINY
     w = synth.make_weights(shape, 6)
     tally = Tally()
-    for n, (ps, P, k) in enumerate(((8, 150, 5), (24, 101, 8), (32, 193, 3), (64, 130, 8), (128, 200, 12))):
+    for n, (ps, P, k) in enumerate(((8, 150, 5), (24, 101, 8), (32, 193, 3), (64, 130, 8), (128, 200, 12), (256, 300, 7))):
         ctx = binding.Context(shape, w, n_pages=(P + 48) // ps + 3, max_seq=P + 40, max_draft=16, page_size=ps,
-                              engine=engine, poison=True)
+                              poison=True)
         orc = oracle.Oracle(shape, w, P + 40)
         prefix = synth.make_prefix(shape, P, 6, request=n)
         orc.prefill(prefix)
