@@ -250,6 +250,30 @@ int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scra
 int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t *resident_clusters,
                                 int32_t clusters_needed, int32_t *out3);
 
+/* ---- the edge-side scheduling model (host code only; no device work) ----
+ *
+ * The verify pass above is what the cloud runs; what decides WHEN it runs and how the draft tokens reach it is the
+ * edge's token-batch pipeline (Sec. 3.2) and its dual-threshold trigger (Sec. 3.3).  These calls make that model
+ * available behind the same ABI.  Times are in any one unit (the paper uses milliseconds). */
+
+/* T of Eq. 6 for the batching B = (b_1 = 1 < b_2 < ... < b_K <= N) of Eq. 1 (boundaries: host, K entries; b_k is the
+ * index of the first draft token of batch k): with t_c = alpha + beta * n and t_ag = gamma * n for a batch of n tokens
+ * (Eq. 2, 3), a batch's generation starts when the previous one's ends (Eq. 4), its transmission when both its own
+ * generation and the previous transmission have ended (Eq. 5); T is the end of the last transmission.
+ * PIPESD_E_INVALID if B is not such a sequence. */
+int32_t pipesd_sched_round_time(int32_t N, double alpha, double beta, double gamma, const int32_t *boundaries,
+                                int32_t K, double *T);
+/* The batching that minimises T (Sec. 4.1, Algorithm 1; optimal by Theorem 4.1): a dynamic programme over the
+ * prefixes of the N draft tokens, O(N^2).  boundaries (host, room for N entries) receives b_1..b_K, *K their number,
+ * *T (nullable) the minimal time.  Among equally good batchings the one the recurrence meets first is returned. */
+int32_t pipesd_sched_optimal_batching(int32_t N, double alpha, double beta, double gamma, int32_t *boundaries,
+                                      int32_t *K, double *T);
+/* One step of the dual-threshold trigger (Sec. 3.3) for a draft token of confidence p = P(D_n): the tentative
+ * cumulative confidence is C1* = C1 * p; verification is triggered (*fire = 1) if C1* <= R1 or p <= R2.  *c1 (in/out,
+ * 1 at the start) is the product over the draft tokens not yet sent to verification: it becomes 1 after a trigger
+ * and C1* otherwise. */
+int32_t pipesd_sched_trigger_step(double *c1, double R1, double R2, double p, int32_t *fire);
+
 /* The same GEMM for callers that cannot allocate device memory.  (The paper has no counterpart: this
  * is a convenience of the library, not a step of the method.)
  *

@@ -90,6 +90,12 @@ _SIGNATURES = {
     "pipesd_gemm_pack": (i32, [vp, vp, i32, i32, vp]),
     "pipesd_gemm_run": (i32, [vp, vp, vp, vp, i32, i32, i32, vp]),
     "pipesd_gemm_run_static": (i32, [vp, vp, vp, i32, i32, i32, vp]),
+    "pipesd_sched_round_time": (i32, [i32, ctypes.c_double, ctypes.c_double, ctypes.c_double, vp, i32,
+                                      ctypes.POINTER(ctypes.c_double)]),
+    "pipesd_sched_optimal_batching": (i32, [i32, ctypes.c_double, ctypes.c_double, ctypes.c_double, vp,
+                                            ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double)]),
+    "pipesd_sched_trigger_step": (i32, [ctypes.POINTER(ctypes.c_double), ctypes.c_double, ctypes.c_double,
+                                        ctypes.c_double, ctypes.POINTER(i32)]),
     "pipesd_debug_attn_split": (i32, [i32, i32, ctypes.POINTER(ctypes.c_int32), i32, ctypes.POINTER(ctypes.c_int32)]),
     "pipesd_debug_req_state": (i32, [vp, i32, ctypes.POINTER(ctypes.c_int32)]),
     "pipesd_debug_wait_timeout": (i32, [vp, i32]),
@@ -370,3 +376,34 @@ def debug_attn_split(total_keys: int, page_size: int, resident_clusters, cluster
     if rc != 0:
         raise PipesdError(rc, "pipesd_debug_attn_split")
     return tuple(out)
+
+
+# ---- the edge-side scheduling model (host code of the library)
+def sched_round_time(N: int, alpha: float, beta: float, gamma: float, boundaries) -> float:
+    b = np.ascontiguousarray(boundaries, np.int32)
+    T = ctypes.c_double()
+    rc = lib().pipesd_sched_round_time(N, alpha, beta, gamma, _np_ptr(b), b.size, ctypes.byref(T))
+    if rc != OK:
+        raise PipesdError(rc, "pipesd_sched_round_time")
+    return T.value
+
+
+def sched_optimal_batching(N: int, alpha: float, beta: float, gamma: float):
+    """(boundaries b_1..b_K as a tuple, minimal T)."""
+    b = np.zeros(max(N, 1), np.int32)
+    K = i32()
+    T = ctypes.c_double()
+    rc = lib().pipesd_sched_optimal_batching(N, alpha, beta, gamma, _np_ptr(b), ctypes.byref(K), ctypes.byref(T))
+    if rc != OK:
+        raise PipesdError(rc, "pipesd_sched_optimal_batching")
+    return tuple(int(x) for x in b[:K.value]), T.value
+
+
+def sched_trigger_step(c1: float, R1: float, R2: float, p: float):
+    """(triggered?, C1 after the step)."""
+    c = ctypes.c_double(c1)
+    fire = i32()
+    rc = lib().pipesd_sched_trigger_step(ctypes.byref(c), R1, R2, p, ctypes.byref(fire))
+    if rc != OK:
+        raise PipesdError(rc, "pipesd_sched_trigger_step")
+    return bool(fire.value), c.value

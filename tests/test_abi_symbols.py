@@ -46,14 +46,15 @@ def test_pure_host_entry_points():
 def test_attention_key_split_plan():
     """The split of a request's keys over clusters and CTAs: a function of the request alone."""
     wide = (48, 45, 41)            # clusters of 8, 9, 10 the device keeps resident (a B200, one query row tile)
-    # 2057 keys: 8 splits of 272 keys are five 64-key tiles per CTA, 9 splits of 240 are four, 10 no fewer
+    # 2057 keys: 8 splits of 272 keys are three 128-key tiles per CTA, 9 splits of 240 are two, 10 no fewer
     assert binding.debug_attn_split(2057, 16, wide, 32) == (1, 9, 240)
     # the wider cluster must still hold the whole request in one wave
     assert binding.debug_attn_split(2057, 16, (48, 31, 31), 32) == (1, 8, 272)
     assert binding.debug_attn_split(2057, 16, (48, 0, 0), 32) == (1, 8, 272)          # widths unavailable
-    assert binding.debug_attn_split(2057, 16, (48, 31, 41), 32) == (1, 10, 208)       # 9 does not fit, 10 does: four tiles
-    # 521 keys: 9 splits of 64 keys are one tile each, 8 splits of 80 are two
-    assert binding.debug_attn_split(521, 16, wide, 8) == (1, 9, 64)
+    assert binding.debug_attn_split(2057, 16, (48, 31, 41), 32) == (1, 10, 208)       # 9 does not fit, 10 does: two tiles
+    # 1030 keys: 9 splits of 128 keys are one tile each, 8 splits of 144 are two; 521 keys: one tile either way
+    assert binding.debug_attn_split(1030, 16, wide, 8) == (1, 9, 128)
+    assert binding.debug_attn_split(521, 16, wide, 8) == (1, 8, 80)
     # short requests: nothing to gain, stay at eight; splits are whole pages
     assert binding.debug_attn_split(9, 16, wide, 8) == (1, 8, 16)
     assert binding.debug_attn_split(100, 8, wide, 8) == (1, 8, 16)
@@ -71,7 +72,7 @@ def test_attention_key_split_plan():
             assert (w == 8) or ncl == 1
             if w > 8:   # widened only for fewer tiles per CTA
                 c8 = -(-(-(-total // 8)) // ps) * ps
-                assert -(-chunk // 64) < -(-c8 // 64)
+                assert -(-chunk // 128) < -(-c8 // 128)
     import pytest
     with pytest.raises(binding.PipesdError):
         binding.debug_attn_split(100, 12, wide, 8)
