@@ -241,14 +241,19 @@ int32_t pipesd_gemm_pack(const void *W, void *packed, int32_t N, int32_t K, void
 int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scratch, int32_t M, int32_t N,
                         int32_t K, void *cuda_stream);
 
+/* CTAs of the attention kernel that the context's device keeps resident at once for a request with this many query
+ * rows per KV head: out2 (host) = {with the whole third ring slot, with the cut-down one} -- the two numbers
+ * pipesd_debug_attn_split takes. */
+int32_t pipesd_debug_attn_slots(pipesd_ctx *ctx, int32_t rows_per_kv_head, int32_t *out2);
 /* Host only, no CUDA call: how the attention kernel splits a request of `total_keys` keys (cached + this pass's
- * rows) at the given page size (tiles of 128 keys).  resident_clusters[0..2] (host) = thread-block clusters of 8, 9 and 10 CTAs the
- * device keeps resident at once for the request's footprint (0 = that width is unavailable), clusters_needed =
- * clusters one layer launches for the request (KV heads x row groups).  out3 (host) receives {clusters sharing the
- * keys, key splits per cluster, keys per split (a multiple of page_size)}.  The split is a function of the request
- * alone, which is what keeps a request's result independent of its batch.  PIPESD_E_INVALID on bad arguments. */
-int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t *resident_clusters,
-                                int32_t clusters_needed, int32_t *out3);
+ * rows) at the given page size into CTAs that each walk tiles of 128 keys.  resident_ctas[0..1] (host) = CTAs of the
+ * kernel the device keeps resident at once for the request's footprint, without and with the cut-down third slot of
+ * the K/V ring; units = CTA groups one layer launches for the request (KV heads x row groups).  out3 (host) receives
+ * {key splits, keys per split (a multiple of page_size), 1 if the cut-down ring suffices}.  The split is a function
+ * of the request and the device alone, which is what keeps a request's result independent of its batch.
+ * PIPESD_E_INVALID on bad arguments. */
+int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t *resident_ctas, int32_t units,
+                                int32_t *out3);
 
 /* ---- the edge-side scheduling model (host code only; no device work) ----
  *

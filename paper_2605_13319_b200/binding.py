@@ -96,6 +96,7 @@ _SIGNATURES = {
                                             ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double)]),
     "pipesd_sched_trigger_step": (i32, [ctypes.POINTER(ctypes.c_double), ctypes.c_double, ctypes.c_double,
                                         ctypes.c_double, ctypes.POINTER(i32)]),
+    "pipesd_debug_attn_slots": (i32, [vp, i32, ctypes.POINTER(ctypes.c_int32)]),
     "pipesd_debug_attn_split": (i32, [i32, i32, ctypes.POINTER(ctypes.c_int32), i32, ctypes.POINTER(ctypes.c_int32)]),
     "pipesd_debug_req_state": (i32, [vp, i32, ctypes.POINTER(ctypes.c_int32)]),
     "pipesd_debug_wait_timeout": (i32, [vp, i32]),
@@ -278,6 +279,11 @@ class Context:
         self._check(lib().pipesd_debug_req_state(self._h, req, out), "pipesd_debug_req_state")
         return tuple(out)
 
+    def debug_attn_slots(self, rows_per_kv_head: int):
+        out = (ctypes.c_int32 * 2)()
+        self._check(lib().pipesd_debug_attn_slots(self._h, rows_per_kv_head, out), "pipesd_debug_attn_slots")
+        return tuple(out)
+
     def debug_wait_timeout(self, limit_us: int):
         self._check(lib().pipesd_debug_wait_timeout(self._h, limit_us), "pipesd_debug_wait_timeout")
 
@@ -368,11 +374,11 @@ def gemm_run_static(packed, x, y, N, K, stream=None):
         raise PipesdError(rc, "pipesd_gemm_run_static")
 
 
-def debug_attn_split(total_keys: int, page_size: int, resident_clusters, clusters_needed: int):
-    """(clusters sharing the keys, key splits per cluster, keys per split) of one request: host arithmetic only."""
-    res = (ctypes.c_int32 * 3)(*[int(x) for x in resident_clusters])
+def debug_attn_split(total_keys: int, page_size: int, resident_ctas, units: int):
+    """(key splits, keys per split, cut-down ring?) of one request: host arithmetic only."""
+    res = (ctypes.c_int32 * 2)(*[int(x) for x in resident_ctas])
     out = (ctypes.c_int32 * 3)()
-    rc = lib().pipesd_debug_attn_split(total_keys, page_size, res, clusters_needed, out)
+    rc = lib().pipesd_debug_attn_split(total_keys, page_size, res, units, out)
     if rc != 0:
         raise PipesdError(rc, "pipesd_debug_attn_split")
     return tuple(out)

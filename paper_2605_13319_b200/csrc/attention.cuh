@@ -1,28 +1,28 @@
 // Multi-query decode attention over a paged bf16 KV cache on the tcgen05 tensor cores: each request contributes a
 // short chunk of query rows (the pending token plus its k drafts) that attend to the cached prefix and, causally,
-// to each other.  The keys are cut into 8 to 10 splits ("split-K") handled by the CTAs of a thread-block cluster;
-// every CTA produces an un-normalised partial output with its reference maximum and sum in its own shared memory,
-// and after a cluster barrier the partials are merged over distributed shared memory and written straight into the
-// output projection's input format -- no partial results in global memory and no separate merge kernel (requests
-// of 4096 keys and more use several clusters and one more merge step).  Tiles of keys that were cached before
-// this pass do not depend on the preceding QKV projection, so their copies are issued before the dependent-launch
-// wait.
+// to each other.  The keys of a request are cut into up to 16 splits ("split-K"), one CTA each; a CTA leaves an
+// un-normalised partial output with its reference maximum and sum in global memory (a few MB that stay in L2),
+// takes a ticket, and the last CTA of a (request, KV head, row group) to arrive merges the splits in split order
+// and writes the result straight into the output projection's input format -- nobody waits for anybody, and a CTA
+// that is not the last one leaves its SM to the next kernel at once.
 //
-// One CTA = one KV head of one request x one key split x up to 128 query rows, where the rows are all (query head
+// One CTA = one KV head of one request x one key split x up to 112 query rows, where the rows are all (query head
 // of the group, chunk row) pairs that share the KV head (GQA).  The keys are on the M side of the MMAs, the (few)
 // query rows on the narrow N side:
 //   S^T[128 keys x N rows] = K_tile[128 x hd] . Q^T[hd x N]          A = K rows from the cache, B = Q
 //   O^T[hd x N rows]      += V_tile^T[hd x 128 keys] . P^T[128 x N]   A = V rows from the cache, B = P
 //   L  [  * x N rows]      += 1[* x 128 keys] . P^T[128 x N]          the softmax denominators, by the same P
-// with S^T, O^T and L in tensor memory (3N columns).  The cache stores, per page and head, the rows in 8-row groups
-// of 8-element pieces ([slot/8][hd/8][slot%8][8]), which IS the operand order of both products (K-major for the
-// first, MN-major for the second): a page lands in shared memory by one bulk copy and is read by the tensor cores
-// as it is.  Q and P are fp32 values split into bf16 hi + lo terms (two MMAs into the same accumulator); K and V
-// are the cache's bf16.
-// Warps 0-3 (one thread per key of a tile, i.e. per tensor-memory lane): masking, the running maximum (a row's
-// reference maximum only moves when the tile's maximum exceeds it by more than 2^8, so that O^T is rarely
-// rescaled), exponentials, P written back as the next MMA's B operand.  Warp 4: bulk copies of the K/V pages and
-// the MMA issue (one thread).  Every wait is bounded and raises the device error word.
+// with S^T (twice: two tiles in flight), O^T and L in tensor memory (4N columns).  The cache stores, per page and
+// head, the rows in 8-row groups of 8-element pieces ([slot/8][hd/8][slot%8][8]), which IS the operand order of
+// both products (K-major for the first, MN-major for the second): a page lands in shared memory by one bulk copy
+// and is read by the tensor cores as it is.  Q and P are fp32 values split into bf16 hi + lo terms (two MMAs into
+// the same accumulator); K and V are the cache's bf16.
+// Warps 0-7: one thread per key of a tile (= tensor-memory lane; warps w and w+4 share a lane quarter and take
+// alternate 16-row column blocks): masking, the running maximum (a row's reference maximum only moves when the
+// tile's maximum exceeds it by more than 2^8, so that O^T is rarely rescaled), exponentials, P written back as the
+// next MMA's B operand.  Warp 8: bulk copies of the K/V pages (a ring of three slots, K0 V0 K1 V1 ...; tiles of keys
+// that were cached before this pass do not depend on the preceding QKV projection and are requested before the
+// dependent-launch wait) and the MMA issue (one thread).  Every wait is bounded and raises the device error word.
 #pragma once
 #include "common.cuh"
 #include "layers.cuh"
@@ -30,11 +30,12 @@
 
 namespace pipesd {
 
-constexpr int kAttnWorkers = 128;           // threads of warps 0-3
+constexpr int kAttnWorkers = 256;           // threads of warps 0-7
 constexpr int kAttnThreads = kAttnWorkers + 32;
 constexpr int kAttnTile = 128;              // keys per tile = M of the MMAs
-constexpr int kAttnMaxRows = 128;           // query rows per CTA (N of the MMAs); more rows: more row groups
-constexpr int kAttnPagesSmem = 512;         // page ids of a CTA's key range kept in shared memory (longer ranges read the table)
+constexpr int kAttnMaxRows = 112;           // query rows per CTA (N of the MMAs; what fits beside the ring); more rows: more row groups
+constexpr int kAttnMaxSplits = 16;          // key splits of one request
+constexpr int kAttnShortTail = 112;         // keys of the second tile up to which the third ring slot is cut down
 constexpr float kAttnLazyRescale = 8.f;     // log2 units by which a tile's maximum may exceed the reference maximum
 
 // Wait for a barrier phase.  Bounded by a try count (each try suspends for a hardware-chosen time; 2^22 of them take
@@ -51,7 +52,6 @@ __device__ __forceinline__ bool attn_wait(uint32_t bar, uint32_t parity) {
     }
     return false;
 }
-
 // The same for a whole warp: every lane waits, and the warp agrees on the outcome (the collective tensor-memory
 // instructions that follow need a warp-uniform control flow).
 __device__ __forceinline__ bool attn_wait_warp(uint32_t bar, uint32_t parity) {
@@ -64,32 +64,35 @@ __device__ __forceinline__ float fast_exp2(float x) {   // 2^x, relative error 2
     return y;
 }
 
-// Shared-memory plan of one CTA with N query rows (a multiple of 16).
+// Shared-memory plan of one CTA with N query rows (a multiple of 16).  K and V tiles travel through a ring of three
+// slots in the order K0 V0 K1 V1 ...: two of a whole tile each and a third of `slot_c` bytes (a whole tile, or less
+// when no CTA of the launch has more than two tiles, the second of at most kAttnShortTail keys: the K/V of such a
+// CTA are then requested in full before the first product starts).
 template <int HD>
 struct AttnSmem {
     static constexpr int kTileBytes = kAttnTile * HD * 2;            // one K or V tile
-    static constexpr int kOnes = 4096;                                // 128 x 16 ones (the denominators' A operand)
-    static constexpr int kSmall = 4 * kAttnMaxRows * 4               // warp maxima [4][128]
-                                  + 4 * kAttnMaxRows * 4             // horizon, reference maximum, rescale factor, Fl
-                                  + 128;                             // barriers, tensor-memory base, flags
+    static constexpr int kOnes = 256;                                 // 16 keys x 8 ones: the denominators' A operand
     __host__ __device__ static constexpr int q_bytes(int N) { return N * HD * 2; }          // hi or lo
     __host__ __device__ static constexpr int p_bytes(int N) { return kAttnTile * N * 2; }   // hi or lo
-    __host__ __device__ static constexpr size_t bytes(int N) {
-        return (size_t)2 * kTileBytes + 2 * q_bytes(N) + 2 * p_bytes(N) + kOnes + kSmall;
+    __host__ __device__ static constexpr int small_bytes(int N) { return 8 * N * 4 + 128; } // warp maxima [4][N], horizon, reference
+                                                                                            // maximum, factor, sums [N] each; barriers
+    __host__ __device__ static constexpr size_t bytes(int N, int slot_c) {
+        return (size_t)kOnes + 2 * kTileBytes + slot_c + 2 * q_bytes(N) + 2 * p_bytes(N) + small_bytes(N);
     }
 };
 
-// Tensor-memory columns of a CTA with N query rows: S^T, O^T and L, N columns each, as a power of two >= 32.
+// Tensor-memory columns of a CTA with N query rows: S^T twice, O^T and L, N columns each, as a power of two >= 32.
 __host__ __device__ constexpr int attn_tmem_cols(int N) {
     int c = 32;
-    while (c < 3 * N) c *= 2;
+    while (c < 4 * N) c *= 2;
     return c;
 }
+static inline int attn_slot_c_bytes(int hd, bool short_tail) { return (short_tail ? kAttnShortTail : kAttnTile) * hd * 2; }
 // Dynamic shared memory to ask for: the plan above, padded so that the CTAs an SM can hold never want more than the
-// SM's 512 tensor-memory columns together (a CTA that waited for columns held by a CTA waiting at a cluster barrier
-// could otherwise wait for ever).
-static inline size_t attn_smem_bytes(int hd, int N) {
-    const size_t need = hd == 128 ? AttnSmem<128>::bytes(N) : AttnSmem<64>::bytes(N);
+// SM's 512 tensor-memory columns together (the allocation instruction blocks until its columns are free).
+static inline size_t attn_smem_bytes(int hd, int N, bool short_tail) {
+    const int sc = attn_slot_c_bytes(hd, short_tail);
+    const size_t need = hd == 128 ? AttnSmem<128>::bytes(N, sc) : AttnSmem<64>::bytes(N, sc);
     const int max_ctas = 512 / attn_tmem_cols(N);
     const size_t floor_ = (size_t)(227 * 1024) / (max_ctas + 1) + 1;
     return need > floor_ ? need : floor_;
@@ -99,61 +102,62 @@ static inline int attn_rows_n(int rows_per_kv_head) {    // N of a CTA that hold
     return (r + 15) / 16 * 16;
 }
 
+// Host: how one request's keys are split.  `units` = CTA groups the request launches per layer (KV heads x row
+// groups); slots[0 | 1] = CTAs of this kernel the device keeps resident at once for the request's row count with the
+// whole | cut-down third ring slot.  As many splits as let all of the request's CTAs run in one wave (at most 16, at
+// most one per 128 keys), then the fewest splits that leave each CTA the same number of 128-key tiles.  A function
+// of the request and the device alone, never of the batch: a request's summation order is the same in every batch.
+struct AttnSplit { int splits, keys_per_split, short_tail; };
+static inline AttnSplit attn_split_plan(int total_keys, int page_size, int units, const int* slots) {
+    auto chunk_of = [&](int s) {
+        const int ch = (total_keys + s - 1) / s;
+        return (ch + page_size - 1) / page_size * page_size;
+    };
+    auto tiles_of = [&](int s) { return (chunk_of(s) + kAttnTile - 1) / kAttnTile; };
+    const int by_keys = (total_keys + kAttnTile - 1) / kAttnTile;
+    AttnSplit p = {1, chunk_of(1), 0};
+    for (int cls = 1; cls >= 0; --cls) {
+        int s = slots[cls] / (units > 0 ? units : 1);
+        s = s > kAttnMaxSplits ? kAttnMaxSplits : s;
+        s = s > by_keys ? by_keys : s;
+        s = s < 1 ? 1 : s;
+        const int t = tiles_of(s);
+        while (s > 1 && tiles_of(s - 1) == t) --s;
+        p.splits = s;
+        p.keys_per_split = chunk_of(s);
+        p.short_tail = cls;
+        if (cls == 0 || p.keys_per_split <= kAttnTile + kAttnShortTail) break;
+    }
+    return p;
+}
+
 // Per-CTA constants of the tile copies.
 struct AttnCtx {
     const uint16_t* kbase;     // K block of page 0 for this layer and KV head
-    const int32_t* bt;         // page ids of the request, indexed from bt_first: shared-memory copy of the CTA's range, or the table
-    int bt_first;
+    const int32_t* bt;         // page ids of the request
     size_t page_stride;        // elements between consecutive pages of a layer
     size_t v_off;              // elements from a K block to the V block of the same page and head
     int page_size;
     int k0, k1;
 };
 
-// Issue (one warp) the copies of one 128-key tile: the rows of a page that belong to one KV head are contiguous in
-// the pool, already in operand order, so every page the tile touches is one bulk copy of K rows (lanes 0-15, one
-// page each) and one of V rows (lanes 16-31), counted in bytes on the barrier.  Whole 8-row groups are copied: the
-// rows of the last group at or beyond k1 are masked (K) and cleared (V) by the consumers.
+// Issue (one warp) the copies of the K rows (kv = 0) or V rows (kv = 1) of one 128-key tile: the rows of a page that
+// belong to one KV head are contiguous in the pool, already in operand order, so every page the tile touches is one
+// bulk copy (lane l takes the l-th page), counted in bytes on the barrier.  Whole 8-row groups are copied: the rows
+// of the last group at or beyond k1 are masked (K) or cleared (V) by the consumers.
 template <int HD>
-__device__ __forceinline__ void attn_issue_tile(const AttnCtx& c, uint32_t k_addr, uint32_t v_addr, uint32_t bar, int j0) {
+__device__ __forceinline__ void attn_issue_tile(const AttnCtx& c, int kv, uint32_t dst, uint32_t bar, int j0) {
     const int lane = threadIdx.x & 31;
     const int j1 = (min(j0 + kAttnTile, c.k1) + 7) & ~7;
-    if (lane == 0) mbar_expect_tx(bar, (uint32_t)(j1 - j0) * (HD * 2) * 2);
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)(j1 - j0) * (HD * 2));
     __syncwarp();
-    const int kv = lane >> 4;
-    for (int pg = lane & 15; ; pg += 16) {
-        const int pidx = j0 / c.page_size + pg;                            // page of the request
-        const int js = max(j0, pidx * c.page_size), je = min(j1, (pidx + 1) * c.page_size);
-        if (js >= je) break;
-        const uint16_t* src = c.kbase + (size_t)c.bt[pidx - c.bt_first] * c.page_stride + (kv ? c.v_off : 0) +
+    const int pidx = j0 / c.page_size + lane;                              // page of the request
+    const int js = max(j0, pidx * c.page_size), je = min(j1, (pidx + 1) * c.page_size);
+    if (js < je) {
+        const uint16_t* src = c.kbase + (size_t)c.bt[pidx] * c.page_stride + (kv ? c.v_off : 0) +
                               (size_t)(js - pidx * c.page_size) * HD;
-        bulk_g2s((kv ? v_addr : k_addr) + (uint32_t)(js - j0) * (HD * 2), src, (uint32_t)(je - js) * (HD * 2), bar);
+        bulk_g2s(dst + (uint32_t)(js - j0) * (HD * 2), src, (uint32_t)(je - js) * (HD * 2), bar);
     }
-}
-
-constexpr int kAttnSplits = 8;        // key splits per cluster of a request whose keys several clusters share
-constexpr int kAttnMaxCluster = 10;   // largest cluster along x (above 8: the non-portable sizes, opted into by the host)
-
-// Host: how one request's keys are split.  `resident[w - 8]` = clusters of width w (8, 9, 10) the device keeps
-// resident at once for this request's shared-memory footprint (0: width unavailable); `need` = clusters the request
-// launches per layer (KV heads x row groups).  One cluster of eight per 2048 keys up to four clusters; a single
-// cluster widens to the smallest width that leaves each CTA the fewest 128-key tiles, as long as all the request's
-// clusters still run in one wave.  Everything here depends on the request alone, never on its batch.
-struct AttnSplit { int clusters, width, keys_per_split; };
-static inline AttnSplit attn_split_plan(int total_keys, int page_size, const int* resident, int need) {
-    AttnSplit p;
-    p.clusters = total_keys / 2048 < 1 ? 1 : (total_keys / 2048 > kMaxSplits / kAttnSplits ? kMaxSplits / kAttnSplits : total_keys / 2048);
-    p.width = kAttnSplits;
-    auto chunk_of = [&](int splits) {
-        const int ch = (total_keys + splits - 1) / splits;
-        return (ch + page_size - 1) / page_size * page_size;
-    };
-    auto tiles_of = [&](int splits) { return (chunk_of(splits) + kAttnTile - 1) / kAttnTile; };
-    if (p.clusters == 1)
-        for (int w = kAttnSplits + 1; w <= kAttnMaxCluster; ++w)
-            if (resident[w - kAttnSplits] >= need && tiles_of(w) < tiles_of(p.width)) p.width = w;
-    p.keys_per_split = chunk_of(p.width * p.clusters);
-    return p;
 }
 
 struct AttnArgs {
@@ -162,21 +166,17 @@ struct AttnArgs {
     const uint16_t* kv_pool;
     int layer, n_pages, page_size, M, Hq, Hkv;
     int n_max;                 // N the launch's shared memory was sized for
+    int slot_c;                // bytes of the ring's third slot
     int row_groups;
-    float* o_part;             // partial results of requests whose keys several clusters share
-    float* m_part;
-    float* l_part;
-    int* tickets;
+    float* o_part;             // partial results: [slot][hd], slot = it_part0 + ((kv head * R + row) * splits + split)
+    float* m_part;             // [slot]
+    float* l_part;             // [slot]
+    int* tickets;              // [item][kv head][row group], zero between launches
     uint16_t* xf_out;          // the output projection's input (split-bf16 fragments)
     int* err;
 };
 
-// grid (cs * max clusters per request, n_kv_heads * row_groups, n_items), cluster (cs,1,1), 8 <= cs <= 10, block 160.
-// A request uses the first it_cs <= cs CTAs of its cluster; the others hold an empty split (exact zeros in the
-// merge), so a request's result does not depend on the cluster size its batch was launched with.
-// A request whose keys are shared by several clusters (long contexts) takes one more step: every cluster
-// writes its merged partial to global memory and the last cluster to arrive (atomic ticket, nobody waits)
-// merges those.
+// grid (max splits of the launch, n_kv_heads * row_groups, n_items), block 288.
 template <int HD>
 __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -185,152 +185,166 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
     pdl_launch_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int item = blockIdx.z;
-    const int cs = (int)cluster_nctaid_x();
-    const int cl = blockIdx.x / cs, rank = blockIdx.x % cs;        // cluster of this (request, head), rank in it
-    const int ncl = a.meta.it_nsplit[item];                        // clusters that share this request's keys
-    if (cl >= ncl) return;                                         // taken by a whole cluster or by none
-    const int S = a.meta.it_cs[item];                              // key splits per cluster of this request (<= cs)
-    const int sp = cl * S + rank;                                  // key split of this CTA (rank < S)
+    // per-request constants: independent loads, in flight together
+    const int nsplit = a.meta.it_nsplit[item];
+    const int rows = a.meta.it_rows[item];
+    const int base = a.meta.it_base[item];
+    const int chunk = a.meta.it_chunk[item];
+    const int row0 = a.meta.it_row0[item];
+    const int part0 = a.meta.it_part0[item];
+    const int req_slot = a.meta.it_slot[item];
+    const int sp = blockIdx.x;                                     // key split of this CTA
+    if (sp >= nsplit) return;
     const int Hkv = a.Hkv, Hq = a.Hq;
     const int kvh = blockIdx.y % Hkv, rg = blockIdx.y / Hkv;
     const int G = Hq / Hkv;
-    const int rows = a.meta.it_rows[item];
     const int R = G * rows;
     const int rho0 = rg * kAttnMaxRows;
-    // the whole cluster shares (item, head, row group): these exits are taken by all CTAs of the cluster or by none
     if (rho0 >= R) return;
     const int n_rows = min(kAttnMaxRows, R - rho0);
     const int N = (n_rows + 15) & ~15;
     if (N > a.n_max) return;
-    const int NG = N / 8;
-    const int base = a.meta.it_base[item];
-    const int total = base + rows, chunk = a.meta.it_chunk[item];
+    const int NG = N / 8, NB = N / 16;
+    const int total = base + rows;
     AttnCtx c;
-    c.k0 = rank < S ? min(sp * chunk, total) : total;
+    c.k0 = min(sp * chunk, total);
     c.k1 = min(c.k0 + chunk, total);
     c.kbase = a.kv_pool + kv_index(a.layer, a.n_pages, 0, 0, Hkv, kvh, a.page_size, 0, HD, 0);
     c.page_stride = (size_t)2 * Hkv * a.page_size * HD;
     c.v_off = (size_t)Hkv * a.page_size * HD;
     c.page_size = a.page_size;
-    c.bt = a.meta.block_tab + (size_t)a.meta.it_slot[item] * a.meta.max_pages;
-    c.bt_first = 0;
+    c.bt = a.meta.block_tab + (size_t)req_slot * a.meta.max_pages;
     const int ntiles = c.k1 > c.k0 ? (c.k1 - c.k0 + kAttnTile - 1) / kAttnTile : 0;
+    const size_t slot0 = (size_t)part0 + ((size_t)kvh * R + rho0) * nsplit;     // + row * nsplit + split
+    const int KSo = (Hq * HD) / 16, NTo = xf_nt(a.M);
 
-    // ---- shared memory
-    unsigned char* k_tile = smem;
-    unsigned char* v_tile = k_tile + SM::kTileBytes;
-    unsigned char* q_hi = v_tile + SM::kTileBytes;
+    // ---- shared memory: the ones come first (the tensor cores read a few KB past them, see below)
+    unsigned char* ones = smem;
+    unsigned char* ring = ones + SM::kOnes;                        // slots 0, 1: a whole tile; slot 2: a.slot_c bytes
+    unsigned char* q_hi = ring + 2 * SM::kTileBytes + a.slot_c;
     unsigned char* q_lo = q_hi + SM::q_bytes(N);
     unsigned char* p_hi = q_lo + SM::q_bytes(N);
     unsigned char* p_lo = p_hi + SM::p_bytes(N);
-    unsigned char* ones = p_lo + SM::p_bytes(N);
-    float* wm = reinterpret_cast<float*>(ones + SM::kOnes);        // [4][128] warp maxima of a tile
-    int* hz = reinterpret_cast<int*>(wm + 4 * kAttnMaxRows);       // [128] last visible key of a row (-1: padding row)
-    float* m_ref = reinterpret_cast<float*>(hz + kAttnMaxRows);    // [128] reference maximum of a row
-    float* alpha = m_ref + kAttnMaxRows;                           // [128] rescale factor of a row for this tile
-    float* Fl = alpha + kAttnMaxRows;                              // [128] the CTA's partial denominators
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(Fl + kAttnMaxRows);   // full, s_full, p_full, pv_done
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4);
+    float* wm = reinterpret_cast<float*>(p_lo + SM::p_bytes(N));   // [4][N] maxima of a tile per lane quarter
+    int* hz = reinterpret_cast<int*>(wm + 4 * N);                  // [N] last visible key of a row (-1: padding row)
+    float* m_ref = reinterpret_cast<float*>(hz + N);               // [N] reference maximum of a row
+    float* alpha = m_ref + N;                                      // [N] rescale factor of a row for this tile
+    float* Fl = alpha + N;                                         // [N] the CTA's partial denominators
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(Fl + N);   // full[3], s_full[2], p_full, pv_done
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 7);
     int* s_flag = reinterpret_cast<int*>(tmem_slot + 1);           // a row's reference maximum moved: rescale
     int* s_last = s_flag + 1;
-    float* Fo = reinterpret_cast<float*>(q_hi);                    // [N][HD]: takes over the Q operands after the tile loop
-    float* Fm = m_ref;
-    const uint32_t bar_full = smem_u32(bars), bar_s = bar_full + 8, bar_p = bar_full + 16, bar_pv = bar_full + 24;
+    const uint32_t bar_full = smem_u32(bars), bar_s = bar_full + 24, bar_p = bar_full + 40, bar_pv = bar_full + 48;
     const uint32_t tmem_cols = (uint32_t)attn_tmem_cols(N);
+    const uint32_t ring_a = smem_u32(ring);
+    auto slot_addr = [&](int i) { return ring_a + (uint32_t)(i % 3) * SM::kTileBytes; };   // ring slot of item i (K_t: 2t, V_t: 2t+1)
 
-    __shared__ int s_pages[kAttnPagesSmem];
-    __shared__ AttnCtx s_ctx;
-    // The page ids of this CTA's key range go to shared memory once: a tile's copies then start without a trip to
-    // the block table first.
-    if (ntiles > 0) {
-        const int p_first = c.k0 / a.page_size, n_pg = (c.k1 - 1) / a.page_size - p_first + 1;
-        if (n_pg <= kAttnPagesSmem) {                              // uniform over the CTA
-            for (int i = tid; i < n_pg; i += kAttnThreads) s_pages[i] = c.bt[p_first + i];
-            c.bt = s_pages;
-            c.bt_first = p_first;
-        }
-    }
-    if (tid == kAttnWorkers) {
-        s_ctx = c;
-        mbar_init(bar_full, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_p, 1);
-        mbar_init(bar_pv, 1);
-        fence_mbar_init();
-    }
-    __syncthreads();
     bool ok = true;
     if (ntiles > 0) {
-        // Tiles made only of keys cached before this pass do not depend on the QKV projection that precedes this
-        // kernel: the first one is requested now, otherwise after the dependency has resolved.
-        const bool early0 = min(c.k0 + kAttnTile, c.k1) <= base;
-        if (warp == 4) {
+        uint32_t tmem = 0;
+        if (warp == 8) {
+            // ---------------- barriers, the first three items of the ring, tensor memory
+            if (lane == 0) {
+                for (int i = 0; i < 7; ++i) mbar_init(bar_full + 8 * i, 1);
+                fence_mbar_init();
+            }
+            __syncwarp();
+            // Items made only of keys cached before this pass do not depend on the QKV projection that precedes this
+            // kernel: they are requested now, the others after the dependency has resolved.
+            const int early_tiles = base >= c.k1 ? ntiles : (base - c.k0) / kAttnTile;      // whole tiles below `base`
+            const int first = ntiles > 1 ? 3 : 2;                                            // items requested up front
+            for (int i = 0; i < first; ++i)
+                if ((i >> 1) < early_tiles) attn_issue_tile<HD>(c, i & 1, slot_addr(i), bar_full + 8 * (i % 3), c.k0 + (i >> 1) * kAttnTile);
             tmem_alloc(smem_u32(tmem_slot), tmem_cols);
             tc_fence_before();
-            if (early0) attn_issue_tile<HD>(s_ctx, smem_u32(k_tile), smem_u32(v_tile), bar_full, c.k0);
+            pdl_wait();
+            for (int i = 0; i < first; ++i)
+                if ((i >> 1) >= early_tiles) attn_issue_tile<HD>(c, i & 1, slot_addr(i), bar_full + 8 * (i % 3), c.k0 + (i >> 1) * kAttnTile);
         } else {
             // operands that do not depend on the predecessor: the ones, the rows' horizons and initial state
-            for (int i = tid; i < SM::kOnes / 4; i += kAttnWorkers) reinterpret_cast<uint32_t*>(ones)[i] = 0x3F803F80u;
-            for (int n = tid; n < kAttnMaxRows; n += kAttnWorkers) {
+            if (tid < SM::kOnes / 4) reinterpret_cast<uint32_t*>(ones)[tid] = 0x3F803F80u;
+            for (int n = tid; n < N; n += kAttnWorkers) {
                 const int rho = rho0 + n;
                 hz[n] = n < n_rows ? base + rho % rows : -1;
                 m_ref[n] = -INFINITY;
             }
-        }
-        pdl_wait();
-        if (warp == 4) {
-            if (!early0) attn_issue_tile<HD>(s_ctx, smem_u32(k_tile), smem_u32(v_tile), bar_full, c.k0);
-        } else {
+            pdl_wait();
             // ---- stage Q (scaled by log2(e)/sqrt(hd)) as the K-major B operand, bf16 hi and lo terms:
-            // piece (row n, k group g) at ((n/8) * HG + g) * 128 + (n%8) * 16
+            // piece (row n, k group g) at ((n/8) * HG + g) * 128 + (n%8) * 16.  Two pieces per thread and step, all
+            // loads of a step in flight together.
             const float scale = rsqrtf((float)HD) * 1.4426950408889634f;   // scores in the log2 domain: p = 2^(s - m)
-            const int row0 = a.meta.it_row0[item];
-            for (int idx = tid; idx < N * HG; idx += kAttnWorkers) {
-                const int n = idx / HG, g = idx % HG;
-                float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                if (n < n_rows) {
-                    const int rho = rho0 + n, gq = rho / rows, r = rho % rows;
-                    const float4* qp = reinterpret_cast<const float4*>(a.q + ((size_t)(row0 + r) * Hq + kvh * G + gq) * HD + g * 8);
-                    const float4 x0 = qp[0], x1 = qp[1];
-                    v[0] = x0.x * scale; v[1] = x0.y * scale; v[2] = x0.z * scale; v[3] = x0.w * scale;
-                    v[4] = x1.x * scale; v[5] = x1.y * scale; v[6] = x1.z * scale; v[7] = x1.w * scale;
-                }
-                uint16_t h[8], l[8];
+            for (int idx0 = tid; idx0 < N * HG; idx0 += 2 * kAttnWorkers) {
+                float4 x[2][2];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) split_bf16(v[i], h[i], l[i]);
-                const uint32_t off = (uint32_t)(((n >> 3) * HG + g) * 128 + (n & 7) * 16);
-                *reinterpret_cast<uint4*>(q_hi + off) = make_uint4(pack2(h[0], h[1]), pack2(h[2], h[3]), pack2(h[4], h[5]), pack2(h[6], h[7]));
-                *reinterpret_cast<uint4*>(q_lo + off) = make_uint4(pack2(l[0], l[1]), pack2(l[2], l[3]), pack2(l[4], l[5]), pack2(l[6], l[7]));
+                for (int u = 0; u < 2; ++u) {
+                    const int idx = idx0 + u * kAttnWorkers, n = idx / HG, g = idx % HG;
+                    x[u][0] = x[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (idx < N * HG && n < n_rows) {
+                        const int rho = rho0 + n, gq = rho / rows, r = rho % rows;
+                        const float4* qp = reinterpret_cast<const float4*>(a.q + ((size_t)(row0 + r) * Hq + kvh * G + gq) * HD + g * 8);
+                        x[u][0] = qp[0];
+                        x[u][1] = qp[1];
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int idx = idx0 + u * kAttnWorkers, n = idx / HG, g = idx % HG;
+                    if (idx >= N * HG) break;
+                    const float v[8] = {x[u][0].x * scale, x[u][0].y * scale, x[u][0].z * scale, x[u][0].w * scale,
+                                        x[u][1].x * scale, x[u][1].y * scale, x[u][1].z * scale, x[u][1].w * scale};
+                    uint16_t h[8], l[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) split_bf16(v[i], h[i], l[i]);
+                    const uint32_t off = (uint32_t)(((n >> 3) * HG + g) * 128 + (n & 7) * 16);
+                    *reinterpret_cast<uint4*>(q_hi + off) = make_uint4(pack2(h[0], h[1]), pack2(h[2], h[3]), pack2(h[4], h[5]), pack2(h[6], h[7]));
+                    *reinterpret_cast<uint4*>(q_lo + off) = make_uint4(pack2(l[0], l[1]), pack2(l[2], l[3]), pack2(l[4], l[5]), pack2(l[6], l[7]));
+                }
             }
             fence_proxy_async_smem();      // the tensor cores read these through the asynchronous proxy
         }
-        __syncthreads();                   // Q, ones and the tensor-memory base are in place
+        __syncthreads();                   // barriers, Q, ones and the tensor-memory base are in place
         tc_fence_after();
-        const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
-        const uint32_t t_S = tmem, t_O = tmem + (uint32_t)N, t_L = tmem + 2u * (uint32_t)N;
+        tmem = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+        const uint32_t t_S = tmem, t_O = tmem + 2u * (uint32_t)N, t_L = tmem + 3u * (uint32_t)N;   // S^T twice, O^T, L
 
-        if (warp == 4) {
-            // ---------------- copies and MMA issue
+        if (warp == 8) {
+            // ---------------- copies and MMA issue.  Ring item i (K_t: 2t, V_t: 2t+1) lives in slot i % 3 and may be
+            // requested once item i - 3 has been read: a K tile by the first product of its tile (s_full), a V tile by
+            // the second (pv_done).  The first product of tile t+1 is issued ahead of the second of tile t.
             const uint32_t idesc_qk = umma_idesc_bf16(128, N, 0, 0), idesc_pv = umma_idesc_bf16(128, N, 1, 1);
-            const uint32_t ka = smem_u32(k_tile), va = smem_u32(v_tile);
             const uint32_t qh = smem_u32(q_hi), ql = smem_u32(q_lo), ph = smem_u32(p_hi), pl = smem_u32(p_lo);
-            const uint64_t ones_desc = umma_desc(smem_u32(ones), 2048, 128);
-            for (int t = 0; t < ntiles; ++t) {
-                const uint32_t par = (uint32_t)t & 1u;
-                if (ok) ok = attn_wait_warp(bar_full, par);                  // K and V rows of tile t have landed
-                if (lane == 0 && ok) {
-                    tc_fence_after();
+            // the denominators' A operand: 16 keys x 8 rows of ones; the other 120 rows of the MMA read whatever follows
+            // in shared memory (the ring) and land in tensor-memory lanes that nobody reads
+            const uint64_t ones_desc = umma_desc(smem_u32(ones), 128, 256);
+            auto issue_qk = [&](int t) {       // S^T[t & 1] = K_t . Q^T
+                const uint32_t ka = slot_addr(2 * t), d = t_S + (uint32_t)((t & 1) * N);
 #pragma unroll
-                    for (int kk = 0; kk < HD / 16; ++kk)
-                        umma_bf16(t_S, umma_desc(ka + kk * 256, 128, HG * 128), umma_desc(qh + kk * 256, 128, HG * 128), idesc_qk, kk > 0);
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    umma_bf16(d, umma_desc(ka + kk * 256, 128, HG * 128), umma_desc(qh + kk * 256, 128, HG * 128), idesc_qk, kk > 0);
 #pragma unroll
-                    for (int kk = 0; kk < HD / 16; ++kk)
-                        umma_bf16(t_S, umma_desc(ka + kk * 256, 128, HG * 128), umma_desc(ql + kk * 256, 128, HG * 128), idesc_qk, 1);
-                    umma_commit(bar_s);
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    umma_bf16(d, umma_desc(ka + kk * 256, 128, HG * 128), umma_desc(ql + kk * 256, 128, HG * 128), idesc_qk, 1);
+                umma_commit(bar_s + 8 * (t & 1));
+            };
+            auto full_wait = [&](int i) { return attn_wait_warp(bar_full + 8 * (i % 3), (uint32_t)(i / 3) & 1u); };
+            auto request = [&](int i) {        // ring item i, if the split has it
+                if ((i >> 1) < ntiles) attn_issue_tile<HD>(c, i & 1, slot_addr(i), bar_full + 8 * (i % 3), c.k0 + (i >> 1) * kAttnTile);
+            };
+            ok = full_wait(0);
+            if (ok && lane == 0) { tc_fence_after(); issue_qk(0); }
+            for (int t = 0; t < ntiles && ok; ++t) {
+                if (t + 1 < ntiles) {
+                    ok = full_wait(2 * t + 2);                                           // K of tile t+1 has landed
+                    // S^T[(t+1) & 1] was last read for tile t-1: free once P of tile t-1 was announced (seen below)
+                    if (ok && lane == 0) { tc_fence_after(); issue_qk(t + 1); }
                 }
-                if (ok) ok = attn_wait_warp(bar_p, par);                     // P of tile t is written (and O^T rescaled)
-                if (lane == 0 && ok) {
+                if (ok) ok = attn_wait_warp(bar_s + 8 * (t & 1), (uint32_t)(t >> 1) & 1u);   // K_t has been read
+                if (ok && t + 1 < ntiles) request(2 * t + 3);                            // V of tile t+1 into K_t's slot
+                if (ok) ok = attn_wait_warp(bar_p, (uint32_t)t & 1u);                    // P of tile t is written (and O^T rescaled)
+                if (ok) ok = full_wait(2 * t + 1);                                       // V of tile t has landed
+                if (ok && lane == 0) {
                     tc_fence_after();
+                    const uint32_t va = slot_addr(2 * t + 1);
                     const int n_valid = min(kAttnTile, c.k1 - (c.k0 + t * kAttnTile));
                     const int n16 = (n_valid + 15) / 16;
                     for (int ks = 0; ks < n16; ++ks) {
@@ -345,43 +359,45 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
                     }
                     umma_commit(bar_pv);
                 }
-                if (!ok) break;
-                if (t + 1 < ntiles) {
-                    ok = attn_wait_warp(bar_pv, par);                   // the tile's operands have been read
-                    if (ok) attn_issue_tile<HD>(s_ctx, ka, va, bar_full, c.k0 + (t + 1) * kAttnTile);
+                if (ok && t + 2 < ntiles) {
+                    ok = attn_wait_warp(bar_pv, (uint32_t)t & 1u);                       // V_t has been read
+                    if (ok) request(2 * t + 4);                                          // K of tile t+2 into V_t's slot
                 }
             }
             if (!ok && a.err && lane == 0) atomicExch(a.err, 3);
         } else {
-            // ---------------- one thread per key of the tile (= tensor-memory lane)
-            const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+            // ---------------- thread = key of the tile (tensor-memory lane 32 * quarter + lane); the two warps of a
+            // lane quarter take alternate 16-row column blocks
+            const int quarter = warp & 3, half = warp >> 2;
+            const int kt = quarter * 32 + lane;                         // key within the tile
+            const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
             for (int t = 0; t < ntiles; ++t) {
-                const uint32_t par = (uint32_t)t & 1u;
-                const int j = c.k0 + t * kAttnTile + tid;               // this thread's key
+                const int j = c.k0 + t * kAttnTile + kt;                // this thread's key
                 const int n_valid = min(kAttnTile, c.k1 - (c.k0 + t * kAttnTile));
+                const uint32_t t_St = t_S + (uint32_t)((t & 1) * N);
                 if (tid == 0) *s_flag = 0;
-                if (ok) ok = attn_wait_warp(bar_s, par);
+                if (ok) ok = attn_wait_warp(bar_s + 8 * (t & 1), (uint32_t)(t >> 1) & 1u);
                 tc_fence_after();
                 const bool need_mask = c.k0 + (t + 1) * kAttnTile - 1 > base || n_valid < kAttnTile;   // CTA-uniform
-                // ---- pass 1: the tile's maximum per row (over the 32 keys of the warp, then over the warps)
-                for (int cb = 0; cb < N / 16; ++cb) {
-                    float s[16];
-                    tmem_ld16(t_S + lane_sel + cb * 16, s);
+                // ---- pass 1: the tile's maximum per row (over the 32 keys of the warp, then over the lane quarters)
+                for (int cu = half; cu < NG; cu += 2) {
+                    float s[8];
+                    tmem_ld8(t_St + lane_sel + cu * 8, s);
                     tmem_ld_wait();
                     float mine = -INFINITY;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
+                    for (int i = 0; i < 8; ++i) {
                         float v = s[i];
-                        if (need_mask && !(j < c.k1 && j <= hz[cb * 16 + i])) v = -INFINITY;
+                        if (need_mask && !(j < c.k1 && j <= hz[cu * 8 + i])) v = -INFINITY;
                         if (!ok) v = -INFINITY;
                         const float wmax = warp_max_redux(v);
                         if (lane == i) mine = wmax;
                     }
-                    if (lane < 16) wm[warp * kAttnMaxRows + cb * 16 + lane] = mine;
+                    if (lane < 8) wm[quarter * N + cu * 8 + lane] = mine;
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(kAttnWorkers) : "memory");
                 if (tid < N) {
-                    const float tmax = fmaxf(fmaxf(wm[tid], wm[kAttnMaxRows + tid]), fmaxf(wm[2 * kAttnMaxRows + tid], wm[3 * kAttnMaxRows + tid]));
+                    const float tmax = fmaxf(fmaxf(wm[tid], wm[N + tid]), fmaxf(wm[2 * N + tid], wm[3 * N + tid]));
                     const float m_old = m_ref[tid];
                     float al = 1.f;
                     if (tmax > -INFINITY) {
@@ -396,7 +412,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
                 tc_fence_after();
                 if (*s_flag && t > 0 && ok) {
                     // ---- a reference maximum moved: rescale the rows' columns of O^T and L (2N columns from t_O)
-                    for (int cb = 0; cb < 2 * N / 16; ++cb) {
+                    for (int cb = half; cb < 2 * NB; cb += 2) {
                         float o[16];
                         tmem_ld16(t_O + lane_sel + cb * 16, o);
                         tmem_ld_wait();
@@ -408,17 +424,17 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
                 }
                 // ---- pass 2: p = 2^(s - reference maximum), written as the MN-major B operand (hi and lo terms):
                 // piece (key group kg, row group g, key) at ((kg * NG + g) * 8 + key % 8) * 16 holds 8 rows
-                for (int cb = 0; cb < N / 16; ++cb) {
-                    float s[16];
-                    tmem_ld16(t_S + lane_sel + cb * 16, s);
+                for (int cu = half; cu < NG; cu += 2) {
+                    float s[8];
+                    tmem_ld8(t_St + lane_sel + cu * 8, s);
                     tmem_ld_wait();
-                    uint32_t hw[8], lw[8];
+                    uint32_t hw[4], lw[4];
 #pragma unroll
-                    for (int i = 0; i < 16; i += 2) {
+                    for (int i = 0; i < 8; i += 2) {
                         float p2[2];
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            const int n = cb * 16 + i + e;
+                            const int n = cu * 8 + i + e;
                             const float mr = m_ref[n];
                             float v = s[i + e];
                             if (need_mask && !(j < c.k1 && j <= hz[n])) v = -INFINITY;
@@ -430,159 +446,133 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
                         hw[i >> 1] = pack2(h0, h1);
                         lw[i >> 1] = pack2(l0, l1);
                     }
-                    const uint32_t off = (uint32_t)((((tid >> 3) * NG + cb * 2) * 8 + (tid & 7)) * 16);
+                    const uint32_t off = (uint32_t)((((kt >> 3) * NG + cu) * 8 + (kt & 7)) * 16);
                     *reinterpret_cast<uint4*>(p_hi + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-                    *reinterpret_cast<uint4*>(p_hi + off + 128) = make_uint4(hw[4], hw[5], hw[6], hw[7]);
                     *reinterpret_cast<uint4*>(p_lo + off) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-                    *reinterpret_cast<uint4*>(p_lo + off + 128) = make_uint4(lw[4], lw[5], lw[6], lw[7]);
                 }
-                // V rows at and beyond the split's end must be finite (P is 0 there, but 0 * NaN is not): cleared
-                if (tid >= n_valid) {
+                // V rows at and beyond the split's end must be finite (P is 0 there, but 0 * NaN is not): cleared, once
+                // the tile's V rows have landed (the copy may bring garbage rows of the last 8-row group)
+                if (n_valid < kAttnTile) {
+                    if (ok) ok = attn_wait_warp(bar_full + 8 * ((2 * t + 1) % 3), (uint32_t)((2 * t + 1) / 3) & 1u);
+                    if (half == 0 && kt >= n_valid && kt < ((n_valid + 15) & ~15)) {
+                        unsigned char* v_tile = ring + ((2 * t + 1) % 3) * SM::kTileBytes;
 #pragma unroll
-                    for (int g = 0; g < HG; ++g)
-                        *reinterpret_cast<uint4*>(v_tile + ((tid >> 3) * HG + g) * 128 + (tid & 7) * 16) = make_uint4(0, 0, 0, 0);
+                        for (int g = 0; g < HG; ++g)
+                            *reinterpret_cast<uint4*>(v_tile + ((kt >> 3) * HG + g) * 128 + (kt & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    }
                 }
                 fence_proxy_async_smem();
                 tc_fence_before();
                 asm volatile("bar.sync 1, %0;" ::"n"(kAttnWorkers) : "memory");
                 if (tid == 0) mbar_arrive(bar_p);
             }
-            // ---- the CTA's partial result: O^T (thread = head dimension) and L (every lane holds all rows' sums)
+            // ---- the CTA's partial result: O^T (thread = head dimension) and L (lanes 0-7 hold all rows' sums)
             if (ok) ok = attn_wait_warp(bar_pv, (uint32_t)(ntiles - 1) & 1u);
             tc_fence_after();
-            for (int cb = 0; cb < N / 16; ++cb) {
+            if (quarter == 0) {
+                for (int cb = half; cb < NB; cb += 2) {
+                    float l[16];
+                    tmem_ld16(t_L + cb * 16, l);
+                    tmem_ld_wait();
+                    if (lane == 0) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const int n = cb * 16 + i;
+                            const float lv = ok ? l[i] : 0.f;
+                            Fl[n] = lv;
+                            if (nsplit > 1 && n < n_rows) {
+                                a.l_part[slot0 + (size_t)n * nsplit + sp] = lv;
+                                a.m_part[slot0 + (size_t)n * nsplit + sp] = m_ref[n];
+                            }
+                        }
+                    }
+                }
+            }
+            if (nsplit == 1) asm volatile("bar.sync 1, %0;" ::"n"(kAttnWorkers) : "memory");     // the sums, for the division below
+            for (int cb = half; cb < NB; cb += 2) {
                 float o[16];
                 tmem_ld16(t_O + lane_sel + cb * 16, o);
                 tmem_ld_wait();
-                if (tid < HD) {
+                if (kt < HD) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) Fo[(size_t)(cb * 16 + i) * HD + tid] = ok ? o[i] : 0.f;
+                    for (int i = 0; i < 16; ++i) {
+                        const int n = cb * 16 + i;
+                        if (n < n_rows) {
+                            const float v = ok ? o[i] : 0.f;
+                            if (nsplit == 1) {      // nothing to merge: normalise and store the output projection's input
+                                const int rho = rho0 + n, gq = rho / rows, r_in = rho % rows;
+                                xf_store_one(a.xf_out, row0 + r_in, (kvh * G + gq) * HD + kt, v / Fl[n], KSo, NTo);
+                            } else {
+                                a.o_part[(slot0 + (size_t)n * nsplit + sp) * HD + kt] = v;
+                            }
+                        }
+                    }
                 }
-            }
-            for (int cb = 0; cb < N / 16; ++cb) {       // thread n keeps row n's sum (its own lane's copy)
-                float l[16];
-                tmem_ld16(t_L + lane_sel + cb * 16, l);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (tid == cb * 16 + i) Fl[tid] = ok ? l[i] : 0.f;
             }
             if (!ok && a.err && lane == 0) atomicExch(a.err, 4);
             tc_fence_before();
         }
         __syncthreads();
-        if (warp == 4) {
+        if (warp == 8) {
             tc_fence_after();
             tmem_dealloc(tmem, tmem_cols);
         }
     } else {
         // empty split: contributes nothing (finite zeros, so the merge can read it unconditionally)
         pdl_wait();
-        for (int i = tid; i < N; i += kAttnThreads) { Fm[i] = -INFINITY; Fl[i] = 0.f; }
-        for (int i = tid; i < N * HD; i += kAttnThreads) Fo[i] = 0.f;
+        for (int i = tid; i < n_rows * HD; i += kAttnThreads) a.o_part[(slot0 + (size_t)(i / HD) * nsplit + sp) * HD + i % HD] = 0.f;
+        for (int i = tid; i < n_rows; i += kAttnThreads) {
+            a.m_part[slot0 + (size_t)i * nsplit + sp] = -INFINITY;
+            a.l_part[slot0 + (size_t)i * nsplit + sp] = 0.f;
+        }
+        __syncthreads();
     }
+    if (nsplit == 1) return;
 
-    // ---- merge the cluster's splits over distributed shared memory; rank r owns rows r, r+cs, ... of the group
-    cluster_sync_all();
-    constexpr int EPT = HD / kAttnWorkers > 0 ? HD / kAttnWorkers : 1;   // output columns per thread
-    const uint32_t fo_a = smem_u32(Fo), fm_a = smem_u32(Fm), fl_a = smem_u32(Fl);
-    const int row0 = a.meta.it_row0[item];
-    const int KSo = (Hq * HD) / 16, NTo = xf_nt(a.M);
-    const size_t slot0 = (size_t)a.meta.it_part0[item] + ((size_t)kvh * R + rho0) * ncl;   // + rl*ncl + cluster
-#pragma unroll 2
-    for (int rl = rank; rl < n_rows; rl += cs) {
-        // all remote reads of a row are issued together: cs maxima, cs sums, cs output values per thread
-        float ms[kAttnMaxCluster], ls[kAttnMaxCluster], ov[EPT][kAttnMaxCluster];
-#pragma unroll
-        for (int r = 0; r < kAttnMaxCluster; ++r) {
-            if (r >= cs) {                       // beyond this launch's cluster: an empty split
-                ms[r] = -INFINITY; ls[r] = 0.f;
-#pragma unroll
-                for (int k = 0; k < EPT; ++k) ov[k][r] = 0.f;
-                continue;
-            }
-            ms[r] = dsmem_ld_f32(dsmem_addr(fm_a + rl * 4, (uint32_t)r));
-            ls[r] = dsmem_ld_f32(dsmem_addr(fl_a + rl * 4, (uint32_t)r));
-#pragma unroll
-            for (int k = 0; k < EPT; ++k) {
-                const int e = tid + k * kAttnWorkers;
-                ov[k][r] = (e < HD && tid < kAttnWorkers) ? dsmem_ld_f32(dsmem_addr(fo_a + (uint32_t)(rl * HD + e) * 4, (uint32_t)r)) : 0.f;
-            }
-        }
-        float m = -INFINITY;
-#pragma unroll
-        for (int r = 0; r < kAttnMaxCluster; ++r) m = fmaxf(m, ms[r]);
-        float den = 0.f, w[kAttnMaxCluster];
-#pragma unroll
-        for (int r = 0; r < kAttnMaxCluster; ++r) {
-            w[r] = (ms[r] == -INFINITY) ? 0.f : exp2f(ms[r] - m);   // an empty split or one beyond the causal horizon
-            den += w[r] * ls[r];
-        }
-        const int rho = rho0 + rl, gq = rho / rows, r_in = rho % rows;
-#pragma unroll
-        for (int k = 0; k < EPT; ++k) {
-            const int e = tid + k * kAttnWorkers;
-            if (e < HD && tid < kAttnWorkers) {
-                float num = 0.f;
-#pragma unroll
-                for (int r = 0; r < kAttnMaxCluster; ++r) num += w[r] * ov[k][r];
-                if (ncl == 1) xf_store_one(a.xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
-                else a.o_part[(slot0 + (size_t)rl * ncl + cl) * HD + e] = num;     // un-normalised, with (m, den)
-            }
-        }
-        if (ncl > 1 && tid == 0) {
-            a.m_part[slot0 + (size_t)rl * ncl + cl] = m;
-            a.l_part[slot0 + (size_t)rl * ncl + cl] = den;
-        }
-    }
-    if (ncl > 1) __threadfence();
-    cluster_sync_all();   // nobody leaves while its shared memory may still be read; partials are published
-    if (ncl == 1) return;
-    // ---- several clusters share the keys: the last one to arrive merges their partials
-    if (rank == 0 && tid == 0) {
+    // ---- the last CTA of this (request, KV head, row group) to arrive merges the splits, in split order
+    // (the barrier above orders the whole CTA's stores before thread 0's fence, and its fence after the ticket orders the
+    // other CTAs' partials before the loads that follow the barrier below)
+    if (tid == 0) {
         int* ticket = a.tickets + ((size_t)item * Hkv + kvh) * a.row_groups + rg;
+        __threadfence();
         const int t = atomicAdd(ticket, 1);
-        const int last = (t == ncl - 1);
+        const int last = (t == nsplit - 1);
         if (last) *ticket = 0;                                   // self-cleaning: ready for the next launch
-        const uint32_t fa = smem_u32(s_last);
-        for (int r = 0; r < cs; ++r) dsmem_st_f32(dsmem_addr(fa, (uint32_t)r), __int_as_float(last));
+        __threadfence();
+        *s_last = last;
     }
-    cluster_sync_all();
+    __syncthreads();
     if (!*s_last) return;
-    __threadfence();
-    for (int rl = rank; rl < n_rows; rl += cs) {
-        float ms[kMaxSplits / kAttnSplits], ls[kMaxSplits / kAttnSplits], ov[EPT][kMaxSplits / kAttnSplits];
+    // warp = row, lane = four columns: one round covers nine rows
+    for (int rl = warp; rl < n_rows; rl += kAttnThreads / 32) {
+        float ms[kAttnMaxSplits], ls[kAttnMaxSplits];
+        float4 ov[kAttnMaxSplits];
+        const size_t sl0 = slot0 + (size_t)rl * nsplit;
 #pragma unroll
-        for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) {
-            const bool on = j < ncl;
-            const size_t sl = slot0 + (size_t)rl * ncl + j;
-            ms[j] = on ? __ldcg(a.m_part + sl) : -INFINITY;
-            ls[j] = on ? __ldcg(a.l_part + sl) : 0.f;
-#pragma unroll
-            for (int k = 0; k < EPT; ++k) {
-                const int e = tid + k * kAttnWorkers;
-                ov[k][j] = (on && e < HD && tid < kAttnWorkers) ? __ldcg(a.o_part + sl * HD + e) : 0.f;
-            }
+        for (int j = 0; j < kAttnMaxSplits; ++j) {               // all loads of the row in flight together
+            const bool on = j < nsplit;
+            ms[j] = on ? __ldcg(a.m_part + sl0 + j) : -INFINITY;
+            ls[j] = on ? __ldcg(a.l_part + sl0 + j) : 0.f;
+            ov[j] = (on && lane < HD / 4) ? __ldcg(reinterpret_cast<const float4*>(a.o_part + (sl0 + j) * HD) + lane)
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         float m = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) m = fmaxf(m, ms[j]);
-        float den = 0.f, w[kMaxSplits / kAttnSplits];
+        for (int j = 0; j < kAttnMaxSplits; ++j) m = fmaxf(m, ms[j]);
+        float den = 0.f;
+        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) {
-            w[j] = (ms[j] == -INFINITY) ? 0.f : exp2f(ms[j] - m);
-            den += w[j] * ls[j];
+        for (int j = 0; j < kAttnMaxSplits; ++j) {
+            const float w = (ms[j] == -INFINITY) ? 0.f : exp2f(ms[j] - m);   // an empty split or one beyond the causal horizon
+            den += w * ls[j];
+            num.x += w * ov[j].x; num.y += w * ov[j].y; num.z += w * ov[j].z; num.w += w * ov[j].w;
         }
-        const int rho = rho0 + rl, gq = rho / rows, r_in = rho % rows;
-#pragma unroll
-        for (int k = 0; k < EPT; ++k) {
-            const int e = tid + k * kAttnWorkers;
-            if (e < HD && tid < kAttnWorkers) {
-                float num = 0.f;
-#pragma unroll
-                for (int j = 0; j < kMaxSplits / kAttnSplits; ++j) num += w[j] * ov[k][j];
-                xf_store_one(a.xf_out, row0 + r_in, (kvh * G + gq) * HD + e, num / den, KSo, NTo);
-            }
+        if (lane < HD / 4) {
+            const int rho = rho0 + rl, gq = rho / rows, r_in = rho % rows;
+            const int col = (kvh * G + gq) * HD + lane * 4;
+            const float inv = 1.f / den;
+            xf_store_pair(reinterpret_cast<uint32_t*>(a.xf_out), row0 + r_in, col, num.x * inv, num.y * inv, KSo, NTo);
+            xf_store_pair(reinterpret_cast<uint32_t*>(a.xf_out), row0 + r_in, col + 2, num.z * inv, num.w * inv, KSo, NTo);
         }
     }
 }

@@ -250,9 +250,8 @@ struct PassMeta {
     const int32_t* it_row0;    // [n_items] first row of the item
     const int32_t* it_rows;    // [n_items] rows of the item (k+1)
     const int32_t* it_base;    // [n_items] cached positions before this pass
-    const int32_t* it_nsplit;  // [n_items] KV splits
+    const int32_t* it_nsplit;  // [n_items] key splits
     const int32_t* it_chunk;   // [n_items] keys per split (multiple of the page size)
-    const int32_t* it_cs;      // [n_items] key splits per cluster (the request's own: 8..10)
     const int32_t* it_part0;   // [n_items] first slot of the item in the attention partial arrays
     const int32_t* block_tab;  // [max_requests][max_pages] page ids, indexed by request slot
     int max_pages;

@@ -48,7 +48,7 @@ struct LayerW {
 
 // Fixed offsets of the per-call metadata block (same layout in pinned host staging and on device).
 struct MetaLayout {
-    size_t row_item, row_pos, row_tok, it_slot, it_row0, it_rows, it_base, it_nsplit, it_chunk, it_cs, it_part0, u, rej, total;
+    size_t row_item, row_pos, row_tok, it_slot, it_row0, it_rows, it_base, it_nsplit, it_chunk, it_part0, u, rej, total;
 };
 
 MetaLayout meta_layout(int max_rows, int max_items) {
@@ -64,7 +64,6 @@ MetaLayout meta_layout(int max_rows, int max_items) {
     m.it_base = take(4 * (size_t)max_items);
     m.it_nsplit = take(4 * (size_t)max_items);
     m.it_chunk = take(4 * (size_t)max_items);
-    m.it_cs = take(4 * (size_t)max_items);
     m.it_part0 = take(4 * (size_t)max_items);
     m.u = take(4 * (size_t)max_rows);
     m.rej = take(sizeof(RejectItem) * (size_t)max_items);
@@ -114,7 +113,7 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     const size_t nssq = (c.d_model + 127) / 128;
     w.ssqA = take(4 * nssq * M);
     w.ssqB = take(4 * nssq * M);
-    const size_t slots = M * c.n_q_heads * (kMaxSplits / kAttnSplits);   // one per (row, head, cluster)
+    const size_t slots = M * c.n_q_heads * kAttnMaxSplits;               // one per (row, head, key split)
     w.o_part = take(4 * slots * c.head_dim);
     w.m_part = take(4 * slots);
     w.l_part = take(4 * slots);
@@ -158,10 +157,13 @@ cudaError_t init_attrs_current_device() {
     cudaError_t e;
     if ((e = gemm_init_attrs()) != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)attn_smem_bytes(128, kAttnMaxRows));
+                             (int)attn_smem_bytes(128, kAttnMaxRows, false));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)attn_smem_bytes(64, kAttnMaxRows));
+    if ((e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes(64, kAttnMaxRows, false));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
 }
 
 int ensure_device_ready() {
@@ -242,8 +244,8 @@ struct pipesd_ctx {
     std::deque<Inflight> inflight;
     int res_buf = 0;
     int last_rows = 0;
-    int attn_occ[kAttnMaxCluster + 1][kAttnMaxRows / 16 + 1] = {};  // [cluster width 9..][query rows / 16]: clusters of the
-                                                                     // attention kernel the device keeps resident at once (0: width unavailable)
+    int attn_slots[kAttnMaxRows / 16 + 1][2] = {};   // [query rows / 16][cut-down third ring slot]: CTAs of the attention
+                                                     // kernel the device keeps resident at once
     uint32_t pf_depth = 32u << 10;   // bytes per successor CTA that a GEMM pulls into L2 for the next GEMM
     std::string err;
     // launch accounting
@@ -268,7 +270,6 @@ struct pipesd_ctx {
         m.it_base = (const int32_t*)(b + ml.it_base);
         m.it_nsplit = (const int32_t*)(b + ml.it_nsplit);
         m.it_chunk = (const int32_t*)(b + ml.it_chunk);
-        m.it_cs = (const int32_t*)(b + ml.it_cs);
         m.it_part0 = (const int32_t*)(b + ml.it_part0);
         m.block_tab = W<int32_t>(ws.block_tab);
         m.max_pages = dv.max_pages;
@@ -388,28 +389,24 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     auto I = [&](size_t off) { return reinterpret_cast<int32_t*>(hm + off); };
     float* hu = reinterpret_cast<float*>(hm + ml.u);
     RejectItem* hr = reinterpret_cast<RejectItem*>(hm + ml.rej);
-    int row = 0, part0 = 0, max_nsplit = 1, u0 = 0, max_cs = kAttnSplits;
+    int row = 0, part0 = 0, max_nsplit = 1, u0 = 0;
+    bool all_short = true;       // no split of the pass has more than two key tiles, the second a short one
     for (int i = 0; i < n_items; ++i) {
         const ItemDesc& it = items[i];
         const int total = it.base + it.rows;
-        // clusters that share the request's keys, key splits per cluster (8..10) and keys per split: from the request
-        // alone (its length, its rows), so that its summation order is the same in every batch
+        // key splits and keys per split: from the request alone (its length, its rows), so that its summation order is
+        // the same in every batch
         const int R_i = it.rows * (c.n_q_heads / c.n_kv_heads);                  // query rows per KV head
-        const int qt_i = attn_rows_n(R_i) / 16;
         const int rg_i = (R_i + kAttnMaxRows - 1) / kAttnMaxRows;
-        int resident[kAttnMaxCluster - kAttnSplits + 1];
-        for (int w = kAttnSplits; w <= kAttnMaxCluster; ++w) resident[w - kAttnSplits] = ctx->attn_occ[w][qt_i];
-        const AttnSplit sp = attn_split_plan(total, c.page_size, resident, c.n_kv_heads * rg_i);
-        const int ncl = sp.clusters, cs_i = sp.width, chunk = sp.keys_per_split;
-        max_cs = std::max(max_cs, cs_i);
-        int nsplit = ncl;   // stored per item: clusters sharing its keys
+        const AttnSplit sp = attn_split_plan(total, c.page_size, c.n_kv_heads * rg_i, ctx->attn_slots[attn_rows_n(R_i) / 16]);
+        const int nsplit = sp.splits, chunk = sp.keys_per_split;
+        if (chunk > kAttnTile + kAttnShortTail) all_short = false;
         I(ml.it_slot)[i] = it.slot;
         I(ml.it_row0)[i] = row;
         I(ml.it_rows)[i] = it.rows;
         I(ml.it_base)[i] = it.base;
         I(ml.it_nsplit)[i] = nsplit;
         I(ml.it_chunk)[i] = chunk;
-        I(ml.it_cs)[i] = cs_i;
         I(ml.it_part0)[i] = part0;
         max_nsplit = std::max(max_nsplit, nsplit);
         part0 += it.rows * c.n_q_heads * nsplit;
@@ -467,7 +464,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     const int maxR = max_item_rows * (Hq / Hkv);                      // query rows that share one KV head
     const int n_max = attn_rows_n(maxR);
     const int row_groups = (maxR + kAttnMaxRows - 1) / kAttnMaxRows;
-    const size_t asmem = attn_smem_bytes(hd, n_max);
+    const size_t asmem = attn_smem_bytes(hd, n_max, all_short);
     GemmArgs base = {};
     base.M = M;
     base.eps = c.rms_eps;
@@ -476,15 +473,15 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     // depth of the L2 hints a kernel issues for its successor's weights (bytes per successor CTA)
     const uint32_t pf_depth = ctx->pf_depth;
     auto launch_attn = [&](int l) -> int {
-        dim3 ag(max_cs * max_nsplit, Hkv * row_groups, n_items);   // cluster = the widest any request of the batch asks for
+        dim3 ag(max_nsplit, Hkv * row_groups, n_items);
         AttnArgs aa = {};
         aa.q = qbuf; aa.meta = meta; aa.kv_pool = ctx->kv_pool;
         aa.layer = l; aa.n_pages = c.n_pages; aa.page_size = c.page_size; aa.M = M; aa.Hq = Hq; aa.Hkv = Hkv;
-        aa.n_max = n_max; aa.row_groups = row_groups;
+        aa.n_max = n_max; aa.slot_c = attn_slot_c_bytes(hd, all_short); aa.row_groups = row_groups;
         aa.o_part = o_part; aa.m_part = m_part; aa.l_part = l_part; aa.tickets = ctx->W<int>(ctx->ws.tickets);
         aa.xf_out = (uint16_t*)xf_attn; aa.err = ctx->err_word();
-        if (hd == 128) CU(launch_pdl_cluster(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, max_cs, aa));
-        else CU(launch_pdl_cluster(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, max_cs, aa));
+        if (hd == 128) CU(launch_pdl(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, aa));
+        else CU(launch_pdl(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, aa));
         ctx->n_launch += 1;
         return PIPESD_OK;
     };
@@ -609,27 +606,29 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
     if (e != cudaSuccess) return bail(PIPESD_E_CUDA);
     if (ensure_device_ready() != PIPESD_OK) return bail(PIPESD_E_CUDA);
 
-    {   // clusters of 9 or 10 CTAs are non-portable sizes: opt in and ask how many such clusters the device keeps
-        // resident for each shared-memory footprint (query row tiles); run_pass widens a request's cluster only if
-        // all of the request's clusters then still run in one wave
-        const bool hd128 = c.head_dim == 128;
-        const void* fn = hd128 ? (const void*)attn_kernel<128> : (const void*)attn_kernel<64>;
-        if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
-            for (int w = kAttnSplits + 1; w <= kAttnMaxCluster; ++w)
-                for (int qt = 1; qt <= kAttnMaxRows / 16; ++qt) {
-                    cudaLaunchConfig_t lc = {};
-                    lc.gridDim = dim3(w, 1, 1);
-                    lc.blockDim = dim3(kAttnThreads);
-                    lc.dynamicSmemBytes = attn_smem_bytes(c.head_dim, 16 * qt);
-                    cudaLaunchAttribute at[1];
-                    at[0].id = cudaLaunchAttributeClusterDimension;
-                    at[0].val.clusterDim.x = w; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-                    lc.attrs = at; lc.numAttrs = 1;
-                    int n_clusters = 0;
-                    if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) == cudaSuccess) ctx->attn_occ[w][qt] = n_clusters;
-                }
-        }
-        (void)cudaGetLastError();
+    {   // CTAs of the attention kernel the device keeps resident at once, per footprint: the key-split plan of a request
+        // aims at one wave.  Counted here from the limits that bind (shared memory, registers, threads, tensor-memory
+        // columns): the runtime's occupancy query answers one CTA per SM for any kernel that allocates tensor memory.
+        int n_sm = 0, smem_sm = 0, smem_rsv = 0, regs_sm = 0, thr_sm = 0;
+        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, c.device) != cudaSuccess || n_sm < 1 ||
+            cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, c.device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&smem_rsv, cudaDevAttrReservedSharedMemoryPerBlock, c.device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, c.device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&thr_sm, cudaDevAttrMaxThreadsPerMultiProcessor, c.device) != cudaSuccess)
+            return bail(PIPESD_E_CUDA);
+        cudaFuncAttributes fa;
+        if (cudaFuncGetAttributes(&fa, c.head_dim == 128 ? (const void*)attn_kernel<128> : (const void*)attn_kernel<64>) != cudaSuccess)
+            return bail(PIPESD_E_CUDA);
+        const int regs_cta = ((fa.numRegs * 32 + 511) / 512 * 512) * (kAttnThreads / 32);     // allocated per warp in units of 512
+        for (int qt = 1; qt <= kAttnMaxRows / 16; ++qt)
+            for (int short_tail = 0; short_tail < 2; ++short_tail) {
+                const size_t smem_cta = attn_smem_bytes(c.head_dim, 16 * qt, short_tail != 0) + fa.sharedSizeBytes + smem_rsv;
+                int per_sm = (int)(smem_sm / smem_cta);
+                per_sm = std::min(per_sm, regs_sm / std::max(1, regs_cta));
+                per_sm = std::min(per_sm, thr_sm / kAttnThreads);
+                per_sm = std::min(per_sm, 512 / attn_tmem_cols(16 * qt));
+                ctx->attn_slots[qt][short_tail] = std::max(1, per_sm) * n_sm;
+            }
     }
     if (const char* e_pf = getenv("PIPESD_PF_KB")) ctx->pf_depth = (uint32_t)atoi(e_pf) << 10;
     ctx->kv_pool = (uint16_t*)mem->kv;
@@ -1153,13 +1152,20 @@ int32_t pipesd_gemm_run(const void* packed, const float* x, float* y, void* scra
     return gemm_run_with_scratch(packed, x, y, scratch, M, N, K, (cudaStream_t)cuda_stream);
 }
 
-int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t* resident_clusters,
-                                int32_t clusters_needed, int32_t* out3) {
-    if (!resident_clusters || !out3 || total_keys < 1 || page_size < 8 || page_size % 8) return PIPESD_E_INVALID;
-    int res[kAttnMaxCluster - kAttnSplits + 1];
-    for (int i = 0; i <= kAttnMaxCluster - kAttnSplits; ++i) res[i] = resident_clusters[i];
-    const AttnSplit p = attn_split_plan(total_keys, page_size, res, clusters_needed);
-    out3[0] = p.clusters; out3[1] = p.width; out3[2] = p.keys_per_split;
+int32_t pipesd_debug_attn_slots(pipesd_ctx* ctx, int32_t rows_per_kv_head, int32_t* out2) {
+    if (!ctx || !out2 || rows_per_kv_head < 1) return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_attn_slots");
+    const int qt = attn_rows_n(rows_per_kv_head) / 16;
+    out2[0] = ctx->attn_slots[qt][0];
+    out2[1] = ctx->attn_slots[qt][1];
+    return PIPESD_OK;
+}
+
+int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t* resident_ctas, int32_t units,
+                                int32_t* out3) {
+    if (!resident_ctas || !out3 || total_keys < 1 || page_size < 8 || page_size % 8 || units < 1) return PIPESD_E_INVALID;
+    const int slots[2] = {resident_ctas[0], resident_ctas[1]};
+    const AttnSplit p = attn_split_plan(total_keys, page_size, units, slots);
+    out3[0] = p.splits; out3[1] = p.keys_per_split; out3[2] = p.short_tail;
     return PIPESD_OK;
 }
 

@@ -44,35 +44,34 @@ def test_pure_host_entry_points():
 
 
 def test_attention_key_split_plan():
-    """The split of a request's keys over clusters and CTAs: a function of the request alone."""
-    wide = (48, 45, 41)            # clusters of 8, 9, 10 the device keeps resident (a B200, one query row tile)
-    # 2057 keys: 8 splits of 272 keys are three 128-key tiles per CTA, 9 splits of 240 are two, 10 no fewer
-    assert binding.debug_attn_split(2057, 16, wide, 32) == (1, 9, 240)
-    # the wider cluster must still hold the whole request in one wave
-    assert binding.debug_attn_split(2057, 16, (48, 31, 31), 32) == (1, 8, 272)
-    assert binding.debug_attn_split(2057, 16, (48, 0, 0), 32) == (1, 8, 272)          # widths unavailable
-    assert binding.debug_attn_split(2057, 16, (48, 31, 41), 32) == (1, 10, 208)       # 9 does not fit, 10 does: two tiles
-    # 1030 keys: 9 splits of 128 keys are one tile each, 8 splits of 144 are two; 521 keys: one tile either way
-    assert binding.debug_attn_split(1030, 16, wide, 8) == (1, 9, 128)
-    assert binding.debug_attn_split(521, 16, wide, 8) == (1, 8, 80)
-    # short requests: nothing to gain, stay at eight; splits are whole pages
-    assert binding.debug_attn_split(9, 16, wide, 8) == (1, 8, 16)
-    assert binding.debug_attn_split(100, 8, wide, 8) == (1, 8, 16)
-    assert binding.debug_attn_split(100, 64, wide, 8) == (1, 8, 64)
-    # one more cluster per 2048 keys, up to four, eight splits each
-    assert binding.debug_attn_split(4096, 16, wide, 32) == (2, 8, 256)
-    assert binding.debug_attn_split(8209, 16, wide, 16) == (4, 8, 272)
-    assert binding.debug_attn_split(40000, 16, wide, 16) == (4, 8, 1264)
+    """The split of a request's keys over CTAs: a function of the request (and the device) alone."""
+    b200 = (148, 296)              # resident CTAs without / with the cut-down third ring slot (head_dim 128, up to 16 rows)
+    # 2057 keys, 32 KV heads: 9 splits fill the wave (296 / 32); 240 keys each are two 128-key tiles, the second short
+    assert binding.debug_attn_split(2057, 16, b200, 32) == (9, 240, 1)
+    # with only the whole-slot footprint resident: 4 splits of 528 keys are five tiles; 4 is the fewest splits with five
+    assert binding.debug_attn_split(2057, 16, (148, 0), 32) == (4, 528, 0)
+    # fewer splits when they leave the same number of tiles: 521 keys, 8 KV heads: at most 5 splits by keys, all of
+    # them one or two tiles -> 112 keys (one tile) needs 5; 3 splits of 176 would be two
+    assert binding.debug_attn_split(521, 16, b200, 8) == (5, 112, 1)
+    # short requests: one split per 128 keys at most
+    assert binding.debug_attn_split(9, 16, b200, 8) == (1, 16, 1)
+    assert binding.debug_attn_split(100, 8, b200, 8) == (1, 104, 1)
+    assert binding.debug_attn_split(300, 64, b200, 8) == (3, 128, 1)
+    # long contexts, few heads: sixteen splits at most; 8209 keys: 16 splits of 528 keys are five tiles each, and so
+    # are 13 splits of 640
+    assert binding.debug_attn_split(8209, 16, (148, 148), 8) == (13, 640, 0)
+    assert binding.debug_attn_split(40000, 16, (148, 148), 8) == (16, 2512, 0)
     # every key is covered, splits are page multiples, whatever the length
     for total in list(range(1, 300)) + [1023, 1024, 1025, 2047, 2048, 4095, 4097, 6143, 6144, 12345]:
         for ps in (8, 16, 24, 64):
-            ncl, w, chunk = binding.debug_attn_split(total, ps, wide, 8)
-            assert 8 <= w <= 10 and 1 <= ncl <= 4 and chunk % ps == 0
-            assert ncl * w * chunk >= total
-            assert (w == 8) or ncl == 1
-            if w > 8:   # widened only for fewer tiles per CTA
-                c8 = -(-(-(-total // 8)) // ps) * ps
-                assert -(-chunk // 128) < -(-c8 // 128)
+            for units in (1, 8, 32):
+                n, chunk, short = binding.debug_attn_split(total, ps, b200, units)
+                assert 1 <= n <= 16 and chunk % ps == 0 and n * chunk >= total
+                assert (n - 1) * chunk < total or n == 1          # no split is wholly empty
+                assert short == (chunk <= 240)
+                if n > 1:   # one split fewer would mean more tiles per CTA
+                    c1 = -(-(-(-total // (n - 1))) // ps) * ps
+                    assert -(-c1 // 128) > -(-chunk // 128)
     import pytest
     with pytest.raises(binding.PipesdError):
-        binding.debug_attn_split(100, 12, wide, 8)
+        binding.debug_attn_split(100, 12, b200, 8)
