@@ -176,9 +176,11 @@ struct AttnArgs {
     int* err;
 };
 
-// grid (max splits of the launch, n_kv_heads * row_groups, n_items), block 288.
+// grid (max splits of the launch, n_kv_heads * row_groups, n_items), block 288.  The register bound is what lets two CTAs
+// share an SM: a CTA's nine warps put three on one of the SM's four register partitions (16K registers each), and two
+// such triples must fit it.
 template <int HD>
-__global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
+__global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a) {
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = AttnSmem<HD>;
     constexpr int HG = HD / 8;                                      // 8-element pieces of a row
@@ -240,6 +242,15 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
     auto slot_addr = [&](int i) { return ring_a + (uint32_t)(i % 3) * SM::kTileBytes; };   // ring slot of item i (K_t: 2t, V_t: 2t+1)
 
     bool ok = true;
+    uint32_t tmem_held = 0;        // tensor memory to give back before leaving, if any (address 0 is a valid one)
+    bool holds_tmem = false;
+    // Tensor memory is released off the critical path: after the partial result has been announced.
+    auto release_tmem = [&]() {
+        if (holds_tmem && warp == 8) {
+            tc_fence_after();
+            tmem_dealloc(tmem_held, tmem_cols);
+        }
+    };
     if (ntiles > 0) {
         uint32_t tmem = 0;
         if (warp == 8) {
@@ -513,10 +524,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
             tc_fence_before();
         }
         __syncthreads();
-        if (warp == 8) {
-            tc_fence_after();
-            tmem_dealloc(tmem, tmem_cols);
-        }
+        tmem_held = tmem;
+        holds_tmem = true;
     } else {
         // empty split: contributes nothing (finite zeros, so the merge can read it unconditionally)
         pdl_wait();
@@ -527,45 +536,51 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(const AttnArgs a) {
         }
         __syncthreads();
     }
-    if (nsplit == 1) return;
+    if (nsplit == 1) { release_tmem(); return; }
 
     // ---- the last CTA of this (request, KV head, row group) to arrive merges the splits, in split order
-    // (the barrier above orders the whole CTA's stores before thread 0's fence, and its fence after the ticket orders the
-    // other CTAs' partials before the loads that follow the barrier below)
+    // (the barrier above orders the whole CTA's stores before thread 0's ticket, a release; the ticket is also an acquire,
+    // and the barrier below orders it before everybody's loads of the other CTAs' partials)
     if (tid == 0) {
         int* ticket = a.tickets + ((size_t)item * Hkv + kvh) * a.row_groups + rg;
-        __threadfence();
-        const int t = atomicAdd(ticket, 1);
+        int t;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(t) : "l"(ticket) : "memory");
         const int last = (t == nsplit - 1);
         if (last) *ticket = 0;                                   // self-cleaning: ready for the next launch
-        __threadfence();
         *s_last = last;
     }
     __syncthreads();
+    release_tmem();
     if (!*s_last) return;
     // warp = row, lane = four columns: one round covers nine rows
     for (int rl = warp; rl < n_rows; rl += kAttnThreads / 32) {
-        float ms[kAttnMaxSplits], ls[kAttnMaxSplits];
-        float4 ov[kAttnMaxSplits];
         const size_t sl0 = slot0 + (size_t)rl * nsplit;
+        float ms[kAttnMaxSplits];
 #pragma unroll
-        for (int j = 0; j < kAttnMaxSplits; ++j) {               // all loads of the row in flight together
-            const bool on = j < nsplit;
-            ms[j] = on ? __ldcg(a.m_part + sl0 + j) : -INFINITY;
-            ls[j] = on ? __ldcg(a.l_part + sl0 + j) : 0.f;
-            ov[j] = (on && lane < HD / 4) ? __ldcg(reinterpret_cast<const float4*>(a.o_part + (sl0 + j) * HD) + lane)
-                                          : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+        for (int j = 0; j < kAttnMaxSplits; ++j) ms[j] = j < nsplit ? __ldcg(a.m_part + sl0 + j) : -INFINITY;
         float m = -INFINITY;
 #pragma unroll
         for (int j = 0; j < kAttnMaxSplits; ++j) m = fmaxf(m, ms[j]);
         float den = 0.f;
         float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int j = 0; j < kAttnMaxSplits; ++j) {
-            const float w = (ms[j] == -INFINITY) ? 0.f : exp2f(ms[j] - m);   // an empty split or one beyond the causal horizon
-            den += w * ls[j];
-            num.x += w * ov[j].x; num.y += w * ov[j].y; num.z += w * ov[j].z; num.w += w * ov[j].w;
+        for (int j0 = 0; j0 < kAttnMaxSplits; j0 += 8) {         // eight splits' loads in flight together, summed in split order
+            if (j0 >= nsplit) break;
+            float ls[8];
+            float4 ov[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const bool on = j0 + j < nsplit;
+                ls[j] = on ? __ldcg(a.l_part + sl0 + j0 + j) : 0.f;
+                ov[j] = (on && lane < HD / 4) ? __ldcg(reinterpret_cast<const float4*>(a.o_part + (sl0 + j0 + j) * HD) + lane)
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float w = (ms[j0 + j] == -INFINITY) ? 0.f : exp2f(ms[j0 + j] - m);   // an empty split or one beyond the causal horizon
+                den += w * ls[j];
+                num.x += w * ov[j].x; num.y += w * ov[j].y; num.z += w * ov[j].z; num.w += w * ov[j].w;
+            }
         }
         if (lane < HD / 4) {
             const int rho = rho0 + rl, gq = rho / rows, r_in = rho % rows;

@@ -14,9 +14,11 @@
 // Activations stay fp32 in the residual stream; the kernel that produces a GEMM input stores it already
 // split into bf16 hi + lo terms in B-fragment order ("xf" arrays), so the matching chunk of activations
 // rides in the same ring stage as its weights (two MMAs, one fp32 accumulator: 2^-17 relative).
-// Split-K: the S CTAs that share a row block form a thread-block cluster.  Each leaves its partial tile
-// in its own shared memory; after a cluster barrier the tiles are summed over distributed shared memory
-// in rank order (deterministic) and the epilogue runs on the sums -- no partial sums in global memory.
+// Split-K: the S CTAs that share a row block form a thread-block cluster.  Each of the block's eight 16-row tiles
+// is owned by one rank; every CTA writes its partial tiles straight into their owners' shared memory (remote
+// stores over distributed shared memory, posted), one cluster barrier follows, and each owner sums what it
+// received in rank order (deterministic) and runs the epilogue -- no partial sums in global memory, no remote
+// loads, and nobody has to wait for anybody after the barrier.
 // Epilogues: plain fp32 output; RoPE + q store + bf16 K/V page append (QKV); residual add + next RMSNorm's
 // gain and sum of squares (O and down projections); SiLU(gate)*up (gate/up projection).  RMSNorm itself
 // never runs as a kernel: the producer stores x*gain and per-block sums of squares, the consumer scales
@@ -31,7 +33,7 @@ constexpr int kGemmConsumers = kGemmConsumerWarps * 32;
 constexpr int kGemmThreads = kGemmConsumers + 32;           // + one producer warp
 constexpr int kGemmKC = 4;                                  // k16 steps per ring stage
 constexpr int kGemmWStage = kGemmKC * 4096;                 // weight bytes per stage
-constexpr int kGemmMinStages = 3, kGemmMaxStages = 6;
+constexpr int kGemmMinStages = 2, kGemmMaxStages = 6;
 constexpr int kGemmCtasPerSm = 3;
 constexpr int kGemmWave = 148 * kGemmCtasPerSm;
 constexpr int kGemmMaxSplit = 8;                            // portable cluster size
@@ -41,7 +43,11 @@ enum GemmMode { kPlain = 0, kQkvRope = 1, kResid = 2, kSwiglu = 3 };
 
 
 __host__ __device__ constexpr int gemm_stage_bytes(int NT) { return kGemmWStage + kGemmKC * NT * 512; }
-__host__ __device__ constexpr int gemm_smem_bytes(int NT, int stages) { return stages * gemm_stage_bytes(NT) + kGemmSmemTail; }
+// partial tiles received from the cluster: [owned tile][source rank][token][16 rows] fp32
+__host__ __device__ constexpr int gemm_recv_bytes(int NT, int S) { return ((8 + S - 1) / S) * S * (NT * 8) * 64; }
+__host__ __device__ constexpr int gemm_smem_bytes(int NT, int stages, int S) {
+    return stages * gemm_stage_bytes(NT) + kGemmSmemTail + gemm_recv_bytes(NT, S);
+}
 
 struct GemmPlan {
     int NT;  // n8 token tiles per token block (1..4)
@@ -87,7 +93,7 @@ static inline GemmPlan gemm_plan(int M, int N, int K) {
     int per_sm = (int)((ctas + 147) / 148);
     if (p.S > 1 && p.NT <= 2) per_sm = kGemmCtasPerSm;
     per_sm = per_sm < 1 ? 1 : (per_sm > kGemmCtasPerSm ? kGemmCtasPerSm : per_sm);
-    int budget = (227 * 1024) / per_sm - 1024 - kGemmSmemTail;
+    int budget = (227 * 1024) / per_sm - 1024 - kGemmSmemTail - gemm_recv_bytes(p.NT, p.S);
     p.stages = budget / gemm_stage_bytes(p.NT);
     p.stages = p.stages < kGemmMinStages ? kGemmMinStages : (p.stages > kGemmMaxStages ? kGemmMaxStages : p.stages);
     return p;
@@ -214,9 +220,11 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
     unsigned char* tail = smem + stages * kStageBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);              // full[stages], empty[stages]
     float* rstd_s = reinterpret_cast<float*>(tail + 128);             // [32]
-    float* tss_s = rstd_s + 32;                                       // [8 tiles][32 tokens]
+    float* tss_s = rstd_s + 32;                                       // rank 0: [8 tiles][32 tokens] sums of squares of the new rows
+    float* recv = reinterpret_cast<float*>(tail + kGemmSmemTail);     // [owned tile][source rank][token MT][row 16]
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * kGemmMaxStages;
+    const uint32_t ssq_bar = full0 + 8 * 2 * kGemmMaxStages;           // rank 0: one arrival per rank once its tile sums are stored
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rb = blockIdx.x / a.S, s = blockIdx.x % a.S, tb = blockIdx.y;   // s == rank in the cluster
     const int ks0 = (int)(((long)a.KS * s) / a.S), ks1 = (int)(((long)a.KS * (s + 1)) / a.S);
@@ -228,6 +236,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
             mbar_init(full0 + 8 * i, 1);
             mbar_init(empty0 + 8 * i, kGemmConsumerWarps);
         }
+        if (MODE == kResid) mbar_init(ssq_bar, (uint32_t)a.S);
         fence_mbar_init();
     }
     __syncthreads();
@@ -372,42 +381,51 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
         if (!ok && a.err && lane == 0) atomicExch(a.err, 2);
         // this CTA has consumed its last weights: from here on HBM idles until the successor streams
         if (ok) l2_prefetch_issue(a.pf, (int)(blockIdx.y * gridDim.x + blockIdx.x), (int)(gridDim.x * gridDim.y), threadIdx.x, kGemmConsumers);
-        // All consumers are past their last ring read before the ring is reused for the partial tile.
-        asm volatile("bar.sync 1, %0;" ::"n"(kGemmConsumers) : "memory");
-        // partial tile P[tile 8][token MT][row 16] (fp32) at the start of the ring
-        float* P = reinterpret_cast<float*>(smem);
+        // Every partial tile goes to the rank that owns the tile (tile % S), into slot [tile / S][this rank] of its receive
+        // buffer: token-major rows of 16 floats, as the epilogue reads them.
         const int g = lane >> 2, t = lane & 3;
+        const uint32_t recv_a = smem_u32(recv);
 #pragma unroll
-        for (int j = 0; j < 2; ++j)
+        for (int j = 0; j < 2; ++j) {
+            const int tile = warp * 2 + j, owner = tile % a.S, q = tile / a.S;
+            const uint32_t slot = recv_a + (uint32_t)((q * a.S + s) * MT * 64);
+            const uint32_t dst = a.S > 1 ? dsmem_addr(slot, (uint32_t)owner) : slot;
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                float* pt = P + ((warp * 2 + j) * MT + nt * 8 + 2 * t) * 16;
-                pt[g] = acc[j][nt][0];
-                pt[16 + g] = acc[j][nt][1];
-                pt[g + 8] = acc[j][nt][2];
-                pt[16 + g + 8] = acc[j][nt][3];
+                const uint32_t pt = dst + (uint32_t)((nt * 8 + 2 * t) * 64);
+                if (a.S > 1) {
+                    dsmem_st_f32(pt + g * 4, acc[j][nt][0]);
+                    dsmem_st_f32(pt + 64 + g * 4, acc[j][nt][1]);
+                    dsmem_st_f32(pt + (g + 8) * 4, acc[j][nt][2]);
+                    dsmem_st_f32(pt + 64 + (g + 8) * 4, acc[j][nt][3]);
+                } else {
+                    float* pl = recv + ((q * a.S + s) * MT + nt * 8 + 2 * t) * 16;
+                    pl[g] = acc[j][nt][0];
+                    pl[16 + g] = acc[j][nt][1];
+                    pl[g + 8] = acc[j][nt][2];
+                    pl[16 + g + 8] = acc[j][nt][3];
+                }
             }
+        }
     }
 
-    // ---------------- cluster reduction + epilogue (all 160 threads reach both barriers, also on errors)
+    // ---------------- cluster reduction + epilogue (all 160 threads reach the barrier, also on errors): after it every
+    // partial of this CTA's tiles has arrived, and nobody writes to or reads from another CTA's shared memory any more
     if (a.S > 1) cluster_sync_all(); else __syncthreads();
     pdl_wait();   // (long satisfied) every thread that touches the predecessors' global data has waited itself
     if (warp < kGemmConsumerWarps) {
         const int row = threadIdx.x & 15, tg = threadIdx.x >> 4;   // 16 lanes = the 16 rows of a tile
-        const uint32_t p_local = smem_base;
         // One tile of the row block: sum the S partial tiles in rank order, then the mode's epilogue.
         // xin / gin / cin / sin_ : prefetched epilogue inputs of this tile, or null to load them here.
         auto epi_tile = [&](int tile, const float* xin, const float* gin, const float* cin, const float* sin_) {
             const int pr = rb * 128 + tile * 16 + row;               // packed row
             float pv[NT][kGemmMaxSplit];
+            const float* rt = recv + (size_t)(tile / a.S) * a.S * MT * 16;    // this tile's partials, one per source rank
 #pragma unroll
             for (int i = 0; i < NT; ++i) {
-                const uint32_t off = (uint32_t)(((tile * MT + tg + 8 * i) * 16 + row) * 4);
 #pragma unroll
-                for (int r = 0; r < kGemmMaxSplit; ++r)      // independent loads, all in flight
-                    pv[i][r] = r < a.S ? (a.S > 1 ? dsmem_ld_f32(dsmem_addr(p_local + off, (uint32_t)r))
-                                                  : *reinterpret_cast<const float*>(smem + off))
-                                       : 0.f;
+                for (int r = 0; r < kGemmMaxSplit; ++r)
+                    pv[i][r] = r < a.S ? rt[(r * MT + tg + 8 * i) * 16 + row] : 0.f;
             }
 #pragma unroll
             for (int i = 0; i < NT; ++i) {
@@ -434,7 +452,7 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
                     q += __shfl_xor_sync(0xffffffffu, q, 4);
                     q += __shfl_xor_sync(0xffffffffu, q, 8);
                     if (row == 0) {
-                        // tile sums go to rank 0's shared memory, which adds the 8 tiles up after the barrier
+                        // tile sums go to rank 0's shared memory, which adds the 8 tiles up once every rank has reported
                         const uint32_t dst = smem_u32(tss_s + tile * 32 + tl);
                         if (a.S > 1) dsmem_st_f32(dsmem_addr(dst, 0u), q); else tss_s[tile * 32 + tl] = q;
                     }
@@ -479,15 +497,37 @@ __global__ void __launch_bounds__(kGemmThreads, kGemmCtasPerSm) gemm_wstream_ker
         } else {
             for (int tile = s; tile < 8; tile += a.S) epi_tile(tile, nullptr, nullptr, nullptr, nullptr);
         }
-    }
-    if (a.S > 1) cluster_sync_all(); else __syncthreads();
-    if (MODE == kResid && s == 0 && threadIdx.x < MT) {
-        const int tok = tok0 + threadIdx.x;
-        if (tok < a.M) {
-            float q = 0.f;
+        if (MODE == kResid) {
+            // Sums of squares of the new rows: every rank has stored its tiles' sums in rank 0's shared memory; one
+            // thread per rank reports that (a release that covers the CTA's stores through the barrier before it) and the
+            // rank is done.  Rank 0 waits for the S reports, adds the eight tiles up in order and writes the block's sum.
+            asm volatile("bar.sync 1, %0;" ::"n"(kGemmConsumers) : "memory");
+            if (threadIdx.x == 0) {
+                if (a.S > 1)
+                    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(dsmem_addr(ssq_bar, 0u)) : "memory");
+                else
+                    mbar_arrive(ssq_bar);
+            }
+            if (s == 0 && threadIdx.x < 32) {
+                bool got = false;
+                for (uint32_t it = 0; it < (1u << 22) && !got; ++it) {
+                    uint32_t okw;
+                    asm volatile(
+                        "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                        : "=r"(okw) : "r"(ssq_bar), "r"(0u) : "memory");
+                    got = okw != 0;
+                }
+                if (!got && a.err && threadIdx.x == 0) atomicExch(a.err, 5);
+                for (int tl = threadIdx.x; tl < MT; tl += 32) {
+                    const int tok = tok0 + tl;
+                    if (tok < a.M) {
+                        float q = 0.f;
 #pragma unroll
-            for (int tile = 0; tile < 8; ++tile) q += tss_s[tile * 32 + threadIdx.x];
-            a.ssq_out[(size_t)rb * a.M + tok] = q;
+                        for (int tile = 0; tile < 8; ++tile) q += tss_s[tile * 32 + tl];
+                        a.ssq_out[(size_t)rb * a.M + tok] = got ? q : 0.f;
+                    }
+                }
+            }
         }
     }
 }
@@ -496,10 +536,10 @@ template <int MODE>
 static inline cudaError_t gemm_launch_mode(const GemmPlan& p, const GemmArgs& a, cudaStream_t st) {
     dim3 grid(p.RB * p.S, p.TB);
     switch (p.NT) {
-        case 1: return launch_pdl_cluster(gemm_wstream_kernel<1, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(1, p.stages), st, p.S, a);
-        case 2: return launch_pdl_cluster(gemm_wstream_kernel<2, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(2, p.stages), st, p.S, a);
-        case 3: return launch_pdl_cluster(gemm_wstream_kernel<3, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(3, p.stages), st, p.S, a);
-        default: return launch_pdl_cluster(gemm_wstream_kernel<4, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(4, p.stages), st, p.S, a);
+        case 1: return launch_pdl_cluster(gemm_wstream_kernel<1, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(1, p.stages, p.S), st, p.S, a);
+        case 2: return launch_pdl_cluster(gemm_wstream_kernel<2, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(2, p.stages, p.S), st, p.S, a);
+        case 3: return launch_pdl_cluster(gemm_wstream_kernel<3, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(3, p.stages, p.S), st, p.S, a);
+        default: return launch_pdl_cluster(gemm_wstream_kernel<4, MODE>, grid, dim3(kGemmThreads), gemm_smem_bytes(4, p.stages, p.S), st, p.S, a);
     }
 }
 
@@ -518,7 +558,7 @@ static inline cudaError_t gemm_launch(int mode, const GemmPlan& p, GemmArgs a, c
 template <int NT, int MODE>
 static inline cudaError_t gemm_set_attr() {
     cudaError_t e = cudaFuncSetAttribute(gemm_wstream_kernel<NT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         gemm_smem_bytes(NT, kGemmMaxStages));
+                                         gemm_smem_bytes(NT, kGemmMaxStages, 7));
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(gemm_wstream_kernel<NT, MODE>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
 }

@@ -619,12 +619,15 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         cudaFuncAttributes fa;
         if (cudaFuncGetAttributes(&fa, c.head_dim == 128 ? (const void*)attn_kernel<128> : (const void*)attn_kernel<64>) != cudaSuccess)
             return bail(PIPESD_E_CUDA);
-        const int regs_cta = ((fa.numRegs * 32 + 511) / 512 * 512) * (kAttnThreads / 32);     // allocated per warp in units of 512
+        // registers: allocated per warp (in units of 512), and a CTA's warps are dealt to the SM's four register
+        // partitions in turn, so the fullest partition binds
+        const int regs_warp = (fa.numRegs * 32 + 511) / 512 * 512;
+        const int warps_part = (kAttnThreads / 32 + 3) / 4;
         for (int qt = 1; qt <= kAttnMaxRows / 16; ++qt)
             for (int short_tail = 0; short_tail < 2; ++short_tail) {
                 const size_t smem_cta = attn_smem_bytes(c.head_dim, 16 * qt, short_tail != 0) + fa.sharedSizeBytes + smem_rsv;
                 int per_sm = (int)(smem_sm / smem_cta);
-                per_sm = std::min(per_sm, regs_sm / std::max(1, regs_cta));
+                per_sm = std::min(per_sm, (regs_sm / 4) / std::max(1, regs_warp * warps_part));
                 per_sm = std::min(per_sm, thr_sm / kAttnThreads);
                 per_sm = std::min(per_sm, 512 / attn_tmem_cols(16 * qt));
                 ctx->attn_slots[qt][short_tail] = std::max(1, per_sm) * n_sm;
