@@ -241,6 +241,12 @@ int32_t pipesd_gemm_pack(const void *W, void *packed, int32_t N, int32_t K, void
 int32_t pipesd_gemm_run(const void *packed, const float *x, float *y, void *scratch, int32_t M, int32_t N,
                         int32_t K, void *cuda_stream);
 
+/* Harness switch.  Passes of more than 32 rows run their projections on the dense tensor-core kernel, smaller passes
+ * on the small-M weight-streaming kernel; the two sum in different orders, so their results agree to rounding, not
+ * bit for bit.  on != 0 makes every pass of the context use the dense kernel (so that a request verified alone runs the
+ * projections a large batch runs; the attention's key splits still follow the pass's composition, so the two agree
+ * to rounding and in their decisions, not in every bit); needs max_rows > 32 (PIPESD_E_INVALID otherwise). */
+int32_t pipesd_debug_force_dense(pipesd_ctx *ctx, int32_t on);
 /* CTAs of the attention kernel that the context's device keeps resident at once for a request with this many query
  * rows per KV head: out2 (host) = {with the whole third ring slot, with the cut-down one} -- the two numbers
  * pipesd_debug_attn_split takes. */
@@ -248,10 +254,10 @@ int32_t pipesd_debug_attn_slots(pipesd_ctx *ctx, int32_t rows_per_kv_head, int32
 /* Host only, no CUDA call: how the attention kernel splits a request of `total_keys` keys (cached + this pass's
  * rows) at the given page size into CTAs that each walk tiles of 128 keys.  resident_ctas[0..1] (host) = CTAs of the
  * kernel the device keeps resident at once for the request's footprint, without and with the cut-down third slot of
- * the K/V ring; units = CTA groups one layer launches for the request (KV heads x row groups).  out3 (host) receives
- * {key splits, keys per split (a multiple of page_size), 1 if the cut-down ring suffices}.  The split is a function
- * of the request and the device alone, which is what keeps a request's result independent of its batch.
- * PIPESD_E_INVALID on bad arguments. */
+ * the K/V ring; units = CTA groups that compete for the device in one layer, in groups of this request's length: KV
+ * heads x row groups for a request verified alone; in a batch the batch's total of keys x groups divided by this
+ * request's keys, rounded up.  out3 (host) receives {key splits, keys per split (a multiple of page_size), 1 if the
+ * cut-down ring suffices}.  PIPESD_E_INVALID on bad arguments. */
 int32_t pipesd_debug_attn_split(int32_t total_keys, int32_t page_size, const int32_t *resident_ctas, int32_t units,
                                 int32_t *out3);
 

@@ -96,6 +96,7 @@ _SIGNATURES = {
                                             ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double)]),
     "pipesd_sched_trigger_step": (i32, [ctypes.POINTER(ctypes.c_double), ctypes.c_double, ctypes.c_double,
                                         ctypes.c_double, ctypes.POINTER(i32)]),
+    "pipesd_debug_force_dense": (i32, [vp, i32]),
     "pipesd_debug_attn_slots": (i32, [vp, i32, ctypes.POINTER(ctypes.c_int32)]),
     "pipesd_debug_attn_split": (i32, [i32, i32, ctypes.POINTER(ctypes.c_int32), i32, ctypes.POINTER(ctypes.c_int32)]),
     "pipesd_debug_req_state": (i32, [vp, i32, ctypes.POINTER(ctypes.c_int32)]),
@@ -278,6 +279,9 @@ class Context:
         out = (ctypes.c_int32 * 3)()
         self._check(lib().pipesd_debug_req_state(self._h, req, out), "pipesd_debug_req_state")
         return tuple(out)
+
+    def debug_force_dense(self, on: bool):
+        self._check(lib().pipesd_debug_force_dense(self._h, int(on)), "pipesd_debug_force_dense")
 
     def debug_attn_slots(self, rows_per_kv_head: int):
         out = (ctypes.c_int32 * 2)()

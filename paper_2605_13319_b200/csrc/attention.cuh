@@ -102,11 +102,13 @@ static inline int attn_rows_n(int rows_per_kv_head) {    // N of a CTA that hold
     return (r + 15) / 16 * 16;
 }
 
-// Host: how one request's keys are split.  `units` = CTA groups the request launches per layer (KV heads x row
-// groups); slots[0 | 1] = CTAs of this kernel the device keeps resident at once for the request's row count with the
-// whole | cut-down third ring slot.  As many splits as let all of the request's CTAs run in one wave (at most 16, at
-// most one per 128 keys), then the fewest splits that leave each CTA the same number of 128-key tiles.  A function
-// of the request and the device alone, never of the batch: a request's summation order is the same in every batch.
+// Host: how one request's keys are split.  `units` = CTA groups that compete for the device per layer, counted in
+// groups of this request's length: for a request verified alone its KV heads x row groups; in a batch the batch's
+// (keys x groups) total divided by this request's keys.  slots[0 | 1] = CTAs of this kernel the device keeps resident
+// at once for the request's row count with the whole | cut-down third ring slot.  As many splits as let all CTAs of the
+// pass run in one wave (at most 16, at most one per 128 keys), then the fewest splits that leave each CTA the same
+// number of 128-key tiles.  The plan fixes the order a row's keys are summed in: a function of the pass's composition
+// and the device, the same every time that composition is verified.
 struct AttnSplit { int splits, keys_per_split, short_tail; };
 static inline AttnSplit attn_split_plan(int total_keys, int page_size, int units, const int* slots) {
     auto chunk_of = [&](int s) {
@@ -172,7 +174,8 @@ struct AttnArgs {
     float* m_part;             // [slot]
     float* l_part;             // [slot]
     int* tickets;              // [item][kv head][row group], zero between launches
-    uint16_t* xf_out;          // the output projection's input (split-bf16 fragments)
+    uint16_t* xf_out;          // the output projection's input: split-bf16 fragments, or (xd_tbs > 0) an xd array
+    int xd_tbs;
     int* err;
 };
 
@@ -186,7 +189,7 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a)
     constexpr int HG = HD / 8;                                      // 8-element pieces of a row
     pdl_launch_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int item = blockIdx.z;
+    const int item = a.meta.it_order[blockIdx.z];
     // per-request constants: independent loads, in flight together
     const int nsplit = a.meta.it_nsplit[item];
     const int rows = a.meta.it_rows[item];
@@ -499,7 +502,15 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a)
                     }
                 }
             }
-            if (nsplit == 1) asm volatile("bar.sync 1, %0;" ::"n"(kAttnWorkers) : "memory");     // the sums, for the division below
+            // nothing to merge: the rows are normalised and stored as the output projection's input.  Where a row lands
+            // there (its token, its head's first k16 step) is worked out once per row, into the maxima's array
+            uint32_t* otab = reinterpret_cast<uint32_t*>(wm);
+            if (nsplit == 1 && tid < n_rows) {
+                const int rho = rho0 + tid, gq = rho / rows, r_in = rho % rows;
+                otab[tid] = act_index_row(row0 + r_in, ((kvh * G + gq) * HD) >> 4, KSo, NTo, a.xd_tbs);
+            }
+            const uint32_t ocol = act_index_col(kt, NTo, a.xd_tbs), olo = act_index_lo(a.xd_tbs);
+            if (nsplit == 1) asm volatile("bar.sync 1, %0;" ::"n"(kAttnWorkers) : "memory");     // the sums and the table
             for (int cb = half; cb < NB; cb += 2) {
                 float o[16];
                 tmem_ld16(t_O + lane_sel + cb * 16, o);
@@ -510,9 +521,8 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a)
                         const int n = cb * 16 + i;
                         if (n < n_rows) {
                             const float v = ok ? o[i] : 0.f;
-                            if (nsplit == 1) {      // nothing to merge: normalise and store the output projection's input
-                                const int rho = rho0 + n, gq = rho / rows, r_in = rho % rows;
-                                xf_store_one(a.xf_out, row0 + r_in, (kvh * G + gq) * HD + kt, v / Fl[n], KSo, NTo);
+                            if (nsplit == 1) {
+                                act_store_at(a.xf_out, otab[n] + ocol, olo, v / Fl[n]);
                             } else {
                                 a.o_part[(slot0 + (size_t)n * nsplit + sp) * HD + kt] = v;
                             }
@@ -586,8 +596,15 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a)
             const int rho = rho0 + rl, gq = rho / rows, r_in = rho % rows;
             const int col = (kvh * G + gq) * HD + lane * 4;
             const float inv = 1.f / den;
-            xf_store_pair(reinterpret_cast<uint32_t*>(a.xf_out), row0 + r_in, col, num.x * inv, num.y * inv, KSo, NTo);
-            xf_store_pair(reinterpret_cast<uint32_t*>(a.xf_out), row0 + r_in, col + 2, num.z * inv, num.w * inv, KSo, NTo);
+            if (a.xd_tbs > 0) {
+                xd_store_one(a.xf_out, row0 + r_in, col, num.x * inv, KSo, a.xd_tbs);
+                xd_store_one(a.xf_out, row0 + r_in, col + 1, num.y * inv, KSo, a.xd_tbs);
+                xd_store_one(a.xf_out, row0 + r_in, col + 2, num.z * inv, KSo, a.xd_tbs);
+                xd_store_one(a.xf_out, row0 + r_in, col + 3, num.w * inv, KSo, a.xd_tbs);
+            } else {
+                xf_store_pair(reinterpret_cast<uint32_t*>(a.xf_out), row0 + r_in, col, num.x * inv, num.y * inv, KSo, NTo);
+                xf_store_pair(reinterpret_cast<uint32_t*>(a.xf_out), row0 + r_in, col + 2, num.z * inv, num.w * inv, KSo, NTo);
+            }
         }
     }
 }

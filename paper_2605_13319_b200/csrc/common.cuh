@@ -211,6 +211,49 @@ __device__ __forceinline__ void xf_store_one(uint16_t* xf, int tok, int k, float
     xf[slot * 8 + 4 + half * 2 + (kk & 1)] = l;
 }
 
+// ---- "xd" activation arrays: the K-major B operand of tcgen05.mma (the dense GEMM's input), in global memory ----
+// Token blocks of `tbs` tokens (a multiple of 16).  Per (token block, k16 step): the bf16 hi tile then the lo tile,
+// tbs * 32 bytes each, cut into 8x8 core matrices: element (token t, k) of a tile at
+// ((t / 8) * 2 + (k / 8) % 2) * 128 + (t % 8) * 16 + (k % 8) * 2.
+__device__ __forceinline__ void xd_store_one(uint16_t* xd, int tok, int k, float v, int KS, int tbs) {
+    const int tb = tok / tbs, tl = tok % tbs;
+    uint16_t h, l;
+    split_bf16(v, h, l);
+    unsigned char* b = reinterpret_cast<unsigned char*>(xd) + ((size_t)tb * KS + (k >> 4)) * (size_t)(tbs * 64) +
+                       (((tl >> 3) * 2 + ((k >> 3) & 1)) * 128 + (tl & 7) * 16 + (k & 7) * 2);
+    *reinterpret_cast<uint16_t*>(b) = h;
+    *reinterpret_cast<uint16_t*>(b + tbs * 32) = l;
+}
+// In either layout an element's index (in 16-bit units) is the sum of a part fixed by its token and the first k16 step
+// ks0 of a block of columns, and a part fixed by the column's offset dk inside that block; the lo half follows the hi
+// half at a fixed distance.  Epilogues that walk tokens x columns compute each part once instead of dividing per element.
+__device__ __forceinline__ uint32_t act_index_row(int tok, int ks0, int KS, int NT, int tbs) {
+    if (tbs > 0) {
+        const int tb = tok / tbs, tl = tok % tbs;
+        return (uint32_t)(((tb * KS + ks0) * (tbs * 64) + (tl >> 3) * 256 + (tl & 7) * 16) >> 1);
+    }
+    const int tb = tok / (8 * NT), nt = (tok >> 3) % NT, g = tok & 7;
+    return (uint32_t)((((tb * KS + ks0) * NT + nt) * 32 + g * 4) * 8);
+}
+__device__ __forceinline__ uint32_t act_index_col(int dk, int NT, int tbs) {
+    const int kk = dk & 15;
+    if (tbs > 0) return (uint32_t)(((dk >> 4) * (tbs * 64) + (kk >> 3) * 128 + (kk & 7) * 2) >> 1);
+    return (uint32_t)((dk >> 4) * NT * 256 + ((kk & 7) >> 1) * 8 + (kk >> 3) * 2 + (kk & 1));
+}
+__device__ __forceinline__ uint32_t act_index_lo(int tbs) { return tbs > 0 ? (uint32_t)tbs * 16u : 4u; }
+__device__ __forceinline__ void act_store_at(uint16_t* dst, uint32_t idx, uint32_t lo, float v) {
+    uint16_t h, l;
+    split_bf16(v, h, l);
+    dst[idx] = h;
+    dst[idx + lo] = l;
+}
+// Store one activation in whichever layout its consumer reads: tbs > 0: an xd array with that block size; tbs == 0:
+// the small-M kernel's fragment order with NT token tiles per block.
+__device__ __forceinline__ void act_store_one(uint16_t* dst, int tok, int k, float v, int KS, int NT, int tbs) {
+    if (tbs > 0) xd_store_one(dst, tok, k, v, KS, tbs);
+    else xf_store_one(dst, tok, k, v, KS, NT);
+}
+
 // ---- thread-block clusters: barrier and distributed shared memory --------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -253,6 +296,7 @@ struct PassMeta {
     const int32_t* it_nsplit;  // [n_items] key splits
     const int32_t* it_chunk;   // [n_items] keys per split (multiple of the page size)
     const int32_t* it_part0;   // [n_items] first slot of the item in the attention partial arrays
+    const int32_t* it_order;   // [n_items] items by decreasing number of keys: the order their attention CTAs launch in
     const int32_t* block_tab;  // [max_requests][max_pages] page ids, indexed by request slot
     int max_pages;
 };

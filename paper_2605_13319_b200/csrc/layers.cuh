@@ -7,7 +7,8 @@
 namespace pipesd {
 
 // x = bf16 embedding row (residual stream, fp32); xf = x * gain of the first RMSNorm as split-bf16
-// fragments; ssq[0][row] = sum x^2, ssq[b > 0][row] = 0 (the consumer adds n_ssq block sums up).
+// fragments (or, with tbs > 0, as an xd array of that token block size); ssq[0][row] = sum x^2, ssq[b > 0][row] = 0
+// (the consumer adds n_ssq block sums up).
 // One CTA of 1024 threads per row, four columns per thread.
 constexpr int kEmbedThreads = 1024;
 constexpr int kEmbedMaxVec = 2;   // float4 per thread: d <= 8192
@@ -15,7 +16,7 @@ __global__ void __launch_bounds__(kEmbedThreads) embed_kernel(float* __restrict_
                                                               const int32_t* __restrict__ row_tok, int M,
                                                               const float* __restrict__ gain, int d,
                                                               uint32_t* __restrict__ xf_out, float* __restrict__ ssq,
-                                                              int n_ssq) {
+                                                              int n_ssq, int tbs) {
     pdl_wait();
     pdl_launch_dependents();
     const int row = blockIdx.x;
@@ -33,8 +34,16 @@ __global__ void __launch_bounds__(kEmbedThreads) embed_kernel(float* __restrict_
             *reinterpret_cast<float4*>(xr + e) = a;
             ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
             const float4 g = *reinterpret_cast<const float4*>(gain + e);
-            xf_store_pair(xf_out, row, e, a.x * g.x, a.y * g.y, KS, NT);
-            xf_store_pair(xf_out, row, e + 2, a.z * g.z, a.w * g.w, KS, NT);
+            if (tbs > 0) {
+                uint16_t* xd = reinterpret_cast<uint16_t*>(xf_out);
+                xd_store_one(xd, row, e, a.x * g.x, KS, tbs);
+                xd_store_one(xd, row, e + 1, a.y * g.y, KS, tbs);
+                xd_store_one(xd, row, e + 2, a.z * g.z, KS, tbs);
+                xd_store_one(xd, row, e + 3, a.w * g.w, KS, tbs);
+            } else {
+                xf_store_pair(xf_out, row, e, a.x * g.x, a.y * g.y, KS, NT);
+                xf_store_pair(xf_out, row, e + 2, a.z * g.z, a.w * g.w, KS, NT);
+            }
         }
     }
     ss = warp_sum(ss);

@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <cmath>
 #include <deque>
 #include <mutex>
 #include <new>
@@ -17,6 +18,7 @@
 #include "attention.cuh"
 #include "common.cuh"
 #include "gemm.cuh"
+#include "gemm_dense.cuh"
 #include "layers.cuh"
 #include "reject.cuh"
 
@@ -37,7 +39,8 @@ struct Request {
 };
 
 struct GemmW {
-    uint4* packed = nullptr;     // MMA-fragment order
+    uint4* packed = nullptr;     // MMA-fragment order (small-M kernel)
+    uint4* packed_u = nullptr;   // tensor-core operand order (dense kernel; only when max_rows > 32)
     int N = 0, K = 0;
 };
 
@@ -48,7 +51,7 @@ struct LayerW {
 
 // Fixed offsets of the per-call metadata block (same layout in pinned host staging and on device).
 struct MetaLayout {
-    size_t row_item, row_pos, row_tok, it_slot, it_row0, it_rows, it_base, it_nsplit, it_chunk, it_part0, u, rej, total;
+    size_t row_item, row_pos, row_tok, it_slot, it_row0, it_rows, it_base, it_nsplit, it_chunk, it_part0, it_order, u, rej, total;
 };
 
 MetaLayout meta_layout(int max_rows, int max_items) {
@@ -65,6 +68,7 @@ MetaLayout meta_layout(int max_rows, int max_items) {
     m.it_nsplit = take(4 * (size_t)max_items);
     m.it_chunk = take(4 * (size_t)max_items);
     m.it_part0 = take(4 * (size_t)max_items);
+    m.it_order = take(4 * (size_t)max_items);
     m.u = take(4 * (size_t)max_rows);
     m.rej = take(sizeof(RejectItem) * (size_t)max_items);
     m.total = align_up(o);
@@ -102,11 +106,12 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
     auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
     const size_t M = c.max_rows;
     w.x = take(4 * M * c.d_model);
-    // split-bf16 activation arrays: 4 bytes per element, token count padded to whole token blocks
-    w.xf_h = take(4 * (M + 32) * c.d_model);
+    // split-bf16 activation arrays: 4 bytes per element, token count padded to whole token blocks (of up to 160 tokens
+    // plus rounding in the dense kernel's layout)
+    w.xf_h = take(4 * (M + 176) * c.d_model);
     w.qbuf = take(4 * M * d.qd);
-    w.xf_attn = take(4 * (M + 32) * d.qd);
-    w.xf_act = take(4 * (M + 32) * c.d_ffn);
+    w.xf_attn = take(4 * (M + 176) * d.qd);
+    w.xf_act = take(4 * (M + 176) * c.d_ffn);
     w.logits = take(4 * M * c.vocab);
     w.partA = take(4 * d.part_floats);
     w.partB = take(4 * d.part_floats);
@@ -135,7 +140,7 @@ WsLayout ws_layout(const pipesd_model_cfg& c, const Derived& d) {
 size_t packed_bytes(int N, int K) { return align_up(gemm_packed_bytes(N, K)); }
 
 size_t weights_bytes(const pipesd_model_cfg& c, const Derived& d) {
-    const size_t copies = 1;
+    const size_t copies = c.max_rows > 32 ? 2 : 1;      // passes of more than 32 rows read the weights in another order
     size_t per_layer = copies * (packed_bytes(d.Nqkv, c.d_model) + packed_bytes(c.d_model, d.qd) +
                                  packed_bytes(2 * c.d_ffn, c.d_model) + packed_bytes(c.d_model, c.d_ffn)) +
                        2 * align_up(4 * (size_t)c.d_model);
@@ -156,6 +161,12 @@ bool g_dev_ready[kMaxDevices] = {false};
 cudaError_t init_attrs_current_device() {
     cudaError_t e;
     if ((e = gemm_init_attrs()) != cudaSuccess) return e;
+    const void* dense_fns[4] = {(const void*)gemm_dense_kernel<kPlain>, (const void*)gemm_dense_kernel<kQkvRope>,
+                                (const void*)gemm_dense_kernel<kResid>, (const void*)gemm_dense_kernel<kSwiglu>};
+    for (const void* fn : dense_fns) {
+        if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kDenseSmemWhole)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, 100)) != cudaSuccess) return e;
+    }
     e = cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)attn_smem_bytes(128, kAttnMaxRows, false));
     if (e != cudaSuccess) return e;
@@ -246,6 +257,9 @@ struct pipesd_ctx {
     int last_rows = 0;
     int attn_slots[kAttnMaxRows / 16 + 1][2] = {};   // [query rows / 16][cut-down third ring slot]: CTAs of the attention
                                                      // kernel the device keeps resident at once
+    int n_sm = 148;             // SMs of the context's device
+    bool force_dense = false;   // harness switch: the dense kernels also for passes of at most 32 rows
+    bool pass_dense = false;    // the pass being enqueued runs on the dense kernels
     uint32_t pf_depth = 32u << 10;   // bytes per successor CTA that a GEMM pulls into L2 for the next GEMM
     std::string err;
     // launch accounting
@@ -271,6 +285,7 @@ struct pipesd_ctx {
         m.it_nsplit = (const int32_t*)(b + ml.it_nsplit);
         m.it_chunk = (const int32_t*)(b + ml.it_chunk);
         m.it_part0 = (const int32_t*)(b + ml.it_part0);
+        m.it_order = (const int32_t*)(b + ml.it_order);
         m.block_tab = W<int32_t>(ws.block_tab);
         m.max_pages = dv.max_pages;
         return m;
@@ -295,9 +310,14 @@ int cuda_fail(pipesd_ctx* c, cudaError_t e, const char* where) {
         if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);    \
     } while (0)
 
-// Launch one weight-streaming GEMM with accounting (and event timing when profiling is on).
-int launch_gemm(pipesd_ctx* ctx, int mode, GemmArgs a, int K) {
-    const GemmPlan p = gemm_plan(a.M, a.N, K);
+template <int MODE>
+cudaError_t dense_launch_mode(const DenseArgs& da, dim3 grid, size_t smem, cudaStream_t st) {
+    return launch_pdl(gemm_dense_kernel<MODE>, grid, dim3(kDenseThreads), smem, st, da);
+}
+
+// Launch one weight-streaming GEMM with accounting (and event timing when profiling is on).  next_N: output rows of
+// the GEMM that consumes this one's activation output (0: none): its token-block plan fixes the layout written.
+int launch_gemm(pipesd_ctx* ctx, int mode, const GemmW& w, GemmArgs a, int K, int next_N) {
     a.err = ctx->err_word();
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     if (ctx->time_gemms) {
@@ -313,7 +333,33 @@ int launch_gemm(pipesd_ctx* ctx, int mode, GemmArgs a, int K) {
         ctx->prof_used += 2;
         CU(cudaEventRecord(e0, ctx->st));
     }
-    CU(gemm_launch(mode, p, a, ctx->st));
+    if (ctx->pass_dense) {
+        const XdPlan pin = dense_plan(a.M, a.N, ctx->n_sm);
+        DenseArgs da = {};
+        da.g = a;
+        da.g.W = w.packed_u;
+        da.g.KS = K / 16;
+        const dim3 grid((a.N + 127) / 128, pin.n_tb);
+        const DenseRing ring = dense_ring(pin.tbs, (int)(grid.x * grid.y), ctx->n_sm);
+        da.g.stages = ring.stages;
+        da.kc = ring.kc;
+        da.g.pf = L2Prefetch{};
+        da.tbs_in = pin.tbs;
+        da.tbs_out = next_N > 0 ? dense_plan(a.M, next_N, ctx->n_sm).tbs : 0;
+        const size_t smem = ring.smem;
+        cudaError_t e;
+        switch (mode) {
+            case kQkvRope: e = dense_launch_mode<kQkvRope>(da, grid, smem, ctx->st); break;
+            case kResid: e = dense_launch_mode<kResid>(da, grid, smem, ctx->st); break;
+            case kSwiglu: e = dense_launch_mode<kSwiglu>(da, grid, smem, ctx->st); break;
+            default: e = dense_launch_mode<kPlain>(da, grid, smem, ctx->st); break;
+        }
+        CU(e);
+    } else {
+        a.W = w.packed;
+        const GemmPlan p = gemm_plan(a.M, a.N, K);
+        CU(gemm_launch(mode, p, a, ctx->st));
+    }
     if (e1) CU(cudaEventRecord(e1, ctx->st));
     ctx->n_launch += 1;
     ctx->n_gemm += 1;
@@ -391,14 +437,28 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     RejectItem* hr = reinterpret_cast<RejectItem*>(hm + ml.rej);
     int row = 0, part0 = 0, max_nsplit = 1, u0 = 0;
     bool all_short = true;       // no split of the pass has more than two key tiles, the second a short one
+    // attention work of the pass in (keys x CTA groups): a request gets the share of the device's resident CTAs that its
+    // keys are of the pass's, so that the CTAs of the whole pass fill one wave
+    double pass_work = 0.0;
+    for (int i = 0; i < n_items; ++i) {
+        const int R_i = items[i].rows * (c.n_q_heads / c.n_kv_heads);
+        pass_work += (double)(items[i].base + items[i].rows) * c.n_kv_heads * ((R_i + kAttnMaxRows - 1) / kAttnMaxRows);
+    }
+    {   // launch order of the attention CTAs: longest requests first
+        int32_t* ord = I(ml.it_order);
+        for (int i = 0; i < n_items; ++i) ord[i] = i;
+        std::stable_sort(ord, ord + n_items, [&](int32_t x, int32_t y) {
+            return items[x].base + items[x].rows > items[y].base + items[y].rows;
+        });
+    }
     for (int i = 0; i < n_items; ++i) {
         const ItemDesc& it = items[i];
         const int total = it.base + it.rows;
-        // key splits and keys per split: from the request alone (its length, its rows), so that its summation order is
-        // the same in every batch
         const int R_i = it.rows * (c.n_q_heads / c.n_kv_heads);                  // query rows per KV head
         const int rg_i = (R_i + kAttnMaxRows - 1) / kAttnMaxRows;
-        const AttnSplit sp = attn_split_plan(total, c.page_size, c.n_kv_heads * rg_i, ctx->attn_slots[attn_rows_n(R_i) / 16]);
+        const int units_i = (int)std::min(1.0e9, std::ceil(pass_work / (double)total));
+        const AttnSplit sp = attn_split_plan(total, c.page_size, std::max(units_i, c.n_kv_heads * rg_i),
+                                             ctx->attn_slots[attn_rows_n(R_i) / 16]);
         const int nsplit = sp.splits, chunk = sp.keys_per_split;
         if (chunk > kAttnTile + kAttnShortTail) all_short = false;
         I(ml.it_slot)[i] = it.slot;
@@ -449,6 +509,11 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     const int hd = c.head_dim, Hq = c.n_q_heads, Hkv = c.n_kv_heads, d = c.d_model, F = c.d_ffn;
     const int n_ssq = (d + 127) / 128;
 
+    // Passes of more than 32 rows run their GEMMs on the dense kernels (every weight byte read once per block of up to 160
+    // tokens); their activation arrays are in that kernel's operand order, with the token block size of the consumer.
+    ctx->pass_dense = ctx->layers[0].qkv.packed_u != nullptr && (M > 32 || ctx->force_dense);
+    const bool dense = ctx->pass_dense;
+    const int tbs_qkv = dense ? dense_plan(M, dv.Nqkv, ctx->n_sm).tbs : 0, tbs_o = dense ? dense_plan(M, d, ctx->n_sm).tbs : 0;
     // Every kernel of the chain is launched with programmatic stream serialisation: it may start while its
     // predecessor drains and blocks in griddepcontrol.wait before touching the predecessor's output.
     {
@@ -456,7 +521,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         CU(launch_pdl(rope_table_kernel, dim3((n + 127) / 128), dim3(128), 0, st, meta, M, hd, log((double)c.rope_base),
                       cs, sn, ctx->W<long long>(ctx->ws.kvoff), c.n_pages, Hkv, c.page_size));
         CU(launch_pdl(embed_kernel, dim3(M), dim3(kEmbedThreads), 0, st, x, (const uint16_t*)ctx->emb, meta.row_tok, M,
-                      (const float*)ctx->layers[0].n1, d, xf_h, ssqA, n_ssq));
+                      (const float*)ctx->layers[0].n1, d, xf_h, ssqA, n_ssq, tbs_qkv));
         ctx->n_launch += 2;
     }
     int max_item_rows = 1;
@@ -479,7 +544,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         aa.layer = l; aa.n_pages = c.n_pages; aa.page_size = c.page_size; aa.M = M; aa.Hq = Hq; aa.Hkv = Hkv;
         aa.n_max = n_max; aa.slot_c = attn_slot_c_bytes(hd, all_short); aa.row_groups = row_groups;
         aa.o_part = o_part; aa.m_part = m_part; aa.l_part = l_part; aa.tickets = ctx->W<int>(ctx->ws.tickets);
-        aa.xf_out = (uint16_t*)xf_attn; aa.err = ctx->err_word();
+        aa.xf_out = (uint16_t*)xf_attn; aa.xd_tbs = tbs_o; aa.err = ctx->err_word();
         if (hd == 128) CU(launch_pdl(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, aa));
         else CU(launch_pdl(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, aa));
         ctx->n_launch += 1;
@@ -489,39 +554,39 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         const LayerW& lw = ctx->layers[l];
         {   // q, k, v = W_qkv . norm(x); RoPE; K/V appended to the pages
             GemmArgs a = base;
-            a.W = lw.qkv.packed; a.xf = (const uint4*)xf_h; a.N = dv.Nqkv; a.ssq_in = ssqA;
+            a.xf = (const uint4*)xf_h; a.N = dv.Nqkv; a.ssq_in = ssqA;
             a.q_out = qbuf; a.kv_pool = ctx->kv_pool; a.cs = cs; a.sn = sn;
             a.row_kvoff = ctx->W<long long>(ctx->ws.kvoff);
             a.Hq = Hq; a.Hkv = Hkv; a.hd = hd; a.layer = l; a.n_pages = c.n_pages; a.page_size = c.page_size;
-            int rc_ = launch_gemm(ctx, kQkvRope, a, d);
+            int rc_ = launch_gemm(ctx, kQkvRope, lw.qkv, a, d, 0);
             if (rc_) return rc_;
         }
         { int rc_ = launch_attn(l); if (rc_) return rc_; }
         {   // x += W_o . attn; xf_h = x * ffn gain; ssqB
             GemmArgs a = base;
-            a.W = lw.o.packed; a.xf = (const uint4*)xf_attn; a.N = d; a.ssq_in = nullptr;
+            a.xf = (const uint4*)xf_attn; a.N = d; a.ssq_in = nullptr;
             a.x = x; a.xf_out = (uint16_t*)xf_h; a.gain_next = lw.n2; a.ssq_out = ssqB;
             a.pf = gemm_prefetch_of(lw.gu.packed, M, 2 * F, d, pf_depth);
-            int rc_ = launch_gemm(ctx, kResid, a, dv.qd);
+            int rc_ = launch_gemm(ctx, kResid, lw.o, a, dv.qd, 2 * F);
             if (rc_) return rc_;
         }
         {   // act = silu(W_g . norm(x)) * (W_u . norm(x))
             GemmArgs a = base;
-            a.W = lw.gu.packed; a.xf = (const uint4*)xf_h; a.N = 2 * F; a.ssq_in = ssqB;
+            a.xf = (const uint4*)xf_h; a.N = 2 * F; a.ssq_in = ssqB;
             a.xf_act = (uint16_t*)xf_act;
             a.pf = gemm_prefetch_of(lw.dn.packed, M, d, F, pf_depth);
-            int rc_ = launch_gemm(ctx, kSwiglu, a, d);
+            int rc_ = launch_gemm(ctx, kSwiglu, lw.gu, a, d, d);
             if (rc_) return rc_;
         }
         {   // x += W_d . act; xf_h = x * (next layer's attention gain | final gain); ssqA
             GemmArgs a = base;
-            a.W = lw.dn.packed; a.xf = (const uint4*)xf_act; a.N = d; a.ssq_in = nullptr;
+            a.xf = (const uint4*)xf_act; a.N = d; a.ssq_in = nullptr;
             a.x = x; a.xf_out = (uint16_t*)xf_h;
             a.gain_next = l + 1 < c.n_layers ? ctx->layers[l + 1].n1 : ctx->final_norm;
             a.ssq_out = ssqA;
             if (l + 1 < c.n_layers) a.pf = gemm_prefetch_of(ctx->layers[l + 1].qkv.packed, M, dv.Nqkv, d, pf_depth);
             else if (want_logits) a.pf = gemm_prefetch_of(ctx->lm.packed, M, c.vocab, d, pf_depth);
-            int rc_ = launch_gemm(ctx, kResid, a, F);
+            int rc_ = launch_gemm(ctx, kResid, lw.dn, a, F, l + 1 < c.n_layers ? dv.Nqkv : c.vocab);
             if (rc_) return rc_;
         }
     }
@@ -531,8 +596,8 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         RowStat* stats = ctx->W<RowStat>(ctx->ws.stats);
         {
             GemmArgs a = base;
-            a.W = ctx->lm.packed; a.xf = (const uint4*)xf_h; a.N = c.vocab; a.ssq_in = ssqA; a.out = logits;
-            int rc_ = launch_gemm(ctx, kPlain, a, d);
+            a.xf = (const uint4*)xf_h; a.N = c.vocab; a.ssq_in = ssqA; a.out = logits;
+            int rc_ = launch_gemm(ctx, kPlain, ctx->lm, a, d, 0);
             if (rc_) return rc_;
         }
         // plain launches from here on: they start after the GEMM has fully completed
@@ -616,6 +681,7 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
             cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, c.device) != cudaSuccess ||
             cudaDeviceGetAttribute(&thr_sm, cudaDevAttrMaxThreadsPerMultiProcessor, c.device) != cudaSuccess)
             return bail(PIPESD_E_CUDA);
+        ctx->n_sm = n_sm;
         cudaFuncAttributes fa;
         if (cudaFuncGetAttributes(&fa, c.head_dim == 128 ? (const void*)attn_kernel<128> : (const void*)attn_kernel<64>) != cudaSuccess)
             return bail(PIPESD_E_CUDA);
@@ -633,7 +699,6 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
                 ctx->attn_slots[qt][short_tail] = std::max(1, per_sm) * n_sm;
             }
     }
-    if (const char* e_pf = getenv("PIPESD_PF_KB")) ctx->pf_depth = (uint32_t)atoi(e_pf) << 10;
     ctx->kv_pool = (uint16_t*)mem->kv;
     ctx->wsp = (char*)mem->workspace;
     for (int i = 0; i < pipesd_ctx::kStages; ++i) {
@@ -668,6 +733,10 @@ int32_t pipesd_ctx_create(const pipesd_model_cfg* cfg, const pipesd_weights* w, 
         int blocks = (int)std::min<size_t>((total + 255) / 256, 148 * 16);
         g.packed = (uint4*)take(gemm_packed_bytes(N, K));
         gemm_pack_kernel<<<blocks, 256, 0, st>>>(ps, g.packed, N, K);
+        if (c.max_rows > 32) {
+            g.packed_u = (uint4*)take(gemm_packed_bytes(N, K));
+            gemm_pack_umma_kernel<<<blocks, 256, 0, st>>>(ps, g.packed_u, N, K);
+        }
     };
     ctx->emb = (uint16_t*)take((size_t)c.vocab * c.d_model * 2);
     if (cudaMemcpyAsync(ctx->emb, w->tok_emb, (size_t)c.vocab * c.d_model * 2, cudaMemcpyDeviceToDevice, st) !=
@@ -1153,6 +1222,14 @@ int32_t pipesd_gemm_run(const void* packed, const float* x, float* y, void* scra
     if (!packed || !x || !y || !scratch || M < 1 || N < 16 || K < 16 || N % 16 || K % 16) return PIPESD_E_INVALID;
     if (ensure_device_ready() != PIPESD_OK) return PIPESD_E_CUDA;
     return gemm_run_with_scratch(packed, x, y, scratch, M, N, K, (cudaStream_t)cuda_stream);
+}
+
+int32_t pipesd_debug_force_dense(pipesd_ctx* ctx, int32_t on) {
+    if (!ctx) return PIPESD_E_INVALID;
+    if (on && ctx->cfg.max_rows <= 32)
+        return fail(ctx, PIPESD_E_INVALID, "pipesd_debug_force_dense: the context keeps no weights in the dense kernel's order (max_rows <= 32)");
+    ctx->force_dense = on != 0;
+    return PIPESD_OK;
 }
 
 int32_t pipesd_debug_attn_slots(pipesd_ctx* ctx, int32_t rows_per_kv_head, int32_t* out2) {

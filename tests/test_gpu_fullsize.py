@@ -247,12 +247,14 @@ def test_7b_ragged_batch_of_32_requests(seven_b):
         row += k + 1
     ctx.kv_rollback([it["req"] for it in items], [0] * n)
     # batch invariance: the same request alone gives the same decision, bit for bit
+    ctx.debug_force_dense(True)       # the kernels the batch of more than 32 rows ran on
     for i in range(n):
         ctx.debug_set_len(items[i]["req"], int(lens[i]))
         (alone,) = ctx.verify([items[i]], flags=binding.Q_HOST)
         assert alone == got[i], f"request {i}: batched {got[i]} != alone {alone}"
         ctx.kv_rollback([items[i]["req"]], [alone[0]])
         assert ctx.req_len(items[i]["req"]) == int(lens[i]) + 1 + alone[0]
+    ctx.debug_force_dense(False)
     print("\n" + tally.report())
     for it in items:
         ctx.req_close(it["req"])

@@ -133,8 +133,17 @@ def test_batched_ragged_verify_and_batch_invariance():
         k = int(ks[i])
         assert logit_rel_err(logits[row:row + k + 1], ref["logits"]).max() < LOGIT_TOL
         tally.check(got[i], ref, ref["logits"], q, u, where=f"request {i}")
+        # alone, on the kernels the batch ran on (more than 32 rows: the dense ones), then on the small-pass kernels
+        ctx.debug_force_dense(True)
         (alone,) = ctx.verify([solo[i]], flags=binding.Q_HOST)
         assert alone == got[i], "batched and single-request results differ"
+        assert logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max() < LOGIT_TOL
+        ctx.debug_force_dense(False)
+        ctx.kv_rollback([solo[i]["req"]], [0])
+        ctx.debug_set_len(solo[i]["req"], int(lens[i]))
+        (small,) = ctx.verify([solo[i]], flags=binding.Q_HOST)
+        assert logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max() < LOGIT_TOL
+        tally.check(small, ref, ref["logits"], q, u, where=f"request {i} alone")
         row += k + 1
     ctx.kv_rollback([it["req"] for it in items], [g[0] for g in got])
     for i in range(n_req):
