@@ -60,6 +60,13 @@ class Tally:
                 f"max rel logit err {self.max_logit_err:.2e}")
 
 
+def decisions_from_logits(logits_rows, item):
+    """The accept/correct rule (CPU checker) applied to given logits rows [k+1, V] of one request: what a second run
+    of the same request must decide, up to decisions that sit inside the tie band."""
+    n, t, margins = oracle.reject(np.asarray(logits_rows, np.float64), item["q"], item["tokens"][1:], item["u"])
+    return dict(n_accepted=n, next_token=t, margins=margins)
+
+
 def draft_inputs(orc, shape, k, sigma, seed, request=0, round_=0, pending=None):
     """One round's inputs from the oracle's own target logits (q = softmax(l + sigma*noise))."""
     if pending is None:

