@@ -54,6 +54,23 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def tensor_peak():
+    """Sustained dense bf16 TFLOP/s (the projections of a large pass run inside a long step)."""
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        return float(json.loads(p.read_text())["bf16_tflops_sustained"]), "measured"
+    return 1400.0, "fallback"
+
+
+def pass_flops(shape, ks):
+    """Tensor-core flops of the projections of one pass as the kernels run them: every activation is a bf16 hi term and
+    a bf16 lo term, so each weight element meets two products per row (2 x 2 flops)."""
+    M = int(np.atleast_1d(ks).sum() + np.atleast_1d(ks).size)
+    d, F, V = shape.d_model, shape.d_ffn, shape.vocab
+    per_layer = (shape.q_dim + 2 * shape.kv_dim) * d + d * shape.q_dim + 3 * F * d
+    return 4.0 * M * (shape.n_layers * per_layer + V * d)
+
+
 def pass_bytes(shape, ks, cached_lens):
     """Algorithmic bytes of one verify pass over the requests (k_i drafts against cached_len_i positions): every
     weight once (bf16), embedding rows of the tokens, K/V of each cached prefix read and of the k_i+1 new rows
@@ -440,6 +457,15 @@ def main():
                                                 "regime": "no dependent-launch overlap (events between launches)"}},
         "clocks": clocks,
     }
+    if sum(ks) + n_req > 32:
+        # a pass of more than 32 rows runs its projections on the dense tensor-core kernel: those are bound by the
+        # tensor cores, the attention by HBM, so neither roofline alone bounds the pass; both fractions are given
+        tp, tp_kind = tensor_peak()
+        tfl = pass_flops(shape, ks) / (ms_step * 1e-3) / 1e12
+        line["roofline"]["kernel"] = "verify pass (chain of gemm_dense_kernel and attn_kernel launches)"
+        line["roofline"]["projections_tensor"] = {"bound": "tensor", "achieved": tfl, "peak": tp, "peak_kind": tp_kind,
+                                                  "unit": "TFLOP/s", "frac": tfl / tp,
+                                                  "note": "projection flops (hi and lo products) over the WHOLE pass time"}
     if world == 1 and not args.no_cpu_baseline:
         sample_reqs = list(range(min(n_req, 4)))
         dt, toks_o = oracle_time(oracle_prepare(shape, weights, lens, ks, sigmas, seed, requests=sample_reqs))
