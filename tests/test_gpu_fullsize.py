@@ -208,7 +208,7 @@ def test_7b_shape_real_prefill_short_prefix(seven_b):
 def test_7b_ragged_batch_of_32_requests(seven_b):
     """32 concurrent requests, prefix ~U[256,4096], k ~U{1..16}, sigma ~U[0.3,2]: ONE batched verify over the
     paged cache, per-request rollback.  The CPU checker covers a standing subset (extremes + others; all 32
-    with PIPESD_FULL=1); every request is also checked bit for bit against the same request verified alone."""
+    with PIPESD_FULL=1); every request is also verified alone and must decide what it decided in the batch (ties counted)."""
     from paper_2605_13319_b200 import binding
     shape, w, ctx, (lens, ks, sig) = seven_b
     V = shape.vocab
