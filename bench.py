@@ -534,9 +534,7 @@ def quick_run(args, ctx, shape, lens, ks, seed, torch):
 # profiles/ (taken on a two-layer model of the same shape -- same per-layer work -- and scaled to a full pass by the
 # layers it covers), with the hash of the kernel sources they were taken on: the figure is reported only while the
 # sources still hash to that value.
-# DRAM bytes per pass (dram__bytes_read.sum + dram__bytes_write.sum over every launch of a pass, ncu): taken on two layers
-# of the workload and scaled by the layer count, 16 x (474.08 + 469.23) MB + 264.14 MB.  Reported only while the
-# kernels' source still hashes to the value the counters were taken with.
+# 7b-k8: 16 x (474.08 + 469.23) MB for the layers + 264.14 MB for the rest of the pass.
 TRAFFIC = {"kernel_source_hash": "36b9b976fc05d1b0", "7b-k8": 15357054464.0}
 
 
