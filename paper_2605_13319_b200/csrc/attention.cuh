@@ -176,6 +176,11 @@ struct AttnArgs {
     int* tickets;              // [item][kv head][row group], zero between launches
     uint16_t* xf_out;          // the output projection's input: split-bf16 fragments, or (xd_tbs > 0) an xd array
     int xd_tbs;
+    // Weights of the projections that follow (nullable): while this kernel runs, HBM carries little besides the K/V
+    // it reads.  Once a CTA's own K/V tiles have all landed, its copy warp asks the L2 for this CTA's share of the
+    // first pf_len[i] bytes at pf_ptr[i] (128-byte lines dealt over the whole grid).  Purely a hint.
+    const unsigned char* pf_ptr[2];
+    size_t pf_len[2];
     int* err;
 };
 
@@ -372,6 +377,17 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a)
                         umma_bf16(t_L, ones_desc, bl, idesc_pv, 1);
                     }
                     umma_commit(bar_pv);
+                }
+                if (ok && t == ntiles - 1) {
+                    // every K/V tile of this CTA has landed and its last products are issued: hints for the weights
+                    // of the projections that follow
+                    const size_t n_thr = (size_t)gridDim.x * gridDim.y * gridDim.z * 32;
+                    const size_t g = (((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 32 + lane;
+#pragma unroll
+                    for (int r = 0; r < 2; ++r)
+                        if (a.pf_ptr[r] != nullptr)
+                            for (size_t o = g * 128; o < a.pf_len[r]; o += n_thr * 128)
+                                asm volatile("prefetch.global.L2 [%0];" ::"l"(a.pf_ptr[r] + o) : "memory");
                 }
                 if (ok && t + 2 < ntiles) {
                     ok = attn_wait_warp(bar_pv, (uint32_t)t & 1u);                       // V_t has been read

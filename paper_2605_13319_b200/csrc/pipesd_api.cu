@@ -260,6 +260,9 @@ struct pipesd_ctx {
     int n_sm = 148;             // SMs of the context's device
     bool force_dense = false;   // harness switch: the dense kernels also for passes of at most 32 rows
     bool pass_dense = false;    // the pass being enqueued runs on the dense kernels
+    // bytes of the O and gate/up weights the attention kernel pulls into L2 once its K/V has landed (measured: all of O
+    // and 16 MB of gate/up; more gains nothing, an SM takes data in only about 1.4 times faster than HBM delivers it)
+    size_t pf_attn[2] = {(size_t)64 << 20, (size_t)16 << 20};
     uint32_t pf_depth = 32u << 10;   // bytes per successor CTA that a GEMM pulls into L2 for the next GEMM
     std::string err;
     // launch accounting
@@ -545,6 +548,13 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         aa.n_max = n_max; aa.slot_c = attn_slot_c_bytes(hd, all_short); aa.row_groups = row_groups;
         aa.o_part = o_part; aa.m_part = m_part; aa.l_part = l_part; aa.tickets = ctx->W<int>(ctx->ws.tickets);
         aa.xf_out = (uint16_t*)xf_attn; aa.xd_tbs = tbs_o; aa.err = ctx->err_word();
+        if (!dense) {
+            const LayerW& lw = ctx->layers[l];
+            aa.pf_ptr[0] = reinterpret_cast<const unsigned char*>(lw.o.packed);
+            aa.pf_len[0] = std::min(gemm_packed_bytes(d, dv.qd), ctx->pf_attn[0]);
+            aa.pf_ptr[1] = reinterpret_cast<const unsigned char*>(lw.gu.packed);
+            aa.pf_len[1] = std::min(gemm_packed_bytes(2 * F, d), ctx->pf_attn[1]);
+        }
         if (hd == 128) CU(launch_pdl(attn_kernel<128>, ag, dim3(kAttnThreads), asmem, st, aa));
         else CU(launch_pdl(attn_kernel<64>, ag, dim3(kAttnThreads), asmem, st, aa));
         ctx->n_launch += 1;
