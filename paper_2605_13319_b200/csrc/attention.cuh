@@ -500,21 +500,21 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a)
             if (ok) ok = attn_wait_warp(bar_pv, (uint32_t)(ntiles - 1) & 1u);
             tc_fence_after();
             if (quarter == 0) {
-                for (int cb = half; cb < NB; cb += 2) {
+                // the column blocks go to the two warps of the quarter the other way round than O^T's below, so that with
+                // one block the denominators are stored by a warp that has no O^T columns to store
+                for (int cb = half ^ 1; cb < NB; cb += 2) {
                     float l[16];
                     tmem_ld16(t_L + cb * 16, l);
                     tmem_ld_wait();
                     if (lane == 0) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int n = cb * 16 + i;
-                            const float lv = ok ? l[i] : 0.f;
-                            Fl[n] = lv;
-                            if (nsplit > 1 && n < n_rows) {
-                                a.l_part[slot0 + (size_t)n * nsplit + sp] = lv;
-                                a.m_part[slot0 + (size_t)n * nsplit + sp] = m_ref[n];
-                            }
-                        }
+                        for (int i = 0; i < 16; ++i) Fl[cb * 16 + i] = ok ? l[i] : 0.f;
+                    }
+                    __syncwarp();
+                    const int n = cb * 16 + lane;
+                    if (nsplit > 1 && lane < 16 && n < n_rows) {         // lane = row: one store each
+                        a.l_part[slot0 + (size_t)n * nsplit + sp] = Fl[n];
+                        a.m_part[slot0 + (size_t)n * nsplit + sp] = m_ref[n];
                     }
                 }
             }
@@ -578,34 +578,37 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a)
     __syncthreads();
     release_tmem();
     if (!*s_last) return;
-    // warp = row, lane = four columns: one round covers nine rows
+    // warp = row, lane = four columns: one round covers nine rows.  All of a row's loads are issued before the first
+    // use (one trip to the L2 for up to kMergeBatch splits): lane j fetches split j's maximum and denominator, every
+    // lane its four columns of each split's numerator; the sums run in split order.
+    constexpr int kMergeBatch = 10;
     for (int rl = warp; rl < n_rows; rl += kAttnThreads / 32) {
         const size_t sl0 = slot0 + (size_t)rl * nsplit;
-        float ms[kAttnMaxSplits];
+        const float m_mine = lane < nsplit ? __ldcg(a.m_part + sl0 + lane) : -INFINITY;
+        const float l_mine = lane < nsplit ? __ldcg(a.l_part + sl0 + lane) : 0.f;
+        float4 ov[kMergeBatch];
 #pragma unroll
-        for (int j = 0; j < kAttnMaxSplits; ++j) ms[j] = j < nsplit ? __ldcg(a.m_part + sl0 + j) : -INFINITY;
-        float m = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < kAttnMaxSplits; ++j) m = fmaxf(m, ms[j]);
+        for (int j = 0; j < kMergeBatch; ++j)
+            ov[j] = (j < nsplit && lane < HD / 4) ? __ldcg(reinterpret_cast<const float4*>(a.o_part + (sl0 + j) * HD) + lane)
+                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float m = warp_max_redux(m_mine);
+        // an empty split, or one beyond the causal horizon, has no maximum and weighs nothing
+        const float w_mine = (m_mine == -INFINITY) ? 0.f : exp2f(m_mine - m);
+        const float wl_mine = w_mine * l_mine;
         float den = 0.f;
         float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int j0 = 0; j0 < kAttnMaxSplits; j0 += 8) {         // eight splits' loads in flight together, summed in split order
-            if (j0 >= nsplit) break;
-            float ls[8];
-            float4 ov[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const bool on = j0 + j < nsplit;
-                ls[j] = on ? __ldcg(a.l_part + sl0 + j0 + j) : 0.f;
-                ov[j] = (on && lane < HD / 4) ? __ldcg(reinterpret_cast<const float4*>(a.o_part + (sl0 + j0 + j) * HD) + lane)
-                                              : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float w = (ms[j0 + j] == -INFINITY) ? 0.f : exp2f(ms[j0 + j] - m);   // an empty split or one beyond the causal horizon
-                den += w * ls[j];
-                num.x += w * ov[j].x; num.y += w * ov[j].y; num.z += w * ov[j].z; num.w += w * ov[j].w;
+        for (int j = 0; j < kMergeBatch; ++j) {
+            const float w = __shfl_sync(0xffffffffu, w_mine, j);
+            den += __shfl_sync(0xffffffffu, wl_mine, j);
+            num.x += w * ov[j].x; num.y += w * ov[j].y; num.z += w * ov[j].z; num.w += w * ov[j].w;
+        }
+        for (int j = kMergeBatch; j < nsplit; ++j) {             // more splits than one batch holds: one by one
+            const float w = __shfl_sync(0xffffffffu, w_mine, j);
+            den += __shfl_sync(0xffffffffu, wl_mine, j);
+            if (lane < HD / 4) {
+                const float4 o = __ldcg(reinterpret_cast<const float4*>(a.o_part + (sl0 + j) * HD) + lane);
+                num.x += w * o.x; num.y += w * o.y; num.z += w * o.z; num.w += w * o.w;
             }
         }
         if (lane < HD / 4) {
