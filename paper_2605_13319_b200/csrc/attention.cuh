@@ -167,6 +167,7 @@ struct AttnArgs {
     PassMeta meta;
     const uint16_t* kv_pool;
     int layer, n_pages, page_size, M, Hq, Hkv;
+    int rows_cap;              // query rows per row group (kAttnMaxRows, or 16 for a batch whose requests have up to 32)
     int n_max;                 // N the launch's shared memory was sized for
     int slot_c;                // bytes of the ring's third slot
     int row_groups;
@@ -209,9 +210,9 @@ __global__ void __launch_bounds__(kAttnThreads, 3) attn_kernel(const AttnArgs a)
     const int kvh = blockIdx.y % Hkv, rg = blockIdx.y / Hkv;
     const int G = Hq / Hkv;
     const int R = G * rows;
-    const int rho0 = rg * kAttnMaxRows;
+    const int rho0 = rg * a.rows_cap;
     if (rho0 >= R) return;
-    const int n_rows = min(kAttnMaxRows, R - rho0);
+    const int n_rows = min(a.rows_cap, R - rho0);
     const int N = (n_rows + 15) & ~15;
     if (N > a.n_max) return;
     const int NG = N / 8, NB = N / 16;

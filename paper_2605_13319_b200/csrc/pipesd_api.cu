@@ -442,10 +442,27 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     bool all_short = true;       // no split of the pass has more than two key tiles, the second a short one
     // attention work of the pass in (keys x CTA groups): a request gets the share of the device's resident CTAs that its
     // keys are of the pass's, so that the CTAs of the whole pass fill one wave
+    // Rows per row group.  A CTA with up to 16 query rows shares its SM with a second one, a CTA with 17..32 does not;
+    // in a batch whose largest request has 17..32 rows per KV head the groups are therefore cut at 16 (requests above 16
+    // rows read their K/V twice) as long as that adds at most an eighth to the K/V the pass reads.
+    int rows_cap = kAttnMaxRows;
+    {
+        int maxR0 = 1;
+        double keys = 0.0, keys16 = 0.0;
+        for (int i = 0; i < n_items; ++i) {
+            const int R_i = items[i].rows * (c.n_q_heads / c.n_kv_heads);
+            maxR0 = std::max(maxR0, R_i);
+            keys += (double)(items[i].base + items[i].rows);
+            keys16 += (double)(items[i].base + items[i].rows) * ((R_i + 15) / 16);
+        }
+        if (n_items > 1 && maxR0 > 16 && maxR0 <= 32 && keys16 <= 1.125 * keys &&
+            ctx->attn_slots[1][0] > ctx->attn_slots[2][0])
+            rows_cap = 16;
+    }
     double pass_work = 0.0;
     for (int i = 0; i < n_items; ++i) {
         const int R_i = items[i].rows * (c.n_q_heads / c.n_kv_heads);
-        pass_work += (double)(items[i].base + items[i].rows) * c.n_kv_heads * ((R_i + kAttnMaxRows - 1) / kAttnMaxRows);
+        pass_work += (double)(items[i].base + items[i].rows) * c.n_kv_heads * ((R_i + rows_cap - 1) / rows_cap);
     }
     {   // launch order of the attention CTAs: longest requests first
         int32_t* ord = I(ml.it_order);
@@ -458,10 +475,10 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         const ItemDesc& it = items[i];
         const int total = it.base + it.rows;
         const int R_i = it.rows * (c.n_q_heads / c.n_kv_heads);                  // query rows per KV head
-        const int rg_i = (R_i + kAttnMaxRows - 1) / kAttnMaxRows;
+        const int rg_i = (R_i + rows_cap - 1) / rows_cap;
         const int units_i = (int)std::min(1.0e9, std::ceil(pass_work / (double)total));
         const AttnSplit sp = attn_split_plan(total, c.page_size, std::max(units_i, c.n_kv_heads * rg_i),
-                                             ctx->attn_slots[attn_rows_n(R_i) / 16]);
+                                             ctx->attn_slots[attn_rows_n(std::min(R_i, rows_cap)) / 16]);
         const int nsplit = sp.splits, chunk = sp.keys_per_split;
         if (chunk > kAttnTile + kAttnShortTail) all_short = false;
         I(ml.it_slot)[i] = it.slot;
@@ -530,8 +547,8 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     int max_item_rows = 1;
     for (auto& it : items) max_item_rows = std::max(max_item_rows, it.rows);
     const int maxR = max_item_rows * (Hq / Hkv);                      // query rows that share one KV head
-    const int n_max = attn_rows_n(maxR);
-    const int row_groups = (maxR + kAttnMaxRows - 1) / kAttnMaxRows;
+    const int n_max = attn_rows_n(std::min(maxR, rows_cap));
+    const int row_groups = (maxR + rows_cap - 1) / rows_cap;
     const size_t asmem = attn_smem_bytes(hd, n_max, all_short);
     GemmArgs base = {};
     base.M = M;
@@ -545,7 +562,7 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
         AttnArgs aa = {};
         aa.q = qbuf; aa.meta = meta; aa.kv_pool = ctx->kv_pool;
         aa.layer = l; aa.n_pages = c.n_pages; aa.page_size = c.page_size; aa.M = M; aa.Hq = Hq; aa.Hkv = Hkv;
-        aa.n_max = n_max; aa.slot_c = attn_slot_c_bytes(hd, all_short); aa.row_groups = row_groups;
+        aa.rows_cap = rows_cap; aa.n_max = n_max; aa.slot_c = attn_slot_c_bytes(hd, all_short); aa.row_groups = row_groups;
         aa.o_part = o_part; aa.m_part = m_part; aa.l_part = l_part; aa.tickets = ctx->W<int>(ctx->ws.tickets);
         aa.xf_out = (uint16_t*)xf_attn; aa.xd_tbs = tbs_o; aa.err = ctx->err_word();
         if (!dense) {
