@@ -443,8 +443,8 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
     // attention work of the pass in (keys x CTA groups): a request gets the share of the device's resident CTAs that its
     // keys are of the pass's, so that the CTAs of the whole pass fill one wave
     // Rows per row group.  A CTA with up to 16 query rows shares its SM with a second one, a CTA with 17..32 does not;
-    // in a batch whose largest request has 17..32 rows per KV head the groups are therefore cut at 16 (requests above 16
-    // rows read their K/V twice) as long as that adds at most an eighth to the K/V the pass reads.
+    // in a pass whose largest request has 17..32 rows per KV head the groups are therefore cut at 16 (requests above 16
+    // rows read their K/V twice) as long as that adds at most an eighth to the K/V the pass reads ...
     int rows_cap = kAttnMaxRows;
     {
         int maxR0 = 1;
@@ -455,7 +455,11 @@ int run_pass(pipesd_ctx* ctx, const std::vector<ItemDesc>& items, bool want_logi
             keys += (double)(items[i].base + items[i].rows);
             keys16 += (double)(items[i].base + items[i].rows) * ((R_i + 15) / 16);
         }
-        if (n_items > 1 && maxR0 > 16 && maxR0 <= 32 && keys16 <= 1.125 * keys &&
+        // ... or at most a tenth to the bytes of the pass (weights once + K/V): a single request of 17 rows at the 7B shape
+        const double kv_key = 4.0 * c.n_layers * c.n_kv_heads * c.head_dim;                     // K and V bytes of a position
+        const double w_bytes = 2.0 * ((double)c.n_layers * ((double)(dv.Nqkv + dv.qd) * c.d_model + 3.0 * c.d_ffn * c.d_model) +
+                                      (double)c.vocab * c.d_model);
+        if (maxR0 > 16 && maxR0 <= 32 && (keys16 <= 1.125 * keys || (keys16 - keys) * kv_key <= 0.1 * (w_bytes + keys * kv_key)) &&
             ctx->attn_slots[1][0] > ctx->attn_slots[2][0])
             rows_cap = 16;
     }
