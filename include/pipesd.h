@@ -142,7 +142,7 @@ const char *pipesd_last_error(const pipesd_ctx *ctx);
  * cloud "only starts a server and executes NAV using the target model", Sec. 4.2, and says nothing about memory.) */
 int32_t pipesd_query_sizes(const pipesd_model_cfg *cfg, pipesd_sizes *out);
 
-/* Create a context = load the target model that performs NAV (Sec. 4.2, cloud component "Target Model"; Sec. 5.1 for
+/* Create a context = load the target model that performs NAV (Sec. 4.2, the target-model component of the cloud side; Sec. 5.1 for
  * the model family): validates cfg, repacks the caller's weights into mem->weights (the caller may free its own
  * weight tensors once pipesd_ctx_sync has returned), zero-initialises metadata.
  * `cuda_stream` is a cudaStream_t (null = the legacy default stream). */
@@ -164,7 +164,7 @@ int32_t pipesd_req_close(pipesd_ctx *ctx, int32_t req);
 int32_t pipesd_req_len(pipesd_ctx *ctx, int32_t req, int32_t *len);
 
 /* Append n prompt tokens (host ids) to the request's cache -- the accepted prefix that every NAV pass runs against
- * (Sec. 2.2: drafts are validated "against the accepted prefix"): the same layer stack as verify, run in chunks of
+ * (Sec. 2.2: the drafts are checked against the prefix accepted so far): the same layer stack as verify, run in chunks of
  * at most min(max_rows, 32) rows, no acceptance step.  If last_logits (host, vocab floats) is non-null it
  * receives the logits of the final position; the call then synchronises. */
 int32_t pipesd_prefill(pipesd_ctx *ctx, int32_t req, const int32_t *tokens, int32_t n, float *last_logits);

@@ -14,7 +14,7 @@ Where the method reaches a result that has a plain definition, this file is that
   definition of "optimal", not the paper's dynamic programme (Algorithm 1), which the library implements and which
   Theorem 4.1 claims to reach the same value.
 * ``trigger_sequence`` follows Sec. 3.3 step by step: C1* = C1 * P(D_n); verification is triggered when C1* <= R1
-  or when P(D_n) <= R2; C1 is the product over the tokens "computed but not yet verified", so it restarts at 1
+  or when P(D_n) <= R2; C1 is the product over the tokens generated since the last verification, so it restarts at 1
   after either kind of trigger.
 """
 from __future__ import annotations
