@@ -431,7 +431,8 @@ def main():
     line = {
         "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16 weights x split-bf16 activations, fp32 accumulate", "data": "synthetic",
+        "vs_baseline": None, "dtype": "bf16", "arithmetic": "bf16 weights x split-bf16 (hi + lo) activations on the tensor cores, fp32 accumulate; K/V bf16",
+        "data": "synthetic",
         "config": cfg,
         "pass": {"bytes": bytes_pass, "gbs": pass_gbs, "frac_of_nominal_8TBs": pass_gbs / NOMINAL_HBM_GBS,
                  "frac_of_measured_copy": pass_gbs / peak},
