@@ -103,12 +103,17 @@ def test_multi_round_verify_rollback_lockstep():
     ctx.close()
 
 
-def test_batched_ragged_verify_and_batch_invariance():
-    """Several requests with different prefix lengths and draft counts in ONE call == each alone == checker."""
+@pytest.mark.parametrize("n_kv_heads", [2, 4])
+def test_batched_ragged_verify_and_batch_invariance(n_kv_heads):
+    """Several requests with different prefix lengths and draft counts in ONE call == each alone == checker.
+    Two query heads per KV head: up to 34 query rows per KV head, one row group; one (MHA): up to 17, which the
+    batch runs as row groups of 16 + 1."""
     from paper_2605_13319_b200 import binding
-    shape = synth.TINY.scaled(name="tiny-gqa", n_kv_heads=2)
+    shape = synth.TINY.scaled(name=f"tiny-kv{n_kv_heads}", n_kv_heads=n_kv_heads)
     n_req = 6
     lens, ks, sig = synth.ragged_requests(3, n_req, 5, 150, 1, 16)
+    if n_kv_heads == 4:
+        ks[1] = 16          # a request of 17 rows: the batch's row groups are cut at 16
     w = synth.make_weights(shape, 2)
     ctx = binding.Context(shape, w, n_pages=(200 // 16 + 2) * n_req * 2, max_seq=200, max_requests=2 * n_req,
                           max_rows=max(33, int(ks.sum() + n_req)), max_draft=16, poison=True)
