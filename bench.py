@@ -535,9 +535,9 @@ def quick_run(args, ctx, shape, lens, ks, seed, torch):
 # profiles/ (taken on a two-layer model of the same shape -- same per-layer work -- and scaled to a full pass by the
 # layers it covers), with the hash of the kernel sources they were taken on: the figure is reported only while the
 # sources still hash to that value.
-# 7b-k8: 16 x (456.06 + 435.78) MB for the layers + 254.46 MB for the rest of the pass, captured with the caches kept
+# 7b-k8: 16 x (455.70 + 434.98) MB for the layers + 254.42 MB for the rest of the pass, captured with the caches kept
 # between launches (ncu --cache-control none): hinted lines are counted where they are fetched, not twice.
-TRAFFIC = {"kernel_source_hash": "8f08418da689238d", "7b-k8": 14523924736.0}
+TRAFFIC = {"kernel_source_hash": "a6d15aa46c461db2", "7b-k8": 14505346816.0}
 
 
 if __name__ == "__main__":
